@@ -1,0 +1,474 @@
+"""Pins of the CPU oracle against facts that do not come from the oracle itself.
+
+Each test fixes a part of oracle/qgalore_oracle.py to something the paper or the
+mathematics determines: published known answers, error bounds, expectations,
+reductions to textbook routines written out here independently, brute force on
+tiny inputs.  CPU only.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle as O
+from paper_2407_08296_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ----------------------------------------------------------------------------- Philox
+def _kat_rows():
+    rows = []
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            rows.append([int(w, 16) for w in line.split()])
+    return rows
+
+
+def test_philox_known_answers():
+    rows = _kat_rows()
+    assert len(rows) == 3
+    for w in rows:
+        out = O.philox4x32_10([np.array([c], dtype=np.uint32) for c in w[:4]], w[4:6])
+        assert [int(o[0]) for o in out] == w[6:10]
+
+
+def test_sr_uniform16_lane_mapping():
+    seed, step = (0x1234 << 32) | 0xABCDEF01, (7 << 32) | 99
+    h = O.sr_uniform16(seed, step, 5, 37)
+    for i, j in [(0, 0), (0, 1), (3, 7), (4, 8), (2, 36), (1, 22)]:
+        x = O.philox4x32_10(
+            [np.array([v], dtype=np.uint32) for v in (j >> 3, i, step & 0xFFFFFFFF, step >> 32)],
+            (seed & 0xFFFFFFFF, seed >> 32))
+        lane = j & 7
+        want = (int(x[lane >> 1][0]) >> (16 * (lane & 1))) & 0xFFFF
+        assert int(h[i, j]) == want
+    # a window taken with (row0, col0) is the same as slicing the whole field
+    win = O.sr_uniform16(seed, step, 2, 11, row0=2, col0=13)
+    assert np.array_equal(win, h[2:4, 13:24])
+    assert h.max() <= 0xFFFF
+
+
+def test_sr_uniform16_is_uniform():
+    h = O.sr_uniform16(5, 3, 2000, 512).astype(np.float64)
+    assert abs(h.mean() - 32767.5) < 4 * 65536 / math.sqrt(12 * h.size)
+    hist = np.bincount((h // 4096).astype(np.int64).ravel(), minlength=16)
+    expect = h.size / 16
+    assert np.all(np.abs(hist - expect) < 5 * math.sqrt(expect))
+
+
+# ----------------------------------------------------------------------------- quantizer (Sec. 3.1)
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("cols", [256, 1376, 85, 600])
+def test_quantizer_half_step_bound_and_range(bits, cols):
+    rng = np.random.default_rng(bits * 1000 + cols)
+    x = (rng.standard_normal((64, cols)) * 0.02).astype(np.float32)
+    q = O.quantize_rtn(x, bits)
+    qlo, qhi = -(1 << (bits - 1)), (1 << (bits - 1)) - 1          # clamp range of the Quant_n equation
+    assert q.codes.min() >= qlo and q.codes.max() <= qhi
+    ngroups = (cols + 255) // 256
+    assert q.scales.shape == (64, ngroups) and q.zeros.shape == (64, ngroups)
+    xh = O.dequantize(q)
+    for k in range(ngroups):
+        a, b = k * 256, min(cols, k * 256 + 256)
+        s = q.scales[:, k:k + 1].astype(np.float64)
+        err = np.abs(xh[:, a:b].astype(np.float64) - x[:, a:b])
+        assert np.all(err <= 0.5 * s * (1 + 1e-3))                  # half a group step
+        seg, cod = x[:, a:b], q.codes[:, a:b]
+        rows = np.arange(64)
+        assert np.all(cod[rows, seg.argmin(axis=1)] == qlo)         # group minimum -> lowest code
+        assert np.all(cod[rows, seg.argmax(axis=1)] == qhi)         # group maximum -> highest code
+        # the scale is (max - min) / (2^n - 1)
+        want = (seg.max(axis=1).astype(np.float64) - seg.min(axis=1)) / ((1 << bits) - 1)
+        assert np.allclose(q.scales[:, k], want, rtol=3e-7)
+    assert np.all(q.zeros == np.rint(q.zeros))
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_requantizing_a_dequantized_tensor_reproduces_codes(bits):
+    rng = np.random.default_rng(11 + bits)
+    x = rng.standard_normal((32, 700)).astype(np.float32)
+    q1 = O.quantize_rtn(x, bits)
+    q2 = O.quantize_rtn(O.dequantize(q1), bits)
+    assert np.array_equal(q1.codes, q2.codes)
+    assert np.allclose(q1.scales, q2.scales, rtol=2.5e-7)
+    assert np.array_equal(q1.zeros, q2.zeros)
+
+
+def test_quantizer_hand_example():
+    # group {0, 1, ..., 255} / 4: min 0, max 63.75, s = 0.25 exactly, z = -128, code = k - 128
+    x = (np.arange(256, dtype=np.float32) / 4)[None, :]
+    q = O.quantize_rtn(x, 8)
+    assert q.scales[0, 0] == np.float32(0.25) and q.zeros[0, 0] == -128
+    assert np.array_equal(q.codes[0], np.arange(256) - 128)
+    assert np.array_equal(O.dequantize(q), x)
+    # INT4: {-7.5, -6.5, ..., 7.5}: s = 1, min * inv = -7.5 -> rint -8 (ties to even), z = 0
+    x4 = (np.arange(16, dtype=np.float32) - 7.5)[None, :]
+    q4 = O.quantize_rtn(x4, 4)
+    assert q4.scales[0, 0] == 1 and q4.zeros[0, 0] == 0
+    # rint(-7.5) = -8, rint(-6.5) = -6, rint(-5.5) = -6 ... ties to even
+    assert np.array_equal(q4.codes[0], np.clip(np.rint(x4[0]), -8, 7).astype(np.int8))
+
+
+def test_quantizer_degenerate_groups():
+    x = np.zeros((3, 300), dtype=np.float32)
+    x[1, :] = 0.5
+    x[2, :256] = -3.0
+    x[2, 256:] = np.linspace(-1, 1, 44, dtype=np.float32)
+    q = O.quantize_rtn(x, 8)
+    assert q.scales[0, 0] == 1 and q.zeros[0, 0] == 0 and np.all(q.codes[0] == 0)
+    assert q.scales[1, 0] == np.float32(0.5) and np.all(q.codes[1] == 1)
+    assert q.scales[2, 0] == 3 and np.all(q.codes[2, :256] == -1)
+    assert np.array_equal(O.dequantize(q)[:, :256], x[:, :256])
+    # a group symmetric about 0 puts min/s and max/s on rounding ties (-127.5, 127.5); with the
+    # reciprocal rounded to binary32 the top code may come out one below the clamp edge
+    assert q.codes[2, 256] == -128 and q.codes[2, 299] in (126, 127)
+    assert np.all(np.abs(O.dequantize(q)[2, 256:] - x[2, 256:]) <= 0.5 * q.scales[2, 1] * (1 + 1e-3))
+
+
+def test_int4_packing_layout():
+    codes = np.array([[-8, 7, 0, -1, 3]], dtype=np.int8)
+    p = O.pack_int4(codes)
+    # byte k = (q[2k] + 8) | (q[2k+1] + 8) << 4 ; odd tail padded with code 0
+    assert p.tolist() == [[0 | (15 << 4), 8 | (7 << 4), 11 | (8 << 4)]]
+    assert np.array_equal(O.unpack_int4(p, 5), codes)
+    rng = np.random.default_rng(0)
+    c = rng.integers(-8, 8, size=(7, 130)).astype(np.int8)
+    assert np.array_equal(O.unpack_int4(O.pack_int4(c), 130), c)
+
+
+# ----------------------------------------------------------------------------- stochastic rounding (Sec. 3.4)
+FRACS = [0.0, 2.0 ** -16, 0.01, 0.25, 0.5, 0.75, 0.99]
+
+
+def _sr_field(rows):
+    """Groups whose scale is exactly 1: element 0 = -100 (min), element 1 = 155 (max), the rest
+    k + frac with 36 columns per fraction.  Two groups per row."""
+    g = np.zeros(256, dtype=np.float32)
+    g[0], g[1] = -100.0, 155.0
+    fr = np.zeros(256, dtype=np.float32)
+    for f_i, f in enumerate(FRACS):
+        cols = 2 + f_i * 36 + np.arange(36)
+        ints = (np.arange(36) * 5 - 90).astype(np.float32)
+        g[cols] = ints + np.float32(f)
+        fr[cols] = f
+    g[2 + 7 * 36:] = 3.0
+    x = np.tile(np.concatenate([g, g])[None, :], (rows, 1))
+    return x, np.concatenate([fr, fr])
+
+
+def test_sr_expectation_equals_input():
+    rows = 100_000                                    # 10^5 draws per element
+    x, _ = _sr_field(rows)
+    q = O.quantize_sr(x, seed=42, step=3)
+    assert np.all(q.scales == 1) and np.all(q.zeros == -28)
+    val = O.dequantize(q).astype(np.float64)          # = floor(x) + up
+    lo = np.floor(x[0].astype(np.float64))
+    assert np.all((val == lo) | (val == lo + 1))      # only floor or ceil ever appear
+    mean = val.mean(axis=0)
+    xt = x[0].astype(np.float64)
+    frac = xt - lo
+    # per element: 4 sigma of a binomial mean; 16-bit draws add a bias below 2^-16
+    sigma = np.sqrt(np.maximum(frac * (1 - frac), 1e-12) / rows)
+    assert np.all(np.abs(mean - xt) <= 4 * sigma + 2.0 ** -16 + 1e-9)
+    # pooled over the 72 columns that share a fraction: E[W_q] = W to 1e-3 LSB
+    for f_i in range(len(FRACS)):
+        cols = np.concatenate([2 + f_i * 36 + np.arange(36), 256 + 2 + f_i * 36 + np.arange(36)])
+        assert abs((mean[cols] - xt[cols]).mean()) < 1e-3
+    # exact integers never move
+    zc = np.concatenate([2 + np.arange(36), 256 + 2 + np.arange(36)])
+    assert np.all(val[:, zc] == xt[zc])
+
+
+def test_sr_accumulates_sub_lsb_updates_where_rtn_loses_them():
+    # Sec. 3.4: a small update vanishes under round-to-nearest and survives, in expectation, under SR.
+    rows = 4
+    base = np.zeros((rows, 256), dtype=np.float32)
+    base[:, 0], base[:, 1] = -100.0, 155.0            # pins the scale at 1
+    base[:, 2:] = 10.0
+    w_rtn, w_sr = base.copy(), base.copy()
+    for step in range(1, 201):
+        for w, fn in ((w_rtn, lambda v: O.quantize_rtn(v, 8)), (w_sr, lambda v: O.quantize_sr(v, 9, step))):
+            upd = w.copy()
+            upd[:, 2:] += np.float32(0.1)             # a tenth of one LSB
+            w[:] = O.dequantize(fn(upd))
+    assert np.all(w_rtn[:, 2:] == 10.0)
+    drift = w_sr[:, 2:].astype(np.float64).mean() - 10.0
+    assert abs(drift - 20.0) < 1.0                    # 200 * 0.1 LSB, std error about 0.13
+
+
+# ----------------------------------------------------------------------------- the step (Sec. 3.5)
+def _dense_adam(grads, lr, b1=0.9, b2=0.999, eps=1e-8):
+    """Textbook Adam (Kingma & Ba, Algorithm 1) on a dense parameter; returns the summed update."""
+    b1, b2, eps, lr = (float(np.float32(v)) for v in (b1, b2, eps, lr))
+    m = np.zeros_like(grads[0], dtype=np.float64)
+    v = np.zeros_like(m)
+    total = np.zeros_like(m)
+    for t, g in enumerate(grads, start=1):
+        m = b1 * m + (1 - b1) * g
+        v = b2 * v + (1 - b2) * g * g
+        total += lr * (m / (1 - b1 ** t)) / (np.sqrt(v / (1 - b2 ** t)) + eps)
+    return total, m, v
+
+
+def _w_q(m, n, seed=0):
+    return O.quantize_rtn(synth.initial_weight(m, n, seed), 8)
+
+
+def _dummy_p(m, r):
+    return O.quantize_rtn(np.zeros((m, r), dtype=np.float32), 4)
+
+
+def test_full_rank_signed_permutation_reduces_to_dense_adam():
+    m, n = 24, 300
+    rng = np.random.default_rng(3)
+    perm = rng.permutation(m)
+    P = np.zeros((m, m))
+    P[perm, np.arange(m)] = rng.choice([-1.0, 1.0], size=m)       # orthonormal, r = m
+    gm = synth.GradientModel(m, n, seed=1)
+    W = _w_q(m, n)
+    M = np.zeros((m, n), dtype=np.float32)
+    V = np.zeros((m, n), dtype=np.float32)
+    grads, w_hat0 = [], O.dequantize(W).astype(np.float64)
+    h = O.Hyper(lr=0.004, alpha=0.25)
+    acc = np.zeros((m, n))
+    for t in (1, 2, 3):
+        gb = gm.sample(t)
+        grads.append(synth.bf16_bits_to_float(gb).astype(np.float64))
+        h.step = t
+        w_before = O.dequantize(W).astype(np.float64)
+        out = O.project_step(gb, _dummy_p(m, m), W, M, V, h, P_override=P)
+        acc += out["W_pre"].astype(np.float64) - w_before              # the applied (pre-rounding) update
+        W, M, V = out["W"], out["M"], out["V"]
+    total, m_d, v_d = _dense_adam(grads, lr=float(np.float32(0.004)) * 0.25)
+    assert np.allclose(-acc, total, rtol=2e-5, atol=3e-8)      # W_pre is binary32: ulp(0.06) = 4e-9 per step
+    # moments live in the rotated basis: P M = dense first moment, |P| V = dense second moment
+    assert np.allclose(P @ M.astype(np.float64), m_d, rtol=1e-5, atol=1e-12)
+    assert np.allclose(np.abs(P) @ V.astype(np.float64), v_d, rtol=1e-5, atol=1e-15)
+    assert w_hat0.shape == (m, n)
+
+
+def test_full_rank_rotation_is_adam_in_rotated_coordinates():
+    m, n = 16, 260
+    Q, _ = np.linalg.qr(np.random.default_rng(5).standard_normal((m, m)))
+    gb = synth.GradientModel(m, n, seed=2).sample(1)
+    G = synth.bf16_bits_to_float(gb).astype(np.float64)
+    W = _w_q(m, n)
+    out = O.project_step(gb, _dummy_p(m, m), W, np.zeros((m, n), np.float32), np.zeros((m, n), np.float32),
+                         O.Hyper(step=1), P_override=Q)
+    total, _, _ = _dense_adam([Q.T @ G], lr=float(np.float32(0.004)) * 0.25)
+    lhs = Q.T @ (out["W_pre"].astype(np.float64) - O.dequantize(W))
+    assert np.allclose(-lhs, total, rtol=1e-4, atol=1e-8)
+
+
+def test_step_tiny_orientation_example():
+    # m = 2, n = 3, r = 1, P = e_1: R is G's first row, the update touches row 0 only.
+    P = O.quantize_rtn(np.array([[1.0], [0.0]], dtype=np.float32), 4)
+    assert np.array_equal(O.dequantize(P), [[1.0], [0.0]])
+    G = np.array([[0.5, -0.25, 2.0], [4.0, 8.0, -16.0]], dtype=np.float32)
+    W = O.quantize_rtn(np.array([[0.0, 0.5, 1.0], [-1.0, 0.0, 1.0]], dtype=np.float32), 8, group=256)
+    out = O.project_step(synth.to_bf16_bits(G), P, W, np.zeros((1, 3), np.float32), np.zeros((1, 3), np.float32),
+                         O.Hyper(lr=0.5, alpha=0.25, step=1))
+    assert np.array_equal(out["R32"], G[:1])
+    assert np.allclose(out["M"], (1 - float(np.float32(0.9))) * G[:1], rtol=1e-6)
+    assert np.allclose(out["V"], (1 - float(np.float32(0.999))) * G[:1] ** 2, rtol=1e-6)  # beta2 travels as binary32
+    assert np.allclose(out["N"], np.sign(G[:1]), atol=1e-6)            # t = 1: N = R / (|R| + eps)
+    w_hat = O.dequantize(W)
+    assert np.allclose(out["W_pre"][0], w_hat[0] - 0.125 * np.sign(G[0]), atol=1e-6)
+    assert np.array_equal(out["W_pre"][1], w_hat[1])
+
+
+def test_step_closed_form_at_t1_and_linearity():
+    m, n, r = 64, 512, 16
+    gb = synth.GradientModel(m, n, seed=4).sample(1)
+    Pq = O.quantize_rtn(synth.random_orthonormal(m, r, seed=4), 4)
+    W = _w_q(m, n, 4)
+    z = np.zeros((r, n), np.float32)
+    out = O.project_step(gb, Pq, W, z, z, O.Hyper(step=1))
+    Pt = O.bf16_round(O.dequantize(Pq)).astype(np.float64)
+    G = synth.bf16_bits_to_float(gb).astype(np.float64)
+    R = Pt.T @ G
+    assert np.allclose(out["R32"], R, rtol=1e-6, atol=1e-12)
+    eps = float(np.float32(1e-8))
+    assert np.allclose(out["N"], R / (np.abs(R) + eps), rtol=1e-5, atol=1e-7)
+    Nb = O.bf16_round(out["N"]).astype(np.float64)
+    want = O.dequantize(W).astype(np.float64) - float(np.float32(0.004)) * 0.25 * (Pt @ Nb)
+    assert np.allclose(out["W_pre"], want, rtol=1e-6, atol=1e-9)
+    # linearity of the projection in G: doubling G (exact in bfloat16) doubles R exactly
+    G2 = synth.to_bf16_bits(2 * synth.bf16_bits_to_float(gb))
+    out2 = O.project_step(G2, Pq, W, z, z, O.Hyper(step=1))
+    assert np.array_equal(out2["R32"], 2 * out["R32"])
+    # and the sum of two integer-valued gradients projects to the sum of the projections
+    rng = np.random.default_rng(8)
+    Ga = rng.integers(-8, 9, size=(m, n)).astype(np.float32)
+    Gb = rng.integers(-8, 9, size=(m, n)).astype(np.float32)
+    Ra, Rb, Rab = (O.project_step(synth.to_bf16_bits(g), Pq, W, z, z, O.Hyper(step=1))["R32"].astype(np.float64)
+                   for g in (Ga, Gb, Ga + Gb))
+    assert np.allclose(Rab, Ra + Rb, rtol=0, atol=2e-5)
+
+
+def test_step_zero_gradient_decays_moments_and_keeps_weights():
+    m, n, r = 32, 600, 8
+    rng = np.random.default_rng(6)
+    Pq = O.quantize_rtn(synth.random_orthonormal(m, r, seed=6), 4)
+    W = _w_q(m, n, 6)
+    M = rng.standard_normal((r, n)).astype(np.float32)
+    V = (rng.standard_normal((r, n)) ** 2).astype(np.float32)
+    # moments that make N = 0 as well: M = 0
+    out = O.project_step(np.zeros((m, n), np.uint16), Pq, W, np.zeros_like(M), V, O.Hyper(step=5, seed=1))
+    assert np.all(out["R32"] == 0) and np.all(out["M"] == 0) and np.all(out["N"] == 0)
+    assert np.array_equal(out["V"], O.fl32(float(np.float32(0.999)) * V.astype(np.float64)))
+    assert np.array_equal(out["W_pre"], O.dequantize(W))
+    mism = out["W"].codes != W.codes
+    assert mism.mean() < 1e-3
+    assert np.all(np.abs(out["W"].codes.astype(int) - W.codes.astype(int)) <= 1)
+    out_m = O.project_step(np.zeros((m, n), np.uint16), Pq, W, M, V, O.Hyper(step=5, seed=1))
+    assert np.array_equal(out_m["M"], O.fl32(float(np.float32(0.9)) * M.astype(np.float64)))
+
+
+def test_step_sr_codes_follow_the_philox_lanes():
+    # the weight codes are floor(T) + [frac(T) * 65536 > h] + z, with h the element's Philox lane
+    m, n, r = 16, 700, 8
+    gb = synth.GradientModel(m, n, seed=7).sample(1)
+    Pq = O.quantize_rtn(synth.random_orthonormal(m, r, seed=7), 4)
+    W = _w_q(m, n, 7)
+    z = np.zeros((r, n), np.float32)
+    seed, t = synth.matrix_seed(3, 5), 17
+    out = O.project_step(gb, Pq, W, z, z, O.Hyper(step=t, seed=seed))
+    T = out["T"].astype(np.float64)
+    h = O.sr_uniform16(seed, t, m, n).astype(np.float64)
+    up = ((T - np.floor(T)) * 65536 > h)
+    zeros = np.repeat(out["W"].zeros, 256, axis=1)[:, :n]
+    want = np.clip(np.floor(T) + up + zeros, -128, 127)
+    assert np.array_equal(out["W"].codes, want.astype(np.int8))
+    assert 0.3 < up.mean() < 0.7
+
+
+# ----------------------------------------------------------------------------- refresh (Sec. 3.5)
+def _jacobi_eigh(A, sweeps=30):
+    """Cyclic Jacobi eigenvalue iteration for a small symmetric matrix (textbook, written out)."""
+    A = A.copy()
+    n = A.shape[0]
+    Vv = np.eye(n)
+    for _ in range(sweeps):
+        off = 0.0
+        for p in range(n - 1):
+            for q in range(p + 1, n):
+                off += A[p, q] ** 2
+                if abs(A[p, q]) < 1e-300:
+                    continue
+                theta = (A[q, q] - A[p, p]) / (2 * A[p, q])
+                tt = math.copysign(1.0, theta) / (abs(theta) + math.sqrt(theta * theta + 1))
+                c = 1 / math.sqrt(tt * tt + 1)
+                s = tt * c
+                J = np.eye(n)
+                J[p, p] = J[q, q] = c
+                J[p, q], J[q, p] = s, -s
+                A = J.T @ A @ J
+                Vv = Vv @ J
+        if off < 1e-30:
+            break
+    w = np.diag(A)
+    order = np.argsort(-w)
+    return w[order], Vv[:, order]
+
+
+def test_refresh_matches_brute_force_jacobi_on_8x8():
+    rng = np.random.default_rng(12)
+    G = synth.bf16_bits_to_float(synth.to_bf16_bits(rng.standard_normal((8, 8)))).astype(np.float64)
+    w, Vv = _jacobi_eigh(G @ G.T)
+    for r in (1, 3, 8):
+        P, Pq, S = O.refresh_subspace(synth.to_bf16_bits(G), r)
+        assert np.allclose(S[:8] ** 2, w, rtol=1e-10)
+        for j in range(r):                                         # distinct singular values: columns match up to sign
+            assert abs(abs(P[:, j].astype(np.float64) @ Vv[:, j]) - 1) < 1e-5
+        piv = np.argmax(np.abs(P), axis=0)
+        assert np.all(P[piv, np.arange(r)] > 0)                    # canonical sign
+        assert Pq.bits == 4 and Pq.codes.shape == (8, r)
+
+
+def test_refresh_orthonormal_energy_and_rank_one():
+    m, n, r = 96, 200, 24
+    gb = synth.GradientModel(m, n, seed=13).sample(1)
+    G = synth.bf16_bits_to_float(gb).astype(np.float64)
+    P, Pq, S = O.refresh_subspace(gb, r)
+    assert np.abs(P.astype(np.float64).T @ P - np.eye(r)).max() <= 1e-5
+    ev = np.sort(np.linalg.eigvalsh(G.T @ G))[::-1]                # singular values by another route
+    captured = np.linalg.norm(P.astype(np.float64).T @ G, "fro") ** 2
+    assert abs(captured - ev[:r].sum()) <= 1e-5 * ev[:r].sum()
+    # INT4 copy stays within half a step of P
+    assert np.all(np.abs(O.dequantize(Pq) - P) <= 0.5 * Pq.scales.max() * (1 + 1e-3))
+    # rank one: G = sigma u v^T gives +-u as the first column
+    rng = np.random.default_rng(14)
+    u = rng.standard_normal(m); u /= np.linalg.norm(u)
+    v = rng.standard_normal(n); v /= np.linalg.norm(v)
+    gb1 = synth.to_bf16_bits(3.0 * np.outer(u, v))
+    P1, _, S1 = O.refresh_subspace(gb1, 2)
+    assert abs(abs(P1[:, 0].astype(np.float64) @ u) - 1) < 1e-4     # bfloat16 rounding of G perturbs u slightly
+    assert abs(S1[0] - 3.0) < 2e-2
+    assert O.principal_angle(P, P) < 1e-7
+    assert abs(O.principal_angle(np.eye(4)[:, :2], np.eye(4)[:, [0, 2]]) - math.pi / 2) < 1e-7
+    c, s = math.cos(0.01), math.sin(0.01)
+    assert abs(O.principal_angle(np.eye(3)[:, :1], np.array([[c], [s], [0.0]])) - 0.01) < 1e-9
+
+
+# ----------------------------------------------------------------------------- similarity and gate (Sec. 3.2)
+def _negated(q):
+    # -(q - z) s = (q' - z') s with q' = -q - 1, z' = -z - 1: stays inside [-8, 7]
+    return O.QTensor((-q.codes.astype(np.int16) - 1).astype(np.int8), q.scales.copy(), -q.zeros - 1, q.bits, q.group)
+
+
+def test_similarity_closed_forms():
+    m, r = 512, 64
+    A = O.quantize_rtn(synth.random_orthonormal(m, r, seed=1, stream=1), 4)
+    B = O.quantize_rtn(synth.random_orthonormal(m, r, seed=1, stream=2), 4)
+    assert abs(O.subspace_similarity(A, A) - 1) < 1e-12
+    nA = _negated(A)
+    assert np.array_equal(O.dequantize(nA), -O.dequantize(A))
+    assert abs(O.subspace_similarity(A, nA) - 1) < 1e-12
+    indep = O.subspace_similarity(A, B)
+    assert abs(indep - math.sqrt(2 / (math.pi * m))) < 0.01         # E|cos| of independent unit vectors
+    perm = O.QTensor(np.roll(A.codes, 1, axis=1), np.roll(A.scales, 0), A.zeros.copy(), 4)
+    assert O.subspace_similarity(A, perm) < 0.1
+    # the leading-columns variant ignores the tail
+    mix = O.QTensor(np.concatenate([A.codes[:, :8], B.codes[:, 8:]], axis=1), A.scales, A.zeros, 4)
+    assert abs(O.subspace_similarity(A, mix, sim_cols=8) - 1) < 1e-12
+    # hand example: a = (1, 0), b = (1, 1)/.. through exact codes
+    a = O.QTensor(np.array([[1], [0]], np.int8), np.ones((2, 1), np.float32), np.zeros((2, 1), np.float32), 4)
+    b = O.QTensor(np.array([[1], [1]], np.int8), np.ones((2, 1), np.float32), np.zeros((2, 1), np.float32), 4)
+    assert abs(O.subspace_similarity(a, b) - 1 / math.sqrt(2)) < 1e-12
+
+
+def test_gate_scripted_sequences():
+    # k = 1: every similarity >= threshold doubles the interval (Sec. 3.2: t -> 2t)
+    st = O.GateState(interval=200)
+    assert O.gate_update(st, 0.39999, 0.4, 1) is False and st.interval == 200
+    assert O.gate_update(st, 0.4, 0.4, 1) is True and st.interval == 400      # ">= 40%": equality counts
+    assert O.gate_update(st, 0.9, 0.4, 1) is True and st.interval == 800
+    # k = 2: needs two in a row, history cleared after a doubling
+    st = O.GateState(interval=200)
+    seq = [0.5, 0.3, 0.5, 0.6, 0.7, 0.8]
+    got = [O.gate_update(st, s, 0.4, 2) for s in seq]
+    assert got == [False, False, False, True, False, True] and st.interval == 800
+    # k = 3 with a dip resets nothing but delays the doubling
+    st = O.GateState(interval=100)
+    got = [O.gate_update(st, s, 0.4, 3) for s in [0.9, 0.9, 0.1, 0.9, 0.9, 0.9]]
+    assert got == [False, False, False, False, False, True] and st.interval == 200
+
+
+# ----------------------------------------------------------------------------- inputs
+def test_synthetic_gradient_recipe():
+    gm = synth.GradientModel(256, 384, seed=0)
+    g = synth.bf16_bits_to_float(gm.sample(1)).astype(np.float64)
+    s = np.linalg.svd(g, compute_uv=False)
+    assert abs(s[0] - 1.0) < 0.02 and abs(s[1] - 0.5) < 0.02       # planted 1/k spectrum on top
+    assert 0.8e-3 < np.std(g - gm.signal()) < 1.2e-3                # noise level 1e-3
+    assert np.array_equal(gm.sample(3), synth.GradientModel(256, 384, seed=0).sample(3))
+    assert not np.array_equal(gm.sample(3), gm.sample(4))
+    assert len(synth.stack_matrices("llama130m")) == 84 and len(synth.stack_matrices("llama7b")) == 224
+    assert sum(s.m * s.n for s in synth.stack_matrices("llama1b")) == 24 * (4 * 2048 * 2048 + 3 * 2048 * 5461)
+    shapes = {(m, n, r): c for m, n, r, c in synth.distinct_shapes("llama1b")}
+    assert shapes == {(2048, 2048, 512): 96, (2048, 5461, 512): 48, (5461, 2048, 512): 24}
