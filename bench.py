@@ -1,0 +1,358 @@
+#!/usr/bin/env python
+"""Throughput of the Q-GaLore optimizer step on a LLaMA-shaped layer stack (one B200 per rank).
+
+A "step" is one pass of the whole hot path (dequantize P, project, Adam, project back, dequantize-
+add, stochastic-rounding requantization) over every 2-D attention/MLP matrix of the stack.
+Prints ONE JSON line: weight elements updated per second, with the per-step roofline, the end-to-end
+figure (gradients copied from pinned host memory every step) and the CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama1b|llama7b|...] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "Q-GaLore optimizer step: weight elements updated/s"
+UNIT = "elements/s"
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained")}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def matrix_flops(m, n, r):
+    return 4.0 * m * n * r                      # two dense contractions of 2 m n r each
+
+
+def matrix_bytes(m, n, r):
+    """Algorithmic HBM bytes of one step of one matrix: G (bf16), W codes read+write, W scale/zero
+    read+write, P codes + scale/zero, M and V fp32 read+write."""
+    ng_n = (n + 255) // 256
+    ng_r = (r + 255) // 256
+    return 2 * m * n + 2 * m * n + 16 * m * ng_n + m * r // 2 + 8 * m * ng_r + 16 * r * n
+
+
+def stack_roofline(specs, peaks):
+    t = 0.0
+    fl = by = 0.0
+    for s in specs:
+        f, b = matrix_flops(s.m, s.n, s.r), matrix_bytes(s.m, s.n, s.r)
+        t += max(f / (peaks["bf16_tflops"] * 1e12), b / (peaks["hbm_gbs"] * 1e9))
+        fl += f
+        by += b
+    return t, fl, by
+
+
+# --------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        rows = [l for (t, l) in self.lines if t0 - 0.05 <= t <= t1 + 0.15] or [l for (_, l) in self.lines]
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- reference arm
+def oracle_sample(workload, steps, warmup):
+    """Times the CPU oracle, as it stands, on one matrix of each distinct shape of the workload and
+    extrapolates by the shape counts.  Returns (elements/s, seconds per stack step, description)."""
+    import oracle as O
+    from paper_2407_08296_b200 import synth
+    shapes = synth.distinct_shapes(workload)
+    per_step = 0.0
+    elements = 0
+    detail = []
+    for (m, n, r, count) in shapes:
+        gm = synth.GradientModel(m, n, seed=0, matrix_index=0)
+        P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=0), 4)
+        W = O.quantize_rtn(synth.initial_weight(m, n, 0), 8)
+        M = np.zeros((r, n), np.float32)
+        V = np.zeros((r, n), np.float32)
+        g = gm.sample(1)
+        best = None
+        for it in range(warmup + steps):
+            t0 = time.perf_counter()
+            out = O.project_step(g, P, W, M, V, O.Hyper(step=it + 1, seed=1))
+            dt = time.perf_counter() - t0
+            W, M, V = out["W"], out["M"], out["V"]
+            if it >= warmup:
+                best = dt if best is None else min(best, dt)
+        per_step += best * count
+        elements += m * n * count
+        detail.append(f"{m}x{n} r{r}: {best:.3f}s x{count}")
+    return elements / per_step, per_step, "one oracle step per distinct shape, extrapolated by shape counts (" + "; ".join(detail) + ")"
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 2))
+    value, per_step, sample = oracle_sample(args.workload, steps, 0 if args.warmup == 0 else 1)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "note": "CPU oracle (numpy/scipy fp64), not a GPU program"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------- our arm
+def build_stack(workload, device, seed=0):
+    """Device-resident synthetic state of the whole stack: bf16 gradients (rank-32 signal + noise),
+    INT8 weights, INT4 projections, zero moments.  Generated with torch on the device (input
+    generation, not the path); quantization goes through the library."""
+    import torch
+    from paper_2407_08296_b200 import binding as B
+    from paper_2407_08296_b200 import synth
+    specs = synth.stack_matrices(workload)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    items = []
+    sig = 1.0 / torch.arange(1, synth.SIGNAL_RANK + 1, device=device, dtype=torch.float32)
+    for s in specs:
+        k = min(synth.SIGNAL_RANK, s.m, s.n)
+        U = torch.linalg.qr(torch.randn(s.m, k, device=device, generator=gen))[0]
+        Vt = torch.linalg.qr(torch.randn(s.n, k, device=device, generator=gen))[0]
+        g32 = (U * sig[:k]) @ Vt.T + synth.NOISE_STD * torch.randn(s.m, s.n, device=device, generator=gen)
+        G = B.empty_matrix(s.m, s.n, torch.bfloat16, device)
+        G.copy_(g32)
+        del g32
+        w32 = B.empty_matrix(s.m, s.n, torch.float32, device)
+        w32.copy_(torch.randn(s.m, s.n, device=device, generator=gen) * synth.WEIGHT_STD)
+        W = B.quantize_int8(w32)
+        del w32
+        p32 = B.empty_matrix(s.m, s.r, torch.float32, device)
+        p32.copy_(torch.linalg.qr(torch.randn(s.m, s.r, device=device, generator=gen))[0])
+        P = B.quantize_int4(p32)
+        del p32
+        M = B.zeros_matrix(s.r, s.n, torch.float32, device)
+        V = B.zeros_matrix(s.r, s.n, torch.float32, device)
+        items.append({"G": G, "P": P, "W": W, "M": M, "V": V, "seed": synth.matrix_seed(seed, s.index), "spec": s})
+    return specs, items
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_08296_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Q-GaLore step has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    B.lib()                                                    # fail loudly if the library is missing
+    peaks, peak_kind = load_peaks()
+
+    # every rank holds and steps its own replica of the stack: matrices are independent units, no collective
+    specs, items = build_stack(args.workload, device, seed=rank)
+    batch = B.StepBatch(items)
+    elements = batch.elements
+    hyper = B.Hyper()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    step_no = 0
+    for _ in range(args.warmup):
+        step_no += 1
+        hyper.step = step_no
+        batch.step(hyper)
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    stream = torch.cuda.current_stream()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.launch_count()
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step_no += 1
+        hyper.step = step_no
+        batch.step(hyper)
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = B.launch_count() - launches0
+    ms_total = ev0.elapsed_time(ev1)
+    clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
+    status = int(batch.status.item())
+
+    tms = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+    ms_total = float(tms.item())
+    ms_per_step = ms_total / args.steps
+    value = elements * world * args.steps / (ms_total * 1e-3)
+
+    # ---- end to end: gradients arrive from pinned host memory every step, the status word is read back
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    h2d = sum(it["G"].shape[0] * it["G"].shape[1] * 2 for it in items)
+    host_g = [torch.empty((it["G"].shape[0], it["G"].shape[1]), dtype=torch.bfloat16).pin_memory() for it in items]
+    for hg, it in zip(host_g, items):
+        hg.copy_(it["G"])
+    host_status = torch.zeros(1, dtype=torch.int32).pin_memory()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        step_no += 1
+        hyper.step = step_no
+        for hg, it in zip(host_g, items):
+            it["G"].copy_(hg, non_blocking=True)
+        batch.step(hyper)
+        host_status.copy_(batch.status, non_blocking=True)
+        stream.synchronize()
+    e1.record(stream)
+    barrier()
+    e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
+    e2e_value = elements * world * e2e_steps / (float(e2e_ms.item()) * 1e-3)
+    del host_g
+
+    if rank == 0:
+        t_roof, flops, nbytes = stack_roofline(specs, peaks)
+        t_roof_nom, _, _ = stack_roofline(specs, NOMINAL)
+        t_c = flops / (peaks["bf16_tflops"] * 1e12)
+        t_m = nbytes / (peaks["hbm_gbs"] * 1e9)
+        sec = ms_per_step * 1e-3
+        if t_c >= t_m:
+            roof = {"bound": "tensor", "achieved": flops / sec / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+        else:
+            roof = {"bound": "hbm", "achieved": nbytes / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["traffic"] = None
+        roof["peak_source"] = peak_kind
+        roof["scope"] = "whole step (all kernels of the stack)"
+        roof["per_matrix_roofline_ms"] = t_roof * 1e3
+        roof["frac_of_per_matrix_roofline"] = t_roof / sec
+        roof["frac_of_nominal_roofline"] = t_roof_nom / sec
+        cpu = None
+        if not args.no_cpu_baseline:
+            v, per_step, sample = oracle_sample(args.workload, 1, 0)
+            cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample,
+                   "host_cpus": os.cpu_count()}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "matrices": len(specs), "elements_per_step": elements,
+                       "rank": specs[0].r, "group": 256, "l2": "inputs larger than L2 (whole stack streams each step)",
+                       "parallelism": f"replica per GPU x{world}, no collective"},
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
+                    "steps": e2e_steps},
+            "gpu_launches": launches, "clocks": clocks, "device_status": status,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="llama1b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

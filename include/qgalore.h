@@ -1,0 +1,186 @@
+/*
+ * qgalore.h - C boundary of the B200 (sm_100a) Q-GaLore per-step optimizer library.
+ *
+ * Q-GaLore (arXiv 2407.08296) keeps each weight matrix W (m x n) in INT8, the GaLore
+ * projection matrix P (m x r) in INT4, and the Adam moments M, V (r x n) of the projected
+ * gradient in the low-rank space.  One optimizer step of one matrix is (Sec. 3.5):
+ *
+ *     P~ = dequant(P)            R = P~^T G          (project the bf16 gradient)
+ *     M, V <- Adam(M, V, R)      N = M^ / (sqrt(V^) + eps)
+ *     W' = dequant(W) - lr * alpha * P~ N            (project back, scale)
+ *     W  <- Quant_8 with stochastic rounding (W')    (Sec. 3.4)
+ *
+ * Common rules for every entry point
+ *   - Return value: 0 (QG_OK) or a negative qg_status.  No exceptions, no allocation, no
+ *     implicit synchronisation: work is enqueued on the caller's stream (a cudaStream_t passed
+ *     as void*, NULL = the default stream) and the call returns.
+ *   - Unless stated otherwise every buffer is DEVICE memory owned by the caller; the library
+ *     neither frees nor retains it.  Structs (qg_qtensor, qg_hyper) are HOST memory read
+ *     during the call.
+ *   - Matrices are row-major with a row pitch ("ld") in ELEMENTS.  Base pointers must be
+ *     16-byte aligned and every row pitch a multiple of 16 bytes, i.e. ld % 8 == 0 for bf16,
+ *     ld % 4 == 0 for fp32, ld % 16 == 0 for INT8 codes, ld % 32 == 0 for INT4 codes.
+ *     Elements between cols and ld are padding: never read as data, never written.
+ *   - Quantization groups (Sec. 3.1, "block-wise", block 256) are runs of `group` consecutive
+ *     elements along a row and restart at every row; a row whose length is not a multiple of
+ *     `group` ends in one shorter group.  scales/zeros are dense [rows][ceil(cols/group)] fp32.
+ *   - INT4 codes are packed two per byte: byte k of a row holds column 2k in its low nibble
+ *     and column 2k+1 in its high nibble, each stored as code + 8 (codes lie in [-8, 7]).
+ *   - A device status word (int32, optional, may be NULL) is OR-ed with QG_DEV_* flags when a
+ *     kernel gives up a bounded wait or an iteration does not converge; it is never cleared
+ *     by the library.
+ */
+#ifndef QGALORE_H_
+#define QGALORE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define QG_API __attribute__((visibility("default")))
+#else
+#define QG_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  QG_OK = 0,
+  QG_INVALID_ARGUMENT = -1,    /* null pointer, non-positive size, bits/group not supported   */
+  QG_UNSUPPORTED_SHAPE = -2,   /* r > m, r not a multiple of 32, r > 2048, size beyond a limit */
+  QG_MISALIGNED = -3,          /* base pointer or row pitch breaks the 16-byte rule            */
+  QG_WORKSPACE_TOO_SMALL = -4,
+  QG_CUDA_ERROR = -5,          /* a CUDA runtime/driver call failed; see qgalore_last_cuda_error */
+  QG_NOT_CONVERGED = -6
+} qg_status;
+
+/* flags OR-ed into the optional device status word */
+#define QG_DEV_WAIT_EXPIRED 1   /* a bounded barrier wait ran out; the tile was abandoned */
+#define QG_DEV_NOT_CONVERGED 2  /* eigen-iteration of the refresh hit its sweep limit     */
+#define QG_DEV_BAD_FACTOR 4     /* Cholesky factor of the refresh met a non-positive pivot */
+
+/* A block-wise quantized matrix (Sec. 3.1; App. A: W = (codes - zeros) * scales). */
+typedef struct {
+  void*   codes;   /* device; bits == 8: int8 [rows][ld]; bits == 4: uint8 [rows][ld / 2]  */
+  float*  scales;  /* device; [rows][ceil(cols / group)]                                    */
+  float*  zeros;   /* device; same shape, integer valued                                    */
+  int64_t rows, cols, ld;
+  int32_t bits;    /* 4 or 8                                                                */
+  int32_t group;   /* 256                                                                   */
+} qg_qtensor;
+
+/* Hyper-parameters of one step.  alpha is GaLore's scale factor (0.25 in Sec. 4.1), the
+ * Adam constants are Kingma & Ba's; step is t >= 1 and enters the bias corrections and the
+ * random-number counter; seed keys the stochastic rounding of this matrix. */
+typedef struct {
+  float    lr, alpha, beta1, beta2, eps, weight_decay;
+  int64_t  step;
+  uint64_t seed;
+} qg_hyper;
+
+/* Optional taps for tests: any non-null pointer receives that intermediate (device, fp32). */
+typedef struct {
+  float* R;      /* r x n, pitch ldmv: projected gradient                     */
+  float* N;      /* r x n, pitch ldmv: Adam direction before bfloat16 rounding */
+  float* W_pre;  /* m x n, pitch W->ld: weight before requantization           */
+} qg_debug;
+
+/* --- Sec. 3.1 / Sec. 3.3: round-to-nearest block-wise quantization ----------------------
+ * dst->codes/scales/zeros receive Quant_4 (resp. Quant_8) of src (fp32, rows x cols, pitch
+ * ld_src).  Per group: s = (max - min) / (2^bits - 1), z = -2^(bits-1) - rint(min / s),
+ * code = clamp(rint(x / s) + z); x / s is evaluated as x * (1 / s) in binary32, ties to even.
+ * A constant group takes z = 0, s = |max| (1 if that is 0).  dst->rows/cols must equal
+ * rows/cols, dst->bits must be 4 (resp. 8).  Bit-exact against the CPU oracle. */
+QG_API int qgalore_quantize_int4(const float* src, int64_t rows, int64_t cols, int64_t ld_src,
+                          const qg_qtensor* dst, void* stream);
+QG_API int qgalore_quantize_int8(const float* src, int64_t rows, int64_t cols, int64_t ld_src,
+                          const qg_qtensor* dst, void* stream);
+
+/* App. A, dequantization line: dst (fp32, pitch ld_dst) = (codes - zeros) * scales. */
+QG_API int qgalore_dequantize(const qg_qtensor* src, float* dst, int64_t ld_dst, void* stream);
+
+/* --- Sec. 3.5 (with Sec. 3.4 for the write-back): one optimizer step of one matrix ------
+ * G       bf16 bit patterns, m x n, pitch ldg                        (read)
+ * P       INT4, m x r                                                (read)
+ * W       INT8, m x n: codes, scales and zeros are replaced          (read + write)
+ * M, V    fp32, r x n, pitch ldmv                                    (read + write)
+ * h       host; step >= 1
+ * workspace  device scratch of at least qgalore_workspace_bytes(QG_OP_PROJECT_STEP, m, n, r)
+ *            bytes, 256-byte aligned; contents are undefined afterwards
+ * status_dev optional device status word
+ * dbg     optional (may be NULL) test taps
+ * Shape limits: 32 <= r <= 2048, r % 32 == 0, r <= m.  Errors are reported before anything
+ * is enqueued; after QG_OK the work is queued on `stream`. */
+QG_API int qgalore_project_step(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r,
+                         const qg_qtensor* P, const qg_qtensor* W,
+                         float* M, float* V, int64_t ldmv, const qg_hyper* h,
+                         void* workspace, size_t workspace_bytes,
+                         int32_t* status_dev, const qg_debug* dbg, void* stream);
+
+/* --- Sec. 3.5, the same step for several matrices (a layer, or a whole stack) in one call ----
+ * Every item is one independent matrix with its own buffers and its own stochastic-rounding
+ * seed; lr, alpha, the Adam constants and the step index come from h (h->seed is ignored).
+ * items is HOST memory.  The workspace (qgalore_workspace_bytes_batched) is shared by the
+ * items, which are processed in order on `stream`.  Validation covers every item before
+ * anything is enqueued. */
+typedef struct {
+  const uint16_t* G; int64_t ldg, m, n, r;
+  qg_qtensor P, W;
+  float* M; float* V; int64_t ldmv;
+  uint64_t seed;
+} qg_step_item;
+
+QG_API int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const qg_hyper* h,
+                                 void* workspace, size_t workspace_bytes,
+                                 int32_t* status_dev, void* stream);
+QG_API size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t count);
+
+/* --- Sec. 3.5 "obtain the projection matrix using SVD" + Sec. 3.3 INT4 storage ------------
+ * Top-r left singular subspace of G (bf16, m x n) by block subspace iteration with
+ * `oversample_cols` extra columns and a Rayleigh-Ritz step, then Quant_4 into P_new.
+ * P_fp32 (optional, m x r fp32, pitch r) receives the basis before quantization.
+ * If P_prev and sim_dev are given, the similarity of Sec. 3.2 between P_prev and P_new over
+ * the leading sim_cols columns is written to *sim_dev. */
+QG_API int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r,
+                             int32_t iters, int32_t oversample_cols, uint64_t seed,
+                             const qg_qtensor* P_new, float* P_fp32,
+                             const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev,
+                             void* workspace, size_t workspace_bytes,
+                             int32_t* status_dev, void* stream);
+
+/* --- Sec. 3.2: cosine similarity between adjacent projection matrices -------------------
+ * *sim_dev = sum_{j < c} |<a_j, b_j>| / (||A[:, :c]||_F ||B[:, :c]||_F), c = sim_cols
+ * (<= 0 means all columns), on the dequantized INT4 matrices A and B (same shape).
+ * workspace: qgalore_workspace_bytes(QG_OP_SIMILARITY, rows, 0, cols) bytes. */
+QG_API int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols,
+                                float* sim_dev, void* workspace, size_t workspace_bytes,
+                                void* stream);
+
+/* --- Sec. 3.2, adaptive lazy update: host-only state machine ----------------------------
+ * Pushes `sim` into `history` (k floats, host) holding *count values; when k values are held
+ * and all are >= threshold, *interval is doubled and the history cleared.  Returns 1 if the
+ * interval was doubled, 0 if not, negative on bad arguments. */
+QG_API int qgalore_gate_update(float sim, float threshold, int32_t k, int32_t* interval,
+                        float* history, int32_t* count);
+
+enum { QG_OP_PROJECT_STEP = 1, QG_OP_REFRESH = 2, QG_OP_SIMILARITY = 3 };
+
+/* Scratch bytes the given operation needs for an m x n matrix at rank r (host, pure).
+ * For QG_OP_REFRESH r is the block width (rank + oversample_cols). */
+QG_API size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r);
+
+QG_API const char* qgalore_status_string(int status);
+/* Text of the last CUDA error this thread met inside the library ("" if none). */
+QG_API const char* qgalore_last_cuda_error(void);
+/* Number of kernels the library has launched from this process (for launch accounting). */
+QG_API uint64_t qgalore_launch_count(void);
+/* Test aid: 0 selects the tensor-core kernels of qgalore_project_step (the default and the
+ * product path), 1 the plain CUDA-core kernels kept to cross-check them.  Not thread safe. */
+QG_API int qgalore_debug_set_step_impl(int impl);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QGALORE_H_ */

@@ -1,0 +1,221 @@
+// extern "C" boundary of the Q-GaLore library: argument validation, scalar preparation and
+// dispatch to the kernels.  Nothing here allocates or synchronises.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "qg_common.cuh"
+
+namespace qg {
+
+static thread_local char g_last_error[256] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+void note_cuda_error(cudaError_t e, const char* where) {
+  snprintf(g_last_error, sizeof(g_last_error), "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
+  (void)cudaGetLastError();  // clear the sticky-less error so that later calls start clean
+}
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+int launch_project_step_simt(const StepArgs& a, cudaStream_t st);
+size_t simt_workspace_bytes(int64_t m, int64_t n, int64_t r);
+int launch_project_step_tc(const StepArgs& a, cudaStream_t st);
+size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r);
+int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters,
+                   uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes,
+                   int32_t* status, cudaStream_t st);
+size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b);
+
+static int g_step_impl = 0;  // 0: tensor-core kernels; 1: CUDA-core kernels (validation aid)
+
+static int check_qtensor(const qg_qtensor* t, int bits) {
+  if (!t || !t->codes || !t->scales || !t->zeros) return QG_INVALID_ARGUMENT;
+  if (t->rows <= 0 || t->cols <= 0 || t->ld < t->cols) return QG_INVALID_ARGUMENT;
+  if (t->bits != bits || t->group != kGroup) return QG_INVALID_ARGUMENT;
+  if (!aligned16(t->codes) || (reinterpret_cast<uintptr_t>(t->scales) & 3u) ||
+      (reinterpret_cast<uintptr_t>(t->zeros) & 3u))
+    return QG_MISALIGNED;
+  if (t->ld % (bits == 8 ? 16 : 32) != 0) return QG_MISALIGNED;
+  return QG_OK;
+}
+
+}  // namespace qg
+
+using namespace qg;
+
+extern "C" {
+
+const char* qgalore_status_string(int status) {
+  switch (status) {
+    case QG_OK: return "ok";
+    case QG_INVALID_ARGUMENT: return "invalid argument";
+    case QG_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case QG_MISALIGNED: return "misaligned pointer or row pitch";
+    case QG_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case QG_CUDA_ERROR: return "CUDA error";
+    case QG_NOT_CONVERGED: return "not converged";
+    default: return "unknown status";
+  }
+}
+
+const char* qgalore_last_cuda_error(void) { return g_last_error; }
+uint64_t qgalore_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+static int quantize_common(int bits, const float* src, int64_t rows, int64_t cols, int64_t ld_src,
+                           const qg_qtensor* dst, void* stream) {
+  if (!src || rows <= 0 || cols <= 0 || ld_src < cols) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(dst, bits);
+  if (rc != QG_OK) return rc;
+  if (dst->rows != rows || dst->cols != cols) return QG_INVALID_ARGUMENT;
+  if (!aligned16(src) || ld_src % 4 != 0) return QG_MISALIGNED;
+  return launch_quantize_rtn(bits, src, rows, cols, ld_src, dst, (cudaStream_t)stream);
+}
+
+int qgalore_quantize_int4(const float* src, int64_t rows, int64_t cols, int64_t ld_src, const qg_qtensor* dst,
+                          void* stream) {
+  return quantize_common(4, src, rows, cols, ld_src, dst, stream);
+}
+
+int qgalore_quantize_int8(const float* src, int64_t rows, int64_t cols, int64_t ld_src, const qg_qtensor* dst,
+                          void* stream) {
+  return quantize_common(8, src, rows, cols, ld_src, dst, stream);
+}
+
+int qgalore_dequantize(const qg_qtensor* src, float* dst, int64_t ld_dst, void* stream) {
+  if (!src || !dst) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(src, src->bits == 4 ? 4 : 8);
+  if (rc != QG_OK) return rc;
+  if (ld_dst < src->cols) return QG_INVALID_ARGUMENT;
+  if (!aligned16(dst) || ld_dst % 4 != 0) return QG_MISALIGNED;
+  return launch_dequantize(src, dst, ld_dst, (cudaStream_t)stream);
+}
+
+size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r) {
+  if (m <= 0 || r <= 0) return 0;
+  switch (op) {
+    case QG_OP_PROJECT_STEP: {
+      if (n <= 0) return 0;
+      const size_t a = simt_workspace_bytes(m, n, r), b = tc_workspace_bytes(m, n, r);
+      return a > b ? a : b;
+    }
+    case QG_OP_REFRESH: return n > 0 ? refresh_workspace_bytes(m, n, r) : 0;
+    case QG_OP_SIMILARITY: return similarity_workspace_bytes(m, r);
+    default: return 0;
+  }
+}
+
+static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
+                             const qg_qtensor* W, float* M, float* V, int64_t ldmv, const qg_hyper* h,
+                             void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
+                             void* stream, bool validate_only) {
+  if (!G || !M || !V || !h || !workspace) return QG_INVALID_ARGUMENT;
+  if (m <= 0 || n <= 0 || r <= 0 || ldg < n || ldmv < n || h->step < 1) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(P, 4);
+  if (rc != QG_OK) return rc;
+  rc = check_qtensor(W, 8);
+  if (rc != QG_OK) return rc;
+  if (P->rows != m || P->cols != r || W->rows != m || W->cols != n) return QG_INVALID_ARGUMENT;
+  if (r % 32 != 0 || r < 32 || r > 2048 || r > m) return QG_UNSUPPORTED_SHAPE;
+  if (m > (1ll << 31) - 1 || n > (1ll << 31) - 1) return QG_UNSUPPORTED_SHAPE;
+  if (!aligned16(G) || !aligned16(M) || !aligned16(V) || ldg % 8 != 0 || ldmv % 4 != 0) return QG_MISALIGNED;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QG_MISALIGNED;
+  if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
+  if (workspace_bytes < qgalore_workspace_bytes(QG_OP_PROJECT_STEP, m, n, r)) return QG_WORKSPACE_TOO_SMALL;
+  if (!std::isfinite(h->lr) || !(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
+    return QG_INVALID_ARGUMENT;
+  if (validate_only) return QG_OK;
+
+  StepArgs a;
+  a.G = G; a.ldg = ldg; a.m = m; a.n = n; a.r = r;
+  a.P = *P; a.W = *W; a.M = M; a.V = V; a.ldmv = ldmv;
+  a.ws = workspace; a.ws_bytes = workspace_bytes; a.status = status_dev;
+  if (dbg) a.dbg = *dbg; else memset(&a.dbg, 0, sizeof(a.dbg));
+  StepScalars& sc = a.sc;
+  sc.beta1 = h->beta1; sc.beta2 = h->beta2;
+  sc.one_minus_beta1 = 1.0f - h->beta1; sc.one_minus_beta2 = 1.0f - h->beta2;
+  sc.bias1 = (float)(1.0 - std::pow((double)h->beta1, (double)h->step));
+  sc.bias2 = (float)(1.0 - std::pow((double)h->beta2, (double)h->step));
+  sc.eps = h->eps;
+  sc.lr_alpha = (float)((double)h->lr * (double)h->alpha);
+  sc.lr_wd = (float)((double)h->lr * (double)h->weight_decay);
+  sc.seed_lo = (uint32_t)(h->seed & 0xFFFFFFFFull); sc.seed_hi = (uint32_t)(h->seed >> 32);
+  sc.step_lo = (uint32_t)((uint64_t)h->step & 0xFFFFFFFFull); sc.step_hi = (uint32_t)((uint64_t)h->step >> 32);
+  if (g_step_impl == 1) return launch_project_step_simt(a, (cudaStream_t)stream);
+  return launch_project_step_tc(a, (cudaStream_t)stream);
+}
+
+int qgalore_project_step(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
+                         const qg_qtensor* W, float* M, float* V, int64_t ldmv, const qg_hyper* h,
+                         void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
+                         void* stream) {
+  return project_step_impl(G, ldg, m, n, r, P, W, M, V, ldmv, h, workspace, workspace_bytes, status_dev, dbg, stream,
+                           false);
+}
+
+size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t count) {
+  size_t need = 0;
+  if (!items) return 0;
+  for (int32_t i = 0; i < count; ++i) {
+    const size_t b = qgalore_workspace_bytes(QG_OP_PROJECT_STEP, items[i].m, items[i].n, items[i].r);
+    need = b > need ? b : need;
+  }
+  return need;
+}
+
+int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const qg_hyper* h, void* workspace,
+                                 size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  if (!items || count <= 0 || !h) return QG_INVALID_ARGUMENT;
+  // first pass validates everything (a dry run of the single-matrix checks), second pass enqueues
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int32_t i = 0; i < count; ++i) {
+      const qg_step_item& it = items[i];
+      qg_hyper hi = *h;
+      hi.seed = it.seed;
+      const int rc = project_step_impl(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &hi,
+                                       workspace, workspace_bytes, status_dev, nullptr, stream, pass == 0);
+      if (rc != QG_OK) return rc;
+    }
+  }
+  return QG_OK;
+}
+
+int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  if (!sim_dev || !workspace) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(A, 4);
+  if (rc != QG_OK) return rc;
+  rc = check_qtensor(B, 4);
+  if (rc != QG_OK) return rc;
+  if (A->rows != B->rows || A->cols != B->cols) return QG_INVALID_ARGUMENT;
+  const int32_t c = (sim_cols <= 0 || sim_cols > A->cols) ? (int32_t)A->cols : sim_cols;
+  if (A->cols > 16384) return QG_UNSUPPORTED_SHAPE;
+  if (workspace_bytes < similarity_workspace_bytes(A->rows, A->cols)) return QG_WORKSPACE_TOO_SMALL;
+  if (reinterpret_cast<uintptr_t>(workspace) & 15u) return QG_MISALIGNED;
+  return launch_similarity(A, B, c, sim_dev, workspace, (cudaStream_t)stream);
+}
+
+int qgalore_gate_update(float sim, float threshold, int32_t k, int32_t* interval, float* history, int32_t* count) {
+  if (k < 1 || !interval || !history || !count || *count < 0 || *count > k || *interval < 1) return QG_INVALID_ARGUMENT;
+  if (*count == k) {                       // keep the last k values
+    for (int i = 1; i < k; ++i) history[i - 1] = history[i];
+    *count = k - 1;
+  }
+  history[(*count)++] = sim;
+  if (*count < k) return 0;
+  for (int i = 0; i < k; ++i)
+    if (!(history[i] >= threshold)) return 0;
+  if (*interval > (1 << 29)) return 0;     // never overflow the interval
+  *interval *= 2;
+  *count = 0;
+  return 1;
+}
+
+/* Test aid: selects the CUDA-core (1) or the tensor-core (0) kernels of qgalore_project_step. */
+int qgalore_debug_set_step_impl(int impl) {
+  if (impl != 0 && impl != 1) return QG_INVALID_ARGUMENT;
+  g_step_impl = impl;
+  return QG_OK;
+}
+
+}  // extern "C"

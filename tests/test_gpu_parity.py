@@ -1,0 +1,181 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Quantizer output is compared bit for bit; the step within the tolerances below."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2407_08296_b200 import binding as B
+from paper_2407_08296_b200 import synth
+
+from parity_utils import (check_direction, check_moments, check_weight_codes, f32_to_device, from_device_q, g_to_device,
+                          to_device_q)
+
+pytestmark = pytest.mark.gpu
+
+MOMENT_TOL = 2e-3        # relative, for M, V, N and R (bf16 operands, fp32 accumulation)
+
+
+# ----------------------------------------------------------------------------- quantizer: bit-exact
+@pytest.mark.parametrize("bits", [4, 8])
+@pytest.mark.parametrize("shape", [(1, 1), (3, 7), (5, 256), (64, 1376), (33, 5461), (128, 128), (17, 600)])
+def test_quantize_bit_exact(bits, shape):
+    rows, cols = shape
+    rng = np.random.default_rng(rows * 7919 + cols + bits)
+    x = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    if rows > 4:
+        x[1, :] = 0.0                 # constant-zero groups
+        x[2, :] = -1.25               # constant groups
+        x[3, : min(cols, 256)] = np.linspace(-1, 1, min(cols, 256), dtype=np.float32)   # symmetric: ties
+        x[4, :] = 1e-41               # subnormal values: scale not a normal number
+    ref = O.quantize_rtn(x, bits)
+    fn = B.quantize_int4 if bits == 4 else B.quantize_int8
+    got = from_device_q(fn(f32_to_device(x)))
+    assert np.array_equal(got.scales.view(np.uint32), ref.scales.view(np.uint32))
+    assert np.array_equal(got.zeros.view(np.uint32), ref.zeros.view(np.uint32))
+    assert np.array_equal(got.codes, ref.codes)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_int4_padding_nibble_and_dequantize(bits):
+    rows, cols = 9, 301
+    x = (np.random.default_rng(5).standard_normal((rows, cols))).astype(np.float32)
+    ref = O.quantize_rtn(x, bits)
+    dq = B.quantize_int4(f32_to_device(x)) if bits == 4 else B.quantize_int8(f32_to_device(x))
+    if bits == 4:
+        packed = dq.codes.cpu().numpy()[:, : (cols + 1) // 2]
+        assert np.array_equal(packed, O.pack_int4(ref.codes))        # odd tail: high nibble holds code 0
+    y = B.dequantize(dq).cpu().numpy()
+    assert np.array_equal(y.view(np.uint32), O.dequantize(ref).view(np.uint32))
+    # dequantize of codes uploaded from the oracle
+    y2 = B.dequantize(to_device_q(ref)).cpu().numpy()
+    assert np.array_equal(y2, O.dequantize(ref))
+
+
+def test_quantize_large_matrix_bit_exact():
+    x = synth.initial_weight(2048, 5461, seed=3)
+    ref = O.quantize_rtn(x, 8)
+    got = from_device_q(B.quantize_int8(f32_to_device(x)))
+    assert np.array_equal(got.codes, ref.codes)
+    assert np.array_equal(got.scales, ref.scales) and np.array_equal(got.zeros, ref.zeros)
+
+
+# ----------------------------------------------------------------------------- similarity
+@pytest.mark.parametrize("m,r,c", [(512, 128, 0), (768, 256, 8), (100, 32, 5), (2048, 512, 0), (4096, 1024, 100)])
+def test_similarity_matches_oracle(m, r, c):
+    A = O.quantize_rtn(synth.random_orthonormal(m, r, seed=m, stream=1), 4)
+    rng = np.random.default_rng(m + r)
+    mix = synth.random_orthonormal(m, r, seed=m, stream=1) + 0.5 * rng.standard_normal((m, r)).astype(np.float32) / np.sqrt(m)
+    Bq = O.quantize_rtn(mix.astype(np.float32), 4)
+    want = O.subspace_similarity(A, Bq, c if c > 0 else None)
+    got = float(B.subspace_similarity(to_device_q(A), to_device_q(Bq), c).item())
+    assert abs(got - want) <= 1e-5
+    same = float(B.subspace_similarity(to_device_q(A), to_device_q(A), c).item())
+    assert abs(same - 1.0) <= 1e-6
+
+
+# ----------------------------------------------------------------------------- the step
+def run_step_case(m, n, r, seed=0, step=1, steps_before=0, wd=0.0, check_taps=True, impl=None):
+    """Teacher-forced single-step parity: upload the oracle's pre-step state, run one GPU step, compare."""
+    gm = synth.GradientModel(m, n, seed=seed, matrix_index=1)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=seed, stream=9), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, seed=seed, matrix_index=1), 8)
+    M = np.zeros((r, n), np.float32)
+    V = np.zeros((r, n), np.float32)
+    sr_seed = synth.matrix_seed(seed, 1)
+    t0 = step - steps_before
+    for t in range(t0, step):          # advance the oracle so that M, V are not trivial
+        out = O.project_step(gm.sample(t), P, W, M, V, O.Hyper(step=t, seed=sr_seed, weight_decay=wd))
+        W, M, V = out["W"], out["M"], out["V"]
+    gb = gm.sample(step)
+    hyp = O.Hyper(step=step, seed=sr_seed, weight_decay=wd)
+    ref = O.project_step(gb, P, W, M, V, hyp)
+
+    dG, dP, dW = g_to_device(gb), to_device_q(P), to_device_q(W)
+    dM, dV = f32_to_device(M), f32_to_device(V)
+    taps = {}
+    if check_taps:
+        taps = {"R": torch.zeros_like(dM), "N": torch.zeros_like(dM),
+                "W_pre": B.zeros_matrix(m, n, torch.float32, "cuda", 1)}
+        # the taps share the pitch of M (R, N) and of W's codes (W_pre)
+        taps["R"] = B.zeros_matrix(r, n, torch.float32)
+        taps["N"] = B.zeros_matrix(r, n, torch.float32)
+        taps["W_pre"] = torch.zeros((m, dW.ld), dtype=torch.float32, device="cuda")[:, :n]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if impl is not None:
+        B.debug_set_step_impl(impl)
+    try:
+        B.project_step(dG, dP, dW, dM, dV, B.Hyper(step=step, seed=sr_seed, weight_decay=wd), status=status,
+                       debug=taps or None)
+        torch.cuda.synchronize()
+    finally:
+        if impl is not None:
+            B.debug_set_step_impl(0)
+    assert int(status.item()) == 0
+    check_moments(dM.cpu().numpy(), ref["M"], "M", MOMENT_TOL)
+    check_moments(dV.cpu().numpy(), ref["V"], "V", MOMENT_TOL)
+    if check_taps:
+        check_moments(taps["R"].cpu().numpy(), ref["R32"], "R", MOMENT_TOL)
+        check_direction(taps["N"].cpu().numpy(), ref["N"], "N", MOMENT_TOL)
+        wpre = taps["W_pre"].cpu().numpy()
+        lsb = np.repeat(ref["W"].scales, 256, axis=1)[:, :n]
+        assert np.abs(wpre - ref["W_pre"]).max() <= 2e-3 * lsb.max(), "pre-rounding weight off by more than 2e-3 LSB"
+    gw = from_device_q(dW)
+    frac = check_weight_codes(gw, ref, sr_seed, step)
+    # padding of the code rows is never written
+    if dW.ld > n:
+        assert int(dW.codes[:, n:].abs().max().item()) == 0
+    return frac
+
+
+SMALL_CASES = [
+    (64, 256, 32), (128, 512, 64), (96, 300, 32), (160, 1376, 64), (512, 1376, 128),
+    (300, 777, 96), (768, 768, 256), (1000, 85, 128), (130, 2736, 128),
+]
+
+
+@pytest.mark.parametrize("m,n,r", SMALL_CASES)
+def test_step_parity_small_and_ragged(m, n, r):
+    run_step_case(m, n, r, seed=m + n + r, step=1)
+
+
+@pytest.mark.parametrize("m,n,r", [(128, 512, 64), (512, 1376, 128)])
+def test_step_parity_cuda_core_kernels(m, n, r):
+    run_step_case(m, n, r, seed=3, step=2, steps_before=1, impl=1)
+
+
+def test_step_parity_after_several_steps_with_weight_decay():
+    run_step_case(256, 1376, 64, seed=11, step=4, steps_before=3, wd=0.1)
+
+
+def test_step_config1_llama60m_mlp():
+    # configs[0]: 512 x 1376, r = 128, one step, seed 0, P from the oracle's refresh of that gradient
+    spec = synth.stack_matrices("llama60m_mlp")[0]
+    gm = synth.GradientModel(spec.m, spec.n, seed=0, matrix_index=0)
+    gb = gm.sample(1)
+    _, P, _ = O.refresh_subspace(gb, spec.r)
+    W = O.quantize_rtn(synth.initial_weight(spec.m, spec.n, 0, 0), 8)
+    z = np.zeros((spec.r, spec.n), np.float32)
+    seed = synth.matrix_seed(0, 0)
+    ref = O.project_step(gb, P, W, z, z, O.Hyper(step=1, seed=seed))
+    dW, dM, dV = to_device_q(W), f32_to_device(z), f32_to_device(z)
+    B.project_step(g_to_device(gb), to_device_q(P), dW, dM, dV, B.Hyper(step=1, seed=seed))
+    torch.cuda.synchronize()
+    check_moments(dM.cpu().numpy(), ref["M"], "M")
+    check_moments(dV.cpu().numpy(), ref["V"], "V")
+    check_weight_codes(from_device_q(dW), ref, seed, 1)
+
+
+def test_step_is_deterministic_and_seeded():
+    m, n, r = 128, 512, 64
+    gb = synth.GradientModel(m, n, seed=1).sample(1)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=1), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 1), 8)
+    z = np.zeros((r, n), np.float32)
+    outs = []
+    for seed in (5, 5, 6):
+        dW, dM, dV = to_device_q(W), f32_to_device(z), f32_to_device(z)
+        B.project_step(g_to_device(gb), to_device_q(P), dW, dM, dV, B.Hyper(step=3, seed=seed))
+        outs.append(dW.codes.cpu().numpy().copy())
+    assert np.array_equal(outs[0], outs[1])           # counter-based randomness: same (seed, step) -> same codes
+    assert not np.array_equal(outs[0], outs[2])
