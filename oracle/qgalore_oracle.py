@@ -274,7 +274,7 @@ class Hyper:
         return g(self.lr), g(self.alpha), g(self.beta1), g(self.beta2), g(self.eps), g(self.weight_decay)
 
 
-def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=None):
+def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=None, N_b_override=None):
     """One Q-GaLore update of one weight matrix (Sec. 3.5, Fig. 4; GaLore projection as cited there).
 
     G_bits : uint16 [m, n] bfloat16 gradient.         P_q : INT4 m x r projection.
@@ -283,6 +283,11 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     W_pre (pre-rounding weight) and T (= W_pre scaled by the new group reciprocal).
     ``P_override`` (float64 m x r) bypasses the INT4 dequantization and the bfloat16
     rounding of P and N; it exists only for the full-rank pin.
+    ``N_b_override`` (float32 r x n, bfloat16-representable) replaces the direction that enters
+    steps 5-6; steps 1-4 are still carried out and returned.  A staged comparison uses it: the
+    direction N = M^ / (sqrt(V^) + eps) amplifies rounding differences of R without bound where
+    sqrt(V^) is of the order of eps, so the weight update of another implementation is checked
+    against steps 5-6 applied to that implementation's own direction.
     """
     lr, alpha, b1, b2, eps, wd = h.as_f32()
     t = int(h.step)
@@ -304,6 +309,8 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     N = m_hat / (np.sqrt(v_hat) + eps)
     N32 = fl32(N)
     N_b = bf16_round(N32) if P_override is None else N32
+    if N_b_override is not None:
+        N_b = np.asarray(N_b_override, dtype=np.float32)
     # 5. project back, scale, add to the dequantized weight (no high-precision master copy)
     D = Pt @ N_b.astype(np.float64)
     W_hat = dequantize(W_q).astype(np.float64)

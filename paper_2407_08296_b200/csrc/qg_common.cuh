@@ -179,7 +179,7 @@ struct StepArgs {
   int32_t* status;
   qg_debug dbg;
 };
-int launch_project_step(const StepArgs& a, cudaStream_t st);
-size_t project_step_workspace_bytes(int64_t m, int64_t n, int64_t r);
+// P~ = bf16((q - z) * s) of an INT4 matrix whose column count is a multiple of 32 (row pitch ld_out elements)
+int launch_dequant_p(const qg_qtensor& P, uint16_t* out, int64_t ld_out, cudaStream_t st);
 
 }  // namespace qg

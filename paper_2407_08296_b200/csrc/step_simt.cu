@@ -162,6 +162,13 @@ struct RequantEpilogue {
 
 }  // namespace
 
+int launch_dequant_p(const qg_qtensor& P, uint16_t* out, int64_t ld_out, cudaStream_t st) {
+  const int64_t threads = P.rows * (P.cols / 8);
+  dequant_p_bf16_kernel<<<(unsigned)ceil_div(threads, 256), 256, 0, st>>>(P, out, ld_out);
+  QG_LAUNCH_CHECK();
+  return QG_OK;
+}
+
 size_t simt_workspace_bytes(int64_t m, int64_t n, int64_t r) {
   const size_t pt = (size_t)round_up(m * r * 2, 256);
   const size_t nb = (size_t)round_up(r * round_up(n, 64) * 2, 256);
@@ -173,9 +180,8 @@ int launch_project_step_simt(const StepArgs& a, cudaStream_t st) {
   uint16_t* Nb = (uint16_t*)((char*)a.ws + round_up(a.m * a.r * 2, 256));
   const int64_t ldn = round_up(a.n, 64);
   {
-    const int64_t threads = a.m * (a.r / 8);
-    dequant_p_bf16_kernel<<<(unsigned)ceil_div(threads, 256), 256, 0, st>>>(a.P, Pt, a.r);
-    QG_LAUNCH_CHECK();
+    const int rc = launch_dequant_p(a.P, Pt, a.r, st);
+    if (rc != QG_OK) return rc;
   }
   {
     AdamEpilogue epi{a.sc, a.M, a.V, a.ldmv, Nb, ldn, a.dbg.R, a.dbg.N, a.n};

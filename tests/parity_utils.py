@@ -56,20 +56,34 @@ def check_moments(gpu, ref, name, tol=2e-3):
     assert np.abs(gpu - ref).max() <= tol * max(np.abs(ref).max(), 1e-300), f"{name}: max error"
 
 
-def check_direction(gpu, ref, name="N", tol=2e-3):
-    """The Adam direction N = M^ / (sqrt(V^) + eps) is ill-conditioned where the projected gradient
-    is within a few eps of zero (at t = 1 it is R / (|R| + eps)), so it is held to the Frobenius bound
-    and to an element-wise bound on all but a vanishing fraction of the elements."""
+def ill_conditioned(ref: dict, hyp) -> np.ndarray:
+    """Elements of the low-rank state where the Adam direction N = M^ / (sqrt(V^) + eps) is
+    ill-conditioned: sqrt(V^) within a factor 1000 of eps.  There a rounding difference dR of the
+    projected gradient moves N by up to eps * dR / (sqrt(V^) + eps)^2, i.e. by O(1) when |R| ~ eps
+    (at t = 1, N = R / (|R| + eps)).  Elsewhere dN <= 1e-6 * dR / eps is far below the tolerance."""
+    _, _, _, b2, eps, _ = hyp.as_f32()
+    v_hat = ref["V"].astype(np.float64) / (1.0 - b2 ** int(hyp.step))
+    return np.sqrt(v_hat) < 1e3 * eps
+
+
+def check_direction(gpu, ref, hyp, name="N", tol=2e-3):
+    """N against the oracle: Frobenius bound on the whole matrix, element-wise bound wherever the
+    direction is well conditioned; the ill-conditioned elements must be rare and of ordinary size."""
     gpu = np.asarray(gpu, dtype=np.float64)
-    ref = np.asarray(ref, dtype=np.float64)
+    want = np.asarray(ref["N"], dtype=np.float64)
     assert np.all(np.isfinite(gpu)), f"{name}: non-finite values"
-    assert rel_fro(gpu, ref) <= tol, f"{name}: relative Frobenius error {rel_fro(gpu, ref):.3e}"
-    off = np.abs(gpu - ref) > tol * np.abs(ref).max()
-    assert off.mean() <= 1e-4, f"{name}: {off.mean():.2e} of the elements off by more than {tol}"
+    ill = ill_conditioned(ref, hyp)
+    assert ill.mean() <= 2e-2, f"{name}: {ill.mean():.2e} of the elements are ill-conditioned"
+    good = ~ill
+    err = np.abs(gpu - want)
+    assert np.linalg.norm(err[good]) <= tol * np.linalg.norm(want[good]), f"{name}: relative Frobenius error"
+    assert err[good].max() <= tol * np.abs(want).max(), f"{name}: max error {err[good].max():.3e}"
+    assert np.abs(gpu).max() <= 10.0 * max(np.abs(want).max(), 1.0), f"{name}: out of range"
+    return float(ill.mean())
 
 
 def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_frac=1e-3):
-    """INT8 weights after one step against the oracle's.
+    """INT8 weights after one step against the oracle's (same direction N_b on both sides).
 
     Scales agree to 1e-5 relative and zero points exactly wherever the group's scaled minimum is
     not at a rounding tie; codes agree except by exactly one level, in at most ``max_frac`` of the
@@ -104,3 +118,83 @@ def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_fr
         ok = near_draw | near_int | near_clamp
         assert np.all(ok[bad]), f"{(bad & ~ok).sum()} code mismatches away from any rounding boundary"
     return float(frac_bad)
+
+
+def check_weight_codes_unforced(gpu_w: O.QTensor, ref: dict, max_frac=5e-3):
+    """End-to-end sanity bound with the oracle's own direction: a handful of ill-conditioned N
+    elements shift whole columns of W' by a few 1e-3 LSB, so codes may differ by one level in
+    slightly more places than with the direction forced; never by more than one level."""
+    ref_w = ref["W"]
+    assert np.allclose(gpu_w.scales, ref_w.scales, rtol=1e-3, atol=0), "W scales (unforced)"
+    diff = np.abs(gpu_w.codes.astype(np.int32) - ref_w.codes.astype(np.int32))
+    n = ref_w.codes.shape[1]
+    gcols = np.repeat(np.arange(ref_w.scales.shape[1]), 256)[:n]
+    same_zero = (gpu_w.zeros == ref_w.zeros)[:, gcols]
+    assert diff[same_zero].max(initial=0) <= 1, "a weight code differs by more than one level (unforced)"
+    frac = float((diff[same_zero] != 0).mean()) if same_zero.any() else 0.0
+    assert frac <= max_frac, f"{frac:.2e} of the weight codes differ (unforced)"
+    return frac
+
+
+class StepTaps:
+    """Device buffers for the optional intermediates of qgalore_project_step."""
+
+    def __init__(self, m, n, r, w_ld):
+        self.R = B.zeros_matrix(r, n, torch.float32)
+        self.N = B.zeros_matrix(r, n, torch.float32)
+        self.W_pre = torch.zeros((m, w_ld), dtype=torch.float32, device="cuda")[:, :n]
+
+    def as_dict(self):
+        return {"R": self.R, "N": self.N, "W_pre": self.W_pre}
+
+
+def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2e-3, impl=None):
+    """Teacher-forced single-step parity of qgalore_project_step against the oracle.
+
+    Stage 1 (steps 1-4): M', V', R and the direction N against the oracle's own.
+    Stage 2 (steps 5-6): the oracle recomputes the weight update from the GPU's bf16 direction, and
+    W', scales, zero points and codes are held to the strict rule of check_weight_codes.
+    Plus the looser end-to-end bound against the oracle's unforced result.  Returns a dict of statistics.
+    """
+    m, n = gb.shape
+    r = P.codes.shape[1]
+    ref = O.project_step(gb, P, W, M, V, hyp)
+    dG, dP, dW = g_to_device(gb), to_device_q(P), to_device_q(W)
+    dM, dV = f32_to_device(M), f32_to_device(V)
+    taps = StepTaps(m, n, r, dW.ld)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if impl is not None:
+        B.debug_set_step_impl(impl)
+    try:
+        B.project_step(dG, dP, dW, dM, dV,
+                       B.Hyper(lr=hyp.lr, alpha=hyp.alpha, beta1=hyp.beta1, beta2=hyp.beta2, eps=hyp.eps,
+                               weight_decay=hyp.weight_decay, step=hyp.step, seed=hyp.seed),
+                       status=status, debug=taps.as_dict())
+        torch.cuda.synchronize()
+    finally:
+        if impl is not None:
+            B.debug_set_step_impl(0)
+    assert int(status.item()) == 0, "device status word"
+    # stage 1
+    check_moments(dM.cpu().numpy(), ref["M"], "M", tol)
+    check_moments(dV.cpu().numpy(), ref["V"], "V", tol)
+    check_moments(taps.R.cpu().numpy(), ref["R32"], "R", tol)
+    n_gpu = taps.N.cpu().numpy()
+    ill = check_direction(n_gpu, ref, hyp, "N", tol)
+    # stage 2: same direction on both sides
+    forced = O.project_step(gb, P, W, M, V, hyp, N_b_override=O.bf16_round(n_gpu))
+    lsb = np.repeat(forced["W"].scales, 256, axis=1)[:, :n]
+    wpre_err = float((np.abs(taps.W_pre.cpu().numpy() - forced["W_pre"]) / lsb).max())
+    assert wpre_err <= 1e-3, f"pre-rounding weight off by {wpre_err:.2e} LSB"
+    gw = from_device_q(dW)
+    frac = check_weight_codes(gw, forced, hyp.seed, hyp.step)
+    frac_unforced = check_weight_codes_unforced(gw, ref)
+    # padding of the rows is never written
+    if dW.ld > n:
+        assert int(dW.codes[:, n:].abs().max().item()) == 0, "padding of the code rows was written"
+    for t in (dM, dV):
+        base = t._base
+        if base is not None and base.shape[1] > n:
+            assert float(base[:, n:].abs().max().item()) == 0.0, "padding of the moment rows was written"
+    return {"mismatch": frac, "mismatch_unforced": frac_unforced, "ill": ill, "wpre_err_lsb": wpre_err,
+            "W": gw, "M": dM.cpu().numpy(), "V": dV.cpu().numpy(), "ref": ref}

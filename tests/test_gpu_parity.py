@@ -8,8 +8,7 @@ import oracle as O
 from paper_2407_08296_b200 import binding as B
 from paper_2407_08296_b200 import synth
 
-from parity_utils import (check_direction, check_moments, check_weight_codes, f32_to_device, from_device_q, g_to_device,
-                          to_device_q)
+from parity_utils import f32_to_device, from_device_q, g_to_device, run_and_check_step, to_device_q
 
 pytestmark = pytest.mark.gpu
 
@@ -75,62 +74,26 @@ def test_similarity_matches_oracle(m, r, c):
 
 
 # ----------------------------------------------------------------------------- the step
-def run_step_case(m, n, r, seed=0, step=1, steps_before=0, wd=0.0, check_taps=True, impl=None):
+def run_step_case(m, n, r, seed=0, step=1, steps_before=0, wd=0.0, impl=None, P=None, matrix_index=1):
     """Teacher-forced single-step parity: upload the oracle's pre-step state, run one GPU step, compare."""
-    gm = synth.GradientModel(m, n, seed=seed, matrix_index=1)
-    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=seed, stream=9), 4)
-    W = O.quantize_rtn(synth.initial_weight(m, n, seed=seed, matrix_index=1), 8)
+    gm = synth.GradientModel(m, n, seed=seed, matrix_index=matrix_index)
+    if P is None:
+        P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=seed, stream=9), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, seed=seed, matrix_index=matrix_index), 8)
     M = np.zeros((r, n), np.float32)
     V = np.zeros((r, n), np.float32)
-    sr_seed = synth.matrix_seed(seed, 1)
-    t0 = step - steps_before
-    for t in range(t0, step):          # advance the oracle so that M, V are not trivial
+    sr_seed = synth.matrix_seed(seed, matrix_index)
+    for t in range(step - steps_before, step):          # advance the oracle so that M, V are not trivial
         out = O.project_step(gm.sample(t), P, W, M, V, O.Hyper(step=t, seed=sr_seed, weight_decay=wd))
         W, M, V = out["W"], out["M"], out["V"]
-    gb = gm.sample(step)
-    hyp = O.Hyper(step=step, seed=sr_seed, weight_decay=wd)
-    ref = O.project_step(gb, P, W, M, V, hyp)
-
-    dG, dP, dW = g_to_device(gb), to_device_q(P), to_device_q(W)
-    dM, dV = f32_to_device(M), f32_to_device(V)
-    taps = {}
-    if check_taps:
-        taps = {"R": torch.zeros_like(dM), "N": torch.zeros_like(dM),
-                "W_pre": B.zeros_matrix(m, n, torch.float32, "cuda", 1)}
-        # the taps share the pitch of M (R, N) and of W's codes (W_pre)
-        taps["R"] = B.zeros_matrix(r, n, torch.float32)
-        taps["N"] = B.zeros_matrix(r, n, torch.float32)
-        taps["W_pre"] = torch.zeros((m, dW.ld), dtype=torch.float32, device="cuda")[:, :n]
-    status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    if impl is not None:
-        B.debug_set_step_impl(impl)
-    try:
-        B.project_step(dG, dP, dW, dM, dV, B.Hyper(step=step, seed=sr_seed, weight_decay=wd), status=status,
-                       debug=taps or None)
-        torch.cuda.synchronize()
-    finally:
-        if impl is not None:
-            B.debug_set_step_impl(0)
-    assert int(status.item()) == 0
-    check_moments(dM.cpu().numpy(), ref["M"], "M", MOMENT_TOL)
-    check_moments(dV.cpu().numpy(), ref["V"], "V", MOMENT_TOL)
-    if check_taps:
-        check_moments(taps["R"].cpu().numpy(), ref["R32"], "R", MOMENT_TOL)
-        check_direction(taps["N"].cpu().numpy(), ref["N"], "N", MOMENT_TOL)
-        wpre = taps["W_pre"].cpu().numpy()
-        lsb = np.repeat(ref["W"].scales, 256, axis=1)[:, :n]
-        assert np.abs(wpre - ref["W_pre"]).max() <= 2e-3 * lsb.max(), "pre-rounding weight off by more than 2e-3 LSB"
-    gw = from_device_q(dW)
-    frac = check_weight_codes(gw, ref, sr_seed, step)
-    # padding of the code rows is never written
-    if dW.ld > n:
-        assert int(dW.codes[:, n:].abs().max().item()) == 0
-    return frac
+    return run_and_check_step(gm.sample(step), P, W, M, V, O.Hyper(step=step, seed=sr_seed, weight_decay=wd),
+                              tol=MOMENT_TOL, impl=impl)
 
 
 SMALL_CASES = [
     (64, 256, 32), (128, 512, 64), (96, 300, 32), (160, 1376, 64), (512, 1376, 128),
-    (300, 777, 96), (768, 768, 256), (1000, 85, 128), (130, 2736, 128),
+    (300, 777, 96), (768, 768, 256), (1000, 85, 128), (130, 2736, 128), (64, 3, 32), (200, 17, 64),
+    (257, 1025, 160),
 ]
 
 
@@ -151,19 +114,15 @@ def test_step_parity_after_several_steps_with_weight_decay():
 def test_step_config1_llama60m_mlp():
     # configs[0]: 512 x 1376, r = 128, one step, seed 0, P from the oracle's refresh of that gradient
     spec = synth.stack_matrices("llama60m_mlp")[0]
-    gm = synth.GradientModel(spec.m, spec.n, seed=0, matrix_index=0)
-    gb = gm.sample(1)
+    gb = synth.GradientModel(spec.m, spec.n, seed=0, matrix_index=0).sample(1)
     _, P, _ = O.refresh_subspace(gb, spec.r)
-    W = O.quantize_rtn(synth.initial_weight(spec.m, spec.n, 0, 0), 8)
-    z = np.zeros((spec.r, spec.n), np.float32)
-    seed = synth.matrix_seed(0, 0)
-    ref = O.project_step(gb, P, W, z, z, O.Hyper(step=1, seed=seed))
-    dW, dM, dV = to_device_q(W), f32_to_device(z), f32_to_device(z)
-    B.project_step(g_to_device(gb), to_device_q(P), dW, dM, dV, B.Hyper(step=1, seed=seed))
-    torch.cuda.synchronize()
-    check_moments(dM.cpu().numpy(), ref["M"], "M")
-    check_moments(dV.cpu().numpy(), ref["V"], "V")
-    check_weight_codes(from_device_q(dW), ref, seed, 1)
+    run_step_case(spec.m, spec.n, spec.r, seed=0, step=1, P=P, matrix_index=0)
+
+
+@pytest.mark.parametrize("m,n,r", [(2048, 2048, 512), (2048, 5461, 512), (5461, 2048, 512)])
+def test_step_parity_llama1b_shapes(m, n, r):
+    # the three distinct shapes of the LLaMA-1B stack at full size, second step (non-trivial moments)
+    run_step_case(m, n, r, seed=4, step=2, steps_before=1)
 
 
 def test_step_is_deterministic_and_seeded():
