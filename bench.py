@@ -172,7 +172,7 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------- our arm
-def build_stack(workload, device, seed=0):
+def build_stack(workload, device, seed=0, layers=0):
     """Device-resident synthetic state of the whole stack: bf16 gradients (rank-32 signal + noise),
     INT8 weights, INT4 projections, zero moments.  Generated with torch on the device (input
     generation, not the path); quantization goes through the library."""
@@ -180,6 +180,8 @@ def build_stack(workload, device, seed=0):
     from paper_2407_08296_b200 import binding as B
     from paper_2407_08296_b200 import synth
     specs = synth.stack_matrices(workload)
+    if layers:
+        specs = [s for s in specs if s.layer < layers]
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
     items = []
@@ -224,8 +226,8 @@ def run_ours(args):
     peaks, peak_kind = load_peaks()
 
     # every rank holds and steps its own replica of the stack: matrices are independent units, no collective
-    specs, items = build_stack(args.workload, device, seed=rank)
-    batch = B.StepBatch(items)
+    specs, items = build_stack(args.workload, device, seed=rank, layers=args.layers)
+    batch = B.StepPlan(items)
     elements = batch.elements
     hyper = B.Hyper()
     torch.cuda.synchronize()
@@ -323,7 +325,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload, "matrices": len(specs), "elements_per_step": elements,
+            "config": {"workload": args.workload + (f"[first {args.layers} layers]" if args.layers else ""), "matrices": len(specs), "elements_per_step": elements,
                        "rank": specs[0].r, "group": 256, "l2": "inputs larger than L2 (whole stack streams each step)",
                        "parallelism": f"replica per GPU x{world}, no collective"},
             "roofline": roof, "cpu_baseline": cpu,
@@ -345,6 +347,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="keep only the first L layers of the stack (small cases for profiler captures); 0 = all")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

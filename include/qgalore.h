@@ -137,6 +137,28 @@ QG_API int qgalore_project_step_batched(const qg_step_item* items, int32_t count
                                  int32_t* status_dev, void* stream);
 QG_API size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t count);
 
+/* --- Sec. 3.5, the step of a fixed list of matrices prepared once ("plan") -------------------------
+ * A training loop steps the same matrices, in the same buffers, thousands of times.  A plan does the
+ * per-matrix set-up once (validation, TMA descriptors, tile tables) and then steps the whole list with
+ * a few grouped kernel launches: consecutive items are packed into chunks that share the workspace, and
+ * each chunk runs as one dequantize-P launch, one projection+Adam launch and one back-projection+
+ * requantization launch over all of its matrices.
+ *   items       HOST; every buffer an item names must stay where it is while the plan lives
+ *   table_dev   DEVICE, 256-byte aligned, qgalore_plan_table_bytes(count) bytes, owned by the caller and
+ *               left untouched by it until qgalore_plan_destroy
+ *   workspace   DEVICE scratch, 1024-byte aligned, at least qgalore_workspace_bytes_batched(items, count)
+ *               bytes; more lets a chunk hold more matrices.  Contents are undefined between steps, but
+ *               the buffer must not move.
+ * qgalore_plan_create copies the table to the device synchronously; it allocates host memory only.
+ * qgalore_plan_step enqueues one optimizer step of every matrix (lr, alpha, the Adam constants and the
+ * step index from h; the stochastic-rounding seed of each matrix from its item) and returns. */
+typedef struct qg_plan qg_plan;
+QG_API size_t qgalore_plan_table_bytes(int32_t count);
+QG_API int qgalore_plan_create(const qg_step_item* items, int32_t count, void* table_dev, size_t table_bytes,
+                        void* workspace, size_t workspace_bytes, qg_plan** plan);
+QG_API int qgalore_plan_step(const qg_plan* plan, const qg_hyper* h, int32_t* status_dev, void* stream);
+QG_API void qgalore_plan_destroy(qg_plan* plan);
+
 /* --- Sec. 3.5 "obtain the projection matrix using SVD" + Sec. 3.3 INT4 storage ------------
  * Top-r left singular subspace of G (bf16, m x n) by block subspace iteration with
  * `oversample_cols` extra columns and a Rayleigh-Ritz step, then Quant_4 into P_new.

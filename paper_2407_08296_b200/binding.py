@@ -74,6 +74,12 @@ def lib() -> C.CDLL:
         L.qgalore_project_step_batched.argtypes = [C.POINTER(_CStepItem), i32, C.POINTER(_CHyper), vp, sz, vp, vp]
         L.qgalore_workspace_bytes_batched.argtypes = [C.POINTER(_CStepItem), i32]
         L.qgalore_workspace_bytes_batched.restype = sz
+        L.qgalore_plan_table_bytes.argtypes = [i32]
+        L.qgalore_plan_table_bytes.restype = sz
+        L.qgalore_plan_create.argtypes = [C.POINTER(_CStepItem), i32, vp, sz, vp, sz, C.POINTER(vp)]
+        L.qgalore_plan_step.argtypes = [vp, C.POINTER(_CHyper), vp, vp]
+        L.qgalore_plan_destroy.argtypes = [vp]
+        L.qgalore_plan_destroy.restype = None
         L.qgalore_refresh_subspace.argtypes = [vp, i64, i64, i64, i64, i32, i32, C.c_uint64, qp, vp, qp, i32, vp,
                                                vp, sz, vp, vp]
         L.qgalore_subspace_similarity.argtypes = [qp, qp, i32, vp, vp, sz, vp]
@@ -274,6 +280,55 @@ class StepBatch:
         _check(lib().qgalore_project_step_batched(self._table, len(self.items), C.byref(hc), _ptr(self.workspace),
                                                   self.workspace.numel(), _ptr(self.status), _stream_ptr(stream)),
                "qgalore_project_step_batched")
+
+
+class StepPlan:
+    """A fixed list of matrices prepared once and stepped many times with grouped launches (Sec. 3.5).
+
+    ``items`` are dicts with G, P, W, M, V and seed.  The plan owns its device table and workspace (torch
+    tensors) and keeps references to the items' tensors, which must not be reallocated while it lives.
+    """
+
+    PREFERRED_WORKSPACE = 64 << 20
+
+    def __init__(self, items: list[dict], workspace_bytes: int | None = None, device=None):
+        self.items = items
+        n = len(items)
+        self._table = (_CStepItem * n)()
+        for k, it in enumerate(items):
+            G, P, W, M, V = it["G"], it["P"], it["W"], it["M"], it["V"]
+            m, ncol = G.shape
+            self._table[k] = _CStepItem(_ptr(G), _matrix_ld(G, "G"), m, ncol, P.cols, P.c_struct(), W.c_struct(),
+                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)))
+        dev = device if device is not None else items[0]["G"].device
+        L = lib()
+        need = int(L.qgalore_workspace_bytes_batched(self._table, n))
+        if workspace_bytes is None:
+            workspace_bytes = max(need, self.PREFERRED_WORKSPACE)
+        self.workspace = torch.empty(max(int(workspace_bytes), 1024), dtype=torch.uint8, device=dev)
+        self.table_dev = torch.empty(int(L.qgalore_plan_table_bytes(n)), dtype=torch.uint8, device=dev)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.elements = sum(int(it["G"].shape[0]) * int(it["G"].shape[1]) for it in items)
+        handle = C.c_void_p()
+        _check(L.qgalore_plan_create(self._table, n, _ptr(self.table_dev), self.table_dev.numel(), _ptr(self.workspace),
+                                     self.workspace.numel(), C.byref(handle)), "qgalore_plan_create")
+        self._handle = handle
+
+    def step(self, hyper: Hyper, stream=None) -> None:
+        hc = hyper.c_struct()
+        _check(lib().qgalore_plan_step(self._handle, C.byref(hc), _ptr(self.status), _stream_ptr(stream)),
+               "qgalore_plan_step")
+
+    def close(self) -> None:
+        if self._handle is not None and self._handle.value:
+            lib().qgalore_plan_destroy(self._handle)
+            self._handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def refresh_subspace(G: torch.Tensor, r: int, iters: int = 12, oversample_cols: int | None = None, seed: int = 0,

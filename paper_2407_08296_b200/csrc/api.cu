@@ -4,6 +4,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <vector>
 
 #include "qg_common.cuh"
 
@@ -26,6 +27,12 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
                    uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes,
                    int32_t* status, cudaStream_t st);
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b);
+struct Plan;
+size_t plan_table_bytes(int32_t count);
+int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t table_bytes, void* workspace,
+                size_t workspace_bytes, Plan** out);
+int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st);
+void plan_destroy(Plan* plan);
 
 static int g_step_impl = 0;  // 0: tensor-core kernels; 1: CUDA-core kernels (validation aid)
 
@@ -105,12 +112,30 @@ size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r) {
   }
 }
 
-static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
-                             const qg_qtensor* W, float* M, float* V, int64_t ldmv, const qg_hyper* h,
-                             void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
-                             void* stream, bool validate_only) {
-  if (!G || !M || !V || !h || !workspace) return QG_INVALID_ARGUMENT;
-  if (m <= 0 || n <= 0 || r <= 0 || ldg < n || ldmv < n || h->step < 1) return QG_INVALID_ARGUMENT;
+static void fill_scalars(const qg_hyper* h, uint64_t seed, StepScalars* sc) {
+  sc->beta1 = h->beta1; sc->beta2 = h->beta2;
+  sc->one_minus_beta1 = 1.0f - h->beta1; sc->one_minus_beta2 = 1.0f - h->beta2;
+  sc->bias1 = (float)(1.0 - std::pow((double)h->beta1, (double)h->step));
+  sc->bias2 = (float)(1.0 - std::pow((double)h->beta2, (double)h->step));
+  sc->eps = h->eps;
+  sc->lr_alpha = (float)((double)h->lr * (double)h->alpha);
+  sc->lr_wd = (float)((double)h->lr * (double)h->weight_decay);
+  sc->seed_lo = (uint32_t)(seed & 0xFFFFFFFFull); sc->seed_hi = (uint32_t)(seed >> 32);
+  sc->step_lo = (uint32_t)((uint64_t)h->step & 0xFFFFFFFFull); sc->step_hi = (uint32_t)((uint64_t)h->step >> 32);
+}
+
+static int check_hyper(const qg_hyper* h) {
+  if (!h || h->step < 1) return QG_INVALID_ARGUMENT;
+  if (!std::isfinite(h->lr) || !(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
+    return QG_INVALID_ARGUMENT;
+  return QG_OK;
+}
+
+// Shape, pointer and alignment rules of one matrix of the step; fills everything of `a` but the scalars.
+static int check_matrix(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
+                        const qg_qtensor* W, float* M, float* V, int64_t ldmv, StepArgs* a) {
+  if (!G || !M || !V) return QG_INVALID_ARGUMENT;
+  if (m <= 0 || n <= 0 || r <= 0 || ldg < n || ldmv < n) return QG_INVALID_ARGUMENT;
   int rc = check_qtensor(P, 4);
   if (rc != QG_OK) return rc;
   rc = check_qtensor(W, 8);
@@ -119,28 +144,29 @@ static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
   if (r % 32 != 0 || r < 32 || r > 2048 || r > m) return QG_UNSUPPORTED_SHAPE;
   if (m > (1ll << 31) - 1 || n > (1ll << 31) - 1) return QG_UNSUPPORTED_SHAPE;
   if (!aligned16(G) || !aligned16(M) || !aligned16(V) || ldg % 8 != 0 || ldmv % 4 != 0) return QG_MISALIGNED;
+  memset(a, 0, sizeof(*a));
+  a->G = G; a->ldg = ldg; a->m = m; a->n = n; a->r = r;
+  a->P = *P; a->W = *W; a->M = M; a->V = V; a->ldmv = ldmv;
+  return QG_OK;
+}
+
+static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
+                             const qg_qtensor* W, float* M, float* V, int64_t ldmv, const qg_hyper* h,
+                             void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
+                             void* stream, bool validate_only) {
+  if (!workspace) return QG_INVALID_ARGUMENT;
+  int rc = check_hyper(h);
+  if (rc != QG_OK) return rc;
+  StepArgs a;
+  rc = check_matrix(G, ldg, m, n, r, P, W, M, V, ldmv, &a);
+  if (rc != QG_OK) return rc;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QG_MISALIGNED;
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
   if (workspace_bytes < qgalore_workspace_bytes(QG_OP_PROJECT_STEP, m, n, r)) return QG_WORKSPACE_TOO_SMALL;
-  if (!std::isfinite(h->lr) || !(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
-    return QG_INVALID_ARGUMENT;
   if (validate_only) return QG_OK;
-
-  StepArgs a;
-  a.G = G; a.ldg = ldg; a.m = m; a.n = n; a.r = r;
-  a.P = *P; a.W = *W; a.M = M; a.V = V; a.ldmv = ldmv;
   a.ws = workspace; a.ws_bytes = workspace_bytes; a.status = status_dev;
-  if (dbg) a.dbg = *dbg; else memset(&a.dbg, 0, sizeof(a.dbg));
-  StepScalars& sc = a.sc;
-  sc.beta1 = h->beta1; sc.beta2 = h->beta2;
-  sc.one_minus_beta1 = 1.0f - h->beta1; sc.one_minus_beta2 = 1.0f - h->beta2;
-  sc.bias1 = (float)(1.0 - std::pow((double)h->beta1, (double)h->step));
-  sc.bias2 = (float)(1.0 - std::pow((double)h->beta2, (double)h->step));
-  sc.eps = h->eps;
-  sc.lr_alpha = (float)((double)h->lr * (double)h->alpha);
-  sc.lr_wd = (float)((double)h->lr * (double)h->weight_decay);
-  sc.seed_lo = (uint32_t)(h->seed & 0xFFFFFFFFull); sc.seed_hi = (uint32_t)(h->seed >> 32);
-  sc.step_lo = (uint32_t)((uint64_t)h->step & 0xFFFFFFFFull); sc.step_hi = (uint32_t)((uint64_t)h->step >> 32);
+  if (dbg) a.dbg = *dbg;
+  fill_scalars(h, h->seed, &a.sc);
   if (g_step_impl == 1) return launch_project_step_simt(a, (cudaStream_t)stream);
   return launch_project_step_tc(a, (cudaStream_t)stream);
 }
@@ -178,6 +204,48 @@ int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const
     }
   }
   return QG_OK;
+}
+
+struct qg_plan {
+  Plan* impl;
+};
+
+size_t qgalore_plan_table_bytes(int32_t count) { return count > 0 ? plan_table_bytes(count) : 0; }
+
+int qgalore_plan_create(const qg_step_item* items, int32_t count, void* table_dev, size_t table_bytes,
+                        void* workspace, size_t workspace_bytes, qg_plan** plan) {
+  if (!items || count <= 0 || !table_dev || !workspace || !plan) return QG_INVALID_ARGUMENT;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) || (reinterpret_cast<uintptr_t>(table_dev) & 255u))
+    return QG_MISALIGNED;
+  std::vector<StepArgs> args((size_t)count);
+  for (int32_t i = 0; i < count; ++i) {
+    const qg_step_item& it = items[i];
+    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &args[i]);
+    if (rc != QG_OK) return rc;
+    args[i].sc.seed_lo = (uint32_t)(it.seed & 0xFFFFFFFFull);
+    args[i].sc.seed_hi = (uint32_t)(it.seed >> 32);
+  }
+  Plan* impl = nullptr;
+  const int rc = plan_create(args.data(), count, table_dev, table_bytes, workspace, workspace_bytes, &impl);
+  if (rc != QG_OK) return rc;
+  *plan = new qg_plan{impl};
+  return QG_OK;
+}
+
+int qgalore_plan_step(const qg_plan* plan, const qg_hyper* h, int32_t* status_dev, void* stream) {
+  if (!plan || !plan->impl) return QG_INVALID_ARGUMENT;
+  const int rc = check_hyper(h);
+  if (rc != QG_OK) return rc;
+  if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
+  StepScalars sc;
+  fill_scalars(h, 0, &sc);
+  return plan_step(plan->impl, sc, status_dev, (cudaStream_t)stream);
+}
+
+void qgalore_plan_destroy(qg_plan* plan) {
+  if (!plan) return;
+  plan_destroy(plan->impl);
+  delete plan;
 }
 
 int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,

@@ -20,6 +20,7 @@
 // Every barrier wait is bounded; on expiry the kernel raises QG_DEV_WAIT_EXPIRED in the status word,
 // stops taking tiles, releases its tensor memory and returns.
 #include <cstring>
+#include <vector>
 
 #include "sm100_ptx.cuh"
 #include "step_epilogue.cuh"
@@ -48,7 +49,6 @@ constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
 //                                 plain stores instead (n_tma_mv / n_tma_w = columns the TMA stores cover).
 struct alignas(64) TcProblem {
   CUtensorMap mapP, mapG, mapN, mapNst, mapM, mapV, mapW, mapMst, mapVst, mapWst;
-  StepScalars sc;
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -59,6 +59,7 @@ struct alignas(64) TcProblem {
   int8_t* w_codes;
   int64_t ldmv, ldw;
   int32_t m, n, r, ngroups, n_tma_mv, n_tma_w;
+  uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles, k1_tile0;
   int32_t k2_mblocks, k2_tiles, k2_tile0;
 };
@@ -66,6 +67,12 @@ static_assert(sizeof(TcProblem) <= 2048, "TcProblem must fit the kernel paramete
 
 __device__ __forceinline__ void raise_wait_expired(int32_t* status) {
   if (status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
+}
+
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
 // ============================================================================================
@@ -77,7 +84,7 @@ struct K1Smem {
   static constexpr int kABytes = 2 * kBoxBytes;            // 128 (r) x 64 (m) bf16
   static constexpr int kBBytes = (BN / 64) * kBoxBytes;    // BN (n) x 64 (m) bf16
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kMvBufs = 3;
+  static constexpr int kMvBufs = BN >= 256 ? 2 : 3;
   static constexpr int kMBytes = kTileM * kChunk * 4;      // 16 KB
   static constexpr int kNBytes = kTileM * kChunk * 2;      // 8 KB
   static constexpr int kMvBufBytes = 2 * kMBytes + kNBytes;
@@ -88,7 +95,7 @@ struct K1Smem {
 template <int BN, bool SINGLE>
 __global__ void __launch_bounds__(224, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table, int nprob,
-                    int total_tiles, int32_t* __restrict__ status) {
+                    int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
   using S = K1Smem<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -138,9 +145,11 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         const TcProblem* p = locate(tile, pi);
-        const int local = tile - p->k1_tile0;
-        const int r0 = (local % p->k1_rblocks) * kTileM, n0 = (local / p->k1_rblocks) * BN;
+        const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
+        const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
         const int kblocks = (p->m + kBK - 1) / kBK;
+        const CUtensorMap* mapP = &p->mapP;
+        const CUtensorMap* mapG = &p->mapG;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % S::kStages;
           const uint32_t ph = (it / S::kStages) & 1;
@@ -149,9 +158,9 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
           uint8_t* sB = sA + S::kABytes;
           mbar_arrive_expect_tx(&full[s], S::kStageBytes);
 #pragma unroll
-          for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, &p->mapP, &full[s], r0 + 64 * h, kb * kBK);
+          for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], r0 + 64 * h, kb * kBK);
 #pragma unroll
-          for (int h = 0; h < BN / 64; ++h) tma_load_2d(sB + h * kBoxBytes, &p->mapG, &full[s], n0 + 64 * h, kb * kBK);
+          for (int h = 0; h < BN / 64; ++h) tma_load_2d(sB + h * kBoxBytes, mapG, &full[s], n0 + 64 * h, kb * kBK);
         }
       }
       if (!ok) raise_wait_expired(status);
@@ -197,16 +206,18 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
         const TcProblem* p = locate(tile, pi);
-        const int local = tile - p->k1_tile0;
-        const int r0 = (local % p->k1_rblocks) * kTileM, n0 = (local / p->k1_rblocks) * BN;
+        const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
+        const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
         const int nchunks = min(BN / kChunk, (p->n - n0 + kChunk - 1) / kChunk);
+        const CUtensorMap* mapM = &p->mapM;
+        const CUtensorMap* mapV = &p->mapV;
         for (int c = 0; c < nchunks; ++c, ++cc) {
           const int b = cc % S::kMvBufs;
           if (!mbar_wait(&mv_empty[b], ((cc / S::kMvBufs) & 1) ^ 1)) { ok = false; break; }
           uint8_t* buf = mv_base + b * S::kMvBufBytes;
           mbar_arrive_expect_tx(&mv_full[b], 2 * S::kMBytes);
-          tma_load_2d(buf, &p->mapM, &mv_full[b], n0 + c * kChunk, r0);
-          tma_load_2d(buf + S::kMBytes, &p->mapV, &mv_full[b], n0 + c * kChunk, r0);
+          tma_load_2d(buf, mapM, &mv_full[b], n0 + c * kChunk, r0);
+          tma_load_2d(buf + S::kMBytes, mapV, &mv_full[b], n0 + c * kChunk, r0);
         }
       }
       if (!ok) raise_wait_expired(status);
@@ -216,16 +227,25 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     const int q = warp & 3;                         // TMEM lane quarter this warp may access
     const int row = q * 32 + lane;                  // accumulator row = row of the r block
     const bool elected = (threadIdx.x == 96);       // first epilogue thread issues the TMA stores
+    const float inv_b1 = 1.0f / sc.bias1, inv_b2 = 1.0f / sc.bias2;
     int pi = 0;
     uint32_t cc = 0, tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
       const TcProblem* p = locate(tile, pi);
-      const int local = tile - p->k1_tile0;
-      const int r0 = (local % p->k1_rblocks) * kTileM, n0 = (local / p->k1_rblocks) * BN;
-      const int nchunks = min(BN / kChunk, (p->n - n0 + kChunk - 1) / kChunk);
-      const StepScalars sc = p->sc;
-      const float inv_b1 = 1.0f / sc.bias1, inv_b2 = 1.0f / sc.bias2;
+      const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
+      const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
+      const int pn = p->n, n_tma = p->n_tma_mv;
+      const int nchunks = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
+      const bool row_ok = r0 + row < p->r;
+      const int64_t ldmv = p->ldmv;
+      float* gM = p->M + (int64_t)(r0 + row) * ldmv;
+      float* gV = p->V + (int64_t)(r0 + row) * ldmv;
+      float* dbgR = p->dbgR ? p->dbgR + (int64_t)(r0 + row) * ldmv : nullptr;
+      float* dbgN = p->dbgN ? p->dbgN + (int64_t)(r0 + row) * ldmv : nullptr;
+      const CUtensorMap* mapMst = &p->mapMst;
+      const CUtensorMap* mapVst = &p->mapVst;
+      const CUtensorMap* mapNst = &p->mapNst;
       const uint32_t ab = tcount & 1;
       ok = named_bar_and(1, 128, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
       if (!ok) break;
@@ -241,7 +261,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         float4* Mrow = reinterpret_cast<float4*>(buf + row * 128);
         float4* Vrow = reinterpret_cast<float4*>(buf + S::kMBytes + row * 128);
         uint2* Nrow = reinterpret_cast<uint2*>(buf + 2 * S::kMBytes + row * 64);
-        const bool tap = (p->dbgR != nullptr || p->dbgN != nullptr) && (r0 + row < p->r);
+        const int col0 = n0 + c * kChunk;
+        const bool special = row_ok && ((dbgR != nullptr) | (dbgN != nullptr) | (col0 + kChunk > n_tma));
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int pj = j ^ (row & 7);             // 128-byte swizzle: 16-byte chunk j lives at j ^ (row % 8)
@@ -252,31 +273,23 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
             const float rr = __uint_as_float(acc[4 * j + e]);
             mm[e] = fmaf(sc.beta1, mm[e], sc.one_minus_beta1 * rr);
             vv[e] = fmaf(sc.beta2, vv[e], sc.one_minus_beta2 * rr * rr);
-            nn[e] = __fdividef(mm[e] * inv_b1, sqrtf(vv[e] * inv_b2) + sc.eps);
+            nn[e] = __fdividef(mm[e] * inv_b1, sqrt_approx(vv[e] * inv_b2) + sc.eps);
           }
           Mrow[pj] = make_float4(mm[0], mm[1], mm[2], mm[3]);
           Vrow[pj] = make_float4(vv[0], vv[1], vv[2], vv[3]);
-          if (n0 + c * kChunk + 4 * j == p->n_tma_mv && r0 + row < p->r) {   // ragged tail: at most 3 columns
-#pragma unroll
-            for (int e = 0; e < 3; ++e) {
-              if (e < p->n - p->n_tma_mv) {
-                p->M[(int64_t)(r0 + row) * p->ldmv + p->n_tma_mv + e] = mm[e];
-                p->V[(int64_t)(r0 + row) * p->ldmv + p->n_tma_mv + e] = vv[e];
-              }
-            }
-          }
           uint2 nb;
           nb.x = (uint32_t)float_to_bf16_bits(nn[0]) | ((uint32_t)float_to_bf16_bits(nn[1]) << 16);
           nb.y = (uint32_t)float_to_bf16_bits(nn[2]) | ((uint32_t)float_to_bf16_bits(nn[3]) << 16);
           // 64-byte swizzle of the bf16 tile: 16-byte chunk (j / 2) lives at (j / 2) ^ ((row / 2) % 4)
           Nrow[(((j >> 1) ^ ((row >> 1) & 3)) << 1) | (j & 1)] = nb;
-          if (tap) {
+          if (special) {                            // ragged tail (at most 3 columns) and the test taps
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const int col = n0 + c * kChunk + 4 * j + e;
-              if (col < p->n) {
-                if (p->dbgR) p->dbgR[(int64_t)(r0 + row) * p->ldmv + col] = __uint_as_float(acc[4 * j + e]);
-                if (p->dbgN) p->dbgN[(int64_t)(r0 + row) * p->ldmv + col] = nn[e];
+              const int col = col0 + 4 * j + e;
+              if (col < pn) {
+                if (col >= n_tma) { gM[col] = mm[e]; gV[col] = vv[e]; }
+                if (dbgR) dbgR[col] = __uint_as_float(acc[4 * j + e]);
+                if (dbgN) dbgN[col] = nn[e];
               }
             }
           }
@@ -284,11 +297,11 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         fence_proxy_async_smem();
         named_bar_sync(1, 128);
         if (elected) {
-          if (n0 + c * kChunk < p->n_tma_mv) {
-            tma_store_2d(&p->mapMst, buf, n0 + c * kChunk, r0);
-            tma_store_2d(&p->mapVst, buf + S::kMBytes, n0 + c * kChunk, r0);
+          if (col0 < n_tma) {
+            tma_store_2d(mapMst, buf, col0, r0);
+            tma_store_2d(mapVst, buf + S::kMBytes, col0, r0);
           }
-          tma_store_2d(&p->mapNst, buf + 2 * S::kMBytes, n0 + c * kChunk, r0);
+          tma_store_2d(mapNst, buf + 2 * S::kMBytes, col0, r0);
           tma_commit_group();
           if (cc >= 1) {                             // the previous chunk's buffer has been read out
             tma_wait_group_read<1>();
@@ -325,19 +338,77 @@ struct K2Smem {
   static constexpr int kCodeBufs = 2;
   static constexpr int kCodeBytes = kTileM * kBN;          // 32 KB of INT8 codes
   static constexpr int kBarOffset = kStages * kStageBytes + kCodeBufs * kCodeBytes;
-  static constexpr int kBytes = kBarOffset + 256 + 1024;
+  static constexpr int kPartOffset = kBarOffset + 256;     // float2 [4 slices][128 rows]: partial min/max
+  static constexpr int kBytes = kPartOffset + 4 * kTileM * 8 + 1024;
+  static constexpr int kEpiWarps = 16;                     // 4 lane quarters x 4 column slices of 64
+  static constexpr int kEpiThreads = kEpiWarps * 32;
+  static constexpr int kThreads = 64 + kEpiThreads;
 };
 
-// Pre-rounding weight of one element: W' = W^ - lr*alpha*D - lr*wd*W^ with W^ = (q - z) * s.
-__device__ __forceinline__ float weight_pre(float qf, float z, float s, float d, const StepScalars& sc) {
-  const float wh = __fmul_rn(__fsub_rn(qf, z), s);
-  return fmaf(-sc.lr_alpha, d, fmaf(-sc.lr_wd, wh, wh));
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves an integer in the low mantissa bits
+
+// 16 consecutive pre-rounding weights W' = W^ - lr*alpha*D - lr*wd*W^, W^ = (q - z) * s, from 16 INT8
+// codes and 16 accumulators.  FAST: q - z is formed without an integer-to-float conversion: the byte
+// (q + 128) is dropped into the mantissa of 2^23 and (2^23 + 128 + z) subtracted, exact for |z| < 2^22.
+template <bool FAST>
+__device__ __forceinline__ void weights16(const uint4 cw, const uint32_t* acc, float z, float s, float lr_alpha,
+                                          float lr_wd, float* w) {
+  const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
+  const float c0 = 8388736.0f + z;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t x = w4[k] ^ 0x80808080u;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      float qz;
+      if (FAST) qz = __fsub_rn(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650 + b)), c0);
+      else qz = __fsub_rn((float)(int8_t)((w4[k] >> (8 * b)) & 0xFFu), z);
+      const float wh = __fmul_rn(qz, s);
+      w[4 * k + b] = fmaf(-lr_alpha, __uint_as_float(acc[4 * k + b]), fmaf(-lr_wd, wh, wh));
+    }
+  }
+}
+
+// Stochastic rounding (Sec. 3.4) of 16 consecutive weights to codes of the new grid.  h holds the 16-bit
+// uniforms of the 16 columns, two per word.  FAST: floor(t) + [frac(t) * 65536 > h] + z equals
+// ceil(t - h / 65536) + z; it is formed as one add in round-up mode onto (2^23 * 1.5 + z), which leaves
+// the code in the low byte.  The subtraction t - h / 65536 rounds by at most 2^-14 for |t| < 2^10, so a
+// decision can differ from the exact one only within that distance of the rounding boundary.
+template <bool FAST>
+__device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& gp, const uint32_t h[8]) {
+  uint32_t bits[16];
+  const float mz = (kMagic + 128.0f) + gp.z;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float t = __fmul_rn(w[j], gp.inv);
+    if (FAST) {
+      // 128 + h / 65536: h dropped into the mantissa of 2^7
+      const float hv = __uint_as_float(__byte_perm(h[j >> 1], 0x43000000u, (j & 1) ? 0x7632 : 0x7610));
+      float y = __fadd_ru(__fsub_rn(t, hv), mz);
+      y = fminf(fmaxf(y, kMagic - 128.0f), kMagic + 127.0f);
+      bits[j] = __float_as_uint(y);
+    } else {
+      const float hf = (float)((h[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
+      const float f = floorf(t);
+      const float up = (__fmul_rn(__fsub_rn(t, f), 65536.0f) > hf) ? 1.0f : 0.0f;
+      const float qv = fminf(fmaxf(__fadd_rn(__fadd_rn(f, up), gp.z), -128.0f), 127.0f);
+      bits[j] = (uint32_t)(int)qv;
+    }
+  }
+  uint32_t o[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t lo = __byte_perm(bits[4 * k], bits[4 * k + 1], 0x0040);
+    const uint32_t hi = __byte_perm(bits[4 * k + 2], bits[4 * k + 3], 0x0040);
+    o[k] = __byte_perm(lo, hi, 0x5410);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 template <bool SINGLE>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(K2Smem::kThreads, 1)
 backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table, int nprob,
-                      int total_tiles, int32_t* __restrict__ status) {
+                      int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
   using S = K2Smem;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -351,13 +422,14 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
   uint64_t* code_full = acc_empty + 2;
   uint64_t* code_empty = code_full + S::kCodeBufs;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(code_empty + S::kCodeBufs);
+  float2* part = reinterpret_cast<float2*>(smem + S::kPartOffset);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const TcProblem* probs = SINGLE ? &single : table;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S::kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], S::kEpiWarps); }
     for (int i = 0; i < S::kCodeBufs; ++i) { mbar_init(&code_full[i], 1); mbar_init(&code_empty[i], 1); }
     fence_mbar_init();
     fence_proxy_async_smem();
@@ -386,14 +458,17 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
         const TcProblem* p = locate(tile, pi);
-        const int local = tile - p->k2_tile0;
-        const int m0 = (local % p->k2_mblocks) * kTileM, n0 = (local / p->k2_mblocks) * S::kBN;
+        const int local = tile - p->k2_tile0, mblocks = p->k2_mblocks;
+        const int m0 = (local % mblocks) * kTileM, n0 = (local / mblocks) * S::kBN;
+        const CUtensorMap* mapW = &p->mapW;
+        const CUtensorMap* mapP = &p->mapP;
+        const CUtensorMap* mapN = &p->mapN;
         const int cb = tcount % S::kCodeBufs;
         if (!mbar_wait(&code_empty[cb], ((tcount / S::kCodeBufs) & 1) ^ 1)) { ok = false; break; }
         uint8_t* cbuf = code_base + cb * S::kCodeBytes;
         mbar_arrive_expect_tx(&code_full[cb], S::kCodeBytes);
-        tma_load_2d(cbuf, &p->mapW, &code_full[cb], n0, m0);
-        tma_load_2d(cbuf + S::kCodeBytes / 2, &p->mapW, &code_full[cb], n0 + 128, m0);
+        tma_load_2d(cbuf, mapW, &code_full[cb], n0, m0);
+        tma_load_2d(cbuf + S::kCodeBytes / 2, mapW, &code_full[cb], n0 + 128, m0);
         const int kblocks = (p->r + kBK - 1) / kBK;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % S::kStages;
@@ -402,9 +477,9 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
           uint8_t* sB = sA + S::kABytes;
           mbar_arrive_expect_tx(&full[s], S::kStageBytes);
 #pragma unroll
-          for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, &p->mapP, &full[s], kb * kBK, m0 + 64 * h);
+          for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], kb * kBK, m0 + 64 * h);
 #pragma unroll
-          for (int h = 0; h < 4; ++h) tma_load_2d(sB + h * kBoxBytes, &p->mapN, &full[s], n0 + 64 * h, kb * kBK);
+          for (int h = 0; h < 4; ++h) tma_load_2d(sB + h * kBoxBytes, mapN, &full[s], n0 + 64 * h, kb * kBK);
         }
       }
       if (!ok) raise_wait_expired(status);
@@ -444,108 +519,120 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       if (!ok) raise_wait_expired(status);
     }
   } else {
-    // ------------------------------------------------------------------ epilogue: one thread = one row = one group
-    const int q = warp & 3;
+    // ------------------------------------------------------------------ epilogue
+    // Sixteen warps: warp (quarter q, slice sl) owns accumulator rows 32q..32q+31 and columns
+    // 64*sl..64*sl+63; a row of the tile is one quantization group, so four threads share a group and
+    // combine their minima and maxima through shared memory.  The 64 pre-rounding weights of a thread
+    // stay in registers between the two passes.
+    const int q = warp & 3, sl = (warp - 2) >> 2;
     const int row = q * 32 + lane;
     const bool elected = (threadIdx.x == 64);
+    const bool no_wd = (sc.lr_wd == 0.0f);
     int pi = 0;
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
       const TcProblem* p = locate(tile, pi);
-      const int local = tile - p->k2_tile0;
-      const int m0 = (local % p->k2_mblocks) * kTileM, nblk = local / p->k2_mblocks, n0 = nblk * S::kBN;
+      const int local = tile - p->k2_tile0, mblocks = p->k2_mblocks;
+      const int m0 = (local % mblocks) * kTileM, nblk = local / mblocks, n0 = nblk * S::kBN;
+      const int pn = p->n, n_tma = p->n_tma_w, ngroups = p->ngroups;
       const int gi = m0 + row;                       // global row
       const bool row_ok = gi < p->m;
-      const int ncols = min(S::kBN, p->n - n0);      // valid columns of this (possibly ragged) group
-      const StepScalars sc = p->sc;
+      const int ncols = min(S::kBN, pn - n0);        // valid columns of this (possibly ragged) group
+      const int64_t ldw = p->ldw;
+      float* g_scale = p->w_scales + (int64_t)gi * ngroups + nblk;
+      float* g_zero = p->w_zeros + (int64_t)gi * ngroups + nblk;
+      int8_t* g_codes = p->w_codes + (int64_t)gi * ldw;
+      float* dbgW = p->dbgW ? p->dbgW + (int64_t)gi * ldw : nullptr;
+      const CUtensorMap* mapWst = &p->mapWst;
+      const uint32_t seed_lo = p->seed_lo, seed_hi = p->seed_hi;
       float s_old = 1.f, z_old = 0.f;
-      if (row_ok) {
-        s_old = __ldg(p->w_scales + (int64_t)gi * p->ngroups + nblk);
-        z_old = __ldg(p->w_zeros + (int64_t)gi * p->ngroups + nblk);
-      }
+      if (row_ok) { s_old = __ldg(g_scale); z_old = __ldg(g_zero); }
       const uint32_t ab = tcount & 1;
       const int cb = tcount % S::kCodeBufs;
       ok = mbar_wait(&code_full[cb], (tcount / S::kCodeBufs) & 1) && mbar_wait(&acc_full[ab], (tcount >> 1) & 1);
-      ok = named_bar_and(1, 128, ok);
+      ok = named_bar_and(1, S::kEpiThreads, ok);
       if (!ok) break;
       tc_fence_after_sync();
       uint8_t* cbuf = code_base + cb * S::kCodeBytes;
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + ab * S::kBN;
-      // codes of column 16*k16 .. +15 of this row: box (k16 / 8), 16-byte chunk (k16 % 8) ^ (row % 8)
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + ab * S::kBN + sl * 64;
+      // codes of columns 16*k16 .. +15 of this row: box (k16 / 8), 16-byte chunk (k16 % 8) ^ (row % 8)
       auto code_ptr = [&](int k16) -> uint4* {
         return reinterpret_cast<uint4*>(cbuf + (k16 >> 3) * (S::kCodeBytes / 2) + row * 128 + (((k16 & 7) ^ (row & 7)) << 4));
       };
 
-      // ---- pass 1: group minimum and maximum of W'
-      float mn = INFINITY, mx = -INFINITY;
-      for (int c = 0; c < S::kBN / kChunk; ++c) {
+      // ---- pass 1: W' of the thread's 64 columns, minimum and maximum
+      float w[64];
+      const bool fast_dq = __all_sync(0xFFFFFFFFu, fabsf(z_old) <= 4.0e6f);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
         uint32_t acc[32];
-        tmem_ld_32x32(tacc + c * kChunk, acc);
+        tmem_ld_32x32(tacc + half * kChunk, acc);
         tmem_ld_wait();
 #pragma unroll
-        for (int hlf = 0; hlf < 2; ++hlf) {
-          const uint4 cw = *code_ptr(2 * c + hlf);
-          const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float qf = (float)(int8_t)((w4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
-            const float w = weight_pre(qf, z_old, s_old, __uint_as_float(acc[16 * hlf + e]), sc);
-            if (c * kChunk + 16 * hlf + e < ncols) { mn = fminf(mn, w); mx = fmaxf(mx, w); }
-          }
+        for (int k = 0; k < 2; ++k) {
+          const uint4 cw = *code_ptr(sl * 4 + half * 2 + k);
+          float* wk = w + half * 32 + k * 16;
+          const float lr_wd = no_wd ? 0.0f : sc.lr_wd;
+          if (fast_dq) weights16<true>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, lr_wd, wk);
+          else weights16<false>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, lr_wd, wk);
         }
       }
-      const GroupParams gp = group_params<8>(mn, mx);
-      if (row_ok) {
-        p->w_scales[(int64_t)gi * p->ngroups + nblk] = gp.s;
-        p->w_zeros[(int64_t)gi * p->ngroups + nblk] = gp.z;
-      }
-
-      // ---- pass 2: stochastic rounding to the new grid, codes written back in place
-      for (int c = 0; c < S::kBN / kChunk; ++c) {
-        uint32_t acc[32];
-        tmem_ld_32x32(tacc + c * kChunk, acc);
-        tmem_ld_wait();
-#pragma unroll
-        for (int hlf = 0; hlf < 2; ++hlf) {
-          uint4* cp = code_ptr(2 * c + hlf);
-          const uint4 cw = *cp;
-          const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
-          uint32_t o4[4] = {0, 0, 0, 0};
-#pragma unroll
-          for (int e8 = 0; e8 < 2; ++e8) {
-            float h[8];
-            sr_lanes8(sc, (uint32_t)gi, (uint32_t)((n0 + c * kChunk + 16 * hlf + 8 * e8) >> 3), h);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int ee = 8 * e8 + e;
-              const float qf = (float)(int8_t)((w4[ee >> 2] >> (8 * (ee & 3))) & 0xFFu);
-              const float w = weight_pre(qf, z_old, s_old, __uint_as_float(acc[16 * hlf + ee]), sc);
-              const int code = (int)sr_code(w, gp, h[e]);
-              o4[ee >> 2] |= (uint32_t)(code & 0xFF) << (8 * (ee & 3));
-              if (p->dbgW && row_ok && (n0 + c * kChunk + 16 * hlf + ee) < p->n)
-                p->dbgW[(int64_t)gi * p->ldw + n0 + c * kChunk + 16 * hlf + ee] = w;
-            }
-          }
-          *cp = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-          if (n0 + c * kChunk + 16 * hlf == p->n_tma_w && row_ok) {          // ragged tail: at most 15 columns
-            int8_t* out = p->w_codes + (int64_t)gi * p->ldw + p->n_tma_w;
-#pragma unroll
-            for (int e = 0; e < 15; ++e)
-              if (e < p->n - p->n_tma_w) out[e] = (int8_t)((o4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
-          }
-        }
-      }
-      tc_fence_before_sync();
+      tc_fence_before_sync();                       // the accumulator buffer can be refilled
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[ab]);
 
+      float mn = INFINITY, mx = -INFINITY;
+      const int myc0 = sl * 64;
+      if (myc0 + 64 <= ncols) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (myc0 + i < ncols) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
+      }
+      part[sl * kTileM + row] = make_float2(mn, mx);
+      named_bar_sync(1, S::kEpiThreads);
+#pragma unroll
+      for (int o = 0; o < 4; ++o) {
+        const float2 pm = part[o * kTileM + row];
+        mn = fminf(mn, pm.x);
+        mx = fmaxf(mx, pm.y);
+      }
+      const GroupParams gp = group_params<8>(mn, mx);
+      if (row_ok && sl == 0) { *g_scale = gp.s; *g_zero = gp.z; }
+
+      // ---- pass 2: stochastic rounding to the new grid, codes written over the old ones in shared memory
+      const bool fast_sr = __all_sync(0xFFFFFFFFu, fabsf(gp.z) <= 1024.0f);
+#pragma unroll
+      for (int k16 = 0; k16 < 4; ++k16) {
+        const int col = n0 + myc0 + 16 * k16;
+        const uint4 x0 = philox4x32_10(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi),
+                                       make_uint2(seed_lo, seed_hi));
+        const uint4 x1 = philox4x32_10(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi),
+                                       make_uint2(seed_lo, seed_hi));
+        const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+        const uint4 out = fast_sr ? sr_codes16<true>(w + 16 * k16, gp, h) : sr_codes16<false>(w + 16 * k16, gp, h);
+        *code_ptr(sl * 4 + k16) = out;
+        if (row_ok && (col == n_tma || dbgW != nullptr)) {   // ragged tail (at most 15 columns), test tap
+          const uint32_t o4[4] = {out.x, out.y, out.z, out.w};
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            if (col + e < pn) {
+              if (col == n_tma) g_codes[col + e] = (int8_t)((o4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
+              if (dbgW) dbgW[col + e] = w[16 * k16 + e];
+            }
+          }
+        }
+      }
+
       // ---- coalesced write-back of the tile's codes
       fence_proxy_async_smem();
-      named_bar_sync(1, 128);
+      named_bar_sync(1, S::kEpiThreads);
       if (elected) {
-        if (n0 < p->n_tma_w) tma_store_2d(&p->mapWst, cbuf, n0, m0);
-        if (n0 + 128 < p->n_tma_w) tma_store_2d(&p->mapWst, cbuf + S::kCodeBytes / 2, n0 + 128, m0);
+        if (n0 < n_tma) tma_store_2d(mapWst, cbuf, n0, m0);
+        if (n0 + 128 < n_tma) tma_store_2d(mapWst, cbuf + S::kCodeBytes / 2, n0 + 128, m0);
         tma_commit_group();
         tma_wait_group_read<0>();
         mbar_arrive(&code_empty[cb]);
@@ -597,23 +684,26 @@ bool make_map(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const vo
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-struct TcWorkspace {
+// Scratch of one matrix: P~ (bf16, m x r, pitch r) then N_b (bf16, r x ldn).
+struct TcScratch {
   uint16_t* Pt;
   uint16_t* Nb;
   int64_t ldn;
 };
 
-TcWorkspace carve(const StepArgs& a) {
-  TcWorkspace w;
-  w.Pt = reinterpret_cast<uint16_t*>(a.ws);
-  w.Nb = reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(a.ws) + round_up(a.m * a.r * 2, 1024));
-  w.ldn = round_up(a.n, 64);
+size_t scratch_pt_bytes(int64_t m, int64_t r) { return (size_t)round_up(m * r * 2, 1024); }
+size_t scratch_nb_bytes(int64_t n, int64_t r) { return (size_t)round_up(r * round_up(n, 64) * 2, 1024); }
+
+TcScratch carve(void* base, int64_t m, int64_t n, int64_t r) {
+  TcScratch w;
+  w.Pt = reinterpret_cast<uint16_t*>(base);
+  w.Nb = reinterpret_cast<uint16_t*>(reinterpret_cast<char*>(base) + scratch_pt_bytes(m, r));
+  w.ldn = round_up(n, 64);
   return w;
 }
 
-int fill_problem(const StepArgs& a, TcProblem* p, int bn) {
+int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   memset(p, 0, sizeof(*p));
-  const TcWorkspace w = carve(a);
   bool ok = true;
   ok &= make_map(&p->mapP, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, a.m, a.r, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapG, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.G, a.n, a.m, a.ldg, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
@@ -633,20 +723,20 @@ int fill_problem(const StepArgs& a, TcProblem* p, int bn) {
                  CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapWst, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, n16 > 0 ? n16 : 16, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
-  p->n_tma_mv = (int32_t)n4;
-  p->n_tma_w = (int32_t)n16;
-  p->M = a.M; p->V = a.V; p->w_codes = reinterpret_cast<int8_t*>(a.W.codes);
   if (!ok) {
     note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
     return QG_CUDA_ERROR;
   }
-  p->sc = a.sc;
+  p->n_tma_mv = (int32_t)n4;
+  p->n_tma_w = (int32_t)n16;
+  p->M = a.M; p->V = a.V; p->w_codes = reinterpret_cast<int8_t*>(a.W.codes);
   p->w_scales = a.W.scales;
   p->w_zeros = a.W.zeros;
   p->dbgR = a.dbg.R; p->dbgN = a.dbg.N; p->dbgW = a.dbg.W_pre;
   p->ldmv = a.ldmv; p->ldw = a.W.ld;
   p->m = (int32_t)a.m; p->n = (int32_t)a.n; p->r = (int32_t)a.r;
   p->ngroups = (int32_t)ceil_div(a.n, kGroup);
+  p->seed_lo = a.sc.seed_lo; p->seed_hi = a.sc.seed_hi;
   p->k1_rblocks = (int32_t)ceil_div(a.r, kTileM);
   p->k1_tiles = p->k1_rblocks * (int32_t)ceil_div(a.n, bn);
   p->k2_mblocks = (int32_t)ceil_div(a.m, kTileM);
@@ -669,38 +759,183 @@ int set_smem(K kernel, int bytes) {
   return QG_OK;
 }
 
-}  // namespace
+// The projection's column-tile width: 256 halves the operand traffic per flop of the 128-wide tile,
+// but only pays once there are enough tiles to occupy every SM.
+int choose_bn(int64_t tiles_at_256) { return tiles_at_256 >= 2 * (int64_t)sm_count() ? 256 : 128; }
 
-size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r) {
-  return (size_t)round_up(m * r * 2, 1024) + (size_t)round_up(r * round_up(n, 64) * 2, 1024);
-}
-
-int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
-  const TcWorkspace w = carve(a);
-  int rc = launch_dequant_p(a.P, w.Pt, a.r, st);
-  if (rc != QG_OK) return rc;
-  TcProblem prob;
-  constexpr int BN = 128;
-  rc = fill_problem(a, &prob, BN);
+template <int BN, bool SINGLE>
+int launch_k1(const TcProblem* single, const TcProblem* table, int nprob, int total_tiles, const StepScalars& sc,
+              int32_t* status, cudaStream_t st) {
+  auto kern = project_adam_kernel<BN, SINGLE>;
+  int rc = set_smem(kern, K1Smem<BN>::kBytes);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
-  {
-    auto kern = project_adam_kernel<BN, true>;
-    rc = set_smem(kern, K1Smem<BN>::kBytes);
-    if (rc != QG_OK) return rc;
-    const int grid = prob.k1_tiles < sms ? prob.k1_tiles : sms;
-    kern<<<grid, 224, K1Smem<BN>::kBytes, st>>>(prob, nullptr, 1, prob.k1_tiles, a.status);
-    QG_LAUNCH_CHECK();
+  const int grid = total_tiles < sms ? total_tiles : sms;
+  static const TcProblem dummy{};
+  kern<<<grid, 224, K1Smem<BN>::kBytes, st>>>(single ? *single : dummy, table, nprob, total_tiles, sc, status);
+  QG_LAUNCH_CHECK();
+  return QG_OK;
+}
+
+template <bool SINGLE>
+int launch_k2(const TcProblem* single, const TcProblem* table, int nprob, int total_tiles, const StepScalars& sc,
+              int32_t* status, cudaStream_t st) {
+  auto kern = backproject_sr_kernel<SINGLE>;
+  int rc = set_smem(kern, K2Smem::kBytes);
+  if (rc != QG_OK) return rc;
+  const int sms = sm_count();
+  const int grid = total_tiles < sms ? total_tiles : sms;
+  static const TcProblem dummy{};
+  kern<<<grid, K2Smem::kThreads, K2Smem::kBytes, st>>>(single ? *single : dummy, table, nprob, total_tiles, sc, status);
+  QG_LAUNCH_CHECK();
+  return QG_OK;
+}
+
+// ---- P~ = bf16(dequant(P)) for a list of matrices in one launch
+struct DequantItem {
+  qg_qtensor P;
+  uint16_t* out;
+  int32_t block0, nblocks;   // blocks of 256 threads, eight columns per thread
+};
+
+__global__ void __launch_bounds__(256)
+dequant_p_grouped_kernel(const DequantItem* __restrict__ items, int nitems) {
+  int lo = 0, hi = nitems - 1;
+  while (lo < hi) {                                  // last item whose block0 <= blockIdx.x
+    const int mid = (lo + hi + 1) >> 1;
+    if (items[mid].block0 <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
   }
-  {
-    auto kern = backproject_sr_kernel<true>;
-    rc = set_smem(kern, K2Smem::kBytes);
-    if (rc != QG_OK) return rc;
-    const int grid = prob.k2_tiles < sms ? prob.k2_tiles : sms;
-    kern<<<grid, 192, K2Smem::kBytes, st>>>(prob, nullptr, 1, prob.k2_tiles, a.status);
+  const DequantItem& it = items[lo];
+  const qg_qtensor& P = it.P;
+  const int ngroups = (int)((P.cols + kGroup - 1) / kGroup);
+  const int64_t chunks = P.cols / 8;
+  const int64_t idx = (int64_t)(blockIdx.x - it.block0) * blockDim.x + threadIdx.x;
+  if (idx >= P.rows * chunks) return;
+  const int64_t row = idx / chunks, c0 = (idx % chunks) * 8;
+  const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)P.codes + row * (P.ld / 2) + (c0 >> 1)));
+  const int g = (int)(c0 / kGroup);
+  const float s = __ldg(P.scales + row * ngroups + g), z = __ldg(P.zeros + row * ngroups + g);
+  float qv[8], v[8];
+  unpack_int4x8(w, qv);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(__fsub_rn(qv[i], z), s);
+  *reinterpret_cast<uint4*>(it.out + row * P.cols + c0) = pack_bf16x8(v);
+}
+
+}  // namespace
+
+size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r) { return scratch_pt_bytes(m, r) + scratch_nb_bytes(n, r); }
+
+int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
+  const TcScratch w = carve(a.ws, a.m, a.n, a.r);
+  int rc = launch_dequant_p(a.P, w.Pt, a.r, st);
+  if (rc != QG_OK) return rc;
+  const int bn = choose_bn(ceil_div(a.r, kTileM) * ceil_div(a.n, 256));
+  TcProblem prob;
+  rc = fill_problem(a, w, &prob, bn);
+  if (rc != QG_OK) return rc;
+  rc = bn == 256 ? launch_k1<256, true>(&prob, nullptr, 1, prob.k1_tiles, a.sc, a.status, st)
+                 : launch_k1<128, true>(&prob, nullptr, 1, prob.k1_tiles, a.sc, a.status, st);
+  if (rc != QG_OK) return rc;
+  return launch_k2<true>(&prob, nullptr, 1, prob.k2_tiles, a.sc, a.status, st);
+}
+
+// ============================================================================================
+// plans: a fixed list of matrices prepared once (tensor maps, tile tables) and stepped many times
+// ============================================================================================
+struct PlanChunk {
+  int first, count;          // items [first, first + count)
+  int k1_tiles, k2_tiles, bn;
+  int dq_blocks;
+};
+
+struct Plan {
+  std::vector<PlanChunk> chunks;
+  TcProblem* table_dev = nullptr;
+  DequantItem* dq_dev = nullptr;
+  int count = 0;
+};
+
+// Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b
+// fit both the caller's workspace and a budget chosen so that N_b, written by the first kernel, is
+// still in the 126 MB L2 when the second kernel reads it.
+constexpr size_t kChunkBudget = 56ull << 20;
+
+size_t plan_table_bytes(int32_t count) {
+  return (size_t)count * (sizeof(TcProblem) + round_up(sizeof(DequantItem), 64)) + 256;
+}
+
+int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t table_bytes, void* workspace,
+                size_t workspace_bytes, Plan** out) {
+  if (table_bytes < plan_table_bytes(count)) return QG_WORKSPACE_TOO_SMALL;
+  std::vector<TcProblem> probs((size_t)count);
+  std::vector<DequantItem> dq((size_t)count);
+  Plan* plan = new Plan();
+  plan->count = count;
+  const size_t budget = workspace_bytes < kChunkBudget ? workspace_bytes : kChunkBudget;
+  int i = 0;
+  while (i < count) {
+    // extent of the chunk
+    size_t used = 0;
+    int j = i;
+    int64_t tiles256 = 0;
+    while (j < count) {
+      const size_t need = tc_workspace_bytes(items[j].m, items[j].n, items[j].r);
+      if (need > workspace_bytes) { delete plan; return QG_WORKSPACE_TOO_SMALL; }
+      if (j > i && used + need > budget) break;
+      used += need;
+      tiles256 += ceil_div(items[j].r, kTileM) * ceil_div(items[j].n, 256);
+      ++j;
+    }
+    PlanChunk ch{};
+    ch.first = i; ch.count = j - i;
+    ch.bn = choose_bn(tiles256);
+    size_t off = 0;
+    for (int k = i; k < j; ++k) {
+      const StepArgs& a = items[k];
+      const TcScratch w = carve(reinterpret_cast<char*>(workspace) + off, a.m, a.n, a.r);
+      off += tc_workspace_bytes(a.m, a.n, a.r);
+      const int rc = fill_problem(a, w, &probs[k], ch.bn);
+      if (rc != QG_OK) { delete plan; return rc; }
+      probs[k].k1_tile0 = ch.k1_tiles; ch.k1_tiles += probs[k].k1_tiles;
+      probs[k].k2_tile0 = ch.k2_tiles; ch.k2_tiles += probs[k].k2_tiles;
+      dq[k].P = a.P; dq[k].out = w.Pt;
+      dq[k].block0 = ch.dq_blocks;
+      dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 8), 256);
+      ch.dq_blocks += dq[k].nblocks;
+    }
+    plan->chunks.push_back(ch);
+    i = j;
+  }
+  plan->table_dev = reinterpret_cast<TcProblem*>(table_dev);
+  plan->dq_dev = reinterpret_cast<DequantItem*>(reinterpret_cast<char*>(table_dev) +
+                                                round_up((int64_t)count * sizeof(TcProblem), 256));
+  cudaError_t e = cudaMemcpy(plan->table_dev, probs.data(), (size_t)count * sizeof(TcProblem), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(plan->dq_dev, dq.data(), (size_t)count * sizeof(DequantItem), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    note_cuda_error(e, "cudaMemcpy(plan table)");
+    delete plan;
+    return QG_CUDA_ERROR;
+  }
+  *out = plan;
+  return QG_OK;
+}
+
+int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st) {
+  for (const PlanChunk& ch : plan->chunks) {
+    dequant_p_grouped_kernel<<<ch.dq_blocks, 256, 0, st>>>(plan->dq_dev + ch.first, ch.count);
     QG_LAUNCH_CHECK();
+    const TcProblem* tab = plan->table_dev + ch.first;
+    int rc = ch.bn == 256 ? launch_k1<256, false>(nullptr, tab, ch.count, ch.k1_tiles, sc, status, st)
+                          : launch_k1<128, false>(nullptr, tab, ch.count, ch.k1_tiles, sc, status, st);
+    if (rc != QG_OK) return rc;
+    rc = launch_k2<false>(nullptr, tab, ch.count, ch.k2_tiles, sc, status, st);
+    if (rc != QG_OK) return rc;
   }
   return QG_OK;
 }
+
+void plan_destroy(Plan* plan) { delete plan; }
 
 }  // namespace qg

@@ -138,3 +138,75 @@ def test_step_is_deterministic_and_seeded():
         outs.append(dW.codes.cpu().numpy().copy())
     assert np.array_equal(outs[0], outs[1])           # counter-based randomness: same (seed, step) -> same codes
     assert not np.array_equal(outs[0], outs[2])
+
+
+# ----------------------------------------------------------------------------- plans (grouped launches)
+def _plan_items(shapes, seed=0, steps_before=1):
+    """Host-side state of a few matrices after ``steps_before`` oracle steps, as (gm, P, W, M, V, sr_seed)."""
+    out = []
+    for idx, (m, n, r) in enumerate(shapes):
+        gm = synth.GradientModel(m, n, seed=seed, matrix_index=idx)
+        P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=seed, stream=idx), 4)
+        W = O.quantize_rtn(synth.initial_weight(m, n, seed, idx), 8)
+        M = np.zeros((r, n), np.float32)
+        V = np.zeros((r, n), np.float32)
+        sr = synth.matrix_seed(seed, idx)
+        for t in range(1, steps_before + 1):
+            o = O.project_step(gm.sample(t), P, W, M, V, O.Hyper(step=t, seed=sr))
+            W, M, V = o["W"], o["M"], o["V"]
+        out.append((gm, P, W, M, V, sr))
+    return out
+
+
+@pytest.mark.parametrize("workspace_bytes", [None, 0])
+def test_plan_step_equals_single_matrix_calls(workspace_bytes):
+    # a plan over ragged and regular shapes gives bit for bit what qgalore_project_step gives per matrix
+    shapes = [(256, 512, 64), (300, 777, 96), (512, 1376, 128), (128, 85, 32), (768, 768, 256), (1024, 2736, 256)]
+    state = _plan_items(shapes, seed=2, steps_before=1)
+    step = 2
+    single, items = [], []
+    for (gm, P, W, M, V, sr) in state:
+        gb = gm.sample(step)
+        dG, dP = g_to_device(gb), to_device_q(P)
+        dW1, dM1, dV1 = to_device_q(W), f32_to_device(M), f32_to_device(V)
+        B.project_step(dG, dP, dW1, dM1, dV1, B.Hyper(step=step, seed=sr))
+        single.append((dW1, dM1, dV1))
+        items.append({"G": dG, "P": dP, "W": to_device_q(W), "M": f32_to_device(M), "V": f32_to_device(V), "seed": sr})
+    if workspace_bytes == 0:     # the minimum: one matrix per chunk
+        workspace_bytes = max(B.workspace_bytes(B.QG_OP_PROJECT_STEP, m, n, r) for (m, n, r) in shapes)
+    plan = B.StepPlan(items, workspace_bytes=workspace_bytes)
+    plan.step(B.Hyper(step=step))
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0
+    for (dW1, dM1, dV1), it in zip(single, items):
+        assert torch.equal(dW1.codes, it["W"].codes)
+        assert torch.equal(dW1.scales, it["W"].scales) and torch.equal(dW1.zeros, it["W"].zeros)
+        assert torch.equal(dM1._base, it["M"]._base) and torch.equal(dV1._base, it["V"]._base)
+    plan.close()
+
+
+def test_plan_free_run_tracks_oracle_moments():
+    # three free-running steps of a small stack: M and V do not depend on W, so they stay on the oracle's trajectory
+    shapes = [(256, 512, 64), (512, 1376, 128)]
+    state = _plan_items(shapes, seed=5, steps_before=0)
+    items = [{"G": g_to_device(gm.sample(1)), "P": to_device_q(P), "W": to_device_q(W), "M": f32_to_device(M),
+              "V": f32_to_device(V), "seed": sr} for (gm, P, W, M, V, sr) in state]
+    plan = B.StepPlan(items)
+    ref = [(W, M, V) for (_, _, W, M, V, _) in state]
+    for t in (1, 2, 3):
+        for k, (gm, P, _, _, _, sr) in enumerate(state):
+            gb = gm.sample(t)
+            items[k]["G"].copy_(torch.from_numpy(gb.view(np.int16)).cuda())
+            o = O.project_step(gb, P, ref[k][0], ref[k][1], ref[k][2], O.Hyper(step=t, seed=sr))
+            ref[k] = (o["W"], o["M"], o["V"])
+        plan.step(B.Hyper(step=t))
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0
+    for k in range(len(state)):
+        m_gpu, v_gpu = items[k]["M"].cpu().numpy(), items[k]["V"].cpu().numpy()
+        assert np.linalg.norm(m_gpu - ref[k][1]) <= MOMENT_TOL * np.linalg.norm(ref[k][1])
+        assert np.linalg.norm(v_gpu - ref[k][2]) <= MOMENT_TOL * np.linalg.norm(ref[k][2])
+        # weights: free-running trajectories differ by re-rolled roundings, but stay within a few levels
+        w_gpu, w_ref = O.dequantize(from_device_q(items[k]["W"])), O.dequantize(ref[k][0])
+        lsb = float(ref[k][0].scales.max())
+        assert np.abs(w_gpu - w_ref).max() <= 4 * lsb
