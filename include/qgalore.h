@@ -202,6 +202,10 @@ QG_API uint64_t qgalore_launch_count(void);
  * product path), 1 the plain CUDA-core kernels kept to cross-check them.  Not thread safe. */
 QG_API int qgalore_debug_set_step_impl(int impl);
 
+/* Diagnostic: writes one text line per tensor-core kernel (registers per thread, thread limit, shared
+ * memory) as the CUDA runtime reports them for the current device into buf (HOST, NUL-terminated). */
+QG_API int qgalore_debug_kernel_info(char* buf, size_t capacity);
+
 #ifdef __cplusplus
 }
 #endif

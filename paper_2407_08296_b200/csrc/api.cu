@@ -33,6 +33,7 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
                 size_t workspace_bytes, Plan** out);
 int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st);
 void plan_destroy(Plan* plan);
+int tc_kernel_info(char* buf, size_t cap);
 
 static int g_step_impl = 0;  // 0: tensor-core kernels; 1: CUDA-core kernels (validation aid)
 
@@ -277,6 +278,12 @@ int qgalore_gate_update(float sim, float threshold, int32_t k, int32_t* interval
   *interval *= 2;
   *count = 0;
   return 1;
+}
+
+int qgalore_debug_kernel_info(char* buf, size_t capacity) {
+  if (!buf || capacity < 2) return QG_INVALID_ARGUMENT;
+  buf[0] = 0;
+  return tc_kernel_info(buf, capacity);
 }
 
 /* Test aid: selects the CUDA-core (1) or the tensor-core (0) kernels of qgalore_project_step. */

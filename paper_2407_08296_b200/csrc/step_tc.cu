@@ -19,6 +19,7 @@
 //
 // Every barrier wait is bounded; on expiry the kernel raises QG_DEV_WAIT_EXPIRED in the status word,
 // stops taking tiles, releases its tensor memory and returns.
+#include <cstdio>
 #include <cstring>
 #include <vector>
 
@@ -40,15 +41,14 @@ constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
 //   mapP    P~  bf16 [m][r]       box 64 x 64, swizzle 128   A operand of both kernels
 //   mapG    G   bf16 [m][ldg]     box 64 x 64, swizzle 128   B operand of the projection
 //   mapN    N_b bf16 [r][ldn]     box 64 x 64, swizzle 128   B operand of the back-projection
-//   mapNst  N_b bf16 [r][ldn]     box 32 x 128, swizzle 64   store from the Adam epilogue
-//   mapM/V  fp32 [r][ldmv]        box 32 x 128, swizzle 128  load of the Adam epilogue
 //   mapW    int8 [m][ldw]         box 128 x 128, swizzle 128 load of the requantizing epilogue
-//   mapMst/Vst/Wst                the same tensors for the stores, with the inner extent rounded DOWN to
-//                                 16 bytes: a TMA store clips at 16-byte granularity, so it would spill into
+//   mapWst                        the same tensor for the store, with the inner extent rounded DOWN to 16
+//                                 bytes: a TMA store clips at 16-byte granularity, so it would spill into
 //                                 the row padding of a ragged matrix; the few tail columns are written with
-//                                 plain stores instead (n_tma_mv / n_tma_w = columns the TMA stores cover).
+//                                 plain stores instead (n_tma_w = columns the TMA store covers).
+// M, V and N_b are read and written by the Adam epilogue with plain vector accesses.
 struct alignas(64) TcProblem {
-  CUtensorMap mapP, mapG, mapN, mapNst, mapM, mapV, mapW, mapMst, mapVst, mapWst;
+  CUtensorMap mapP, mapG, mapN, mapW, mapWst;
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -57,8 +57,9 @@ struct alignas(64) TcProblem {
   float* M;
   float* V;
   int8_t* w_codes;
-  int64_t ldmv, ldw;
-  int32_t m, n, r, ngroups, n_tma_mv, n_tma_w;
+  uint16_t* nb;                        // N_b, bf16 r x ldn (scratch)
+  int64_t ldmv, ldw, ldn;
+  int32_t m, n, r, ngroups, n_tma_w;
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles, k1_tile0;
   int32_t k2_mblocks, k2_tiles, k2_tile0;
@@ -80,43 +81,50 @@ __device__ __forceinline__ float sqrt_approx(float x) {
 // ============================================================================================
 template <int BN>
 struct K1Smem {
-  static constexpr int kStages = 3;
   static constexpr int kABytes = 2 * kBoxBytes;            // 128 (r) x 64 (m) bf16
   static constexpr int kBBytes = (BN / 64) * kBoxBytes;    // BN (n) x 64 (m) bf16
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kMvBufs = BN >= 256 ? 2 : 3;
-  static constexpr int kMBytes = kTileM * kChunk * 4;      // 16 KB
-  static constexpr int kNBytes = kTileM * kChunk * 2;      // 8 KB
-  static constexpr int kMvBufBytes = 2 * kMBytes + kNBytes;
-  static constexpr int kBarOffset = kStages * kStageBytes + kMvBufs * kMvBufBytes;
+  static constexpr int kStages = (192 * 1024) / kStageBytes;
+  static constexpr int kBarOffset = kStages * kStageBytes;
   static constexpr int kBytes = kBarOffset + 256 + 1024;   // barriers + slack for 1024-byte alignment
+  static constexpr int kEpiWarps = 8;                      // 4 lane quarters x 2 halves of 16 lanes
+  static constexpr int kThreads = 64 + kEpiWarps * 32;
 };
 
+// The Adam update of Sec. 3.5 on one element: M <- b1 M + (1-b1) R, V <- b2 V + (1-b2) R^2,
+// N = (M / (1 - b1^t)) / (sqrt(V / (1 - b2^t)) + eps)   (Kingma & Ba; eps outside the root).
+__device__ __forceinline__ float adam1(const StepScalars& sc, float inv_b1, float inv_b2, float r, float& m, float& v) {
+  m = fmaf(sc.beta1, m, sc.one_minus_beta1 * r);
+  v = fmaf(sc.beta2, v, sc.one_minus_beta2 * r * r);
+  return __fdividef(m * inv_b1, sqrt_approx(v * inv_b2) + sc.eps);
+}
+
+// The epilogue reads the accumulator in the 16-lane x 256-bit shape: thread t holds, per group of
+// eight columns, the column pair 2(t%4), 2(t%4)+1 of rows t/4 and t/4 + 8.  A quad of threads therefore
+// covers 32 contiguous bytes of a row of M, V (fp32): every global access of the epilogue moves whole
+// 32-byte sectors without staging through shared memory, and M, V of the next two 32-column chunks
+// are prefetched into registers (64 KB in flight per SM) while the current one is computed.
 template <int BN, bool SINGLE>
-__global__ void __launch_bounds__(224, 1)
+__global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table, int nprob,
                     int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
   using S = K1Smem<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
-  uint8_t* mv_base = smem + S::kStages * S::kStageBytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::kBarOffset);
   uint64_t* full = bars;                         // [kStages]
   uint64_t* empty = bars + S::kStages;           // [kStages]
   uint64_t* acc_full = bars + 2 * S::kStages;    // [2]
   uint64_t* acc_empty = acc_full + 2;            // [2]
-  uint64_t* mv_full = acc_empty + 2;             // [kMvBufs]
-  uint64_t* mv_empty = mv_full + S::kMvBufs;     // [kMvBufs]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mv_empty + S::kMvBufs);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const TcProblem* probs = SINGLE ? &single : table;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S::kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
-    for (int i = 0; i < S::kMvBufs; ++i) { mbar_init(&mv_full[i], 1); mbar_init(&mv_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], S::kEpiWarps); }
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -198,123 +206,103 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       }
       if (!ok) raise_wait_expired(status);
     }
-  } else if (warp == 2) {
-    // ------------------------------------------------------------------ loader of the M, V chunks
-    if (lane == 0) {
-      int pi = 0;
-      uint32_t cc = 0;
-      bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const TcProblem* p = locate(tile, pi);
-        const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
-        const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
-        const int nchunks = min(BN / kChunk, (p->n - n0 + kChunk - 1) / kChunk);
-        const CUtensorMap* mapM = &p->mapM;
-        const CUtensorMap* mapV = &p->mapV;
-        for (int c = 0; c < nchunks; ++c, ++cc) {
-          const int b = cc % S::kMvBufs;
-          if (!mbar_wait(&mv_empty[b], ((cc / S::kMvBufs) & 1) ^ 1)) { ok = false; break; }
-          uint8_t* buf = mv_base + b * S::kMvBufBytes;
-          mbar_arrive_expect_tx(&mv_full[b], 2 * S::kMBytes);
-          tma_load_2d(buf, mapM, &mv_full[b], n0 + c * kChunk, r0);
-          tma_load_2d(buf + S::kMBytes, mapV, &mv_full[b], n0 + c * kChunk, r0);
-        }
-      }
-      if (!ok) raise_wait_expired(status);
-    }
   } else {
     // ------------------------------------------------------------------ epilogue: Adam on the tile
-    const int q = warp & 3;                         // TMEM lane quarter this warp may access
-    const int row = q * 32 + lane;                  // accumulator row = row of the r block
-    const bool elected = (threadIdx.x == 96);       // first epilogue thread issues the TMA stores
+    const int q = warp & 3, hh = (warp - 2) >> 2;   // TMEM lane quarter of this warp, 16-lane half within it
+    const int lrow = q * 32 + hh * 16 + (lane >> 2); // first of the thread's two tile rows (the other: + 8)
+    const int lcol = 2 * (lane & 3);                 // first column of the thread's pair within a group of 8
+    const uint32_t lane_addr = (uint32_t)(q * 32 + hh * 16) << 16;
     const float inv_b1 = 1.0f / sc.bias1, inv_b2 = 1.0f / sc.bias2;
     int pi = 0;
-    uint32_t cc = 0, tcount = 0;
+    uint32_t tcount = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
       const TcProblem* p = locate(tile, pi);
       const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
       const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
-      const int pn = p->n, n_tma = p->n_tma_mv;
-      const int nchunks = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
-      const bool row_ok = r0 + row < p->r;
-      const int64_t ldmv = p->ldmv;
-      float* gM = p->M + (int64_t)(r0 + row) * ldmv;
-      float* gV = p->V + (int64_t)(r0 + row) * ldmv;
-      float* dbgR = p->dbgR ? p->dbgR + (int64_t)(r0 + row) * ldmv : nullptr;
-      float* dbgN = p->dbgN ? p->dbgN + (int64_t)(r0 + row) * ldmv : nullptr;
-      const CUtensorMap* mapMst = &p->mapMst;
-      const CUtensorMap* mapVst = &p->mapVst;
-      const CUtensorMap* mapNst = &p->mapNst;
-      const uint32_t ab = tcount & 1;
-      ok = named_bar_and(1, 128, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
-      if (!ok) break;
-      tc_fence_after_sync();
-      for (int c = 0; c < nchunks; ++c, ++cc) {
-        const int b = cc % S::kMvBufs;
-        ok = named_bar_and(1, 128, mbar_wait(&mv_full[b], (cc / S::kMvBufs) & 1));
-        if (!ok) break;
-        uint32_t acc[32];
-        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + c * kChunk, acc);
-        tmem_ld_wait();
-        uint8_t* buf = mv_base + b * S::kMvBufBytes;
-        float4* Mrow = reinterpret_cast<float4*>(buf + row * 128);
-        float4* Vrow = reinterpret_cast<float4*>(buf + S::kMBytes + row * 128);
-        uint2* Nrow = reinterpret_cast<uint2*>(buf + 2 * S::kMBytes + row * 64);
-        const int col0 = n0 + c * kChunk;
-        const bool special = row_ok && ((dbgR != nullptr) | (dbgN != nullptr) | (col0 + kChunk > n_tma));
+      const int pn = p->n;
+      const int nch = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
+      const int cmax = pn - n0 - lcol;               // offset `off` (from n0 + lcol) is a valid column iff off < cmax
+      const int64_t ldmv = p->ldmv, ldn = p->ldn;
+      float* Mr[2]; float* Vr[2]; uint16_t* Nr[2]; float* tapR[2]; float* tapN[2];
+      bool rok[2];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int pj = j ^ (row & 7);             // 128-byte swizzle: 16-byte chunk j lives at j ^ (row % 8)
-          float4 m4 = Mrow[pj], v4 = Vrow[pj];
-          float mm[4] = {m4.x, m4.y, m4.z, m4.w}, vv[4] = {v4.x, v4.y, v4.z, v4.w}, nn[4];
+      for (int a = 0; a < 2; ++a) {
+        const int64_t gr = r0 + lrow + 8 * a;
+        rok[a] = gr < p->r;
+        Mr[a] = p->M + gr * ldmv + n0 + lcol;
+        Vr[a] = p->V + gr * ldmv + n0 + lcol;
+        Nr[a] = p->nb + gr * ldn + n0 + lcol;
+        tapR[a] = p->dbgR ? p->dbgR + gr * ldmv + n0 + lcol : nullptr;
+        tapN[a] = p->dbgN ? p->dbgN + gr * ldmv + n0 + lcol : nullptr;
+      }
+      float2 sm[3][8], sv[3][8];                     // three chunks of M, V: index 2k + a
+      auto load_chunk = [&](int c, float2* m, float2* v) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float rr = __uint_as_float(acc[4 * j + e]);
-            mm[e] = fmaf(sc.beta1, mm[e], sc.one_minus_beta1 * rr);
-            vv[e] = fmaf(sc.beta2, vv[e], sc.one_minus_beta2 * rr * rr);
-            nn[e] = __fdividef(mm[e] * inv_b1, sqrt_approx(vv[e] * inv_b2) + sc.eps);
-          }
-          Mrow[pj] = make_float4(mm[0], mm[1], mm[2], mm[3]);
-          Vrow[pj] = make_float4(vv[0], vv[1], vv[2], vv[3]);
-          uint2 nb;
-          nb.x = (uint32_t)float_to_bf16_bits(nn[0]) | ((uint32_t)float_to_bf16_bits(nn[1]) << 16);
-          nb.y = (uint32_t)float_to_bf16_bits(nn[2]) | ((uint32_t)float_to_bf16_bits(nn[3]) << 16);
-          // 64-byte swizzle of the bf16 tile: 16-byte chunk (j / 2) lives at (j / 2) ^ ((row / 2) % 4)
-          Nrow[(((j >> 1) ^ ((row >> 1) & 3)) << 1) | (j & 1)] = nb;
-          if (special) {                            // ragged tail (at most 3 columns) and the test taps
+        for (int k = 0; k < 4; ++k)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int col = col0 + 4 * j + e;
-              if (col < pn) {
-                if (col >= n_tma) { gM[col] = mm[e]; gV[col] = vv[e]; }
-                if (dbgR) dbgR[col] = __uint_as_float(acc[4 * j + e]);
-                if (dbgN) dbgN[col] = nn[e];
+          for (int a = 0; a < 2; ++a) {
+            const int off = kChunk * c + 8 * k;
+            float2 mm = make_float2(0.f, 0.f), vv = make_float2(0.f, 0.f);
+            if (rok[a]) {
+              if (off + 1 < cmax) {
+                mm = __ldcs(reinterpret_cast<const float2*>(Mr[a] + off));
+                vv = __ldcs(reinterpret_cast<const float2*>(Vr[a] + off));
+              } else if (off < cmax) {
+                mm.x = __ldcs(Mr[a] + off);
+                vv.x = __ldcs(Vr[a] + off);
               }
             }
+            m[2 * k + a] = mm;
+            v[2 * k + a] = vv;
           }
-        }
-        fence_proxy_async_smem();
-        named_bar_sync(1, 128);
-        if (elected) {
-          if (col0 < n_tma) {
-            tma_store_2d(mapMst, buf, col0, r0);
-            tma_store_2d(mapVst, buf + S::kMBytes, col0, r0);
-          }
-          tma_store_2d(mapNst, buf + 2 * S::kMBytes, col0, r0);
-          tma_commit_group();
-          if (cc >= 1) {                             // the previous chunk's buffer has been read out
-            tma_wait_group_read<1>();
-            mbar_arrive(&mv_empty[(cc - 1) % S::kMvBufs]);
-          }
+      };
+      load_chunk(0, sm[0], sv[0]);
+      if (nch > 1) load_chunk(1, sm[1], sv[1]);
+
+      const uint32_t ab = tcount & 1;
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
+      if (!ok) break;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int c = 0; c < BN / kChunk; ++c) {
+        if (c < nch) {
+          if (c + 2 < nch) load_chunk(c + 2, sm[(c + 2) % 3], sv[(c + 2) % 3]);
+          uint32_t acc[16];
+          tmem_ld_16x256b_x4(tmem_base + lane_addr + ab * BN + c * kChunk, acc);
+          tmem_ld_wait();
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {
+              const int off = kChunk * c + 8 * k;
+              float2 mm = sm[c % 3][2 * k + a], vv = sv[c % 3][2 * k + a];
+              const float ra = __uint_as_float(acc[4 * k + 2 * a]), rb = __uint_as_float(acc[4 * k + 2 * a + 1]);
+              const float na = adam1(sc, inv_b1, inv_b2, ra, mm.x, vv.x);
+              const float nb = adam1(sc, inv_b1, inv_b2, rb, mm.y, vv.y);
+              if (rok[a]) {
+                if (off + 1 < cmax) {
+                  __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
+                  __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
+                  *reinterpret_cast<uint32_t*>(Nr[a] + off) =
+                      (uint32_t)float_to_bf16_bits(na) | ((uint32_t)float_to_bf16_bits(nb) << 16);
+                  if (tapR[a]) { tapR[a][off] = ra; tapR[a][off + 1] = rb; }
+                  if (tapN[a]) { tapN[a][off] = na; tapN[a][off + 1] = nb; }
+                } else if (off < cmax) {             // odd n: the last column stands alone
+                  Mr[a][off] = mm.x;
+                  Vr[a][off] = vv.x;
+                  Nr[a][off] = float_to_bf16_bits(na);
+                  if (tapR[a]) tapR[a][off] = ra;
+                  if (tapN[a]) tapN[a][off] = na;
+                }
+              }
+            }
         }
       }
-      if (!ok) break;
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&acc_empty[ab]);
     }
-    if (elected) tma_wait_group<0>();
     if (!ok && lane == 0) raise_wait_expired(status);
   }
 
@@ -350,7 +338,7 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves an integ
 // 16 consecutive pre-rounding weights W' = W^ - lr*alpha*D - lr*wd*W^, W^ = (q - z) * s, from 16 INT8
 // codes and 16 accumulators.  FAST: q - z is formed without an integer-to-float conversion: the byte
 // (q + 128) is dropped into the mantissa of 2^23 and (2^23 + 128 + z) subtracted, exact for |z| < 2^22.
-template <bool FAST>
+template <bool FAST, bool NOWD>
 __device__ __forceinline__ void weights16(const uint4 cw, const uint32_t* acc, float z, float s, float lr_alpha,
                                           float lr_wd, float* w) {
   const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
@@ -364,7 +352,7 @@ __device__ __forceinline__ void weights16(const uint4 cw, const uint32_t* acc, f
       if (FAST) qz = __fsub_rn(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650 + b)), c0);
       else qz = __fsub_rn((float)(int8_t)((w4[k] >> (8 * b)) & 0xFFu), z);
       const float wh = __fmul_rn(qz, s);
-      w[4 * k + b] = fmaf(-lr_alpha, __uint_as_float(acc[4 * k + b]), fmaf(-lr_wd, wh, wh));
+      w[4 * k + b] = fmaf(-lr_alpha, __uint_as_float(acc[4 * k + b]), NOWD ? wh : fmaf(-lr_wd, wh, wh));
     }
   }
 }
@@ -374,9 +362,39 @@ __device__ __forceinline__ void weights16(const uint4 cw, const uint32_t* acc, f
 // ceil(t - h / 65536) + z; it is formed as one add in round-up mode onto (2^23 * 1.5 + z), which leaves
 // the code in the low byte.  The subtraction t - h / 65536 rounds by at most 2^-14 for |t| < 2^10, so a
 // decision can differ from the exact one only within that distance of the rounding boundary.
+// Four 32-bit integers -> four signed bytes with saturation (first argument in the lowest byte).
+__device__ __forceinline__ uint32_t pack_sat_s8x4(int c0, int c1, int c2, int c3) {
+  uint32_t hi, out;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(c3), "r"(c2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(c1), "r"(c0), "r"(hi));
+  return out;
+}
+
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float d;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// Philox4x32-10 with the ten round keys given (key schedule hoisted out of the per-block calls) and
+// each 32 x 32 -> 64 bit product taken as one wide multiply.
+__device__ __forceinline__ uint4 philox_rounds(uint4 c, const uint32_t* kx, const uint32_t* ky) {
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint64_t p0 = (uint64_t)c.x * 0xD2511F53ull, p1 = (uint64_t)c.z * 0xCD9E8D57ull;
+    c = make_uint4((uint32_t)(p1 >> 32) ^ c.y ^ kx[i], (uint32_t)p1, (uint32_t)(p0 >> 32) ^ c.w ^ ky[i], (uint32_t)p0);
+  }
+  return c;
+}
+
 template <bool FAST>
 __device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& gp, const uint32_t h[8]) {
-  uint32_t bits[16];
+  int code[16];
   const float mz = (kMagic + 128.0f) + gp.z;
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
@@ -384,24 +402,19 @@ __device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& g
     if (FAST) {
       // 128 + h / 65536: h dropped into the mantissa of 2^7
       const float hv = __uint_as_float(__byte_perm(h[j >> 1], 0x43000000u, (j & 1) ? 0x7632 : 0x7610));
-      float y = __fadd_ru(__fsub_rn(t, hv), mz);
-      y = fminf(fmaxf(y, kMagic - 128.0f), kMagic + 127.0f);
-      bits[j] = __float_as_uint(y);
+      const float y = __fadd_ru(__fsub_rn(t, hv), mz);       // kMagic + ceil(t - h / 65536) + z
+      code[j] = __float_as_int(y) - 0x4B400000;               // may be -129 or 128: the pack saturates
     } else {
       const float hf = (float)((h[j >> 1] >> (16 * (j & 1))) & 0xFFFFu);
       const float f = floorf(t);
       const float up = (__fmul_rn(__fsub_rn(t, f), 65536.0f) > hf) ? 1.0f : 0.0f;
       const float qv = fminf(fmaxf(__fadd_rn(__fadd_rn(f, up), gp.z), -128.0f), 127.0f);
-      bits[j] = (uint32_t)(int)qv;
+      code[j] = (int)qv;
     }
   }
   uint32_t o[4];
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const uint32_t lo = __byte_perm(bits[4 * k], bits[4 * k + 1], 0x0040);
-    const uint32_t hi = __byte_perm(bits[4 * k + 2], bits[4 * k + 3], 0x0040);
-    o[k] = __byte_perm(lo, hi, 0x5410);
-  }
+  for (int k = 0; k < 4; ++k) o[k] = pack_sat_s8x4(code[4 * k], code[4 * k + 1], code[4 * k + 2], code[4 * k + 3]);
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
@@ -522,8 +535,9 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
     // ------------------------------------------------------------------ epilogue
     // Sixteen warps: warp (quarter q, slice sl) owns accumulator rows 32q..32q+31 and columns
     // 64*sl..64*sl+63; a row of the tile is one quantization group, so four threads share a group and
-    // combine their minima and maxima through shared memory.  The 64 pre-rounding weights of a thread
-    // stay in registers between the two passes.
+    // combine their minima and maxima through shared memory.  The pre-rounding weights are written
+    // back over the accumulator in tensor memory between the two passes (registers are the scarce
+    // resource with 18 warps on the SM: 5 warps share one 16K-register scheduler partition).
     const int q = warp & 3, sl = (warp - 2) >> 2;
     const int row = q * 32 + lane;
     const bool elected = (threadIdx.x == 64);
@@ -561,37 +575,37 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
         return reinterpret_cast<uint4*>(cbuf + (k16 >> 3) * (S::kCodeBytes / 2) + row * 128 + (((k16 & 7) ^ (row & 7)) << 4));
       };
 
-      // ---- pass 1: W' of the thread's 64 columns, minimum and maximum
-      float w[64];
+      // ---- pass 1: W' of the thread's 64 columns, written back over the accumulator; minimum and maximum
       const bool fast_dq = __all_sync(0xFFFFFFFFu, fabsf(z_old) <= 4.0e6f);
+      const int myc0 = sl * 64;
+      float mn = INFINITY, mx = -INFINITY;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t acc[32];
+        float w[32];
         tmem_ld_32x32(tacc + half * kChunk, acc);
         tmem_ld_wait();
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
           const uint4 cw = *code_ptr(sl * 4 + half * 2 + k);
-          float* wk = w + half * 32 + k * 16;
-          const float lr_wd = no_wd ? 0.0f : sc.lr_wd;
-          if (fast_dq) weights16<true>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, lr_wd, wk);
-          else weights16<false>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, lr_wd, wk);
+          float* wk = w + k * 16;
+          if (fast_dq && no_wd) weights16<true, true>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, 0.f, wk);
+          else if (fast_dq) weights16<true, false>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, sc.lr_wd, wk);
+          else weights16<false, false>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, sc.lr_wd, wk);
         }
-      }
-      tc_fence_before_sync();                       // the accumulator buffer can be refilled
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[ab]);
-
-      float mn = INFINITY, mx = -INFINITY;
-      const int myc0 = sl * 64;
-      if (myc0 + 64 <= ncols) {
+        if (myc0 + half * kChunk + kChunk <= ncols) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
-      } else {
+          for (int i = 0; i < 32; i += 2) { mn = min3(mn, w[i], w[i + 1]); mx = max3(mx, w[i], w[i + 1]); }
+        } else {
 #pragma unroll
-        for (int i = 0; i < 64; ++i)
-          if (myc0 + i < ncols) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
+          for (int i = 0; i < 32; ++i)
+            if (myc0 + half * kChunk + i < ncols) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(w[i]);
+        tmem_st_32x32(tacc + half * kChunk, acc);
       }
+      tmem_st_wait();
       part[sl * kTileM + row] = make_float2(mn, mx);
       named_bar_sync(1, S::kEpiThreads);
 #pragma unroll
@@ -605,23 +619,37 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
 
       // ---- pass 2: stochastic rounding to the new grid, codes written over the old ones in shared memory
       const bool fast_sr = __all_sync(0xFFFFFFFFu, fabsf(gp.z) <= 1024.0f);
+      uint32_t kx[10], ky[10];
 #pragma unroll
-      for (int k16 = 0; k16 < 4; ++k16) {
-        const int col = n0 + myc0 + 16 * k16;
-        const uint4 x0 = philox4x32_10(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi),
-                                       make_uint2(seed_lo, seed_hi));
-        const uint4 x1 = philox4x32_10(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi),
-                                       make_uint2(seed_lo, seed_hi));
-        const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-        const uint4 out = fast_sr ? sr_codes16<true>(w + 16 * k16, gp, h) : sr_codes16<false>(w + 16 * k16, gp, h);
-        *code_ptr(sl * 4 + k16) = out;
-        if (row_ok && (col == n_tma || dbgW != nullptr)) {   // ragged tail (at most 15 columns), test tap
-          const uint32_t o4[4] = {out.x, out.y, out.z, out.w};
+      for (int i = 0; i < 10; ++i) { kx[i] = seed_lo + (uint32_t)i * 0x9E3779B9u; ky[i] = seed_hi + (uint32_t)i * 0xBB67AE85u; }
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            if (col + e < pn) {
-              if (col == n_tma) g_codes[col + e] = (int8_t)((o4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
-              if (dbgW) dbgW[col + e] = w[16 * k16 + e];
+      for (int half = 0; half < 2; ++half) {
+        uint32_t wbits[32];
+        tmem_ld_32x32(tacc + half * kChunk, wbits);
+        tmem_ld_wait();
+        if (half == 1) {                              // last read of this accumulator buffer
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        }
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk) {
+          const int k16 = half * 2 + kk;
+          const int col = n0 + myc0 + 16 * k16;
+          const float* w = reinterpret_cast<const float*>(wbits) + 16 * kk;
+          const uint4 x0 = philox_rounds(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
+          const uint4 x1 = philox_rounds(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
+          const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+          const uint4 out = fast_sr ? sr_codes16<true>(w, gp, h) : sr_codes16<false>(w, gp, h);
+          *code_ptr(sl * 4 + k16) = out;
+          if (row_ok && (col == n_tma || dbgW != nullptr)) {   // ragged tail (at most 15 columns), test tap
+            const uint32_t o4[4] = {out.x, out.y, out.z, out.w};
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              if (col + e < pn) {
+                if (col == n_tma) g_codes[col + e] = (int8_t)((o4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
+                if (dbgW) dbgW[col + e] = w[e];
+              }
             }
           }
         }
@@ -708,32 +736,22 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   ok &= make_map(&p->mapP, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, a.m, a.r, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapG, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.G, a.n, a.m, a.ldg, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapN, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Nb, a.n, a.r, w.ldn, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapNst, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Nb, a.n, a.r, w.ldn, kChunk, kTileM,
-                 CU_TENSOR_MAP_SWIZZLE_64B);
-  ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, a.n, a.r, a.ldmv, kChunk, kTileM,
-                 CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, a.n, a.r, a.ldmv, kChunk, kTileM,
-                 CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
-  const int64_t n4 = a.n & ~int64_t(3), n16 = a.n & ~int64_t(15);
-  ok &= make_map(&p->mapMst, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, n4 > 0 ? n4 : 4, a.r, a.ldmv, kChunk, kTileM,
-                 CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapVst, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, n4 > 0 ? n4 : 4, a.r, a.ldmv, kChunk, kTileM,
-                 CU_TENSOR_MAP_SWIZZLE_128B);
+  const int64_t n16 = a.n & ~int64_t(15);
   ok &= make_map(&p->mapWst, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, n16 > 0 ? n16 : 16, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) {
     note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
     return QG_CUDA_ERROR;
   }
-  p->n_tma_mv = (int32_t)n4;
   p->n_tma_w = (int32_t)n16;
   p->M = a.M; p->V = a.V; p->w_codes = reinterpret_cast<int8_t*>(a.W.codes);
   p->w_scales = a.W.scales;
   p->w_zeros = a.W.zeros;
   p->dbgR = a.dbg.R; p->dbgN = a.dbg.N; p->dbgW = a.dbg.W_pre;
-  p->ldmv = a.ldmv; p->ldw = a.W.ld;
+  p->nb = w.Nb;
+  p->ldmv = a.ldmv; p->ldw = a.W.ld; p->ldn = w.ldn;
   p->m = (int32_t)a.m; p->n = (int32_t)a.n; p->r = (int32_t)a.r;
   p->ngroups = (int32_t)ceil_div(a.n, kGroup);
   p->seed_lo = a.sc.seed_lo; p->seed_hi = a.sc.seed_hi;
@@ -772,7 +790,7 @@ int launch_k1(const TcProblem* single, const TcProblem* table, int nprob, int to
   const int sms = sm_count();
   const int grid = total_tiles < sms ? total_tiles : sms;
   static const TcProblem dummy{};
-  kern<<<grid, 224, K1Smem<BN>::kBytes, st>>>(single ? *single : dummy, table, nprob, total_tiles, sc, status);
+  kern<<<grid, K1Smem<BN>::kThreads, K1Smem<BN>::kBytes, st>>>(single ? *single : dummy, table, nprob, total_tiles, sc, status);
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
@@ -937,5 +955,30 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
 }
 
 void plan_destroy(Plan* plan) { delete plan; }
+
+// Registers, thread limit and shared memory of the tensor-core kernels as the loaded module reports them.
+int tc_kernel_info(char* buf, size_t cap) {
+  size_t used = 0;
+  auto add = [&](const char* name, const void* fn, int threads, int dyn_smem) {
+    cudaFuncAttributes at{};
+    const cudaError_t e = cudaFuncGetAttributes(&at, fn);
+    int n = 0;
+    if (e != cudaSuccess) {
+      n = snprintf(buf + used, cap - used, "%s: %s\n", name, cudaGetErrorName(e));
+      (void)cudaGetLastError();
+    } else {
+      n = snprintf(buf + used, cap - used, "%s: regs %d, max threads %d, launched with %d threads, dynamic smem %d, static smem %zu, local %zu\n",
+                   name, at.numRegs, at.maxThreadsPerBlock, threads, dyn_smem, at.sharedSizeBytes, at.localSizeBytes);
+    }
+    if (n > 0) used = (used + (size_t)n < cap) ? used + (size_t)n : cap - 1;
+  };
+  add("project_adam<128,single>", (const void*)project_adam_kernel<128, true>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
+  add("project_adam<256,single>", (const void*)project_adam_kernel<256, true>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
+  add("project_adam<128,table>", (const void*)project_adam_kernel<128, false>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
+  add("project_adam<256,table>", (const void*)project_adam_kernel<256, false>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
+  add("backproject_sr<single>", (const void*)backproject_sr_kernel<true>, K2Smem::kThreads, K2Smem::kBytes);
+  add("backproject_sr<table>", (const void*)backproject_sr_kernel<false>, K2Smem::kThreads, K2Smem::kBytes);
+  return QG_OK;
+}
 
 }  // namespace qg
