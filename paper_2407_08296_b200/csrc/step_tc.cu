@@ -36,11 +36,19 @@ constexpr int kBK = 64;                 // K extent of one pipeline stage (eleme
 constexpr int kBoxBytes = 64 * kBK * 2; // one TMA box of an operand: 64 x kBK bf16 = 8 KB
 constexpr int kTileM = 128;             // accumulator rows (TMEM lanes)
 constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
+constexpr int kPrefetch = 10;           // K blocks by which the L2 prefetch of G runs ahead of the staged loads
 
 // One matrix of the step, as the kernels see it.  Tensor maps (row-major tensors, inner extent first):
-//   mapP    P~  bf16 [m][r]       box 64 x 64, swizzle 128   A operand of both kernels
-//   mapG    G   bf16 [m][ldg]     box 64 x 64, swizzle 128   B operand of the projection
-//   mapN    N_b bf16 [r][ldn]     box 64 x 64, swizzle 128   B operand of the back-projection
+//   mapP    P~  bf16 [m][r]       box 64 x 64, swizzle 128   A operand of the projection (2-D, exact bounds)
+//   mapG    G   bf16 [m][ldg]     box 64 x 64, swizzle 128   B operand of the projection (2-D, exact bounds)
+//   mapP3   P~  as (64, m, r/64)  box 64 x 64 x 2            the same operand tiles in ONE copy each: an
+//   mapG3   G   as (64, m, n/64)  box 64 x 64 x BN/64        MN-major tile is a row of 64-column chunks, and
+//   mapN3   N_b as (64, r, ldn/64) box 64 x 64 x 4           the third dimension walks the chunks
+//   mapPk   P~  bf16 [m][r]       box 64 x 128, swizzle 128  A operand of the back-projection (K-major)
+// The 3-D views hold whole chunks only; a tile that touches a ragged last chunk (r or n not a multiple
+// of 64) is loaded chunk by chunk through the 2-D maps, whose bounds are exact.  One copy per operand
+// matters because a single thread issues them: with six copies per K block that thread, not the tensor
+// pipe, set the pace.
 //   mapW    int8 [m][ldw]         box 128 x 128, swizzle 128 load of the requantizing epilogue
 //   mapWst                        the same tensor for the store, with the inner extent rounded DOWN to 16
 //                                 bytes: a TMA store clips at 16-byte granularity, so it would spill into
@@ -48,7 +56,7 @@ constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
 //                                 plain stores instead (n_tma_w = columns the TMA store covers).
 // M, V and N_b are read and written by the Adam epilogue with plain vector accesses.
 struct alignas(64) TcProblem {
-  CUtensorMap mapP, mapG, mapN, mapW, mapWst;
+  CUtensorMap mapP, mapG, mapP3, mapG3, mapN3, mapPk, mapW, mapWst;
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -60,6 +68,7 @@ struct alignas(64) TcProblem {
   uint16_t* nb;                        // N_b, bf16 r x ldn (scratch)
   int64_t ldmv, ldw, ldn;
   int32_t m, n, r, ngroups, n_tma_w;
+  int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles, k1_tile0;
   int32_t k2_mblocks, k2_tiles, k2_tile0;
@@ -158,17 +167,53 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         const int kblocks = (p->m + kBK - 1) / kBK;
         const CUtensorMap* mapP = &p->mapP;
         const CUtensorMap* mapG = &p->mapG;
+        const CUtensorMap* mapP3 = &p->mapP3;
+        const CUtensorMap* mapG3 = &p->mapG3;
+        // whole-chunk tiles take one 3-D copy per operand; chunks past the end of a 3-D view read as zero
+        const bool a3 = (p->r_whole == p->r) || (r0 + kTileM <= p->r_whole);
+        const bool b3 = (p->n_whole == p->n) || (n0 + BN <= p->n_whole);
+        // G comes from HBM with a latency the few shared-memory stages cannot cover; its boxes are
+        // therefore pulled into L2 kPrefetch K blocks ahead (across the tile boundary), so that the
+        // staged loads only see L2 latency.  P~ was just written by the dequantize kernel and is in L2.
+        const CUtensorMap* mapG3n = nullptr;
+        int n0_2 = 0, kblocks2 = 0;
+        if (tile + (int)gridDim.x < total_tiles) {
+          int pi2 = pi;
+          const TcProblem* p2 = locate(tile + gridDim.x, pi2);
+          n0_2 = ((tile + (int)gridDim.x - p2->k1_tile0) / p2->k1_rblocks) * BN;
+          kblocks2 = (p2->m + kBK - 1) / kBK;
+          if (n0_2 + 64 <= p2->n_whole) mapG3n = &p2->mapG3;
+        }
+        if (tile == (int)blockIdx.x && n0 + 64 <= p->n_whole) {
+          for (int kb = 0; kb < min(kPrefetch, kblocks); ++kb) tma_prefetch_l2_3d(mapG3, 0, kb * kBK, n0 / 64);
+        }
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          {
+            const int t = kb + kPrefetch;
+            if (t < kblocks) {
+              if (n0 + 64 <= p->n_whole) tma_prefetch_l2_3d(mapG3, 0, t * kBK, n0 / 64);
+            } else if (mapG3n != nullptr && t - kblocks < kblocks2) {
+              tma_prefetch_l2_3d(mapG3n, 0, (t - kblocks) * kBK, n0_2 / 64);
+            }
+          }
           const int s = it % S::kStages;
           const uint32_t ph = (it / S::kStages) & 1;
           if (!mbar_wait(&empty[s], ph ^ 1)) { ok = false; break; }
           uint8_t* sA = stage_base + s * S::kStageBytes;
           uint8_t* sB = sA + S::kABytes;
           mbar_arrive_expect_tx(&full[s], S::kStageBytes);
+          if (a3) {
+            tma_load_3d(sA, mapP3, &full[s], 0, kb * kBK, r0 / 64);
+          } else {
 #pragma unroll
-          for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], r0 + 64 * h, kb * kBK);
+            for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], r0 + 64 * h, kb * kBK);
+          }
+          if (b3) {
+            tma_load_3d(sB, mapG3, &full[s], 0, kb * kBK, n0 / 64);
+          } else {
 #pragma unroll
-          for (int h = 0; h < BN / 64; ++h) tma_load_2d(sB + h * kBoxBytes, mapG, &full[s], n0 + 64 * h, kb * kBK);
+            for (int h = 0; h < BN / 64; ++h) tma_load_2d(sB + h * kBoxBytes, mapG, &full[s], n0 + 64 * h, kb * kBK);
+          }
         }
       }
       if (!ok) raise_wait_expired(status);
@@ -177,6 +222,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(kTileM, BN, true, true);
+      const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), kBoxBytes, 1024);
+      const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
       int pi = 0;
       uint32_t it = 0, tcount = 0;
       bool ok = true;
@@ -191,15 +238,12 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
           const int s = it % S::kStages;
           if (!mbar_wait(&full[s], (it / S::kStages) & 1)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint32_t aA = smem_u32(stage_base + s * S::kStageBytes);
-          const uint32_t aB = aA + S::kABytes;
+          // both operands are MN-major: 16 K indices = two 8-index groups of 1024 bytes each; the start
+          // address field counts 16-byte units, so a stage or K step is an add on the descriptor
+          const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
+          const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            // both operands are MN-major: 16 K indices = two 8-index groups of 1024 bytes each
-            const uint64_t da = umma_smem_desc_sw128(aA + k * 2048, kBoxBytes, 1024);
-            const uint64_t db = umma_smem_desc_sw128(aB + k * 2048, kBoxBytes, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
-          }
+          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, da + k * (2048 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
           umma_commit(&empty[s]);
         }
         if (ok) umma_commit(&acc_full[ab]);
@@ -474,8 +518,8 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
         const int local = tile - p->k2_tile0, mblocks = p->k2_mblocks;
         const int m0 = (local % mblocks) * kTileM, n0 = (local / mblocks) * S::kBN;
         const CUtensorMap* mapW = &p->mapW;
-        const CUtensorMap* mapP = &p->mapP;
-        const CUtensorMap* mapN = &p->mapN;
+        const CUtensorMap* mapPk = &p->mapPk;
+        const CUtensorMap* mapN3 = &p->mapN3;
         const int cb = tcount % S::kCodeBufs;
         if (!mbar_wait(&code_empty[cb], ((tcount / S::kCodeBufs) & 1) ^ 1)) { ok = false; break; }
         uint8_t* cbuf = code_base + cb * S::kCodeBytes;
@@ -489,10 +533,8 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
           uint8_t* sA = stage_base + s * S::kStageBytes;
           uint8_t* sB = sA + S::kABytes;
           mbar_arrive_expect_tx(&full[s], S::kStageBytes);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], kb * kBK, m0 + 64 * h);
-#pragma unroll
-          for (int h = 0; h < 4; ++h) tma_load_2d(sB + h * kBoxBytes, mapN, &full[s], n0 + 64 * h, kb * kBK);
+          tma_load_2d(sA, mapPk, &full[s], kb * kBK, m0);
+          tma_load_3d(sB, mapN3, &full[s], 0, kb * kBK, n0 / 64);
         }
       }
       if (!ok) raise_wait_expired(status);
@@ -501,6 +543,8 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc_bf16(kTileM, S::kBN, false, true);
+      const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), 16, 1024);
+      const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
       int pi = 0;
       uint32_t it = 0, tcount = 0;
       bool ok = true;
@@ -515,16 +559,12 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
           const int s = it % S::kStages;
           if (!mbar_wait(&full[s], (it / S::kStages) & 1)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint32_t aA = smem_u32(stage_base + s * S::kStageBytes);
-          const uint32_t aB = aA + S::kABytes;
+          // A is K-major (rows of 128 bytes, 16 K indices = 32 bytes further along the row),
+          // B is MN-major (16 K indices = two 8-index groups of 1024 bytes)
+          const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
+          const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            // A is K-major (rows of 128 bytes, 16 K indices = 32 bytes further along the row),
-            // B is MN-major (16 K indices = two 8-index groups of 1024 bytes)
-            const uint64_t da = umma_smem_desc_sw128(aA + k * 32, 16, 1024);
-            const uint64_t db = umma_smem_desc_sw128(aB + k * 2048, kBoxBytes, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0);
-          }
+          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, da + k * (32 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
           umma_commit(&empty[s]);
         }
         if (ok) umma_commit(&acc_full[ab]);
@@ -712,6 +752,22 @@ bool make_map(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const vo
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// A row-major bf16 matrix [rows][pitch] seen as (64 columns, rows, chunks): element (x, y, z) is column
+// 64 z + x of row y.  A box 64 x box_rows x box_chunks lands in shared memory as box_chunks consecutive
+// [box_rows][64] slabs, i.e. the MN-major 128-byte-swizzled operand layout.
+bool make_map_chunked(CUtensorMap* map, const void* base, int64_t rows, int64_t chunks, int64_t pitch_elems, int box_rows,
+                      int box_chunks) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)chunks};
+  const cuuint64_t gstr[2] = {(cuuint64_t)pitch_elems * 2, 128};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_chunks};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Scratch of one matrix: P~ (bf16, m x r, pitch r) then N_b (bf16, r x ldn).
 struct TcScratch {
   uint16_t* Pt;
@@ -735,7 +791,13 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   bool ok = true;
   ok &= make_map(&p->mapP, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, a.m, a.r, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapG, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.G, a.n, a.m, a.ldg, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapN, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Nb, a.n, a.r, w.ldn, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapPk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, a.m, a.r, 64, kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
+  const int64_t r_whole = a.r & ~int64_t(63), n_whole = a.n & ~int64_t(63);
+  ok &= make_map_chunked(&p->mapP3, w.Pt, a.m, r_whole > 0 ? r_whole / 64 : 1, a.r, kBK, 2);
+  ok &= make_map_chunked(&p->mapG3, a.G, a.m, n_whole > 0 ? n_whole / 64 : 1, a.ldg, kBK, bn / 64);
+  ok &= make_map_chunked(&p->mapN3, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 4);
+  p->r_whole = (int32_t)r_whole;
+  p->n_whole = (int32_t)n_whole;
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
   const int64_t n16 = a.n & ~int64_t(15);
