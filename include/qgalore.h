@@ -158,6 +158,12 @@ QG_API int qgalore_plan_create(const qg_step_item* items, int32_t count, void* t
                         void* workspace, size_t workspace_bytes, qg_plan** plan);
 QG_API int qgalore_plan_step(const qg_plan* plan, const qg_hyper* h, int32_t* status_dev, void* stream);
 QG_API void qgalore_plan_destroy(qg_plan* plan);
+/* Measurement aid: the same step as qgalore_plan_step with a CUDA event recorded before and after every
+ * kernel launch on `stream`; waits for the step to finish (the one entry point that synchronises, and
+ * that creates and destroys events).  kernel_ms[0..2] (HOST) receive the summed device time of the
+ * dequantize-P, projection+Adam and back-projection+requantize launches, kernel_launches[0..2] their counts. */
+QG_API int qgalore_plan_step_timed(const qg_plan* plan, const qg_hyper* h, int32_t* status_dev, void* stream,
+                            float* kernel_ms, int32_t* kernel_launches);
 
 /* --- Sec. 3.5 "obtain the projection matrix using SVD" + Sec. 3.3 INT4 storage ------------
  * Top-r left singular subspace of G (bf16, m x n) by block subspace iteration with

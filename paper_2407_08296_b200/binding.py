@@ -78,6 +78,7 @@ def lib() -> C.CDLL:
         L.qgalore_plan_table_bytes.restype = sz
         L.qgalore_plan_create.argtypes = [C.POINTER(_CStepItem), i32, vp, sz, vp, sz, C.POINTER(vp)]
         L.qgalore_plan_step.argtypes = [vp, C.POINTER(_CHyper), vp, vp]
+        L.qgalore_plan_step_timed.argtypes = [vp, C.POINTER(_CHyper), vp, vp, C.POINTER(C.c_float), C.POINTER(i32)]
         L.qgalore_plan_destroy.argtypes = [vp]
         L.qgalore_plan_destroy.restype = None
         L.qgalore_refresh_subspace.argtypes = [vp, i64, i64, i64, i64, i32, i32, C.c_uint64, qp, vp, qp, i32, vp,
@@ -318,6 +319,16 @@ class StepPlan:
         hc = hyper.c_struct()
         _check(lib().qgalore_plan_step(self._handle, C.byref(hc), _ptr(self.status), _stream_ptr(stream)),
                "qgalore_plan_step")
+
+    def step_timed(self, hyper: Hyper, stream=None) -> tuple[list[float], list[int]]:
+        """One step with events around every launch; returns (ms per kernel kind, launches per kernel kind)
+        for [dequantize-P, projection+Adam, back-projection+requantize].  Blocks until the step is done."""
+        hc = hyper.c_struct()
+        ms = (C.c_float * 3)()
+        cnt = (C.c_int32 * 3)()
+        _check(lib().qgalore_plan_step_timed(self._handle, C.byref(hc), _ptr(self.status), _stream_ptr(stream), ms, cnt),
+               "qgalore_plan_step_timed")
+        return [float(x) for x in ms], [int(x) for x in cnt]
 
     def close(self) -> None:
         if self._handle is not None and self._handle.value:

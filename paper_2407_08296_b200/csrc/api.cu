@@ -31,7 +31,9 @@ struct Plan;
 size_t plan_table_bytes(int32_t count);
 int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t table_bytes, void* workspace,
                 size_t workspace_bytes, Plan** out);
-int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st);
+int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st, cudaEvent_t* ev);
+int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st, float* ms,
+                    int32_t* launches);
 void plan_destroy(Plan* plan);
 int tc_kernel_info(char* buf, size_t cap);
 
@@ -240,7 +242,17 @@ int qgalore_plan_step(const qg_plan* plan, const qg_hyper* h, int32_t* status_de
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
   StepScalars sc;
   fill_scalars(h, 0, &sc);
-  return plan_step(plan->impl, sc, status_dev, (cudaStream_t)stream);
+  return plan_step(plan->impl, sc, status_dev, (cudaStream_t)stream, nullptr);
+}
+
+int qgalore_plan_step_timed(const qg_plan* plan, const qg_hyper* h, int32_t* status_dev, void* stream,
+                            float* kernel_ms, int32_t* kernel_launches) {
+  if (!plan || !plan->impl || !kernel_ms || !kernel_launches) return QG_INVALID_ARGUMENT;
+  const int rc = check_hyper(h);
+  if (rc != QG_OK) return rc;
+  StepScalars sc;
+  fill_scalars(h, 0, &sc);
+  return plan_step_timed(plan->impl, sc, status_dev, (cudaStream_t)stream, kernel_ms, kernel_launches);
 }
 
 void qgalore_plan_destroy(qg_plan* plan) {

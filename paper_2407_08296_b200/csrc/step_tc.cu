@@ -1002,18 +1002,52 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
   return QG_OK;
 }
 
-int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st) {
+// One step of every chunk.  With `ev` (4 events per chunk, created by the caller) an event is recorded
+// before the chunk's first kernel and after each of its three kernels.
+int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st, cudaEvent_t* ev) {
+  size_t c = 0;
   for (const PlanChunk& ch : plan->chunks) {
+    if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 0], st));
     dequant_p_grouped_kernel<<<ch.dq_blocks, 256, 0, st>>>(plan->dq_dev + ch.first, ch.count);
     QG_LAUNCH_CHECK();
+    if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 1], st));
     const TcProblem* tab = plan->table_dev + ch.first;
     int rc = ch.bn == 256 ? launch_k1<256, false>(nullptr, tab, ch.count, ch.k1_tiles, sc, status, st)
                           : launch_k1<128, false>(nullptr, tab, ch.count, ch.k1_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
+    if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 2], st));
     rc = launch_k2<false>(nullptr, tab, ch.count, ch.k2_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
+    if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 3], st));
+    ++c;
   }
   return QG_OK;
+}
+
+// One step with an event pair around every launch; blocks until the step has finished.
+// ms[0..2] receive the summed durations of the dequantize, projection and back-projection launches,
+// launches[0..2] their counts.
+int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st, float* ms,
+                    int32_t* launches) {
+  const size_t nch = plan->chunks.size();
+  std::vector<cudaEvent_t> ev(4 * nch, nullptr);
+  int rc = QG_OK;
+  for (auto& e : ev)
+    if (cudaEventCreate(&e) != cudaSuccess) rc = QG_CUDA_ERROR;
+  if (rc == QG_OK) rc = plan_step(plan, sc, status, st, ev.data());
+  if (rc == QG_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = QG_CUDA_ERROR;
+  for (int k = 0; k < 3; ++k) { ms[k] = 0.f; launches[k] = 0; }
+  if (rc == QG_OK) {
+    for (size_t c = 0; c < nch; ++c)
+      for (int k = 0; k < 3; ++k) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, ev[4 * c + k], ev[4 * c + k + 1]) == cudaSuccess) { ms[k] += t; launches[k] += 1; }
+      }
+  }
+  for (auto& e : ev)
+    if (e) cudaEventDestroy(e);
+  (void)cudaGetLastError();
+  return rc;
 }
 
 void plan_destroy(Plan* plan) { delete plan; }
