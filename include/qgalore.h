@@ -186,6 +186,27 @@ QG_API int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B,
                                 float* sim_dev, void* workspace, size_t workspace_bytes,
                                 void* stream);
 
+/* --- The same statistic for callers that cannot allocate device memory (the paper has no counterpart: this
+ * is a convenience of the library).  Some code that wants the similarity runs where cudaMalloc is
+ * not an option: inside a framework's optimizer hook that must not touch the caching allocator, in a process
+ * whose memory budget was handed out up front, or on a stream that is being recorded.  For them the scratch
+ * of the two reduction kernels sits in a fixed array inside the library instead of a caller workspace, so
+ * the call takes only its inputs and the output scalar and never calls cudaMalloc, cudaFree or any
+ * allocating routine.
+ *   - Limit: qgalore_workspace_bytes(QG_OP_SIMILARITY, rows, 0, cols) must not exceed
+ *     qgalore_subspace_similarity_static_max_bytes() (2 MiB: e.g. 11008 x 1024 fits, 16384 x 2048 does not);
+ *     larger shapes return QG_WORKSPACE_TOO_SMALL and enqueue nothing.  Every GPU on which the library is
+ *     loaded keeps those 2 MiB reserved until the process ends.
+ *   - The first call on each device looks up the array's device address (a runtime query, made with that
+ *     device current); make that first call before you start capturing a stream.
+ *   - All calls on a device share the one array.  Nothing in it has to be zero on entry (the first kernel
+ *     rewrites every word the second reads), but two calls that overlap on the GPU - different streams, or
+ *     different host threads - race on it and return garbage: serialise them.
+ * Results are identical to qgalore_subspace_similarity on the same inputs. */
+QG_API int qgalore_subspace_similarity_static(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols,
+                                       float* sim_dev, void* stream);
+QG_API size_t qgalore_subspace_similarity_static_max_bytes(void);
+
 /* --- Sec. 3.2, adaptive lazy update: host-only state machine ----------------------------
  * Pushes `sim` into `history` (k floats, host) holding *count values; when k values are held
  * and all are >= threshold, *interval is doubled and the history cleared.  Returns 1 if the

@@ -84,6 +84,8 @@ def lib() -> C.CDLL:
         L.qgalore_refresh_subspace.argtypes = [vp, i64, i64, i64, i64, i32, i32, C.c_uint64, qp, vp, qp, i32, vp,
                                                vp, sz, vp, vp]
         L.qgalore_subspace_similarity.argtypes = [qp, qp, i32, vp, vp, sz, vp]
+        L.qgalore_subspace_similarity_static.argtypes = [qp, qp, i32, vp, vp]
+        L.qgalore_subspace_similarity_static_max_bytes.restype = sz
         L.qgalore_gate_update.argtypes = [C.c_float, C.c_float, i32, C.POINTER(i32), C.POINTER(C.c_float),
                                           C.POINTER(i32)]
         L.qgalore_workspace_bytes.argtypes = [C.c_int, i64, i64, i64]
@@ -376,6 +378,19 @@ def subspace_similarity(A: QTensor, B: QTensor, sim_cols: int = 0, out: torch.Te
     ac, bc = A.c_struct(), B.c_struct()
     _check(lib().qgalore_subspace_similarity(C.byref(ac), C.byref(bc), sim_cols, _ptr(out), _ptr(workspace),
                                              workspace.numel(), _stream_ptr(stream)), "qgalore_subspace_similarity")
+    return out
+
+
+def subspace_similarity_static(A: QTensor, B: QTensor, sim_cols: int = 0, out: torch.Tensor | None = None,
+                               stream=None) -> torch.Tensor:
+    """Same result as subspace_similarity, for callers that may not allocate: the scratch is a fixed array
+    inside the library (shapes needing more than 2 MiB are refused), so pass ``out`` and nothing is allocated.
+    Calls on one device share that array and must not overlap."""
+    if out is None:
+        out = torch.zeros(1, dtype=torch.float32, device=A.codes.device)
+    ac, bc = A.c_struct(), B.c_struct()
+    _check(lib().qgalore_subspace_similarity_static(C.byref(ac), C.byref(bc), sim_cols, _ptr(out), _stream_ptr(stream)),
+           "qgalore_subspace_similarity_static")
     return out
 
 

@@ -256,3 +256,42 @@ int launch_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t c, float
 }
 
 }  // namespace qg
+
+// ------------------------------------------------------------------------ similarity without a caller workspace
+// The scratch of the two similarity kernels lives in this fixed device array instead of memory the
+// caller allocates.  Every device that loads the library carries these 2 MiB until the process exits.
+namespace {
+constexpr size_t kStaticSimilarityBytes = 2u << 20;
+static __device__ __align__(256) unsigned char g_similarity_scratch[kStaticSimilarityBytes];
+constexpr int kMaxDevices = 64;
+void* g_similarity_scratch_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal
+}  // namespace
+
+extern "C" QG_API size_t qgalore_subspace_similarity_static_max_bytes(void) { return kStaticSimilarityBytes; }
+
+extern "C" QG_API int qgalore_subspace_similarity_static(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols,
+                                                         float* sim_dev, void* stream) {
+  using namespace qg;
+  if (!A || !B || !sim_dev) return QG_INVALID_ARGUMENT;
+  for (const qg_qtensor* t : {A, B}) {
+    if (!t->codes || !t->scales || !t->zeros || t->rows <= 0 || t->cols <= 0 || t->ld < t->cols) return QG_INVALID_ARGUMENT;
+    if (t->bits != 4 || t->group != kGroup) return QG_INVALID_ARGUMENT;
+    if (!aligned16(t->codes) || t->ld % 32 != 0) return QG_MISALIGNED;
+  }
+  if (A->rows != B->rows || A->cols != B->cols) return QG_INVALID_ARGUMENT;
+  if (A->cols > 16384) return QG_UNSUPPORTED_SHAPE;
+  // the shape must fit the fixed array: report it as a workspace that cannot be made larger
+  if (similarity_workspace_bytes(A->rows, A->cols) > kStaticSimilarityBytes) return QG_WORKSPACE_TOO_SMALL;
+  int dev = 0;
+  QG_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return QG_UNSUPPORTED_SHAPE;
+  if (!g_similarity_scratch_ptr[dev]) {
+    // In host code the array's name is only a handle; the kernels need its address on the current device.
+    void* p = nullptr;
+    QG_CUDA_TRY(cudaGetSymbolAddress(&p, g_similarity_scratch));
+    g_similarity_scratch_ptr[dev] = p;
+  }
+  const int32_t c = (sim_cols <= 0 || sim_cols > A->cols) ? (int32_t)A->cols : sim_cols;
+  // the first kernel overwrites every scratch word the second one reads, so nothing has to be cleared
+  return launch_similarity(A, B, c, sim_dev, g_similarity_scratch_ptr[dev], (cudaStream_t)stream);
+}
