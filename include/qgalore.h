@@ -144,7 +144,7 @@ QG_API size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t
  * each chunk runs as one dequantize-P launch, one projection+Adam launch and one back-projection+
  * requantization launch over all of its matrices.
  *   items       HOST; every buffer an item names must stay where it is while the plan lives
- *   table_dev   DEVICE, 256-byte aligned, qgalore_plan_table_bytes(count) bytes, owned by the caller and
+ *   table_dev   DEVICE, 256-byte aligned, qgalore_plan_table_bytes(items, count) bytes, owned by the caller and
  *               left untouched by it until qgalore_plan_destroy
  *   workspace   DEVICE scratch, 1024-byte aligned, at least qgalore_workspace_bytes_batched(items, count)
  *               bytes; more lets a chunk hold more matrices.  Contents are undefined between steps, but
@@ -153,7 +153,7 @@ QG_API size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t
  * qgalore_plan_step enqueues one optimizer step of every matrix (lr, alpha, the Adam constants and the
  * step index from h; the stochastic-rounding seed of each matrix from its item) and returns. */
 typedef struct qg_plan qg_plan;
-QG_API size_t qgalore_plan_table_bytes(int32_t count);
+QG_API size_t qgalore_plan_table_bytes(const qg_step_item* items, int32_t count);  /* 0 if an item is invalid */
 QG_API int qgalore_plan_create(const qg_step_item* items, int32_t count, void* table_dev, size_t table_bytes,
                         void* workspace, size_t workspace_bytes, qg_plan** plan);
 QG_API int qgalore_plan_step(const qg_plan* plan, const qg_hyper* h, int32_t* status_dev, void* stream);

@@ -74,7 +74,7 @@ def lib() -> C.CDLL:
         L.qgalore_project_step_batched.argtypes = [C.POINTER(_CStepItem), i32, C.POINTER(_CHyper), vp, sz, vp, vp]
         L.qgalore_workspace_bytes_batched.argtypes = [C.POINTER(_CStepItem), i32]
         L.qgalore_workspace_bytes_batched.restype = sz
-        L.qgalore_plan_table_bytes.argtypes = [i32]
+        L.qgalore_plan_table_bytes.argtypes = [C.POINTER(_CStepItem), i32]
         L.qgalore_plan_table_bytes.restype = sz
         L.qgalore_plan_create.argtypes = [C.POINTER(_CStepItem), i32, vp, sz, vp, sz, C.POINTER(vp)]
         L.qgalore_plan_step.argtypes = [vp, C.POINTER(_CHyper), vp, vp]
@@ -309,7 +309,7 @@ class StepPlan:
         if workspace_bytes is None:
             workspace_bytes = max(need, self.PREFERRED_WORKSPACE)
         self.workspace = torch.empty(max(int(workspace_bytes), 1024), dtype=torch.uint8, device=dev)
-        self.table_dev = torch.empty(int(L.qgalore_plan_table_bytes(n)), dtype=torch.uint8, device=dev)
+        self.table_dev = torch.empty(max(int(L.qgalore_plan_table_bytes(self._table, n)), 256), dtype=torch.uint8, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.elements = sum(int(it["G"].shape[0]) * int(it["G"].shape[1]) for it in items)
         handle = C.c_void_p()

@@ -28,7 +28,7 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
                    int32_t* status, cudaStream_t st);
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b);
 struct Plan;
-size_t plan_table_bytes(int32_t count);
+size_t plan_table_bytes(const StepArgs* items, int32_t count);
 int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t table_bytes, void* workspace,
                 size_t workspace_bytes, Plan** out);
 int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStream_t st, cudaEvent_t* ev);
@@ -213,21 +213,33 @@ struct qg_plan {
   Plan* impl;
 };
 
-size_t qgalore_plan_table_bytes(int32_t count) { return count > 0 ? plan_table_bytes(count) : 0; }
+static int plan_args(const qg_step_item* items, int32_t count, std::vector<StepArgs>* args) {
+  args->resize((size_t)count);
+  for (int32_t i = 0; i < count; ++i) {
+    const qg_step_item& it = items[i];
+    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &(*args)[i]);
+    if (rc != QG_OK) return rc;
+    (*args)[i].sc.seed_lo = (uint32_t)(it.seed & 0xFFFFFFFFull);
+    (*args)[i].sc.seed_hi = (uint32_t)(it.seed >> 32);
+  }
+  return QG_OK;
+}
+
+size_t qgalore_plan_table_bytes(const qg_step_item* items, int32_t count) {
+  if (!items || count <= 0) return 0;
+  std::vector<StepArgs> args;
+  if (plan_args(items, count, &args) != QG_OK) return 0;
+  return plan_table_bytes(args.data(), count);
+}
 
 int qgalore_plan_create(const qg_step_item* items, int32_t count, void* table_dev, size_t table_bytes,
                         void* workspace, size_t workspace_bytes, qg_plan** plan) {
   if (!items || count <= 0 || !table_dev || !workspace || !plan) return QG_INVALID_ARGUMENT;
   if ((reinterpret_cast<uintptr_t>(workspace) & 1023u) || (reinterpret_cast<uintptr_t>(table_dev) & 255u))
     return QG_MISALIGNED;
-  std::vector<StepArgs> args((size_t)count);
-  for (int32_t i = 0; i < count; ++i) {
-    const qg_step_item& it = items[i];
-    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &args[i]);
-    if (rc != QG_OK) return rc;
-    args[i].sc.seed_lo = (uint32_t)(it.seed & 0xFFFFFFFFull);
-    args[i].sc.seed_hi = (uint32_t)(it.seed >> 32);
-  }
+  std::vector<StepArgs> args;
+  const int rca = plan_args(items, count, &args);
+  if (rca != QG_OK) return rca;
   Plan* impl = nullptr;
   const int rc = plan_create(args.data(), count, table_dev, table_bytes, workspace, workspace_bytes, &impl);
   if (rc != QG_OK) return rc;

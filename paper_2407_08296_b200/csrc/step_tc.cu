@@ -21,6 +21,8 @@
 // stops taking tiles, releases its tensor memory and returns.
 #include <cstdio>
 #include <cstring>
+#include <algorithm>
+#include <queue>
 #include <vector>
 
 #include "sm100_ptx.cuh"
@@ -70,10 +72,36 @@ struct alignas(64) TcProblem {
   int32_t m, n, r, ngroups, n_tma_w;
   int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
-  int32_t k1_rblocks, k1_tiles, k1_tile0;
-  int32_t k2_mblocks, k2_tiles, k2_tile0;
+  int32_t k1_rblocks, k1_tiles;
+  int32_t k2_mblocks, k2_tiles;
 };
 static_assert(sizeof(TcProblem) <= 2048, "TcProblem must fit the kernel parameter space");
+
+// The tiles one CTA works through.  A single matrix is walked round-robin (tile = block, block + grid, ...);
+// a plan carries a precomputed list per CTA, (problem, tile within the problem) pairs in entries
+// [start[block], start[block + 1]): tiles differ in cost by the K extent of their matrix, and a
+// longest-first assignment on the host keeps the CTAs level where round-robin left the slowest one with
+// 1.6 times the average work.
+struct TileSchedule {
+  const int32_t* start;
+  const int2* items;
+};
+
+template <bool SINGLE>
+struct TileWalk {
+  int idx, end, stride;
+  const int2* items;
+  __device__ TileWalk(const TileSchedule& s, int total_tiles) {
+    if (SINGLE) { idx = blockIdx.x; end = total_tiles; stride = gridDim.x; items = nullptr; }
+    else { idx = s.start[blockIdx.x]; end = s.start[blockIdx.x + 1]; stride = 1; items = s.items; }
+  }
+  __device__ bool valid() const { return idx < end; }
+  __device__ bool has_next() const { return idx + stride < end; }
+  __device__ int2 at(int i) const { return SINGLE ? make_int2(0, i) : items[i]; }
+  __device__ int2 cur() const { return at(idx); }
+  __device__ int2 next() const { return at(idx + stride); }
+  __device__ void advance() { idx += stride; }
+};
 
 __device__ __forceinline__ void raise_wait_expired(int32_t* status) {
   if (status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
@@ -115,8 +143,8 @@ __device__ __forceinline__ float adam1(const StepScalars& sc, float inv_b1, floa
 // are prefetched into registers (64 KB in flight per SM) while the current one is computed.
 template <int BN, bool SINGLE>
 __global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
-project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table, int nprob,
-                    int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
+project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
+                    const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
   using S = K1Smem<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -146,23 +174,18 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // tile -> (problem, r block, n block); consecutive tiles share the n block, so that the G tile
+  // tile -> (r block, n block) of its problem; consecutive tiles share the n block, so that the G tile
   // one of them brings from HBM serves the others from L2
-  auto locate = [&](int tile, int& pi) -> const TcProblem* {
-    if (SINGLE) return probs;
-    while (pi + 1 < nprob && tile >= probs[pi].k1_tile0 + probs[pi].k1_tiles) ++pi;
-    return probs + pi;
-  };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int pi = 0;
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-        const TcProblem* p = locate(tile, pi);
-        const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
+      for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance()) {
+        const int2 item = tw.cur();
+        const TcProblem* p = probs + item.x;
+        const int local = item.y, rblocks = p->k1_rblocks;
         const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
         const int kblocks = (p->m + kBK - 1) / kBK;
         const CUtensorMap* mapP = &p->mapP;
@@ -177,14 +200,14 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         // staged loads only see L2 latency.  P~ was just written by the dequantize kernel and is in L2.
         const CUtensorMap* mapG3n = nullptr;
         int n0_2 = 0, kblocks2 = 0;
-        if (tile + (int)gridDim.x < total_tiles) {
-          int pi2 = pi;
-          const TcProblem* p2 = locate(tile + gridDim.x, pi2);
-          n0_2 = ((tile + (int)gridDim.x - p2->k1_tile0) / p2->k1_rblocks) * BN;
+        if (tw.has_next()) {
+          const int2 item2 = tw.next();
+          const TcProblem* p2 = probs + item2.x;
+          n0_2 = (item2.y / p2->k1_rblocks) * BN;
           kblocks2 = (p2->m + kBK - 1) / kBK;
           if (n0_2 + 64 <= p2->n_whole) mapG3n = &p2->mapG3;
         }
-        if (tile == (int)blockIdx.x && n0 + 64 <= p->n_whole) {
+        if (it == 0 && n0 + 64 <= p->n_whole) {
           for (int kb = 0; kb < min(kPrefetch, kblocks); ++kb) tma_prefetch_l2_3d(mapG3, 0, kb * kBK, n0 / 64);
         }
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -224,11 +247,10 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       constexpr uint32_t idesc = umma_idesc_bf16(kTileM, BN, true, true);
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), kBoxBytes, 1024);
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
-      int pi = 0;
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
-        const TcProblem* p = locate(tile, pi);
+      for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
+        const TcProblem* p = probs + tw.cur().x;
         const int kblocks = (p->m + kBK - 1) / kBK;
         const uint32_t ab = tcount & 1;
         if (!mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
@@ -257,12 +279,12 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     const int lcol = 2 * (lane & 3);                 // first column of the thread's pair within a group of 8
     const uint32_t lane_addr = (uint32_t)(q * 32 + hh * 16) << 16;
     const float inv_b1 = 1.0f / sc.bias1, inv_b2 = 1.0f / sc.bias2;
-    int pi = 0;
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
-      const TcProblem* p = locate(tile, pi);
-      const int local = tile - p->k1_tile0, rblocks = p->k1_rblocks;
+    for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
+      const int2 item = tw.cur();
+      const TcProblem* p = probs + item.x;
+      const int local = item.y, rblocks = p->k1_rblocks;
       const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
       const int pn = p->n;
       const int nch = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
@@ -464,8 +486,8 @@ __device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& g
 
 template <bool SINGLE>
 __global__ void __launch_bounds__(K2Smem::kThreads, 1)
-backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table, int nprob,
-                      int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
+backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
+                      const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
   using S = K2Smem;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -500,22 +522,17 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // tile -> (problem, m block, n block); consecutive tiles share the n block of N_b
-  auto locate = [&](int tile, int& pi) -> const TcProblem* {
-    if (SINGLE) return probs;
-    while (pi + 1 < nprob && tile >= probs[pi].k2_tile0 + probs[pi].k2_tiles) ++pi;
-    return probs + pi;
-  };
+  // tile -> (m block, n block) of its problem; consecutive tiles share the n block of N_b
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int pi = 0;
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
-        const TcProblem* p = locate(tile, pi);
-        const int local = tile - p->k2_tile0, mblocks = p->k2_mblocks;
+      for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
+        const int2 item = tw.cur();
+        const TcProblem* p = probs + item.x;
+        const int local = item.y, mblocks = p->k2_mblocks;
         const int m0 = (local % mblocks) * kTileM, n0 = (local / mblocks) * S::kBN;
         const CUtensorMap* mapW = &p->mapW;
         const CUtensorMap* mapPk = &p->mapPk;
@@ -545,11 +562,10 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       constexpr uint32_t idesc = umma_idesc_bf16(kTileM, S::kBN, false, true);
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), 16, 1024);
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
-      int pi = 0;
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
-        const TcProblem* p = locate(tile, pi);
+      for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
+        const TcProblem* p = probs + tw.cur().x;
         const int kblocks = (p->r + kBK - 1) / kBK;
         const uint32_t ab = tcount & 1;
         if (!mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
@@ -582,12 +598,12 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
     const int row = q * 32 + lane;
     const bool elected = (threadIdx.x == 64);
     const bool no_wd = (sc.lr_wd == 0.0f);
-    int pi = 0;
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++tcount) {
-      const TcProblem* p = locate(tile, pi);
-      const int local = tile - p->k2_tile0, mblocks = p->k2_mblocks;
+    for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
+      const int2 item = tw.cur();
+      const TcProblem* p = probs + item.x;
+      const int local = item.y, mblocks = p->k2_mblocks;
       const int m0 = (local % mblocks) * kTileM, nblk = local / mblocks, n0 = nblk * S::kBN;
       const int pn = p->n, n_tma = p->n_tma_w, ngroups = p->ngroups;
       const int gi = m0 + row;                       // global row
@@ -844,29 +860,29 @@ int set_smem(K kernel, int bytes) {
 int choose_bn(int64_t tiles_at_256) { return tiles_at_256 >= 2 * (int64_t)sm_count() ? 256 : 128; }
 
 template <int BN, bool SINGLE>
-int launch_k1(const TcProblem* single, const TcProblem* table, int nprob, int total_tiles, const StepScalars& sc,
-              int32_t* status, cudaStream_t st) {
+int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
+              int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
   auto kern = project_adam_kernel<BN, SINGLE>;
   int rc = set_smem(kern, K1Smem<BN>::kBytes);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
-  const int grid = total_tiles < sms ? total_tiles : sms;
+  const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
   static const TcProblem dummy{};
-  kern<<<grid, K1Smem<BN>::kThreads, K1Smem<BN>::kBytes, st>>>(single ? *single : dummy, table, nprob, total_tiles, sc, status);
+  kern<<<grid, K1Smem<BN>::kThreads, K1Smem<BN>::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
 
 template <bool SINGLE>
-int launch_k2(const TcProblem* single, const TcProblem* table, int nprob, int total_tiles, const StepScalars& sc,
-              int32_t* status, cudaStream_t st) {
+int launch_k2(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
+              int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
   auto kern = backproject_sr_kernel<SINGLE>;
   int rc = set_smem(kern, K2Smem::kBytes);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
-  const int grid = total_tiles < sms ? total_tiles : sms;
+  const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
   static const TcProblem dummy{};
-  kern<<<grid, K2Smem::kThreads, K2Smem::kBytes, st>>>(single ? *single : dummy, table, nprob, total_tiles, sc, status);
+  kern<<<grid, K2Smem::kThreads, K2Smem::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
@@ -914,10 +930,11 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
   TcProblem prob;
   rc = fill_problem(a, w, &prob, bn);
   if (rc != QG_OK) return rc;
-  rc = bn == 256 ? launch_k1<256, true>(&prob, nullptr, 1, prob.k1_tiles, a.sc, a.status, st)
-                 : launch_k1<128, true>(&prob, nullptr, 1, prob.k1_tiles, a.sc, a.status, st);
+  const TileSchedule none{nullptr, nullptr};
+  rc = bn == 256 ? launch_k1<256, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
+                 : launch_k1<128, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
   if (rc != QG_OK) return rc;
-  return launch_k2<true>(&prob, nullptr, 1, prob.k2_tiles, a.sc, a.status, st);
+  return launch_k2<true>(&prob, nullptr, none, 0, prob.k2_tiles, a.sc, a.status, st);
 }
 
 // ============================================================================================
@@ -927,29 +944,68 @@ struct PlanChunk {
   int first, count;          // items [first, first + count)
   int k1_tiles, k2_tiles, bn;
   int dq_blocks;
+  int k1_grid, k2_grid;
+  size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
 };
 
 struct Plan {
   std::vector<PlanChunk> chunks;
   TcProblem* table_dev = nullptr;
   DequantItem* dq_dev = nullptr;
+  int32_t* sched_dev = nullptr;
   int count = 0;
 };
+
+// Longest-processing-time-first assignment of tiles to `grid` CTAs: tiles in order of decreasing cost (ties
+// keep their order, which keeps tiles that share an operand block next to each other), each to the CTA with
+// the least work so far.  Appends start[grid + 1] and the (problem, tile) pairs to `buf`.
+void schedule_tiles(const std::vector<int2>& tiles, const std::vector<float>& cost, int grid, std::vector<int32_t>& buf,
+                    size_t* start_off, size_t* items_off) {
+  std::vector<int> order(tiles.size());
+  for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost[a] > cost[b]; });
+  using Load = std::pair<float, int>;                         // (work so far, CTA)
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+  for (int c = 0; c < grid; ++c) heap.push({0.f, c});
+  std::vector<std::vector<int>> per_cta((size_t)grid);
+  for (int t : order) {
+    Load l = heap.top();
+    heap.pop();
+    per_cta[(size_t)l.second].push_back(t);
+    heap.push({l.first + cost[t], l.second});
+  }
+  *start_off = buf.size();
+  int32_t run = 0;
+  for (int c = 0; c < grid; ++c) { buf.push_back(run); run += (int32_t)per_cta[(size_t)c].size(); }
+  buf.push_back(run);
+  if (buf.size() & 1) buf.push_back(0);                      // int2 alignment of the pairs
+  *items_off = buf.size();
+  for (int c = 0; c < grid; ++c)
+    for (int t : per_cta[(size_t)c]) { buf.push_back(tiles[t].x); buf.push_back(tiles[t].y); }
+}
 
 // Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b
 // fit both the caller's workspace and a budget chosen so that N_b, written by the first kernel, is
 // still in the 126 MB L2 when the second kernel reads it.
 constexpr size_t kChunkBudget = 56ull << 20;
 
-size_t plan_table_bytes(int32_t count) {
-  return (size_t)count * (sizeof(TcProblem) + round_up(sizeof(DequantItem), 64)) + 256;
+size_t plan_table_bytes(const StepArgs* items, int32_t count) {
+  size_t sched = 0;                                           // int32 words: pairs of every tile + starts per chunk
+  for (int32_t i = 0; i < count; ++i) {
+    const int64_t k1 = ceil_div(items[i].r, kTileM) * ceil_div(items[i].n, 128);
+    const int64_t k2 = ceil_div(items[i].m, kTileM) * ceil_div(items[i].n, K2Smem::kBN);
+    sched += (size_t)(2 * (k1 + k2)) + 2 * (size_t)(sm_count() + 3);
+  }
+  return (size_t)round_up((int64_t)count * sizeof(TcProblem), 256) + (size_t)round_up((int64_t)count * sizeof(DequantItem), 256) +
+         sched * sizeof(int32_t) + 256;
 }
 
 int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t table_bytes, void* workspace,
                 size_t workspace_bytes, Plan** out) {
-  if (table_bytes < plan_table_bytes(count)) return QG_WORKSPACE_TOO_SMALL;
+  if (table_bytes < plan_table_bytes(items, count)) return QG_WORKSPACE_TOO_SMALL;
   std::vector<TcProblem> probs((size_t)count);
   std::vector<DequantItem> dq((size_t)count);
+  std::vector<int32_t> sched;
   Plan* plan = new Plan();
   plan->count = count;
   const size_t budget = workspace_bytes < kChunkBudget ? workspace_bytes : kChunkBudget;
@@ -971,28 +1027,47 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     ch.first = i; ch.count = j - i;
     ch.bn = choose_bn(tiles256);
     size_t off = 0;
+    std::vector<int2> t1, t2;
+    std::vector<float> c1, c2;
     for (int k = i; k < j; ++k) {
       const StepArgs& a = items[k];
       const TcScratch w = carve(reinterpret_cast<char*>(workspace) + off, a.m, a.n, a.r);
       off += tc_workspace_bytes(a.m, a.n, a.r);
       const int rc = fill_problem(a, w, &probs[k], ch.bn);
       if (rc != QG_OK) { delete plan; return rc; }
-      probs[k].k1_tile0 = ch.k1_tiles; ch.k1_tiles += probs[k].k1_tiles;
-      probs[k].k2_tile0 = ch.k2_tiles; ch.k2_tiles += probs[k].k2_tiles;
+      ch.k1_tiles += probs[k].k1_tiles;
+      ch.k2_tiles += probs[k].k2_tiles;
+      // cost of a tile in K blocks of its main loop, plus a constant for its epilogue and hand-over
+      for (int t = 0; t < probs[k].k1_tiles; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(a.m, kBK) + 6.f); }
+      for (int t = 0; t < probs[k].k2_tiles; ++t) { t2.push_back(make_int2(k - i, t)); c2.push_back((float)ceil_div(a.r, kBK) + 6.f); }
       dq[k].P = a.P; dq[k].out = w.Pt;
       dq[k].block0 = ch.dq_blocks;
       dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 8), 256);
       ch.dq_blocks += dq[k].nblocks;
     }
+    ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
+    ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
+    schedule_tiles(t1, c1, ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);
+    if (sched.size() & 1) sched.push_back(0);
+    schedule_tiles(t2, c2, ch.k2_grid, sched, &ch.k2_start_off, &ch.k2_items_off);
+    if (sched.size() & 1) sched.push_back(0);
     plan->chunks.push_back(ch);
     i = j;
   }
   plan->table_dev = reinterpret_cast<TcProblem*>(table_dev);
   plan->dq_dev = reinterpret_cast<DequantItem*>(reinterpret_cast<char*>(table_dev) +
                                                 round_up((int64_t)count * sizeof(TcProblem), 256));
+  plan->sched_dev = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(plan->dq_dev) +
+                                               round_up((int64_t)count * sizeof(DequantItem), 256));
+  if (reinterpret_cast<char*>(plan->sched_dev + sched.size()) > reinterpret_cast<char*>(table_dev) + table_bytes) {
+    delete plan;
+    return QG_WORKSPACE_TOO_SMALL;
+  }
   cudaError_t e = cudaMemcpy(plan->table_dev, probs.data(), (size_t)count * sizeof(TcProblem), cudaMemcpyHostToDevice);
   if (e == cudaSuccess)
     e = cudaMemcpy(plan->dq_dev, dq.data(), (size_t)count * sizeof(DequantItem), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess)
+    e = cudaMemcpy(plan->sched_dev, sched.data(), sched.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) {
     note_cuda_error(e, "cudaMemcpy(plan table)");
     delete plan;
@@ -1012,11 +1087,13 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
     QG_LAUNCH_CHECK();
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 1], st));
     const TcProblem* tab = plan->table_dev + ch.first;
-    int rc = ch.bn == 256 ? launch_k1<256, false>(nullptr, tab, ch.count, ch.k1_tiles, sc, status, st)
-                          : launch_k1<128, false>(nullptr, tab, ch.count, ch.k1_tiles, sc, status, st);
+    const TileSchedule s1{plan->sched_dev + ch.k1_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k1_items_off)};
+    const TileSchedule s2{plan->sched_dev + ch.k2_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k2_items_off)};
+    int rc = ch.bn == 256 ? launch_k1<256, false>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
+                          : launch_k1<128, false>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 2], st));
-    rc = launch_k2<false>(nullptr, tab, ch.count, ch.k2_tiles, sc, status, st);
+    rc = launch_k2<false>(nullptr, tab, s2, ch.k2_grid, ch.k2_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 3], st));
     ++c;
