@@ -166,11 +166,20 @@ QG_API int qgalore_plan_step_timed(const qg_plan* plan, const qg_hyper* h, int32
                             float* kernel_ms, int32_t* kernel_launches);
 
 /* --- Sec. 3.5 "obtain the projection matrix using SVD" + Sec. 3.3 INT4 storage ------------
- * Top-r left singular subspace of G (bf16, m x n) by block subspace iteration with
- * `oversample_cols` extra columns and a Rayleigh-Ritz step, then Quant_4 into P_new.
- * P_fp32 (optional, m x r fp32, pitch r) receives the basis before quantization.
- * If P_prev and sim_dev are given, the similarity of Sec. 3.2 between P_prev and P_new over
- * the leading sim_cols columns is written to *sim_dev. */
+ * Top-r left singular vectors of G (bf16, m x n, pitch ldg) by block subspace iteration on G G^T with a
+ * block of b = r + oversample_cols columns (`iters` multiplications by G G^T, each followed by a block
+ * Gram-Schmidt orthonormalisation) and a Rayleigh-Ritz step (eigenvectors of the projected b x b matrix by
+ * a Jacobi iteration in fp64), then Quant_4 into P_new.  Each column carries the sign that makes its
+ * largest-magnitude entry positive.
+ *   P_new      INT4, m x r, ld == r; written
+ *   P_fp32     optional (may be NULL): m x r fp32, pitch r, receives the vectors before quantization
+ *   P_prev, sim_dev  if both given, the similarity of Sec. 3.2 between P_prev and P_new over the leading
+ *              sim_cols columns (<= 0: all) is written to *sim_dev
+ *   workspace  qgalore_workspace_bytes(QG_OP_REFRESH, m, n, b) bytes, 256-byte aligned
+ *   status_dev optional; receives QG_DEV_NOT_CONVERGED / QG_DEV_BAD_FACTOR
+ * Shape rules: r % 32 == 0, b % 64 == 0, b <= min(m, n), b <= 4096.  Typical use: b = 2 r, iters = 12.
+ * The Adam moments and the step count are not touched.  The random start block is drawn from Philox
+ * keyed by `seed`. */
 QG_API int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r,
                              int32_t iters, int32_t oversample_cols, uint64_t seed,
                              const qg_qtensor* P_new, float* P_fp32,

@@ -350,10 +350,16 @@ def refresh_subspace(G: torch.Tensor, r: int, iters: int = 12, oversample_cols: 
                      status: torch.Tensor | None = None, stream=None) -> QTensor:
     """New INT4 projection matrix from the top-r left singular subspace of G (Sec. 3.5, Sec. 3.3)."""
     m, n = G.shape
-    if oversample_cols is None:
-        oversample_cols = min(r, min(m, n) - r)
+    if oversample_cols is None:     # block of 2 r columns, in whole panels of 64, never wider than the matrix
+        block = min((2 * r + 63) // 64 * 64, min(m, n) // 64 * 64)
+        oversample_cols = max(block - r, 0)
     if P_new is None:
         P_new = QTensor.empty(m, r, 4, G.device)
+        if P_new.ld != r:               # the refresh writes a densely packed P (ld == r)
+            ng = (r + GROUP - 1) // GROUP
+            P_new = QTensor(torch.full((m, r // 2), 0x88, dtype=torch.uint8, device=G.device),
+                            torch.zeros((m, ng), dtype=torch.float32, device=G.device),
+                            torch.zeros((m, ng), dtype=torch.float32, device=G.device), m, r, r, 4)
     if workspace is None:
         workspace = torch.empty(workspace_bytes(QG_OP_REFRESH, m, n, r + oversample_cols), dtype=torch.uint8,
                                 device=G.device)

@@ -23,9 +23,9 @@ int launch_project_step_simt(const StepArgs& a, cudaStream_t st);
 size_t simt_workspace_bytes(int64_t m, int64_t n, int64_t r);
 int launch_project_step_tc(const StepArgs& a, cudaStream_t st);
 size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r);
-int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters,
-                   uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes,
-                   int32_t* status, cudaStream_t st);
+int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
+                   uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
+                   cudaStream_t st);
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b);
 struct Plan;
 size_t plan_table_bytes(const StepArgs* items, int32_t count);
@@ -109,7 +109,11 @@ size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r) {
       const size_t a = simt_workspace_bytes(m, n, r), b = tc_workspace_bytes(m, n, r);
       return a > b ? a : b;
     }
-    case QG_OP_REFRESH: return n > 0 ? refresh_workspace_bytes(m, n, r) : 0;
+    case QG_OP_REFRESH: {
+      if (n <= 0) return 0;
+      const size_t a = refresh_workspace_bytes(m, n, r), s = similarity_workspace_bytes(m, r);
+      return a > s ? a : s;
+    }
     case QG_OP_SIMILARITY: return similarity_workspace_bytes(m, r);
     default: return 0;
   }
@@ -271,6 +275,40 @@ void qgalore_plan_destroy(qg_plan* plan) {
   if (!plan) return;
   plan_destroy(plan->impl);
   delete plan;
+}
+
+int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
+                             int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
+                             const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  if (!G || !workspace || m <= 0 || n <= 0 || r <= 0 || ldg < n || iters < 0 || oversample_cols < 0)
+    return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(P_new, 4);
+  if (rc != QG_OK) return rc;
+  if (P_new->rows != m || P_new->cols != r || P_new->ld != r) return QG_INVALID_ARGUMENT;
+  if (P_prev) {
+    rc = check_qtensor(P_prev, 4);
+    if (rc != QG_OK) return rc;
+    if (P_prev->rows != m || P_prev->cols != r) return QG_INVALID_ARGUMENT;
+  }
+  const int64_t b = r + oversample_cols;
+  // the block is handled in panels of 64 columns and cannot be wider than the matrix is tall or wide
+  if (r % 32 != 0 || b % 64 != 0 || b > m || b > n || b > 4096 || m > (1ll << 31) - 1 || n > (1ll << 31) - 1)
+    return QG_UNSUPPORTED_SHAPE;
+  if (!aligned16(G) || ldg % 8 != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return QG_MISALIGNED;
+  if (P_fp32 && !aligned16(P_fp32)) return QG_MISALIGNED;
+  if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
+  if (workspace_bytes < qgalore_workspace_bytes(QG_OP_REFRESH, m, n, b)) return QG_WORKSPACE_TOO_SMALL;
+  constexpr int kJacobiSweeps = 12;
+  rc = launch_refresh(G, ldg, m, n, r, b, iters, kJacobiSweeps, seed, P_new, P_fp32, workspace, workspace_bytes,
+                      status_dev, (cudaStream_t)stream);
+  if (rc != QG_OK) return rc;
+  if (P_prev && sim_dev) {
+    const int32_t c = (sim_cols <= 0 || sim_cols > r) ? (int32_t)r : sim_cols;
+    // the refresh has finished with its scratch by the time this runs on the same stream
+    return launch_similarity(P_prev, P_new, c, sim_dev, workspace, (cudaStream_t)stream);
+  }
+  return QG_OK;
 }
 
 int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,

@@ -1,0 +1,396 @@
+// Subspace refresh (Sec. 3.5: "obtain the projection matrix using SVD"; Sec. 3.3: INT4 storage).
+//
+// The top-r left singular vectors of the gradient G (m x n, bf16) are found without a full SVD:
+// block subspace iteration on G G^T with a block of b = r + oversample columns, followed by a
+// Rayleigh-Ritz step that rotates the converged block onto the singular vectors.
+//
+//   Q <- orth(Gaussian m x b)
+//   repeat iters times:   Z = G^T Q  (n x b);   Y = G Z  (m x b);   Q <- orth(Y)
+//   Z = G^T Q;   T = Z^T Z  (b x b, fp64);   T = X diag(lambda) X^T;   P = Q X[:, top r]
+//
+// Everything heavy is a GEMM (one generic fp32 kernel, fp64 accumulation for T).  orth() is block
+// Gram-Schmidt over panels of 64 columns, each projection done twice, the panel itself by two rounds of
+// Cholesky QR.  The eigenvectors of T come from a one-sided (Hestenes) Jacobi iteration in fp64 with a
+// round-robin pair ordering, one launch per round of b/2 disjoint column pairs.  Each column of P is then
+// given the sign that makes its largest entry positive, and P is quantized to INT4 (Quant_4).
+//
+// The arithmetic is plain fp32/fp64 on the CUDA cores: the singular values next to the r-th one sit in the
+// noise bulk of the gradient with relative gaps of 1e-4..1e-3, and resolving that subspace to 1e-2 rad
+// needs fp32-faithful products (bf16 tensor-core products do not get there).
+#include <cmath>
+
+#include "qg_common.cuh"
+
+namespace qg {
+
+namespace {
+
+constexpr int kPanel = 64;    // columns orthonormalised together
+constexpr int kGT = 64;       // GEMM tile (square), 16 x 16 threads, 4 x 4 outputs each
+constexpr int kGK = 16;
+
+__device__ __forceinline__ float ld_as_float(const uint16_t* p, int64_t i) { return bf16_bits_to_float(p[i]); }
+__device__ __forceinline__ float ld_as_float(const float* p, int64_t i) { return p[i]; }
+
+// C[M x N] = alpha * A * B + beta * C.  A(i, k) = A[i * sa_m + k * sa_k], B(k, j) = B[k * sb_k + j * sb_n],
+// C(i, j) = C[i * ldc + j].  TA is uint16_t (bfloat16 bits) or float; ACC/TC float or double.
+template <class TA, class ACC, class TC>
+__global__ void __launch_bounds__(256)
+gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* __restrict__ B, int64_t sb_k, int64_t sb_n,
+            TC* __restrict__ C, int64_t ldc, int M, int N, int K, ACC alpha, ACC beta) {
+  __shared__ __align__(16) float As[kGK][kGT + 4];
+  __shared__ __align__(16) float Bs[kGK][kGT + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int64_t m0 = (int64_t)blockIdx.y * kGT, n0 = (int64_t)blockIdx.x * kGT;
+  ACC acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = (ACC)0;
+  const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
+  for (int k0 = 0; k0 < K; k0 += kGK) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      int mm, kk;
+      if (a_m_fast) { mm = tid & 63; kk = (tid >> 6) + 4 * e; } else { kk = tid & 15; mm = (tid >> 4) + 16 * e; }
+      const int64_t gm = m0 + mm, gk = k0 + kk;
+      As[kk][mm] = (gm < M && gk < K) ? ld_as_float(A, gm * sa_m + gk * sa_k) : 0.f;
+      int nn, kb;
+      if (b_n_fast) { nn = tid & 63; kb = (tid >> 6) + 4 * e; } else { kb = tid & 15; nn = (tid >> 4) + 16 * e; }
+      const int64_t gn = n0 + nn, gkb = k0 + kb;
+      Bs[kb][nn] = (gn < N && gkb < K) ? B[gkb * sb_k + gn * sb_n] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kGK; ++kk) {
+      const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] += (ACC)a[i] * (ACC)b[j];
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t gm = m0 + ty * 4 + i;
+    if (gm >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t gn = n0 + tx * 4 + j;
+      if (gn >= N) continue;
+      TC* c = C + gm * ldc + gn;
+      const ACC v = alpha * acc[i][j] + (beta != (ACC)0 ? beta * (ACC)(*c) : (ACC)0);
+      *c = (TC)v;
+    }
+  }
+}
+
+template <class TA, class ACC, class TC>
+int gemm(const TA* A, int64_t sa_m, int64_t sa_k, const float* B, int64_t sb_k, int64_t sb_n, TC* C, int64_t ldc, int64_t M,
+         int64_t N, int64_t K, ACC alpha, ACC beta, cudaStream_t st) {
+  if (M <= 0 || N <= 0) return QG_OK;
+  dim3 grid((unsigned)ceil_div(N, kGT), (unsigned)ceil_div(M, kGT));
+  gemm_kernel<TA, ACC, TC><<<grid, 256, 0, st>>>(A, sa_m, sa_k, B, sb_k, sb_n, C, ldc, (int)M, (int)N, (int)K, alpha, beta);
+  QG_LAUNCH_CHECK();
+  return QG_OK;
+}
+
+// ---- Gaussian start block: Q[i][j] ~ N(0, 1) from Philox4x32-10 (counter (j / 4, i, 0, 0x51)) and Box-Muller
+__global__ void __launch_bounds__(256)
+gaussian_kernel(float* __restrict__ Q, int64_t ld, int64_t rows, int64_t cols, uint32_t seed_lo, uint32_t seed_hi) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t quads = cols / 4;
+  if (idx >= rows * quads) return;
+  const int64_t i = idx / quads, jq = idx % quads;
+  const uint4 x = philox4x32_10(make_uint4((uint32_t)jq, (uint32_t)i, 0u, 0x51u), make_uint2(seed_lo, seed_hi));
+  const float u0 = ((float)x.x + 0.5f) * 2.3283064365386963e-10f, u1 = ((float)x.y + 0.5f) * 2.3283064365386963e-10f;
+  const float u2 = ((float)x.z + 0.5f) * 2.3283064365386963e-10f, u3 = ((float)x.w + 0.5f) * 2.3283064365386963e-10f;
+  const float r0 = sqrtf(-2.f * logf(u0)), r1 = sqrtf(-2.f * logf(u2));
+  float s0, c0, s1, c1;
+  sincospif(2.f * u1, &s0, &c0);
+  sincospif(2.f * u3, &s1, &c1);
+  *reinterpret_cast<float4*>(Q + i * ld + 4 * jq) = make_float4(r0 * c0, r0 * s0, r1 * c1, r1 * s1);
+}
+
+// ---- Cholesky factor of a 64 x 64 Gram matrix and the inverse of the factor, one CTA of 64 threads, fp64.
+// S (row-major fp32) = L L^T;  Linv = L^-1 (lower triangular, row-major fp32).  A non-positive pivot raises
+// QG_DEV_BAD_FACTOR and is replaced by a tiny positive number so that the run continues with finite values.
+__global__ void __launch_bounds__(64)
+chol64_inverse_kernel(const float* __restrict__ S, float* __restrict__ Linv, int32_t* __restrict__ status) {
+  __shared__ double L[kPanel][kPanel + 1];
+  const int t = threadIdx.x;
+  for (int i = 0; i < kPanel; ++i) L[i][t] = (double)S[i * kPanel + t];
+  __syncthreads();
+  for (int k = 0; k < kPanel; ++k) {
+    if (t == 0) {
+      double d = L[k][k];
+      if (!(d > 0.0)) { if (status) atomicOr(status, QG_DEV_BAD_FACTOR); d = 1e-30; }
+      L[k][k] = sqrt(d);
+    }
+    __syncthreads();
+    if (t > k) L[t][k] /= L[k][k];
+    __syncthreads();
+    if (t > k)
+      for (int j = k + 1; j <= t; ++j) L[t][j] -= L[t][k] * L[j][k];
+    __syncthreads();
+  }
+  // column t of L^-1 by forward substitution (L x = e_t), kept by its thread
+  double x[kPanel];
+  for (int i = 0; i < kPanel; ++i) {
+    double v = 0.0;
+    if (i >= t) {
+      v = (i == t) ? 1.0 : 0.0;
+      for (int j = t; j < i; ++j) v -= L[i][j] * x[j];
+      v /= L[i][i];
+    }
+    x[i] = v;
+    Linv[i * kPanel + t] = (float)v;
+  }
+}
+
+// ---- one-sided Jacobi on the rows of two b x b fp64 matrices (T symmetric, so its rows are its columns;
+// XT holds X transposed).  Round `rnd` of a sweep pairs the b indices by the round-robin tournament
+// schedule; block k rotates rows (p, q) of T and of XT so that the two rows of T become orthogonal.
+__device__ __forceinline__ void tournament_pair(int nitems, int rnd, int k, int& p, int& q) {
+  const int mod = nitems - 1;
+  if (k == 0) { p = nitems - 1; q = rnd % mod; }
+  else { p = (rnd + k) % mod; q = (rnd - k + mod) % mod; }
+  if (p > q) { const int t = p; p = q; q = t; }
+}
+
+__global__ void __launch_bounds__(128)
+jacobi_round_kernel(double* __restrict__ T, double* __restrict__ XT, int b, int rnd, double* __restrict__ off_max,
+                    const int32_t* __restrict__ done) {
+  if (*done) return;
+  int p, q;
+  tournament_pair(b, rnd, blockIdx.x, p, q);
+  double* tp = T + (int64_t)p * b;
+  double* tq = T + (int64_t)q * b;
+  double a = 0.0, c = 0.0, d = 0.0;
+  for (int i = threadIdx.x; i < b; i += blockDim.x) {
+    const double x = tp[i], y = tq[i];
+    a += x * x; d += y * y; c += x * y;
+  }
+  __shared__ double red[3][4];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+    d += __shfl_xor_sync(0xFFFFFFFFu, d, o);
+    c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+  }
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = a; red[1][threadIdx.x >> 5] = d; red[2][threadIdx.x >> 5] = c; }
+  __syncthreads();
+  a = red[0][0] + red[0][1] + red[0][2] + red[0][3];
+  d = red[1][0] + red[1][1] + red[1][2] + red[1][3];
+  c = red[2][0] + red[2][1] + red[2][2] + red[2][3];
+  const double denom = sqrt(a * d);
+  const double rel = denom > 0.0 ? fabs(c) / denom : 0.0;
+  if (threadIdx.x == 0 && rel > 0.0) {
+    // off_max is only ever compared, so the monotone integer view of a non-negative double serves atomicMax
+    atomicMax(reinterpret_cast<unsigned long long*>(off_max), (unsigned long long)__double_as_longlong(rel));
+  }
+  if (rel < 1e-15) return;
+  const double zeta = (d - a) / (2.0 * c);
+  const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+  const double cs = 1.0 / sqrt(1.0 + tt * tt), sn = cs * tt;
+  double* xp = XT + (int64_t)p * b;
+  double* xq = XT + (int64_t)q * b;
+  for (int i = threadIdx.x; i < b; i += blockDim.x) {
+    const double x = tp[i], y = tq[i];
+    tp[i] = cs * x - sn * y;
+    tq[i] = sn * x + cs * y;
+    const double u = xp[i], v = xq[i];
+    xp[i] = cs * u - sn * v;
+    xq[i] = sn * u + cs * v;
+  }
+}
+
+__global__ void jacobi_sweep_end_kernel(double* off_max, int32_t* done, double tol, int last, int32_t* status) {
+  if (*done) return;
+  if (*off_max <= tol) *done = 1;
+  else if (last && status) atomicOr(status, QG_DEV_NOT_CONVERGED);
+  *off_max = 0.0;
+}
+
+__global__ void __launch_bounds__(256)
+identity64_kernel(double* __restrict__ XT, int b) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < (int64_t)b * b) XT[idx] = (idx / b == idx % b) ? 1.0 : 0.0;
+}
+
+// lambda_j = norm of row j of the rotated T (= |eigenvalue j|); rank_j = its position in descending order
+__global__ void __launch_bounds__(128)
+row_norm_kernel(const double* __restrict__ T, int b, double* __restrict__ lam) {
+  const double* row = T + (int64_t)blockIdx.x * b;
+  double s = 0.0;
+  for (int i = threadIdx.x; i < b; i += blockDim.x) s += row[i] * row[i];
+  __shared__ double red[4];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) lam[blockIdx.x] = sqrt(red[0] + red[1] + red[2] + red[3]);
+}
+
+// Xsel[i][rank_j] = X[i][j] = XT[j][i] for the r largest lambda_j
+__global__ void __launch_bounds__(256)
+select_top_kernel(const double* __restrict__ XT, const double* __restrict__ lam, int b, int r, float* __restrict__ Xsel) {
+  const int j = blockIdx.x;
+  const double lj = lam[j];
+  __shared__ int s_rank;
+  if (threadIdx.x == 0) s_rank = 0;
+  __syncthreads();
+  int cnt = 0;
+  for (int k = threadIdx.x; k < b; k += blockDim.x) {
+    const double lk = lam[k];
+    cnt += (lk > lj || (lk == lj && k < j)) ? 1 : 0;
+  }
+  atomicAdd(&s_rank, cnt);
+  __syncthreads();
+  const int rank = s_rank;
+  if (rank >= r) return;
+  for (int i = threadIdx.x; i < b; i += blockDim.x) Xsel[(int64_t)i * r + rank] = (float)XT[(int64_t)j * b + i];
+}
+
+// Each column of P gets the sign that makes its largest-magnitude entry positive; optional copy to P_out.
+__global__ void __launch_bounds__(256)
+sign_fix_kernel(float* __restrict__ P, int64_t m, int r, float* __restrict__ P_out) {
+  const int j = blockIdx.x;
+  float best = 0.f, bestv = 0.f;
+  for (int64_t i = threadIdx.x; i < m; i += blockDim.x) {
+    const float v = P[i * r + j];
+    if (fabsf(v) > best) { best = fabsf(v); bestv = v; }
+  }
+  __shared__ float sb[256], sv[256];
+  sb[threadIdx.x] = best; sv[threadIdx.x] = bestv;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o && sb[threadIdx.x + o] > sb[threadIdx.x]) { sb[threadIdx.x] = sb[threadIdx.x + o]; sv[threadIdx.x] = sv[threadIdx.x + o]; }
+    __syncthreads();
+  }
+  const float sgn = sv[0] < 0.f ? -1.f : 1.f;
+  for (int64_t i = threadIdx.x; i < m; i += blockDim.x) {
+    const float v = P[i * r + j] * sgn;
+    P[i * r + j] = v;
+    if (P_out) P_out[i * r + j] = v;
+  }
+}
+
+struct RefreshWs {
+  float *Q, *Y, *Z, *Wp, *Cb, *S, *Linv, *Xsel, *P32;
+  double *T, *XT, *lam, *off;
+  int32_t* done;
+};
+
+size_t carve_refresh(void* base, int64_t m, int64_t n, int64_t b, int64_t r, RefreshWs* w) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) { void* p = base ? (char*)base + off : nullptr; off += (size_t)round_up((int64_t)bytes, 256); return p; };
+  RefreshWs t{};
+  t.T = (double*)take((size_t)b * b * 8);
+  t.XT = (double*)take((size_t)b * b * 8);
+  t.lam = (double*)take((size_t)b * 8);
+  t.off = (double*)take(8);
+  t.done = (int32_t*)take(4);
+  t.Q = (float*)take((size_t)m * b * 4);
+  t.Y = (float*)take((size_t)m * b * 4);
+  t.Z = (float*)take((size_t)n * b * 4);
+  t.Wp = (float*)take((size_t)m * kPanel * 4);
+  t.Cb = (float*)take((size_t)b * kPanel * 4);
+  t.S = (float*)take((size_t)kPanel * kPanel * 4);
+  t.Linv = (float*)take((size_t)kPanel * kPanel * 4);
+  t.Xsel = (float*)take((size_t)b * r * 4);
+  t.P32 = (float*)take((size_t)m * r * 4);
+  if (w) *w = t;
+  return off;
+}
+
+// Q <- orthonormal basis of the columns of Y (m x b, both pitch b), panel by panel.
+int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cudaStream_t st) {
+  for (int64_t j0 = 0; j0 < b; j0 += kPanel) {
+    float* Yj = w.Y + j0;
+    float* Qj = w.Q + j0;
+    int rc;
+    for (int pass = 0; pass < 2 && j0 > 0; ++pass) {
+      // C = Q[:, :j0]^T Yj   (j0 x 64);   Yj -= Q[:, :j0] C
+      rc = gemm<float, float, float>(w.Q, 1, b, Yj, b, 1, w.Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st);
+      if (rc != QG_OK) return rc;
+      rc = gemm<float, float, float>(w.Q, b, 1, w.Cb, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st);
+      if (rc != QG_OK) return rc;
+    }
+    // two rounds of Cholesky QR on the panel: Yj -> Wp -> Qj
+    const float* src = Yj; int64_t lds = b;
+    float* dst = w.Wp; int64_t ldd = kPanel;
+    for (int pass = 0; pass < 2; ++pass) {
+      rc = gemm<float, float, float>(src, 1, lds, src, lds, 1, w.S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st);
+      if (rc != QG_OK) return rc;
+      chol64_inverse_kernel<<<1, 64, 0, st>>>(w.S, w.Linv, status);
+      QG_LAUNCH_CHECK();
+      // dst = src * Linv^T:  B(k, j) = Linv[j][k]
+      rc = gemm<float, float, float>(src, lds, 1, w.Linv, 1, kPanel, dst, ldd, m, kPanel, kPanel, 1.f, 0.f, st);
+      if (rc != QG_OK) return rc;
+      src = w.Wp; lds = kPanel; dst = Qj; ldd = b;
+    }
+  }
+  return QG_OK;
+}
+
+}  // namespace
+
+size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b) { return carve_refresh(nullptr, m, n, b, b, nullptr); }
+
+int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
+                   uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
+                   cudaStream_t st) {
+  RefreshWs w;
+  if (carve_refresh(ws, m, n, b, r, &w) > ws_bytes) return QG_WORKSPACE_TOO_SMALL;
+  int rc;
+  // start block
+  {
+    const int64_t threads = m * (b / 4);
+    gaussian_kernel<<<(unsigned)ceil_div(threads, 256), 256, 0, st>>>(w.Y, b, m, b, (uint32_t)seed, (uint32_t)(seed >> 32));
+    QG_LAUNCH_CHECK();
+    rc = orthonormalize(w, m, b, status, st);
+    if (rc != QG_OK) return rc;
+  }
+  for (int it = 0; it <= iters; ++it) {
+    // Z = G^T Q
+    rc = gemm<uint16_t, float, float>(G, 1, ldg, w.Q, b, 1, w.Z, b, n, b, m, 1.f, 0.f, st);
+    if (rc != QG_OK) return rc;
+    if (it == iters) break;
+    // Y = G Z
+    rc = gemm<uint16_t, float, float>(G, ldg, 1, w.Z, b, 1, w.Y, b, m, b, n, 1.f, 0.f, st);
+    if (rc != QG_OK) return rc;
+    rc = orthonormalize(w, m, b, status, st);
+    if (rc != QG_OK) return rc;
+  }
+  // Rayleigh-Ritz: T = Z^T Z in fp64, eigenvectors by one-sided Jacobi
+  rc = gemm<float, double, double>(w.Z, 1, b, w.Z, b, 1, w.T, b, b, b, n, 1.0, 0.0, st);
+  if (rc != QG_OK) return rc;
+  identity64_kernel<<<(unsigned)ceil_div(b * b, 256), 256, 0, st>>>(w.XT, (int)b);
+  QG_LAUNCH_CHECK();
+  QG_CUDA_TRY(cudaMemsetAsync(w.off, 0, 8, st));
+  QG_CUDA_TRY(cudaMemsetAsync(w.done, 0, 4, st));
+  for (int sw = 0; sw < sweeps; ++sw) {
+    for (int rnd = 0; rnd < (int)b - 1; ++rnd) {
+      jacobi_round_kernel<<<(unsigned)(b / 2), 128, 0, st>>>(w.T, w.XT, (int)b, rnd, w.off, w.done);
+      QG_LAUNCH_CHECK();
+    }
+    jacobi_sweep_end_kernel<<<1, 1, 0, st>>>(w.off, w.done, 1e-9, sw == sweeps - 1, status);
+    QG_LAUNCH_CHECK();
+  }
+  row_norm_kernel<<<(unsigned)b, 128, 0, st>>>(w.T, (int)b, w.lam);
+  QG_LAUNCH_CHECK();
+  select_top_kernel<<<(unsigned)b, 256, 0, st>>>(w.XT, w.lam, (int)b, (int)r, w.Xsel);
+  QG_LAUNCH_CHECK();
+  // P = Q Xsel
+  rc = gemm<float, float, float>(w.Q, b, 1, w.Xsel, r, 1, w.P32, r, m, r, b, 1.f, 0.f, st);
+  if (rc != QG_OK) return rc;
+  sign_fix_kernel<<<(unsigned)r, 256, 0, st>>>(w.P32, m, (int)r, P_fp32);
+  QG_LAUNCH_CHECK();
+  return launch_quantize_rtn(4, w.P32, m, r, r, P_new, st);
+}
+
+}  // namespace qg

@@ -73,6 +73,69 @@ def test_similarity_matches_oracle(m, r, c):
     assert abs(same - 1.0) <= 1e-6
 
 
+# ----------------------------------------------------------------------------- refresh
+def run_refresh_case(m, n, r, seed=0, iters=12):
+    gb = synth.GradientModel(m, n, seed=seed, matrix_index=0).sample(1)
+    P_ref, _, sv = O.refresh_subspace(gb, r)
+    dG = g_to_device(gb)
+    P32 = torch.zeros((m, r), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P_new = B.refresh_subspace(dG, r, iters=iters, seed=seed + 1, P_fp32=P32, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device status word"
+    Pg = P32.cpu().numpy().astype(np.float64)
+    assert np.all(np.isfinite(Pg))
+    # orthonormal columns, each with its largest entry positive
+    assert np.abs(Pg.T @ Pg - np.eye(r)).max() <= 1e-4
+    piv = np.argmax(np.abs(Pg), axis=0)
+    assert np.all(Pg[piv, np.arange(r)] > 0)
+    # the subspace is the oracle's (exact SVD) to a largest principal angle below 1e-2 rad
+    angle = O.principal_angle(P_ref, Pg)
+    assert angle < 1e-2, f"largest principal angle {angle:.3e} rad"
+    # it captures the energy of the top-r singular values
+    G = O.bf16_bits_to_f32(gb).astype(np.float64)
+    energy = np.linalg.norm(Pg.T @ G) ** 2
+    assert abs(energy - np.sum(sv[:r] ** 2)) <= 1e-5 * np.sum(sv[:r] ** 2)
+    # the leading, well separated singular vectors agree one by one (up to the sign convention both sides share)
+    lead = np.abs(np.sum(P_ref[:, :8].astype(np.float64) * Pg[:, :8], axis=0))
+    assert lead.min() > 0.999, f"leading vectors: {lead}"
+    # and what was stored is Quant_4 of exactly those vectors
+    want = O.quantize_rtn(P32.cpu().numpy(), 4)
+    got = from_device_q(P_new)
+    assert np.array_equal(got.codes, want.codes) and np.array_equal(got.scales, want.scales)
+    assert np.array_equal(got.zeros, want.zeros)
+    return angle, P_new
+
+
+@pytest.mark.parametrize("m,n,r", [(256, 320, 64), (320, 256, 64), (512, 1376, 128), (768, 768, 256)])
+def test_refresh_subspace_matches_exact_svd(m, n, r):
+    run_refresh_case(m, n, r, seed=m + r)
+
+
+def test_refresh_reports_similarity_with_previous_projection():
+    m, n, r = 256, 512, 64
+    gm = synth.GradientModel(m, n, seed=9, matrix_index=0)
+    dG = g_to_device(gm.sample(1))
+    P1 = B.refresh_subspace(dG, r, seed=1)
+    sim = torch.zeros(1, dtype=torch.float32, device="cuda")
+    dG2 = g_to_device(gm.sample(2))                       # same planted subspace, fresh noise
+    P2 = B.refresh_subspace(dG2, r, seed=2, P_prev=P1, sim_cols=8, sim=sim)
+    torch.cuda.synchronize()
+    want = O.subspace_similarity(from_device_q(P1), from_device_q(P2), 8)
+    assert abs(float(sim.item()) - want) <= 1e-5
+    assert float(sim.item()) > 0.9                         # the leading planted directions persist
+
+
+def test_refresh_rejects_bad_block_widths():
+    dG = torch.zeros((128, 256), dtype=torch.int16, device="cuda")
+    with pytest.raises(B.QgError) as e:
+        B.refresh_subspace(dG, 64, oversample_cols=32)     # block of 96 columns: not a multiple of 64
+    assert e.value.status == B.QG_UNSUPPORTED_SHAPE
+    with pytest.raises(B.QgError) as e:
+        B.refresh_subspace(dG, 64, oversample_cols=128)    # block wider than the matrix is tall
+    assert e.value.status == B.QG_UNSUPPORTED_SHAPE
+
+
 # ----------------------------------------------------------------------------- the step
 def run_step_case(m, n, r, seed=0, step=1, steps_before=0, wd=0.0, impl=None, P=None, matrix_index=1):
     """Teacher-forced single-step parity: upload the oracle's pre-step state, run one GPU step, compare."""
