@@ -238,6 +238,11 @@ QG_API uint64_t qgalore_launch_count(void);
  * product path), 1 the plain CUDA-core kernels kept to cross-check them.  Not thread safe. */
 QG_API int qgalore_debug_set_step_impl(int impl);
 
+/* Test aid: plans created after this call run their back-projection as CTA pairs (tcgen05 cta_group::2,
+ * 256 x 256 tiles per pair) if `on` is non-zero, one CTA per 128 x 256 tile otherwise (the default).  Both give
+ * the same results bit for bit.  Not thread safe. */
+QG_API int qgalore_debug_set_pair_mode(int on);
+
 /* Diagnostic: writes one text line per tensor-core kernel (registers per thread, thread limit, shared
  * memory) as the CUDA runtime reports them for the current device into buf (HOST, NUL-terminated). */
 QG_API int qgalore_debug_kernel_info(char* buf, size_t capacity);

@@ -36,6 +36,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
                     int32_t* launches);
 void plan_destroy(Plan* plan);
 int tc_kernel_info(char* buf, size_t cap);
+int set_pair_mode(int on);
 
 static int g_step_impl = 0;  // 0: tensor-core kernels; 1: CUDA-core kernels (validation aid)
 
@@ -347,6 +348,8 @@ int qgalore_debug_kernel_info(char* buf, size_t capacity) {
   buf[0] = 0;
   return tc_kernel_info(buf, capacity);
 }
+
+int qgalore_debug_set_pair_mode(int on) { return set_pair_mode(on); }
 
 /* Test aid: selects the CUDA-core (1) or the tensor-core (0) kernels of qgalore_project_step. */
 int qgalore_debug_set_step_impl(int impl) {

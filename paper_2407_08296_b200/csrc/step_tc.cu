@@ -23,6 +23,7 @@
 #include <cstring>
 #include <algorithm>
 #include <queue>
+#include <type_traits>
 #include <vector>
 
 #include "sm100_ptx.cuh"
@@ -58,7 +59,7 @@ constexpr int kPrefetch = 10;           // K blocks by which the L2 prefetch of 
 //                                 plain stores instead (n_tma_w = columns the TMA store covers).
 // M, V and N_b are read and written by the Adam epilogue with plain vector accesses.
 struct alignas(64) TcProblem {
-  CUtensorMap mapP, mapG, mapP3, mapG3, mapN3, mapPk, mapW, mapWst;
+  CUtensorMap mapP, mapG, mapP3, mapG3, mapN3, mapN3h, mapPk, mapW, mapWst;
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -74,6 +75,7 @@ struct alignas(64) TcProblem {
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles;
   int32_t k2_mblocks, k2_tiles;
+  int32_t k2_mpairs, k2p_tiles;        // the same in 256-row blocks, for CTA pairs
 };
 static_assert(sizeof(TcProblem) <= 2048, "TcProblem must fit the kernel parameter space");
 
@@ -85,6 +87,7 @@ static_assert(sizeof(TcProblem) <= 2048, "TcProblem must fit the kernel paramete
 struct TileSchedule {
   const int32_t* start;
   const int2* items;
+  int32_t ctas;          // CTAs that share one list (2 when the kernel runs as CTA pairs)
 };
 
 template <bool SINGLE>
@@ -93,7 +96,7 @@ struct TileWalk {
   const int2* items;
   __device__ TileWalk(const TileSchedule& s, int total_tiles) {
     if (SINGLE) { idx = blockIdx.x; end = total_tiles; stride = gridDim.x; items = nullptr; }
-    else { idx = s.start[blockIdx.x]; end = s.start[blockIdx.x + 1]; stride = 1; items = s.items; }
+    else { idx = s.start[blockIdx.x / s.ctas]; end = s.start[blockIdx.x / s.ctas + 1]; stride = 1; items = s.items; }
   }
   __device__ bool valid() const { return idx < end; }
   __device__ bool has_next() const { return idx + stride < end; }
@@ -394,9 +397,22 @@ struct K2Smem {
   static constexpr int kBarOffset = kStages * kStageBytes + kCodeBufs * kCodeBytes;
   static constexpr int kPartOffset = kBarOffset + 256;     // float2 [4 slices][128 rows]: partial min/max
   static constexpr int kBytes = kPartOffset + 4 * kTileM * 8 + 1024;
-  static constexpr int kEpiWarps = 16;                     // 4 lane quarters x 4 column slices of 64
+  static constexpr int kEpiWarps = 16;                     // two groups of 4 lane quarters x 2 column slices of 128
   static constexpr int kEpiThreads = kEpiWarps * 32;
+  static constexpr int kGroupWarps = 8;
+  static constexpr int kGroupThreads = kGroupWarps * 32;
   static constexpr int kThreads = 64 + kEpiThreads;
+};
+
+// The same kernel run by CTA pairs: 256 (m) x 256 (n) per pair, each CTA stages its own 128 rows of A and its
+// half (128 columns) of B.
+struct K2PairSmem : K2Smem {
+  static constexpr int kStages = 4;
+  static constexpr int kBBytes = 2 * kBoxBytes;            // this CTA's 128 (n) x 64 (r) half of B
+  static constexpr int kStageBytes = kABytes + kBBytes;    // 32 KB
+  static constexpr int kBarOffset = kStages * kStageBytes + kCodeBufs * kCodeBytes;
+  static constexpr int kPartOffset = kBarOffset + 256;
+  static constexpr int kBytes = kPartOffset + 4 * kTileM * 8 + 1024;
 };
 
 constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves an integer in the low mantissa bits
@@ -484,11 +500,13 @@ __device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& g
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-template <bool SINGLE>
+template <bool SINGLE, int CTAS>
 __global__ void __launch_bounds__(K2Smem::kThreads, 1)
 backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
                       const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
-  using S = K2Smem;
+  static_assert(CTAS == 1 || !SINGLE, "CTA pairs run from a plan only");
+  using S = typename std::conditional<CTAS == 2, K2PairSmem, K2Smem>::type;
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;   // 0 = the pair's leader, which issues the MMAs
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
@@ -508,21 +526,24 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S::kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], S::kEpiWarps); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], CTAS * S::kGroupWarps); }
     for (int i = 0; i < S::kCodeBufs; ++i) { mbar_init(&code_full[i], 1); mbar_init(&code_empty[i], 1); }
     fence_mbar_init();
     fence_proxy_async_smem();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 512);
-    tmem_relinquish();
+    if (CTAS == 2) { tmem_alloc_pair(tmem_slot, 512); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();              // the peer's barriers exist before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // tile -> (m block, n block) of its problem; consecutive tiles share the n block of N_b
+  // tile -> (m block, n block) of its problem; consecutive tiles share the n block of N_b.  A pair takes two
+  // adjacent m blocks, this CTA the one of its rank; the leader's `full` barriers count the loads of both CTAs
+  // and its `acc_empty` barriers the epilogue warps of both.
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -532,34 +553,34 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
         const int2 item = tw.cur();
         const TcProblem* p = probs + item.x;
-        const int local = item.y, mblocks = p->k2_mblocks;
-        const int m0 = (local % mblocks) * kTileM, n0 = (local / mblocks) * S::kBN;
-        const CUtensorMap* mapW = &p->mapW;
+        const int local = item.y, mblocks = CTAS == 2 ? p->k2_mpairs : p->k2_mblocks;
+        const int m0 = (local % mblocks) * (CTAS * kTileM) + (int)rank * kTileM, n0 = (local / mblocks) * S::kBN;
         const CUtensorMap* mapPk = &p->mapPk;
-        const CUtensorMap* mapN3 = &p->mapN3;
-        const int cb = tcount % S::kCodeBufs;
-        if (!mbar_wait(&code_empty[cb], ((tcount / S::kCodeBufs) & 1) ^ 1)) { ok = false; break; }
-        uint8_t* cbuf = code_base + cb * S::kCodeBytes;
-        mbar_arrive_expect_tx(&code_full[cb], S::kCodeBytes);
-        tma_load_2d(cbuf, mapW, &code_full[cb], n0, m0);
-        tma_load_2d(cbuf + S::kCodeBytes / 2, mapW, &code_full[cb], n0 + 128, m0);
+        const CUtensorMap* mapN3 = CTAS == 2 ? &p->mapN3h : &p->mapN3;
         const int kblocks = (p->r + kBK - 1) / kBK;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % S::kStages;
           if (!mbar_wait(&empty[s], ((it / S::kStages) & 1) ^ 1)) { ok = false; break; }
           uint8_t* sA = stage_base + s * S::kStageBytes;
           uint8_t* sB = sA + S::kABytes;
-          mbar_arrive_expect_tx(&full[s], S::kStageBytes);
-          tma_load_2d(sA, mapPk, &full[s], kb * kBK, m0);
-          tma_load_3d(sB, mapN3, &full[s], 0, kb * kBK, n0 / 64);
+          if (CTAS == 2) {
+            if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * S::kStageBytes);
+            const uint32_t lead_full = mapa_u32(smem_u32(&full[s]), 0);
+            tma_load_2d_pair(sA, mapPk, lead_full, kb * kBK, m0);
+            tma_load_3d_pair(sB, mapN3, lead_full, 0, kb * kBK, n0 / 64 + 2 * (int)rank);
+          } else {
+            mbar_arrive_expect_tx(&full[s], S::kStageBytes);
+            tma_load_2d(sA, mapPk, &full[s], kb * kBK, m0);
+            tma_load_3d(sB, mapN3, &full[s], 0, kb * kBK, n0 / 64);
+          }
         }
       }
       if (!ok) raise_wait_expired(status);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, S::kBN, false, true);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(CTAS * kTileM, S::kBN, false, true);
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), 16, 1024);
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
       uint32_t it = 0, tcount = 0;
@@ -568,44 +589,73 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
         const TcProblem* p = probs + tw.cur().x;
         const int kblocks = (p->r + kBK - 1) / kBK;
         const uint32_t ab = tcount & 1;
-        if (!mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
+        if (!(CTAS == 2 ? mbar_wait_cluster(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)
+                        : mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1))) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + ab * S::kBN;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % S::kStages;
-          if (!mbar_wait(&full[s], (it / S::kStages) & 1)) { ok = false; break; }
+          if (!(CTAS == 2 ? mbar_wait_cluster(&full[s], (it / S::kStages) & 1) : mbar_wait(&full[s], (it / S::kStages) & 1))) {
+            ok = false;
+            break;
+          }
           tc_fence_after_sync();
           // A is K-major (rows of 128 bytes, 16 K indices = 32 bytes further along the row),
           // B is MN-major (16 K indices = two 8-index groups of 1024 bytes)
           const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
           const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, da + k * (32 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
-          umma_commit(&empty[s]);
+          for (int k = 0; k < kBK / 16; ++k) {
+            if (CTAS == 2) umma_bf16_pair(d_tmem, da + k * (32 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
+            else umma_bf16(d_tmem, da + k * (32 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
+          }
+          if (CTAS == 2) umma_commit_pair(&empty[s]); else umma_commit(&empty[s]);
         }
-        if (ok) umma_commit(&acc_full[ab]);
+        if (ok) { if (CTAS == 2) umma_commit_pair(&acc_full[ab]); else umma_commit(&acc_full[ab]); }
       }
       if (!ok) raise_wait_expired(status);
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    // Sixteen warps: warp (quarter q, slice sl) owns accumulator rows 32q..32q+31 and columns
-    // 64*sl..64*sl+63; a row of the tile is one quantization group, so four threads share a group and
-    // combine their minima and maxima through shared memory.  The pre-rounding weights are written
-    // back over the accumulator in tensor memory between the two passes (registers are the scarce
-    // resource with 18 warps on the SM: 5 warps share one 16K-register scheduler partition).
-    const int q = warp & 3, sl = (warp - 2) >> 2;
+    // Sixteen warps in two groups of eight; group g takes the tiles whose accumulator buffer is g, so the
+    // two groups work on different tiles and one fills the other's waits (scale loads, barriers, the
+    // hand-over to the TMA store).  Within a group, warp (quarter q, slice sl) owns accumulator rows
+    // 32q..32q+31 and columns 128*sl..128*sl+127; a row of the tile is one quantization group, so two threads
+    // share a group and combine their minima and maxima through shared memory.  The pre-rounding weights
+    // are written back over the accumulator in tensor memory between the two passes (registers are the
+    // scarce resource with 18 warps on the SM: 5 warps share one 16K-register scheduler partition).
+    const int grp = (warp - 2) >> 3;
+    const int q = warp & 3, sl = ((warp - 2) >> 2) & 1;
     const int row = q * 32 + lane;
-    const bool elected = (threadIdx.x == 64);
+    const bool elected = (threadIdx.x == 64 + grp * S::kGroupThreads);
+    const int bar_id = 1 + grp;
     const bool no_wd = (sc.lr_wd == 0.0f);
+    float2* gpart = part + grp * 2 * kTileM;
+    uint8_t* cbuf = code_base + grp * S::kCodeBytes;   // the group's own buffer for the INT8 codes of its tile
+    // the codes of a tile are fetched by the group itself: the first tile here, each later one as soon as
+    // the previous tile's codes have been consumed (after pass 1), so the fetch overlaps pass 2
+    auto fetch_codes = [&](int2 it2) {
+      const TcProblem* p2 = probs + it2.x;
+      const int mb2 = CTAS == 2 ? p2->k2_mpairs : p2->k2_mblocks;
+      const int m2 = (it2.y % mb2) * (CTAS * kTileM) + (int)rank * kTileM, n2 = (it2.y / mb2) * S::kBN;
+      mbar_arrive_expect_tx(&code_full[grp], S::kCodeBytes);
+      tma_load_2d(cbuf, &p2->mapW, &code_full[grp], n2, m2);
+      tma_load_2d(cbuf + S::kCodeBytes / 2, &p2->mapW, &code_full[grp], n2 + 128, m2);
+    };
+    {
+      TileWalk<SINGLE> first(sched, total_tiles);
+      if (grp == 1) first.advance();
+      if (elected && first.valid()) fetch_codes(first.cur());
+    }
     uint32_t tcount = 0;
     bool ok = true;
     for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
+      if ((int)(tcount & 1) != grp) continue;
       const int2 item = tw.cur();
       const TcProblem* p = probs + item.x;
-      const int local = item.y, mblocks = p->k2_mblocks;
-      const int m0 = (local % mblocks) * kTileM, nblk = local / mblocks, n0 = nblk * S::kBN;
-      const int pn = p->n, n_tma = p->n_tma_w, ngroups = p->ngroups;
+      const int local = item.y, mblocks = CTAS == 2 ? p->k2_mpairs : p->k2_mblocks;
+      const int m0 = (local % mblocks) * (CTAS * kTileM) + (int)rank * kTileM, nblk = local / mblocks, n0 = nblk * S::kBN;
+      const int pn = p->n, ngroups = p->ngroups;
       const int gi = m0 + row;                       // global row
       const bool row_ok = gi < p->m;
       const int ncols = min(S::kBN, pn - n0);        // valid columns of this (possibly ragged) group
@@ -614,59 +664,69 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       float* g_zero = p->w_zeros + (int64_t)gi * ngroups + nblk;
       int8_t* g_codes = p->w_codes + (int64_t)gi * ldw;
       float* dbgW = p->dbgW ? p->dbgW + (int64_t)gi * ldw : nullptr;
-      const CUtensorMap* mapWst = &p->mapWst;
       const uint32_t seed_lo = p->seed_lo, seed_hi = p->seed_hi;
       float s_old = 1.f, z_old = 0.f;
       if (row_ok) { s_old = __ldg(g_scale); z_old = __ldg(g_zero); }
-      const uint32_t ab = tcount & 1;
-      const int cb = tcount % S::kCodeBufs;
-      ok = mbar_wait(&code_full[cb], (tcount / S::kCodeBufs) & 1) && mbar_wait(&acc_full[ab], (tcount >> 1) & 1);
-      ok = named_bar_and(1, S::kEpiThreads, ok);
+      const uint32_t ab = tcount & 1;                // == grp: a group always drains the same accumulator buffer
+      ok = mbar_wait(&code_full[grp], (tcount >> 1) & 1) && mbar_wait(&acc_full[ab], (tcount >> 1) & 1);
+      ok = named_bar_and(bar_id, S::kGroupThreads, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      uint8_t* cbuf = code_base + cb * S::kCodeBytes;
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + ab * S::kBN + sl * 64;
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + ab * S::kBN + sl * 128;
       // codes of columns 16*k16 .. +15 of this row: box (k16 / 8), 16-byte chunk (k16 % 8) ^ (row % 8)
       auto code_ptr = [&](int k16) -> uint4* {
         return reinterpret_cast<uint4*>(cbuf + (k16 >> 3) * (S::kCodeBytes / 2) + row * 128 + (((k16 & 7) ^ (row & 7)) << 4));
       };
 
-      // ---- pass 1: W' of the thread's 64 columns, written back over the accumulator; minimum and maximum
+      // ---- pass 1: W' of the thread's 128 columns, written back over the accumulator; minimum and maximum.
+      // Pieces of 16 columns, the tensor-memory load of the next piece in flight while one is computed.
       const bool fast_dq = __all_sync(0xFFFFFFFFu, fabsf(z_old) <= 4.0e6f);
-      const int myc0 = sl * 64;
+      const int myc0 = sl * 128;
       float mn = INFINITY, mx = -INFINITY;
+      auto pass1_piece = [&](int pc, const uint32_t* acc) {
+        float w[16];
+        const uint4 cw = *code_ptr(sl * 8 + pc);
+        if (fast_dq && no_wd) weights16<true, true>(cw, acc, z_old, s_old, sc.lr_alpha, 0.f, w);
+        else if (fast_dq) weights16<true, false>(cw, acc, z_old, s_old, sc.lr_alpha, sc.lr_wd, w);
+        else weights16<false, false>(cw, acc, z_old, s_old, sc.lr_alpha, sc.lr_wd, w);
+        if (myc0 + 16 * pc + 16 <= ncols) {
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t acc[32];
-        float w[32];
-        tmem_ld_32x32(tacc + half * kChunk, acc);
-        tmem_ld_wait();
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-          const uint4 cw = *code_ptr(sl * 4 + half * 2 + k);
-          float* wk = w + k * 16;
-          if (fast_dq && no_wd) weights16<true, true>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, 0.f, wk);
-          else if (fast_dq) weights16<true, false>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, sc.lr_wd, wk);
-          else weights16<false, false>(cw, acc + 16 * k, z_old, s_old, sc.lr_alpha, sc.lr_wd, wk);
-        }
-        if (myc0 + half * kChunk + kChunk <= ncols) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 2) { mn = min3(mn, w[i], w[i + 1]); mx = max3(mx, w[i], w[i + 1]); }
+          for (int i = 0; i < 16; i += 2) { mn = min3(mn, w[i], w[i + 1]); mx = max3(mx, w[i], w[i + 1]); }
         } else {
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (myc0 + half * kChunk + i < ncols) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
+          for (int i = 0; i < 16; ++i)
+            if (myc0 + 16 * pc + i < ncols) { mn = fminf(mn, w[i]); mx = fmaxf(mx, w[i]); }
         }
+        uint32_t wb[16];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) acc[i] = __float_as_uint(w[i]);
-        tmem_st_32x32(tacc + half * kChunk, acc);
+        for (int i = 0; i < 16; ++i) wb[i] = __float_as_uint(w[i]);
+        tmem_st_32x16(tacc + 16 * pc, wb);
+      };
+      {
+        uint32_t a0[16], a1[16];
+        tmem_ld_32x16(tacc, a0);
+        tmem_ld_wait();
+#pragma unroll 1
+        for (int pc = 0; pc < 8; pc += 2) {
+          tmem_ld_32x16(tacc + 16 * (pc + 1), a1);
+          pass1_piece(pc, a0);
+          tmem_ld_wait();
+          if (pc + 2 < 8) tmem_ld_32x16(tacc + 16 * (pc + 2), a0);
+          pass1_piece(pc + 1, a1);
+          tmem_ld_wait();
+        }
       }
       tmem_st_wait();
-      part[sl * kTileM + row] = make_float2(mn, mx);
-      named_bar_sync(1, S::kEpiThreads);
-#pragma unroll
-      for (int o = 0; o < 4; ++o) {
-        const float2 pm = part[o * kTileM + row];
+      gpart[sl * kTileM + row] = make_float2(mn, mx);
+      fence_proxy_async_smem();                         // the old codes have been read: the buffer may be refilled
+      named_bar_sync(bar_id, S::kGroupThreads);
+      if (elected) {
+        TileWalk<SINGLE> nx = tw;
+        nx.advance();
+        if (nx.valid()) { nx.advance(); if (nx.valid()) fetch_codes(nx.cur()); }
+      }
+      {
+        const float2 pm = gpart[(sl ^ 1) * kTileM + row];
         mn = fminf(mn, pm.x);
         mx = fmaxf(mx, pm.y);
       }
@@ -678,59 +738,63 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       uint32_t kx[10], ky[10];
 #pragma unroll
       for (int i = 0; i < 10; ++i) { kx[i] = seed_lo + (uint32_t)i * 0x9E3779B9u; ky[i] = seed_hi + (uint32_t)i * 0xBB67AE85u; }
+      auto pass2_piece = [&](int pc, const uint32_t* wbits) {
+        const int col = n0 + myc0 + 16 * pc;
+        const float* w = reinterpret_cast<const float*>(wbits);
+        const uint4 x0 = philox_rounds(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
+        const uint4 x1 = philox_rounds(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
+        const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+        const uint4 out = fast_sr ? sr_codes16<true>(w, gp, h) : sr_codes16<false>(w, gp, h);
+        // sixteen new codes of this row, straight to global memory (the two halves of a 32-byte sector are
+        // written by consecutive pieces and merge in L2); the ragged end of a row byte by byte
+        if (row_ok && col + 16 <= pn) {
+          *reinterpret_cast<uint4*>(g_codes + col) = out;
+        } else if (row_ok && col < pn) {
+          const uint32_t o4[4] = {out.x, out.y, out.z, out.w};
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t wbits[32];
-        tmem_ld_32x32(tacc + half * kChunk, wbits);
-        tmem_ld_wait();
-        if (half == 1) {                              // last read of this accumulator buffer
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&acc_empty[ab]);
+          for (int e = 0; e < 15; ++e)
+            if (col + e < pn) g_codes[col + e] = (int8_t)((o4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
         }
+        if (dbgW != nullptr && row_ok) {
 #pragma unroll
-        for (int kk = 0; kk < 2; ++kk) {
-          const int k16 = half * 2 + kk;
-          const int col = n0 + myc0 + 16 * k16;
-          const float* w = reinterpret_cast<const float*>(wbits) + 16 * kk;
-          const uint4 x0 = philox_rounds(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
-          const uint4 x1 = philox_rounds(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
-          const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-          const uint4 out = fast_sr ? sr_codes16<true>(w, gp, h) : sr_codes16<false>(w, gp, h);
-          *code_ptr(sl * 4 + k16) = out;
-          if (row_ok && (col == n_tma || dbgW != nullptr)) {   // ragged tail (at most 15 columns), test tap
-            const uint32_t o4[4] = {out.x, out.y, out.z, out.w};
-#pragma unroll
-            for (int e = 0; e < 16; ++e) {
-              if (col + e < pn) {
-                if (col == n_tma) g_codes[col + e] = (int8_t)((o4[e >> 2] >> (8 * (e & 3))) & 0xFFu);
-                if (dbgW) dbgW[col + e] = w[e];
-              }
+          for (int e = 0; e < 16; ++e)
+            if (col + e < pn) dbgW[col + e] = w[e];
+        }
+      };
+      {
+        uint32_t a0[16], a1[16];
+        tmem_ld_32x16(tacc, a0);
+        tmem_ld_wait();
+#pragma unroll 1
+        for (int pc = 0; pc < 8; pc += 2) {
+          tmem_ld_32x16(tacc + 16 * (pc + 1), a1);
+          pass2_piece(pc, a0);
+          tmem_ld_wait();
+          if (pc + 2 < 8) {
+            tmem_ld_32x16(tacc + 16 * (pc + 2), a0);
+          } else {                                      // every read of this accumulator buffer has landed
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+              if (CTAS == 2) mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[ab]), 0));
+              else mbar_arrive(&acc_empty[ab]);
             }
           }
+          pass2_piece(pc + 1, a1);
+          tmem_ld_wait();
         }
       }
 
-      // ---- coalesced write-back of the tile's codes
-      fence_proxy_async_smem();
-      named_bar_sync(1, S::kEpiThreads);
-      if (elected) {
-        if (n0 < n_tma) tma_store_2d(mapWst, cbuf, n0, m0);
-        if (n0 + 128 < n_tma) tma_store_2d(mapWst, cbuf + S::kCodeBytes / 2, n0 + 128, m0);
-        tma_commit_group();
-        tma_wait_group_read<0>();
-        mbar_arrive(&code_empty[cb]);
-      }
     }
-    if (elected) tma_wait_group<0>();
     if (!ok && lane == 0) raise_wait_expired(status);
   }
 
   tc_fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();              // neither CTA leaves while the other may still signal it
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 512);
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, 512); else tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -812,6 +876,7 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   ok &= make_map_chunked(&p->mapP3, w.Pt, a.m, r_whole > 0 ? r_whole / 64 : 1, a.r, kBK, 2);
   ok &= make_map_chunked(&p->mapG3, a.G, a.m, n_whole > 0 ? n_whole / 64 : 1, a.ldg, kBK, bn / 64);
   ok &= make_map_chunked(&p->mapN3, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 4);
+  ok &= make_map_chunked(&p->mapN3h, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 2);
   p->r_whole = (int32_t)r_whole;
   p->n_whole = (int32_t)n_whole;
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
@@ -837,6 +902,8 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->k1_tiles = p->k1_rblocks * (int32_t)ceil_div(a.n, bn);
   p->k2_mblocks = (int32_t)ceil_div(a.m, kTileM);
   p->k2_tiles = p->k2_mblocks * (int32_t)ceil_div(a.n, K2Smem::kBN);
+  p->k2_mpairs = (p->k2_mblocks + 1) / 2;
+  p->k2p_tiles = p->k2_mpairs * (int32_t)ceil_div(a.n, K2Smem::kBN);
   return QG_OK;
 }
 
@@ -873,16 +940,31 @@ int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedul
   return QG_OK;
 }
 
-template <bool SINGLE>
+template <bool SINGLE, int CTAS>
 int launch_k2(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
               int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
-  auto kern = backproject_sr_kernel<SINGLE>;
-  int rc = set_smem(kern, K2Smem::kBytes);
+  using S = typename std::conditional<CTAS == 2, K2PairSmem, K2Smem>::type;
+  auto kern = backproject_sr_kernel<SINGLE, CTAS>;
+  int rc = set_smem(kern, S::kBytes);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
   const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
   static const TcProblem dummy{};
-  kern<<<grid, K2Smem::kThreads, K2Smem::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
+  if (CTAS == 1) {
+    kern<<<grid, S::kThreads, S::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
+  } else {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(S::kThreads);
+    cfg.dynamicSmemBytes = S::kBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    QG_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, dummy, table, sched, total_tiles, sc, status));
+  }
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
@@ -930,11 +1012,11 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
   TcProblem prob;
   rc = fill_problem(a, w, &prob, bn);
   if (rc != QG_OK) return rc;
-  const TileSchedule none{nullptr, nullptr};
+  const TileSchedule none{nullptr, nullptr, 1};
   rc = bn == 256 ? launch_k1<256, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
                  : launch_k1<128, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
   if (rc != QG_OK) return rc;
-  return launch_k2<true>(&prob, nullptr, none, 0, prob.k2_tiles, a.sc, a.status, st);
+  return launch_k2<true, 1>(&prob, nullptr, none, 0, prob.k2_tiles, a.sc, a.status, st);
 }
 
 // ============================================================================================
@@ -942,9 +1024,9 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
 // ============================================================================================
 struct PlanChunk {
   int first, count;          // items [first, first + count)
-  int k1_tiles, k2_tiles, bn;
+  int k1_tiles, k2_tiles, k2p_tiles, bn;
   int dq_blocks;
-  int k1_grid, k2_grid;
+  int k1_grid, k2_grid, pairs;
   size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
 };
 
@@ -983,6 +1065,9 @@ void schedule_tiles(const std::vector<int2>& tiles, const std::vector<float>& co
   for (int c = 0; c < grid; ++c)
     for (int t : per_cta[(size_t)c]) { buf.push_back(tiles[t].x); buf.push_back(tiles[t].y); }
 }
+
+// 1: the back-projection of a plan runs as CTA pairs (cta_group::2); 0: one CTA per tile.  Read when a plan is created.
+int g_pair_mode = 0;
 
 // Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b
 // fit both the caller's workspace and a budget chosen so that N_b, written by the first kernel, is
@@ -1039,17 +1124,21 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       ch.k2_tiles += probs[k].k2_tiles;
       // cost of a tile in K blocks of its main loop, plus a constant for its epilogue and hand-over
       for (int t = 0; t < probs[k].k1_tiles; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(a.m, kBK) + 6.f); }
-      for (int t = 0; t < probs[k].k2_tiles; ++t) { t2.push_back(make_int2(k - i, t)); c2.push_back((float)ceil_div(a.r, kBK) + 6.f); }
+      const int k2n = g_pair_mode ? probs[k].k2p_tiles : probs[k].k2_tiles;
+      for (int t = 0; t < k2n; ++t) { t2.push_back(make_int2(k - i, t)); c2.push_back((float)ceil_div(a.r, kBK) + 6.f); }
+      ch.k2p_tiles += probs[k].k2p_tiles;
       dq[k].P = a.P; dq[k].out = w.Pt;
       dq[k].block0 = ch.dq_blocks;
       dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 8), 256);
       ch.dq_blocks += dq[k].nblocks;
     }
     ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
-    ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
+    ch.pairs = g_pair_mode;
+    if (ch.pairs) ch.k2_grid = 2 * (ch.k2p_tiles < sm_count() / 2 ? ch.k2p_tiles : sm_count() / 2);   // CTA pairs
+    else ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
     schedule_tiles(t1, c1, ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);
     if (sched.size() & 1) sched.push_back(0);
-    schedule_tiles(t2, c2, ch.k2_grid, sched, &ch.k2_start_off, &ch.k2_items_off);
+    schedule_tiles(t2, c2, ch.pairs ? ch.k2_grid / 2 : ch.k2_grid, sched, &ch.k2_start_off, &ch.k2_items_off);
     if (sched.size() & 1) sched.push_back(0);
     plan->chunks.push_back(ch);
     i = j;
@@ -1087,13 +1176,15 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
     QG_LAUNCH_CHECK();
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 1], st));
     const TcProblem* tab = plan->table_dev + ch.first;
-    const TileSchedule s1{plan->sched_dev + ch.k1_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k1_items_off)};
-    const TileSchedule s2{plan->sched_dev + ch.k2_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k2_items_off)};
+    const TileSchedule s1{plan->sched_dev + ch.k1_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k1_items_off), 1};
+    const TileSchedule s2{plan->sched_dev + ch.k2_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k2_items_off),
+                          ch.pairs ? 2 : 1};
     int rc = ch.bn == 256 ? launch_k1<256, false>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
                           : launch_k1<128, false>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 2], st));
-    rc = launch_k2<false>(nullptr, tab, s2, ch.k2_grid, ch.k2_tiles, sc, status, st);
+    rc = ch.pairs ? launch_k2<false, 2>(nullptr, tab, s2, ch.k2_grid, ch.k2p_tiles, sc, status, st)
+                  : launch_k2<false, 1>(nullptr, tab, s2, ch.k2_grid, ch.k2_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 3], st));
     ++c;
@@ -1128,6 +1219,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
 }
 
 void plan_destroy(Plan* plan) { delete plan; }
+int set_pair_mode(int on) { g_pair_mode = on ? 1 : 0; return QG_OK; }
 
 // Registers, thread limit and shared memory of the tensor-core kernels as the loaded module reports them.
 int tc_kernel_info(char* buf, size_t cap) {
@@ -1149,8 +1241,9 @@ int tc_kernel_info(char* buf, size_t cap) {
   add("project_adam<256,single>", (const void*)project_adam_kernel<256, true>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
   add("project_adam<128,table>", (const void*)project_adam_kernel<128, false>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
   add("project_adam<256,table>", (const void*)project_adam_kernel<256, false>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
-  add("backproject_sr<single>", (const void*)backproject_sr_kernel<true>, K2Smem::kThreads, K2Smem::kBytes);
-  add("backproject_sr<table>", (const void*)backproject_sr_kernel<false>, K2Smem::kThreads, K2Smem::kBytes);
+  add("backproject_sr<single>", (const void*)backproject_sr_kernel<true, 1>, K2Smem::kThreads, K2Smem::kBytes);
+  add("backproject_sr<table>", (const void*)backproject_sr_kernel<false, 1>, K2Smem::kThreads, K2Smem::kBytes);
+  add("backproject_sr<table, pairs>", (const void*)backproject_sr_kernel<false, 2>, K2Smem::kThreads, K2PairSmem::kBytes);
   return QG_OK;
 }
 
