@@ -242,6 +242,9 @@ QG_API int qgalore_debug_set_step_impl(int impl);
  * 256 x 256 tiles per pair) if `on` is non-zero, one CTA per 128 x 256 tile otherwise (the default).  Both give
  * the same results bit for bit.  Not thread safe. */
 QG_API int qgalore_debug_set_pair_mode(int on);
+/* Test aid: scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks
+ * mean fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
+QG_API int qgalore_debug_set_chunk_budget(size_t bytes);
 
 /* Diagnostic: writes one text line per tensor-core kernel (registers per thread, thread limit, shared
  * memory) as the CUDA runtime reports them for the current device into buf (HOST, NUL-terminated). */

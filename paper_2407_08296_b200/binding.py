@@ -292,7 +292,7 @@ class StepPlan:
     tensors) and keeps references to the items' tensors, which must not be reallocated while it lives.
     """
 
-    PREFERRED_WORKSPACE = 64 << 20
+    PREFERRED_WORKSPACE = 264 << 20
 
     def __init__(self, items: list[dict], workspace_bytes: int | None = None, device=None):
         self.items = items

@@ -1069,10 +1069,11 @@ void schedule_tiles(const std::vector<int2>& tiles, const std::vector<float>& co
 // 1: the back-projection of a plan runs as CTA pairs (cta_group::2); 0: one CTA per tile.  Read when a plan is created.
 int g_pair_mode = 0;
 
-// Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b
-// fit both the caller's workspace and a budget chosen so that N_b, written by the first kernel, is
-// still in the 126 MB L2 when the second kernel reads it.
-constexpr size_t kChunkBudget = 56ull << 20;
+// Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b fit
+// both the caller's workspace and this budget.  Few, long launches win: with two or three tiles per CTA the
+// fill and drain of the software pipelines cost a third of a launch, which outweighs keeping N_b (written by
+// the first kernel, read by the second) inside the 126 MB L2.
+size_t g_chunk_budget = 256ull << 20;
 
 size_t plan_table_bytes(const StepArgs* items, int32_t count) {
   size_t sched = 0;                                           // int32 words: pairs of every tile + starts per chunk
@@ -1093,7 +1094,7 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
   std::vector<int32_t> sched;
   Plan* plan = new Plan();
   plan->count = count;
-  const size_t budget = workspace_bytes < kChunkBudget ? workspace_bytes : kChunkBudget;
+  const size_t budget = workspace_bytes < g_chunk_budget ? workspace_bytes : g_chunk_budget;
   int i = 0;
   while (i < count) {
     // extent of the chunk
@@ -1220,6 +1221,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
 
 void plan_destroy(Plan* plan) { delete plan; }
 int set_pair_mode(int on) { g_pair_mode = on ? 1 : 0; return QG_OK; }
+int set_chunk_budget(size_t bytes) { g_chunk_budget = bytes; return QG_OK; }
 
 // Registers, thread limit and shared memory of the tensor-core kernels as the loaded module reports them.
 int tc_kernel_info(char* buf, size_t cap) {
