@@ -238,10 +238,11 @@ QG_API uint64_t qgalore_launch_count(void);
  * product path), 1 the plain CUDA-core kernels kept to cross-check them.  Not thread safe. */
 QG_API int qgalore_debug_set_step_impl(int impl);
 
-/* Test aid: plans created after this call run their back-projection as CTA pairs (tcgen05 cta_group::2,
- * 256 x 256 tiles per pair) if `on` is non-zero, one CTA per 128 x 256 tile otherwise (the default).  Both give
- * the same results bit for bit.  Not thread safe. */
-QG_API int qgalore_debug_set_pair_mode(int on);
+/* Test aid: which kernels of plans created after this call run as CTA pairs (tcgen05 cta_group::2, 256 x 256
+ * tiles per pair): bit 0 the back-projection, bit 1 the projection (where every rank of a chunk is a multiple of
+ * 256).  0 = one CTA per 128 x 256 tile; the default is 2.  Every setting gives the same results bit for bit.
+ * Not thread safe. */
+QG_API int qgalore_debug_set_pair_mode(int mask);
 /* Test aid: scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks
  * mean fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
 QG_API int qgalore_debug_set_chunk_budget(size_t bytes);

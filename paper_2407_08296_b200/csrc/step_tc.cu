@@ -39,7 +39,6 @@ constexpr int kBK = 64;                 // K extent of one pipeline stage (eleme
 constexpr int kBoxBytes = 64 * kBK * 2; // one TMA box of an operand: 64 x kBK bf16 = 8 KB
 constexpr int kTileM = 128;             // accumulator rows (TMEM lanes)
 constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
-constexpr int kPrefetch = 10;           // K blocks by which the L2 prefetch of G runs ahead of the staged loads
 
 // One matrix of the step, as the kernels see it.  Tensor maps (row-major tensors, inner extent first):
 //   mapP    P~  bf16 [m][r]       box 64 x 64, swizzle 128   A operand of the projection (2-D, exact bounds)
@@ -59,7 +58,7 @@ constexpr int kPrefetch = 10;           // K blocks by which the L2 prefetch of 
 //                                 plain stores instead (n_tma_w = columns the TMA store covers).
 // M, V and N_b are read and written by the Adam epilogue with plain vector accesses.
 struct alignas(64) TcProblem {
-  CUtensorMap mapP, mapG, mapP3, mapG3, mapN3, mapN3h, mapPk, mapW, mapWst;
+  CUtensorMap mapP, mapG, mapP3, mapG3, mapG3h, mapN3, mapN3h, mapPk, mapW, mapWst;
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -74,6 +73,7 @@ struct alignas(64) TcProblem {
   int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles;
+  int32_t k1_rpairs, k1p_tiles;        // the same in 256-row blocks of r (256-column tiles), for CTA pairs
   int32_t k2_mblocks, k2_tiles;
   int32_t k2_mpairs, k2p_tiles;        // the same in 256-row blocks, for CTA pairs
 };
@@ -119,10 +119,10 @@ __device__ __forceinline__ float sqrt_approx(float x) {
 // ============================================================================================
 // Kernel 1: projection + Adam
 // ============================================================================================
-template <int BN>
+template <int BN, int CTAS = 1>
 struct K1Smem {
   static constexpr int kABytes = 2 * kBoxBytes;            // 128 (r) x 64 (m) bf16
-  static constexpr int kBBytes = (BN / 64) * kBoxBytes;    // BN (n) x 64 (m) bf16
+  static constexpr int kBBytes = (BN / 64 / CTAS) * kBoxBytes;   // this CTA's share of BN (n) x 64 (m) bf16
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kStages = (192 * 1024) / kStageBytes;
   static constexpr int kBarOffset = kStages * kStageBytes;
@@ -144,11 +144,14 @@ __device__ __forceinline__ float adam1(const StepScalars& sc, float inv_b1, floa
 // covers 32 contiguous bytes of a row of M, V (fp32): every global access of the epilogue moves whole
 // 32-byte sectors without staging through shared memory, and M, V of the next two 32-column chunks
 // are prefetched into registers (64 KB in flight per SM) while the current one is computed.
-template <int BN, bool SINGLE>
+template <int BN, bool SINGLE, int CTAS>
 __global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
                     const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
-  using S = K1Smem<BN>;
+  static_assert(CTAS == 1 || (!SINGLE && BN == 256), "CTA pairs run from a plan, on 256-column tiles");
+  using S = K1Smem<BN, CTAS>;
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;   // 0 = the pair's leader, which issues the MMAs
+  constexpr int BNC = BN / CTAS;                 // columns of the B tile this CTA stages
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* stage_base = smem;
@@ -164,21 +167,24 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < S::kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], S::kEpiWarps); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], CTAS * S::kEpiWarps); }
     fence_mbar_init();
     fence_proxy_async_smem();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 2 * BN);
-    tmem_relinquish();
+    if (CTAS == 2) { tmem_alloc_pair(tmem_slot, 2 * BN); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_slot, 2 * BN); tmem_relinquish(); }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();              // the peer's barriers exist before anything signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
   // tile -> (r block, n block) of its problem; consecutive tiles share the n block, so that the G tile
-  // one of them brings from HBM serves the others from L2
+  // one of them brings from HBM serves the others from L2.  A pair takes two adjacent r blocks (this CTA the
+  // one of its rank) and splits the columns of the G tile: each CTA stages its own 128 rows of P~^T and its
+  // half of G, the leader's MMA (M = 256) reads both halves.
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -188,57 +194,55 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance()) {
         const int2 item = tw.cur();
         const TcProblem* p = probs + item.x;
-        const int local = item.y, rblocks = p->k1_rblocks;
-        const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
+        const int local = item.y, rblocks = CTAS == 2 ? p->k1_rpairs : p->k1_rblocks;
+        const int r0 = (local % rblocks) * (CTAS * kTileM) + (int)rank * kTileM;
+        const int n0 = (local / rblocks) * BN + (int)rank * BNC;      // first column this CTA stages
         const int kblocks = (p->m + kBK - 1) / kBK;
         const CUtensorMap* mapP = &p->mapP;
         const CUtensorMap* mapG = &p->mapG;
         const CUtensorMap* mapP3 = &p->mapP3;
-        const CUtensorMap* mapG3 = &p->mapG3;
+        const CUtensorMap* mapG3 = CTAS == 2 ? &p->mapG3h : &p->mapG3;
         // whole-chunk tiles take one 3-D copy per operand; chunks past the end of a 3-D view read as zero
         const bool a3 = (p->r_whole == p->r) || (r0 + kTileM <= p->r_whole);
-        const bool b3 = (p->n_whole == p->n) || (n0 + BN <= p->n_whole);
-        // G comes from HBM with a latency the few shared-memory stages cannot cover; its boxes are
-        // therefore pulled into L2 kPrefetch K blocks ahead (across the tile boundary), so that the
-        // staged loads only see L2 latency.  P~ was just written by the dequantize kernel and is in L2.
-        const CUtensorMap* mapG3n = nullptr;
-        int n0_2 = 0, kblocks2 = 0;
-        if (tw.has_next()) {
-          const int2 item2 = tw.next();
-          const TcProblem* p2 = probs + item2.x;
-          n0_2 = (item2.y / p2->k1_rblocks) * BN;
-          kblocks2 = (p2->m + kBK - 1) / kBK;
-          if (n0_2 + 64 <= p2->n_whole) mapG3n = &p2->mapG3;
-        }
-        if (it == 0 && n0 + 64 <= p->n_whole) {
-          for (int kb = 0; kb < min(kPrefetch, kblocks); ++kb) tma_prefetch_l2_3d(mapG3, 0, kb * kBK, n0 / 64);
-        }
+        const bool b3 = (p->n_whole == p->n) || (n0 + BNC <= p->n_whole);
+        // (An L2 prefetch of G a few K blocks ahead was tried and removed: the extra TMA instruction per K
+        // block cost the single producer thread more than the hidden latency was worth.)
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
-          {
-            const int t = kb + kPrefetch;
-            if (t < kblocks) {
-              if (n0 + 64 <= p->n_whole) tma_prefetch_l2_3d(mapG3, 0, t * kBK, n0 / 64);
-            } else if (mapG3n != nullptr && t - kblocks < kblocks2) {
-              tma_prefetch_l2_3d(mapG3n, 0, (t - kblocks) * kBK, n0_2 / 64);
-            }
-          }
           const int s = it % S::kStages;
           const uint32_t ph = (it / S::kStages) & 1;
           if (!mbar_wait(&empty[s], ph ^ 1)) { ok = false; break; }
           uint8_t* sA = stage_base + s * S::kStageBytes;
           uint8_t* sB = sA + S::kABytes;
-          mbar_arrive_expect_tx(&full[s], S::kStageBytes);
-          if (a3) {
-            tma_load_3d(sA, mapP3, &full[s], 0, kb * kBK, r0 / 64);
-          } else {
+          if (CTAS == 2) {
+            // the leader's barrier counts the bytes of both CTAs; every copy lands in the issuing CTA only
+            if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * S::kStageBytes);
+            const uint32_t lead_full = mapa_u32(smem_u32(&full[s]), 0);
+            if (a3) {
+              tma_load_3d_pair(sA, mapP3, lead_full, 0, kb * kBK, r0 / 64);
+            } else {
 #pragma unroll
-            for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], r0 + 64 * h, kb * kBK);
-          }
-          if (b3) {
-            tma_load_3d(sB, mapG3, &full[s], 0, kb * kBK, n0 / 64);
-          } else {
+              for (int h = 0; h < 2; ++h) tma_load_2d_pair(sA + h * kBoxBytes, mapP, lead_full, r0 + 64 * h, kb * kBK);
+            }
+            if (b3) {
+              tma_load_3d_pair(sB, mapG3, lead_full, 0, kb * kBK, n0 / 64);
+            } else {
 #pragma unroll
-            for (int h = 0; h < BN / 64; ++h) tma_load_2d(sB + h * kBoxBytes, mapG, &full[s], n0 + 64 * h, kb * kBK);
+              for (int h = 0; h < BNC / 64; ++h) tma_load_2d_pair(sB + h * kBoxBytes, mapG, lead_full, n0 + 64 * h, kb * kBK);
+            }
+          } else {
+            mbar_arrive_expect_tx(&full[s], S::kStageBytes);
+            if (a3) {
+              tma_load_3d(sA, mapP3, &full[s], 0, kb * kBK, r0 / 64);
+            } else {
+#pragma unroll
+              for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], r0 + 64 * h, kb * kBK);
+            }
+            if (b3) {
+              tma_load_3d(sB, mapG3, &full[s], 0, kb * kBK, n0 / 64);
+            } else {
+#pragma unroll
+              for (int h = 0; h < BN / 64; ++h) tma_load_2d(sB + h * kBoxBytes, mapG, &full[s], n0 + 64 * h, kb * kBK);
+            }
           }
         }
       }
@@ -246,8 +250,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, BN, true, true);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(CTAS * kTileM, BN, true, true);
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), kBoxBytes, 1024);
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
       uint32_t it = 0, tcount = 0;
@@ -256,22 +260,29 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         const TcProblem* p = probs + tw.cur().x;
         const int kblocks = (p->m + kBK - 1) / kBK;
         const uint32_t ab = tcount & 1;
-        if (!mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
+        if (!(CTAS == 2 ? mbar_wait_cluster(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)
+                        : mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1))) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + ab * BN;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % S::kStages;
-          if (!mbar_wait(&full[s], (it / S::kStages) & 1)) { ok = false; break; }
+          if (!(CTAS == 2 ? mbar_wait_cluster(&full[s], (it / S::kStages) & 1) : mbar_wait(&full[s], (it / S::kStages) & 1))) {
+            ok = false;
+            break;
+          }
           tc_fence_after_sync();
           // both operands are MN-major: 16 K indices = two 8-index groups of 1024 bytes each; the start
           // address field counts 16-byte units, so a stage or K step is an add on the descriptor
           const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
           const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, da + k * (2048 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
-          umma_commit(&empty[s]);
+          for (int k = 0; k < kBK / 16; ++k) {
+            if (CTAS == 2) umma_bf16_pair(d_tmem, da + k * (2048 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
+            else umma_bf16(d_tmem, da + k * (2048 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
+          }
+          if (CTAS == 2) umma_commit_pair(&empty[s]); else umma_commit(&empty[s]);
         }
-        if (ok) umma_commit(&acc_full[ab]);
+        if (ok) { if (CTAS == 2) umma_commit_pair(&acc_full[ab]); else umma_commit(&acc_full[ab]); }
       }
       if (!ok) raise_wait_expired(status);
     }
@@ -287,8 +298,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
       const int2 item = tw.cur();
       const TcProblem* p = probs + item.x;
-      const int local = item.y, rblocks = p->k1_rblocks;
-      const int r0 = (local % rblocks) * kTileM, n0 = (local / rblocks) * BN;
+      const int local = item.y, rblocks = CTAS == 2 ? p->k1_rpairs : p->k1_rblocks;
+      const int r0 = (local % rblocks) * (CTAS * kTileM) + (int)rank * kTileM, n0 = (local / rblocks) * BN;
       const int pn = p->n;
       const int nch = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
       const int cmax = pn - n0 - lcol;               // offset `off` (from n0 + lcol) is a valid column iff off < cmax
@@ -370,16 +381,20 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&acc_empty[ab]);
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[ab]), 0));
+        else mbar_arrive(&acc_empty[ab]);
+      }
     }
     if (!ok && lane == 0) raise_wait_expired(status);
   }
 
   tc_fence_before_sync();
   __syncthreads();
+  if (CTAS == 2) cluster_sync_all();              // neither CTA leaves while the other may still signal it
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 2 * BN);
+    if (CTAS == 2) tmem_dealloc_pair(tmem_base, 2 * BN); else tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 
@@ -875,6 +890,7 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   const int64_t r_whole = a.r & ~int64_t(63), n_whole = a.n & ~int64_t(63);
   ok &= make_map_chunked(&p->mapP3, w.Pt, a.m, r_whole > 0 ? r_whole / 64 : 1, a.r, kBK, 2);
   ok &= make_map_chunked(&p->mapG3, a.G, a.m, n_whole > 0 ? n_whole / 64 : 1, a.ldg, kBK, bn / 64);
+  ok &= make_map_chunked(&p->mapG3h, a.G, a.m, n_whole > 0 ? n_whole / 64 : 1, a.ldg, kBK, 2);
   ok &= make_map_chunked(&p->mapN3, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 4);
   ok &= make_map_chunked(&p->mapN3h, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 2);
   p->r_whole = (int32_t)r_whole;
@@ -900,6 +916,8 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->seed_lo = a.sc.seed_lo; p->seed_hi = a.sc.seed_hi;
   p->k1_rblocks = (int32_t)ceil_div(a.r, kTileM);
   p->k1_tiles = p->k1_rblocks * (int32_t)ceil_div(a.n, bn);
+  p->k1_rpairs = (p->k1_rblocks + 1) / 2;
+  p->k1p_tiles = p->k1_rpairs * (int32_t)ceil_div(a.n, 256);
   p->k2_mblocks = (int32_t)ceil_div(a.m, kTileM);
   p->k2_tiles = p->k2_mblocks * (int32_t)ceil_div(a.n, K2Smem::kBN);
   p->k2_mpairs = (p->k2_mblocks + 1) / 2;
@@ -926,16 +944,31 @@ int set_smem(K kernel, int bytes) {
 // but only pays once there are enough tiles to occupy every SM.
 int choose_bn(int64_t tiles_at_256) { return tiles_at_256 >= 2 * (int64_t)sm_count() ? 256 : 128; }
 
-template <int BN, bool SINGLE>
+template <int BN, bool SINGLE, int CTAS>
 int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
               int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
-  auto kern = project_adam_kernel<BN, SINGLE>;
-  int rc = set_smem(kern, K1Smem<BN>::kBytes);
+  using S = K1Smem<BN, CTAS>;
+  auto kern = project_adam_kernel<BN, SINGLE, CTAS>;
+  int rc = set_smem(kern, S::kBytes);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
   const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
   static const TcProblem dummy{};
-  kern<<<grid, K1Smem<BN>::kThreads, K1Smem<BN>::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
+  if (CTAS == 1) {
+    kern<<<grid, S::kThreads, S::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
+  } else {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(S::kThreads);
+    cfg.dynamicSmemBytes = S::kBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    QG_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, dummy, table, sched, total_tiles, sc, status));
+  }
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
@@ -1013,8 +1046,8 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
   rc = fill_problem(a, w, &prob, bn);
   if (rc != QG_OK) return rc;
   const TileSchedule none{nullptr, nullptr, 1};
-  rc = bn == 256 ? launch_k1<256, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
-                 : launch_k1<128, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
+  rc = bn == 256 ? launch_k1<256, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
+                 : launch_k1<128, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
   if (rc != QG_OK) return rc;
   return launch_k2<true, 1>(&prob, nullptr, none, 0, prob.k2_tiles, a.sc, a.status, st);
 }
@@ -1026,7 +1059,7 @@ struct PlanChunk {
   int first, count;          // items [first, first + count)
   int k1_tiles, k2_tiles, k2p_tiles, bn;
   int dq_blocks;
-  int k1_grid, k2_grid, pairs;
+  int k1_grid, k2_grid, pairs, k1_pairs, k1p_tiles;
   size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
 };
 
@@ -1066,8 +1099,9 @@ void schedule_tiles(const std::vector<int2>& tiles, const std::vector<float>& co
     for (int t : per_cta[(size_t)c]) { buf.push_back(tiles[t].x); buf.push_back(tiles[t].y); }
 }
 
-// 1: the back-projection of a plan runs as CTA pairs (cta_group::2); 0: one CTA per tile.  Read when a plan is created.
-int g_pair_mode = 0;
+// bit 0: the back-projection of a plan runs as CTA pairs (cta_group::2); bit 1: the projection does.  Read when a
+// plan is created.
+int g_pair_mode = 2;
 
 // Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b fit
 // both the caller's workspace and this budget.  Few, long launches win: with two or three tiles per CTA the
@@ -1112,6 +1146,11 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     PlanChunk ch{};
     ch.first = i; ch.count = j - i;
     ch.bn = choose_bn(tiles256);
+    // the projection runs as CTA pairs when asked to, on 256-column tiles, if every rank of the chunk fills
+    // whole 256-row pairs
+    ch.k1_pairs = (g_pair_mode & 2) && ch.bn == 256;
+    for (int k = i; k < j && ch.k1_pairs; ++k)
+      if (items[k].r % 256 != 0) ch.k1_pairs = 0;
     size_t off = 0;
     std::vector<int2> t1, t2;
     std::vector<float> c1, c2;
@@ -1124,8 +1163,10 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       ch.k1_tiles += probs[k].k1_tiles;
       ch.k2_tiles += probs[k].k2_tiles;
       // cost of a tile in K blocks of its main loop, plus a constant for its epilogue and hand-over
-      for (int t = 0; t < probs[k].k1_tiles; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(a.m, kBK) + 6.f); }
-      const int k2n = g_pair_mode ? probs[k].k2p_tiles : probs[k].k2_tiles;
+      const int k1n = ch.k1_pairs ? probs[k].k1p_tiles : probs[k].k1_tiles;
+      for (int t = 0; t < k1n; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(a.m, kBK) + 6.f); }
+      ch.k1p_tiles += probs[k].k1p_tiles;
+      const int k2n = (g_pair_mode & 1) ? probs[k].k2p_tiles : probs[k].k2_tiles;
       for (int t = 0; t < k2n; ++t) { t2.push_back(make_int2(k - i, t)); c2.push_back((float)ceil_div(a.r, kBK) + 6.f); }
       ch.k2p_tiles += probs[k].k2p_tiles;
       dq[k].P = a.P; dq[k].out = w.Pt;
@@ -1133,11 +1174,12 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 8), 256);
       ch.dq_blocks += dq[k].nblocks;
     }
-    ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
-    ch.pairs = g_pair_mode;
+    if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
+    else ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
+    ch.pairs = g_pair_mode & 1;
     if (ch.pairs) ch.k2_grid = 2 * (ch.k2p_tiles < sm_count() / 2 ? ch.k2p_tiles : sm_count() / 2);   // CTA pairs
     else ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
-    schedule_tiles(t1, c1, ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);
+    schedule_tiles(t1, c1, ch.k1_pairs ? ch.k1_grid / 2 : ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);
     if (sched.size() & 1) sched.push_back(0);
     schedule_tiles(t2, c2, ch.pairs ? ch.k2_grid / 2 : ch.k2_grid, sched, &ch.k2_start_off, &ch.k2_items_off);
     if (sched.size() & 1) sched.push_back(0);
@@ -1177,11 +1219,13 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
     QG_LAUNCH_CHECK();
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 1], st));
     const TcProblem* tab = plan->table_dev + ch.first;
-    const TileSchedule s1{plan->sched_dev + ch.k1_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k1_items_off), 1};
+    const TileSchedule s1{plan->sched_dev + ch.k1_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k1_items_off),
+                          ch.k1_pairs ? 2 : 1};
     const TileSchedule s2{plan->sched_dev + ch.k2_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k2_items_off),
                           ch.pairs ? 2 : 1};
-    int rc = ch.bn == 256 ? launch_k1<256, false>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
-                          : launch_k1<128, false>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
+    int rc = ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st)
+             : ch.bn == 256 ? launch_k1<256, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
+                            : launch_k1<128, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 2], st));
     rc = ch.pairs ? launch_k2<false, 2>(nullptr, tab, s2, ch.k2_grid, ch.k2p_tiles, sc, status, st)
@@ -1220,7 +1264,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
 }
 
 void plan_destroy(Plan* plan) { delete plan; }
-int set_pair_mode(int on) { g_pair_mode = on ? 1 : 0; return QG_OK; }
+int set_pair_mode(int mask) { g_pair_mode = mask & 3; return QG_OK; }
 int set_chunk_budget(size_t bytes) { g_chunk_budget = bytes; return QG_OK; }
 
 // Registers, thread limit and shared memory of the tensor-core kernels as the loaded module reports them.
@@ -1239,10 +1283,11 @@ int tc_kernel_info(char* buf, size_t cap) {
     }
     if (n > 0) used = (used + (size_t)n < cap) ? used + (size_t)n : cap - 1;
   };
-  add("project_adam<128,single>", (const void*)project_adam_kernel<128, true>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
-  add("project_adam<256,single>", (const void*)project_adam_kernel<256, true>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
-  add("project_adam<128,table>", (const void*)project_adam_kernel<128, false>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
-  add("project_adam<256,table>", (const void*)project_adam_kernel<256, false>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
+  add("project_adam<128,single>", (const void*)project_adam_kernel<128, true, 1>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
+  add("project_adam<256,single>", (const void*)project_adam_kernel<256, true, 1>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
+  add("project_adam<128,table>", (const void*)project_adam_kernel<128, false, 1>, K1Smem<128>::kThreads, K1Smem<128>::kBytes);
+  add("project_adam<256,table>", (const void*)project_adam_kernel<256, false, 1>, K1Smem<256>::kThreads, K1Smem<256>::kBytes);
+  add("project_adam<256,table,pairs>", (const void*)project_adam_kernel<256, false, 2>, K1Smem<256, 2>::kThreads, K1Smem<256, 2>::kBytes);
   add("backproject_sr<single>", (const void*)backproject_sr_kernel<true, 1>, K2Smem::kThreads, K2Smem::kBytes);
   add("backproject_sr<table>", (const void*)backproject_sr_kernel<false, 1>, K2Smem::kThreads, K2Smem::kBytes);
   add("backproject_sr<table, pairs>", (const void*)backproject_sr_kernel<false, 2>, K2Smem::kThreads, K2PairSmem::kBytes);

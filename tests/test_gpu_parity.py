@@ -273,3 +273,37 @@ def test_plan_free_run_tracks_oracle_moments():
         w_gpu, w_ref = O.dequantize(from_device_q(items[k]["W"])), O.dequantize(ref[k][0])
         lsb = float(ref[k][0].scales.max())
         assert np.abs(w_gpu - w_ref).max() <= 4 * lsb
+
+
+def _clone_items(items):
+    return [{"G": it["G"], "P": it["P"], "W": it["W"].clone(), "M": it["M"]._base.clone()[:, :it["M"].shape[1]],
+             "V": it["V"]._base.clone()[:, :it["V"].shape[1]], "seed": it["seed"]} for it in items]
+
+
+@pytest.mark.parametrize("mask", [1, 2, 3])   # compared with mask 0
+def test_cta_pair_kernels_equal_single_cta_kernels(mask):
+    # two layers of the LLaMA-1B stack (14 matrices, r = 512): the cta_group::2 variants of the two GEMM kernels
+    # must reproduce the one-CTA kernels bit for bit (same products, same accumulation order, same epilogues)
+    import ctypes
+    import bench
+    _, base = bench.build_stack("llama1b", torch.device("cuda", 0), seed=3, layers=2)
+    set_mode = B.lib().qgalore_debug_set_pair_mode
+    set_mode.argtypes = [ctypes.c_int]
+    results = []
+    try:
+        for m in (0, mask):
+            set_mode(m)
+            items = _clone_items(base)
+            plan = B.StepPlan(items)
+            for t in (1, 2):
+                plan.step(B.Hyper(step=t))
+            torch.cuda.synchronize()
+            assert int(plan.status.item()) == 0
+            plan.close()
+            results.append(items)
+    finally:
+        set_mode(2)                                        # the library's default
+    for a, b in zip(*results):
+        assert torch.equal(a["W"].codes, b["W"].codes)
+        assert torch.equal(a["W"].scales, b["W"].scales) and torch.equal(a["W"].zeros, b["W"].zeros)
+        assert torch.equal(a["M"], b["M"]) and torch.equal(a["V"], b["V"])
