@@ -131,12 +131,40 @@ struct K1Smem {
   static constexpr int kThreads = 64 + kEpiWarps * 32;
 };
 
-// The Adam update of Sec. 3.5 on one element: M <- b1 M + (1-b1) R, V <- b2 V + (1-b2) R^2,
+// The Adam update of Sec. 3.5: M <- b1 M + (1-b1) R, V <- b2 V + (1-b2) R^2,
 // N = (M / (1 - b1^t)) / (sqrt(V / (1 - b2^t)) + eps)   (Kingma & Ba; eps outside the root).
-__device__ __forceinline__ float adam1(const StepScalars& sc, float inv_b1, float inv_b2, float r, float& m, float& v) {
-  m = fmaf(sc.beta1, m, sc.one_minus_beta1 * r);
-  v = fmaf(sc.beta2, v, sc.one_minus_beta2 * r * r);
-  return __fdividef(m * inv_b1, sqrt_approx(v * inv_b2) + sc.eps);
+// Packed fp32 pairs (one instruction for two lanes of a float2).
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(*reinterpret_cast<uint64_t*>(&d)) : "l"(*reinterpret_cast<uint64_t*>(&a)), "l"(*reinterpret_cast<uint64_t*>(&b)));
+  return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(*reinterpret_cast<uint64_t*>(&d)) : "l"(*reinterpret_cast<uint64_t*>(&a)), "l"(*reinterpret_cast<uint64_t*>(&b)));
+  return d;
+}
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;"
+      : "=l"(*reinterpret_cast<uint64_t*>(&d))
+      : "l"(*reinterpret_cast<uint64_t*>(&a)), "l"(*reinterpret_cast<uint64_t*>(&b)), "l"(*reinterpret_cast<uint64_t*>(&c)));
+  return d;
+}
+
+// Constants of the Adam update in the form the epilogue uses them: with k_v = bias1^2 / bias2 and
+// eps_b = eps * bias1,  N = (M / bias1) / (sqrt(V / bias2) + eps) = M / (sqrt(V * k_v) + eps_b).
+struct AdamConsts {
+  float2 b1, b2, omb1, omb2, kv, epsb;
+};
+
+// Adam on two adjacent elements: m, v are updated in place, the direction is returned.
+__device__ __forceinline__ float2 adam2(const AdamConsts& c, float2 r, float2& m, float2& v) {
+  m = fma2(c.b1, m, mul2(c.omb1, r));
+  v = fma2(c.b2, v, mul2(mul2(c.omb2, r), r));
+  const float2 q = mul2(v, c.kv);
+  const float2 den = add2(make_float2(sqrt_approx(q.x), sqrt_approx(q.y)), c.epsb);
+  return make_float2(__fdividef(m.x, den.x), __fdividef(m.y, den.y));
 }
 
 // The epilogue reads the accumulator in the 16-lane x 256-bit shape: thread t holds, per group of
@@ -292,7 +320,11 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     const int lrow = q * 32 + hh * 16 + (lane >> 2); // first of the thread's two tile rows (the other: + 8)
     const int lcol = 2 * (lane & 3);                 // first column of the thread's pair within a group of 8
     const uint32_t lane_addr = (uint32_t)(q * 32 + hh * 16) << 16;
-    const float inv_b1 = 1.0f / sc.bias1, inv_b2 = 1.0f / sc.bias2;
+    AdamConsts ac;
+    ac.b1 = make_float2(sc.beta1, sc.beta1); ac.b2 = make_float2(sc.beta2, sc.beta2);
+    ac.omb1 = make_float2(sc.one_minus_beta1, sc.one_minus_beta1); ac.omb2 = make_float2(sc.one_minus_beta2, sc.one_minus_beta2);
+    ac.kv = make_float2(sc.bias1 * sc.bias1 / sc.bias2, sc.bias1 * sc.bias1 / sc.bias2);
+    ac.epsb = make_float2(sc.eps * sc.bias1, sc.eps * sc.bias1);
     uint32_t tcount = 0;
     bool ok = true;
     for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
@@ -317,6 +349,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         tapN[a] = p->dbgN ? p->dbgN + gr * ldmv + n0 + lcol : nullptr;
       }
       float2 sm[3][8], sv[3][8];                     // three chunks of M, V: index 2k + a
+      // interior tiles (every row and column valid, no test taps) take a path without per-access predicates
+      const bool interior = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr;
       auto load_chunk = [&](int c, float2* m, float2* v) {
 #pragma unroll
         for (int k = 0; k < 4; ++k)
@@ -324,7 +358,10 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
           for (int a = 0; a < 2; ++a) {
             const int off = kChunk * c + 8 * k;
             float2 mm = make_float2(0.f, 0.f), vv = make_float2(0.f, 0.f);
-            if (rok[a]) {
+            if (interior) {
+              mm = __ldcs(reinterpret_cast<const float2*>(Mr[a] + off));
+              vv = __ldcs(reinterpret_cast<const float2*>(Vr[a] + off));
+            } else if (rok[a]) {
               if (off + 1 < cmax) {
                 mm = __ldcs(reinterpret_cast<const float2*>(Mr[a] + off));
                 vv = __ldcs(reinterpret_cast<const float2*>(Vr[a] + off));
@@ -357,23 +394,26 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
             for (int a = 0; a < 2; ++a) {
               const int off = kChunk * c + 8 * k;
               float2 mm = sm[c % 3][2 * k + a], vv = sv[c % 3][2 * k + a];
-              const float ra = __uint_as_float(acc[4 * k + 2 * a]), rb = __uint_as_float(acc[4 * k + 2 * a + 1]);
-              const float na = adam1(sc, inv_b1, inv_b2, ra, mm.x, vv.x);
-              const float nb = adam1(sc, inv_b1, inv_b2, rb, mm.y, vv.y);
-              if (rok[a]) {
+              const float2 rr = make_float2(__uint_as_float(acc[4 * k + 2 * a]), __uint_as_float(acc[4 * k + 2 * a + 1]));
+              const float2 nn = adam2(ac, rr, mm, vv);
+              const __nv_bfloat162 nb2 = __floats2bfloat162_rn(nn.x, nn.y);
+              if (interior) {
+                __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
+                __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
+                *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
+              } else if (rok[a]) {
                 if (off + 1 < cmax) {
                   __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
                   __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
-                  *reinterpret_cast<uint32_t*>(Nr[a] + off) =
-                      (uint32_t)float_to_bf16_bits(na) | ((uint32_t)float_to_bf16_bits(nb) << 16);
-                  if (tapR[a]) { tapR[a][off] = ra; tapR[a][off + 1] = rb; }
-                  if (tapN[a]) { tapN[a][off] = na; tapN[a][off + 1] = nb; }
+                  *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
+                  if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
+                  if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
                 } else if (off < cmax) {             // odd n: the last column stands alone
                   Mr[a][off] = mm.x;
                   Vr[a][off] = vv.x;
-                  Nr[a][off] = float_to_bf16_bits(na);
-                  if (tapR[a]) tapR[a][off] = ra;
-                  if (tapN[a]) tapN[a][off] = na;
+                  Nr[a][off] = float_to_bf16_bits(nn.x);
+                  if (tapR[a]) tapR[a][off] = rr.x;
+                  if (tapN[a]) tapN[a][off] = nn.x;
                 }
               }
             }
