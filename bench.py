@@ -69,7 +69,10 @@ def dq_units(m, n, r):
 # DRAM bytes per launch of the dominant kernels from the committed ncu capture (profiles/), per weight
 # element of the captured launch, so that it scales to the launches timed here.  None = no valid capture
 # for the kernels as they stand.
-NCU_TRAFFIC_PER_ELEMENT = {"project_adam": None, "backproject_sr": None}
+NCU_TRAFFIC_PER_ELEMENT = {
+    # profiles/project_adam_and_backproject_sr_llama1b_4layers.md: 1231 MB resp. 526 MB over 201.3 M elements
+    "llama1b": {"project_adam": 1231.0e6 / 201.3184e6, "backproject_sr": 526.6e6 / 201.3184e6},
+}
 
 
 def stack_roofline(specs, peaks):
@@ -351,7 +354,7 @@ def run_ours(args):
         else:
             roof = {"bound": "hbm", "achieved": k_bytes / k_sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        tpe = NCU_TRAFFIC_PER_ELEMENT.get(names[dom])
+        tpe = NCU_TRAFFIC_PER_ELEMENT.get(args.workload, {}).get(names[dom])
         roof["traffic"] = None if tpe is None else tpe * elements * args.steps / max(kcount[dom], 1)
         roof["kernel"] = names[dom]
         roof["launches"] = kcount[dom]
