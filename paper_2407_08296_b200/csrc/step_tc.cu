@@ -1046,9 +1046,12 @@ int launch_k2(const TcProblem* single, const TcProblem* table, const TileSchedul
 struct DequantItem {
   qg_qtensor P;
   uint16_t* out;
-  int32_t block0, nblocks;   // blocks of 256 threads, eight columns per thread
+  int32_t block0, nblocks;   // blocks of 256 threads, 32 columns per thread
 };
 
+// One thread converts 32 consecutive columns of a row (16 bytes of codes -> 64 bytes of bf16): the stored
+// nibble (code + 8) is dropped into the mantissa of 2^23 and (2^23 + 8 + z) subtracted, which gives q - z
+// exactly without an integer-to-float conversion.
 __global__ void __launch_bounds__(256)
 dequant_p_grouped_kernel(const DequantItem* __restrict__ items, int nitems) {
   int lo = 0, hi = nitems - 1;
@@ -1057,20 +1060,37 @@ dequant_p_grouped_kernel(const DequantItem* __restrict__ items, int nitems) {
     if (items[mid].block0 <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
   }
   const DequantItem& it = items[lo];
-  const qg_qtensor& P = it.P;
-  const int ngroups = (int)((P.cols + kGroup - 1) / kGroup);
-  const int64_t chunks = P.cols / 8;
-  const int64_t idx = (int64_t)(blockIdx.x - it.block0) * blockDim.x + threadIdx.x;
-  if (idx >= P.rows * chunks) return;
-  const int64_t row = idx / chunks, c0 = (idx % chunks) * 8;
-  const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)P.codes + row * (P.ld / 2) + (c0 >> 1)));
-  const int g = (int)(c0 / kGroup);
-  const float s = __ldg(P.scales + row * ngroups + g), z = __ldg(P.zeros + row * ngroups + g);
-  float qv[8], v[8];
-  unpack_int4x8(w, qv);
+  const uint32_t cols = (uint32_t)it.P.cols, rows = (uint32_t)it.P.rows;
+  const uint32_t per_row = cols / 32, ngroups = (cols + kGroup - 1) / kGroup;
+  const uint32_t idx = (blockIdx.x - (uint32_t)it.block0) * blockDim.x + threadIdx.x;
+  if (idx >= rows * per_row) return;
+  const uint32_t row = idx / per_row, c0 = (idx - row * per_row) * 32;
+  const uint4 w4 = __ldg(reinterpret_cast<const uint4*>((const uint8_t*)it.P.codes + (size_t)row * (it.P.ld / 2) + (c0 >> 1)));
+  const uint32_t g = c0 / kGroup;
+  const float s = __ldg(it.P.scales + (size_t)row * ngroups + g), z = __ldg(it.P.zeros + (size_t)row * ngroups + g);
+  const float c = 8388616.0f + z;                    // 2^23 + 8 + z, exact for |z| < 2^22
+  const bool fast = fabsf(z) < 4.0e6f;
+  const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
+  uint4* out = reinterpret_cast<uint4*>(it.out + (size_t)row * cols + c0);
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(__fsub_rn(qv[i], z), s);
-  *reinterpret_cast<uint4*>(it.out + row * P.cols + c0) = pack_bf16x8(v);
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t lo4 = w[k] & 0x0F0F0F0Fu, hi4 = (w[k] >> 4) & 0x0F0F0F0Fu;   // even and odd columns, one per byte
+    float v[8];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      float qe, qo;
+      if (fast) {
+        qe = __fsub_rn(__uint_as_float(__byte_perm(lo4, 0x4B000000u, 0x7650 + b)), c);
+        qo = __fsub_rn(__uint_as_float(__byte_perm(hi4, 0x4B000000u, 0x7650 + b)), c);
+      } else {
+        qe = __fsub_rn((float)((int)((lo4 >> (8 * b)) & 0xFu) - 8), z);
+        qo = __fsub_rn((float)((int)((hi4 >> (8 * b)) & 0xFu) - 8), z);
+      }
+      v[2 * b] = __fmul_rn(qe, s);
+      v[2 * b + 1] = __fmul_rn(qo, s);
+    }
+    out[k] = pack_bf16x8(v);
+  }
 }
 
 }  // namespace
@@ -1211,7 +1231,7 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       ch.k2p_tiles += probs[k].k2p_tiles;
       dq[k].P = a.P; dq[k].out = w.Pt;
       dq[k].block0 = ch.dq_blocks;
-      dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 8), 256);
+      dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 32), 256);
       ch.dq_blocks += dq[k].nblocks;
     }
     if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
