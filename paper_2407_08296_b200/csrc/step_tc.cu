@@ -480,6 +480,25 @@ __device__ __forceinline__ void weights16(const uint4 cw, const uint32_t* acc, f
                                           float lr_wd, float* w) {
   const uint32_t w4[4] = {cw.x, cw.y, cw.z, cw.w};
   const float c0 = 8388736.0f + z;
+  if (FAST && NOWD) {
+    // the common case, two elements per instruction: (q - z), times s, minus lr*alpha*D
+    const float2 mc0 = make_float2(-c0, -c0), s2 = make_float2(s, s), mla = make_float2(-lr_alpha, -lr_alpha);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const uint32_t x = w4[k] ^ 0x80808080u;
+#pragma unroll
+      for (int b = 0; b < 4; b += 2) {
+        const float2 v = make_float2(__uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650 + b)),
+                                     __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7651 + b)));
+        const float2 wh = mul2(add2(v, mc0), s2);
+        const float2 d = make_float2(__uint_as_float(acc[4 * k + b]), __uint_as_float(acc[4 * k + b + 1]));
+        const float2 r = fma2(mla, d, wh);
+        w[4 * k + b] = r.x;
+        w[4 * k + b + 1] = r.y;
+      }
+    }
+    return;
+  }
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const uint32_t x = w4[k] ^ 0x80808080u;
@@ -533,6 +552,29 @@ template <bool FAST>
 __device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& gp, const uint32_t h[8]) {
   int code[16];
   const float mz = (kMagic + 128.0f) + gp.z;
+  if (FAST) {
+    const float2 inv2 = make_float2(gp.inv, gp.inv), mz2 = make_float2(mz, mz);
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+      // 128 + h / 65536 of the two columns (h dropped into the mantissa of 2^7), negated by the sign bit
+      const float2 mhv = make_float2(__uint_as_float(__byte_perm(h[j >> 1], 0xC3000000u, 0x7610)),
+                                     __uint_as_float(__byte_perm(h[j >> 1], 0xC3000000u, 0x7632)));
+      const float2 t = mul2(make_float2(w[j], w[j + 1]), inv2);
+      float2 y;                                             // kMagic + ceil(t - h / 65536) + z, per lane
+      {
+        const float2 u = add2(t, mhv);
+        asm("add.rp.f32x2 %0, %1, %2;"
+            : "=l"(*reinterpret_cast<uint64_t*>(&y))
+            : "l"(*reinterpret_cast<const uint64_t*>(&u)), "l"(*reinterpret_cast<const uint64_t*>(&mz2)));
+      }
+      code[j] = __float_as_int(y.x) - 0x4B400000;           // may be -129 or 128: the pack saturates
+      code[j + 1] = __float_as_int(y.y) - 0x4B400000;
+    }
+    uint32_t o[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) o[k] = pack_sat_s8x4(code[4 * k], code[4 * k + 1], code[4 * k + 2], code[4 * k + 3]);
+    return make_uint4(o[0], o[1], o[2], o[3]);
+  }
 #pragma unroll
   for (int j = 0; j < 16; ++j) {
     const float t = __fmul_rn(w[j], gp.inv);
