@@ -52,13 +52,12 @@ constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
 // matters because a single thread issues them: with six copies per K block that thread, not the tensor
 // pipe, set the pace.
 //   mapW    int8 [m][ldw]         box 128 x 128, swizzle 128 load of the requantizing epilogue
-//   mapWst                        the same tensor for the store, with the inner extent rounded DOWN to 16
-//                                 bytes: a TMA store clips at 16-byte granularity, so it would spill into
-//                                 the row padding of a ragged matrix; the few tail columns are written with
-//                                 plain stores instead (n_tma_w = columns the TMA store covers).
-// M, V and N_b are read and written by the Adam epilogue with plain vector accesses.
+//   mapM, mapV  fp32 [r][ldmv]    box 32 x 16, swizzle 128   the Adam epilogue's reads of the old moments
+// Everything the epilogues write (M, V, N_b, the INT8 codes, scales and zero points) goes out with plain
+// vector stores: a TMA store clips at 16-byte granularity and would spill into the row padding of a ragged
+// matrix.
 struct alignas(64) TcProblem {
-  CUtensorMap mapP, mapG, mapP3, mapG3, mapG3h, mapN3, mapN3h, mapPk, mapW, mapWst;
+  CUtensorMap mapP, mapG, mapP3, mapG3, mapG3h, mapN3, mapN3h, mapPk, mapW, mapM, mapV;
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -69,7 +68,7 @@ struct alignas(64) TcProblem {
   int8_t* w_codes;
   uint16_t* nb;                        // N_b, bf16 r x ldn (scratch)
   int64_t ldmv, ldw, ldn;
-  int32_t m, n, r, ngroups, n_tma_w;
+  int32_t m, n, r, ngroups;
   int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles;
@@ -124,10 +123,17 @@ struct K1Smem {
   static constexpr int kABytes = 2 * kBoxBytes;            // 128 (r) x 64 (m) bf16
   static constexpr int kBBytes = (BN / 64 / CTAS) * kBoxBytes;   // this CTA's share of BN (n) x 64 (m) bf16
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = (192 * 1024) / kStageBytes;
-  static constexpr int kBarOffset = kStages * kStageBytes;
-  static constexpr int kBytes = kBarOffset + 256 + 1024;   // barriers + slack for 1024-byte alignment
   static constexpr int kEpiWarps = 8;                      // 4 lane quarters x 2 halves of 16 lanes
+  // every epilogue warp stages its own 16 rows x 32 columns of M and of V per accumulator chunk, kMvSlots
+  // chunks deep, through TMA
+  static constexpr int kMvSlots = kStageBytes > 32 * 1024 ? 2 : 3;
+  static constexpr int kMvArrayBytes = 16 * kChunk * 4;    // 2 KB: one array's piece of a chunk
+  static constexpr int kMvSlotBytes = 2 * kMvArrayBytes;   // M then V
+  static constexpr int kMvBytes = kEpiWarps * kMvSlots * kMvSlotBytes;
+  static constexpr int kStages = (224 * 1024 - kMvBytes) / kStageBytes;
+  static constexpr int kMvOffset = kStages * kStageBytes;
+  static constexpr int kBarOffset = kMvOffset + kMvBytes;
+  static constexpr int kBytes = kBarOffset + 512 + 1024;   // barriers + slack for 1024-byte alignment
   static constexpr int kThreads = 64 + kEpiWarps * 32;
 };
 
@@ -169,9 +175,9 @@ __device__ __forceinline__ float2 adam2(const AdamConsts& c, float2 r, float2& m
 
 // The epilogue reads the accumulator in the 16-lane x 256-bit shape: thread t holds, per group of
 // eight columns, the column pair 2(t%4), 2(t%4)+1 of rows t/4 and t/4 + 8.  A quad of threads therefore
-// covers 32 contiguous bytes of a row of M, V (fp32): every global access of the epilogue moves whole
-// 32-byte sectors without staging through shared memory, and M, V of the next two 32-column chunks
-// are prefetched into registers (64 KB in flight per SM) while the current one is computed.
+// covers 32 contiguous bytes of a row of M, V (fp32): every global store of the epilogue writes whole
+// 32-byte sectors straight from registers.  The old M, V come the other way through shared memory, by
+// TMA, several chunks ahead (see the epilogue).
 template <int BN, bool SINGLE, int CTAS>
 __global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
@@ -188,7 +194,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
   uint64_t* empty = bars + S::kStages;           // [kStages]
   uint64_t* acc_full = bars + 2 * S::kStages;    // [2]
   uint64_t* acc_empty = acc_full + 2;            // [2]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* mv_full = acc_empty + 2;             // [kEpiWarps][kMvSlots]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mv_full + S::kEpiWarps * S::kMvSlots);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const TcProblem* probs = SINGLE ? &single : table;
@@ -196,6 +203,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
   if (threadIdx.x == 0) {
     for (int i = 0; i < S::kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], CTAS * S::kEpiWarps); }
+    for (int i = 0; i < S::kEpiWarps * S::kMvSlots; ++i) mbar_init(&mv_full[i], 1);
     fence_mbar_init();
     fence_proxy_async_smem();
   }
@@ -317,15 +325,67 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
   } else {
     // ------------------------------------------------------------------ epilogue: Adam on the tile
     const int q = warp & 3, hh = (warp - 2) >> 2;   // TMEM lane quarter of this warp, 16-lane half within it
-    const int lrow = q * 32 + hh * 16 + (lane >> 2); // first of the thread's two tile rows (the other: + 8)
+    const int wrow = q * 32 + hh * 16;               // first of the warp's 16 tile rows
+    const int lrow = wrow + (lane >> 2);             // first of the thread's two tile rows (the other: + 8)
     const int lcol = 2 * (lane & 3);                 // first column of the thread's pair within a group of 8
-    const uint32_t lane_addr = (uint32_t)(q * 32 + hh * 16) << 16;
+    const uint32_t lane_addr = (uint32_t)wrow << 16;
     AdamConsts ac;
     ac.b1 = make_float2(sc.beta1, sc.beta1); ac.b2 = make_float2(sc.beta2, sc.beta2);
     ac.omb1 = make_float2(sc.one_minus_beta1, sc.one_minus_beta1); ac.omb2 = make_float2(sc.one_minus_beta2, sc.one_minus_beta2);
     ac.kv = make_float2(sc.bias1 * sc.bias1 / sc.bias2, sc.bias1 * sc.bias1 / sc.bias2);
     ac.epsb = make_float2(sc.eps * sc.bias1, sc.eps * sc.bias1);
-    uint32_t tcount = 0;
+
+    // M and V reach the warp through shared memory: one TMA copy per array brings the warp's 16 rows x 32
+    // columns of a chunk (rows of 128 bytes, 128-byte swizzle; columns and rows past the matrix read as
+    // zero), kMvSlots chunks ahead of the one being computed and across tile boundaries.  Loads that wait
+    // in registers cannot run that far ahead: a warp has six scoreboards to track them with, and a wait for
+    // one chunk's registers also waits for the younger loads that share its scoreboard.
+    const int ew = warp - 2;
+    uint8_t* mv_base = smem + S::kMvOffset + ew * (S::kMvSlots * S::kMvSlotBytes);
+    uint64_t* my_full = mv_full + ew * S::kMvSlots;
+    // byte offset of the thread's column pair of 8-column group k in a staged row: 16-byte unit
+    // (2k + (lane & 3) / 2) ^ (row % 8), then 8 bytes for the odd pair; both of the thread's rows have the
+    // same row % 8
+    const uint32_t swz = (uint32_t)(lane >> 2), half8 = (uint32_t)(lane & 1) * 8u, unit0 = (uint32_t)((lane >> 1) & 1);
+    const uint32_t row_off = (uint32_t)(lane >> 2) * 128u;
+
+    struct Cursor {                                  // a (tile, chunk) position in this CTA's work list
+      TileWalk<SINGLE> tw;
+      const TcProblem* p;
+      int c, nch, x0, y0;
+      __device__ Cursor(const TileSchedule& sch, int total) : tw(sch, total), p(nullptr), c(0), nch(0), x0(0), y0(0) {}
+    };
+    auto enter_tile = [&](Cursor& cu) {
+      if (!cu.tw.valid()) return;
+      const int2 item = cu.tw.cur();
+      cu.p = probs + item.x;
+      const int rblocks = CTAS == 2 ? cu.p->k1_rpairs : cu.p->k1_rblocks;
+      cu.y0 = (item.y % rblocks) * (CTAS * kTileM) + (int)rank * kTileM + wrow;
+      cu.x0 = (item.y / rblocks) * BN;
+      cu.nch = min(BN / kChunk, (cu.p->n - cu.x0 + kChunk - 1) / kChunk);
+      cu.c = 0;
+    };
+    auto next_chunk = [&](Cursor& cu) {
+      if (++cu.c >= cu.nch) { cu.tw.advance(); enter_tile(cu); }
+    };
+    Cursor ld(sched, total_tiles);                   // the next chunk to request
+    enter_tile(ld);
+    uint32_t ld_slot = 0, in_flight = 0;
+    auto request = [&]() {                           // one lane: the two copies of chunk `ld` into slot ld_slot
+      if (lane == 0) {
+        uint8_t* dst = mv_base + ld_slot * S::kMvSlotBytes;
+        mbar_arrive_expect_tx(&my_full[ld_slot], S::kMvSlotBytes);
+        tma_load_2d(dst, &ld.p->mapM, &my_full[ld_slot], ld.x0 + kChunk * ld.c, ld.y0);
+        tma_load_2d(dst + S::kMvArrayBytes, &ld.p->mapV, &my_full[ld_slot], ld.x0 + kChunk * ld.c, ld.y0);
+      }
+      ld_slot = (ld_slot + 1 == (uint32_t)S::kMvSlots) ? 0u : ld_slot + 1;
+      ++in_flight;
+      next_chunk(ld);
+    };
+#pragma unroll 1
+    for (int i = 0; i < S::kMvSlots && ld.tw.valid(); ++i) request();
+
+    uint32_t tcount = 0, slot = 0, slot_phase = 0;
     bool ok = true;
     for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
       const int2 item = tw.cur();
@@ -348,82 +408,86 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         tapR[a] = p->dbgR ? p->dbgR + gr * ldmv + n0 + lcol : nullptr;
         tapN[a] = p->dbgN ? p->dbgN + gr * ldmv + n0 + lcol : nullptr;
       }
-      float2 sm[3][8], sv[3][8];                     // three chunks of M, V: index 2k + a
       // interior tiles (every row and column valid, no test taps) take a path without per-access predicates
       const bool interior = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr;
-      auto load_chunk = [&](int c, float2* m, float2* v) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            const int off = kChunk * c + 8 * k;
-            float2 mm = make_float2(0.f, 0.f), vv = make_float2(0.f, 0.f);
-            if (interior) {
-              mm = __ldcs(reinterpret_cast<const float2*>(Mr[a] + off));
-              vv = __ldcs(reinterpret_cast<const float2*>(Vr[a] + off));
-            } else if (rok[a]) {
-              if (off + 1 < cmax) {
-                mm = __ldcs(reinterpret_cast<const float2*>(Mr[a] + off));
-                vv = __ldcs(reinterpret_cast<const float2*>(Vr[a] + off));
-              } else if (off < cmax) {
-                mm.x = __ldcs(Mr[a] + off);
-                vv.x = __ldcs(Vr[a] + off);
-              }
-            }
-            m[2 * k + a] = mm;
-            v[2 * k + a] = vv;
-          }
-      };
-      load_chunk(0, sm[0], sv[0]);
-      if (nch > 1) load_chunk(1, sm[1], sv[1]);
 
       const uint32_t ab = tcount & 1;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
       if (!ok) break;
       tc_fence_after_sync();
+#pragma unroll 1
+      for (int c = 0; c < nch; ++c) {
+        // this chunk's M and V from the warp's slot into registers (index 2k + a), then the slot goes back
+        // to the copy engine for the chunk kMvSlots further on
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&my_full[slot], slot_phase));
+        if (!ok) break;
+        --in_flight;
+        float2 sm[8], sv[8];
+        {
+          const uint8_t* src = mv_base + slot * S::kMvSlotBytes + row_off + half8;
 #pragma unroll
-      for (int c = 0; c < BN / kChunk; ++c) {
-        if (c < nch) {
-          if (c + 2 < nch) load_chunk(c + 2, sm[(c + 2) % 3], sv[(c + 2) % 3]);
-          uint32_t acc[16];
-          tmem_ld_16x256b_x4(tmem_base + lane_addr + ab * BN + c * kChunk, acc);
-          tmem_ld_wait();
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t u = (((uint32_t)(2 * k) + unit0) ^ swz) << 4;
 #pragma unroll
             for (int a = 0; a < 2; ++a) {
-              const int off = kChunk * c + 8 * k;
-              float2 mm = sm[c % 3][2 * k + a], vv = sv[c % 3][2 * k + a];
-              const float2 rr = make_float2(__uint_as_float(acc[4 * k + 2 * a]), __uint_as_float(acc[4 * k + 2 * a + 1]));
-              const float2 nn = adam2(ac, rr, mm, vv);
-              const __nv_bfloat162 nb2 = __floats2bfloat162_rn(nn.x, nn.y);
-              if (interior) {
+              sm[2 * k + a] = *reinterpret_cast<const float2*>(src + a * 1024 + u);
+              sv[2 * k + a] = *reinterpret_cast<const float2*>(src + S::kMvArrayBytes + a * 1024 + u);
+            }
+          }
+        }
+        if (++slot == (uint32_t)S::kMvSlots) { slot = 0; slot_phase ^= 1u; }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (ld.tw.valid()) request();
+
+        uint32_t acc[16];
+        tmem_ld_16x256b_x4(tmem_base + lane_addr + ab * BN + c * kChunk, acc);
+        tmem_ld_wait();
+        if (c + 1 == nch) {                           // every read of this accumulator buffer has landed
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            if (CTAS == 2) mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[ab]), 0));
+            else mbar_arrive(&acc_empty[ab]);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            const int off = kChunk * c + 8 * k;
+            float2 mm = sm[2 * k + a], vv = sv[2 * k + a];
+            const float2 rr = make_float2(__uint_as_float(acc[4 * k + 2 * a]), __uint_as_float(acc[4 * k + 2 * a + 1]));
+            const float2 nn = adam2(ac, rr, mm, vv);
+            const __nv_bfloat162 nb2 = __floats2bfloat162_rn(nn.x, nn.y);
+            if (interior) {
+              __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
+              __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
+              *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
+            } else if (rok[a]) {
+              if (off + 1 < cmax) {
                 __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
                 __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
                 *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
-              } else if (rok[a]) {
-                if (off + 1 < cmax) {
-                  __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
-                  __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
-                  *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
-                  if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
-                  if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
-                } else if (off < cmax) {             // odd n: the last column stands alone
-                  Mr[a][off] = mm.x;
-                  Vr[a][off] = vv.x;
-                  Nr[a][off] = float_to_bf16_bits(nn.x);
-                  if (tapR[a]) tapR[a][off] = rr.x;
-                  if (tapN[a]) tapN[a][off] = nn.x;
-                }
+                if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
+                if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
+              } else if (off < cmax) {             // odd n: the last column stands alone
+                Mr[a][off] = mm.x;
+                Vr[a][off] = vv.x;
+                Nr[a][off] = float_to_bf16_bits(nn.x);
+                if (tapR[a]) tapR[a][off] = rr.x;
+                if (tapN[a]) tapN[a][off] = nn.x;
               }
             }
-        }
+          }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) {
-        if (CTAS == 2) mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[ab]), 0));
-        else mbar_arrive(&acc_empty[ab]);
+    }
+    if (!ok) {
+      // a wait ran out: let the copies still on their way into this warp's slots land (bounded) before the
+      // CTA gives its shared memory back
+      for (; in_flight > 0; --in_flight) {
+        mbar_wait(&my_full[slot], slot_phase);
+        if (++slot == (uint32_t)S::kMvSlots) { slot = 0; slot_phase ^= 1u; }
       }
     }
     if (!ok && lane == 0) raise_wait_expired(status);
@@ -979,14 +1043,12 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->n_whole = (int32_t)n_whole;
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
-  const int64_t n16 = a.n & ~int64_t(15);
-  ok &= make_map(&p->mapWst, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, n16 > 0 ? n16 : 16, a.m, a.W.ld, 128, kTileM,
-                 CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, a.n, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, a.n, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) {
     note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
     return QG_CUDA_ERROR;
   }
-  p->n_tma_w = (int32_t)n16;
   p->M = a.M; p->V = a.V; p->w_codes = reinterpret_cast<int8_t*>(a.W.codes);
   p->w_scales = a.W.scales;
   p->w_zeros = a.W.zeros;
