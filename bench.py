@@ -66,12 +66,26 @@ def dq_units(m, n, r):
     return 0.0, m * r // 2 + 8 * m * ((r + 255) // 256)
 
 
-# DRAM bytes per launch of the dominant kernels from the committed ncu capture (profiles/), per weight
-# element of the captured launch, so that it scales to the launches timed here.  None = no valid capture
-# for the kernels as they stand.
+# Lane-operations per weight element that the requantizing epilogue of the back-projection cannot avoid,
+# counted from the definitions (scalar 32-bit operations, no credit for packed pairs): Philox4x32-10 for
+# eight 16-bit uniforms = 10 rounds x (2 wide multiplies + 2 three-input XORs) = 5 per element; byte -> float,
+# minus zero point, times scale, minus lr*alpha*D = 4; minimum and maximum = 2; times 1/s', uniform -> float,
+# subtract, round up, clamp, pack = 6.
+K2_ALU_OPS_PER_ELEMENT = 17
+ALU_LANES_PER_SM_CLOCK = 128            # 4 schedulers x 32 lanes issue one instruction per clock
+
+
+def k2_alu_ops(m, n, r):
+    return float(K2_ALU_OPS_PER_ELEMENT) * m * n
+
+
+# DRAM bytes per launch of the kernels from the committed ncu capture (profiles/), per weight element of
+# the captured launch, so that it scales to the launches timed here.  None = no valid capture for the
+# kernels as they stand.
 NCU_TRAFFIC_PER_ELEMENT = {
-    # profiles/project_adam_and_backproject_sr_llama1b_4layers.md: 1231 MB resp. 526 MB over 201.3 M elements
-    "llama1b": {"project_adam": 1231.0e6 / 201.3184e6, "backproject_sr": 526.6e6 / 201.3184e6},
+    # profiles/project_adam_and_backproject_sr_llama1b_4layers.md: 1214.6, 527.7 and 48.7 MB over 201.3 M elements
+    "llama1b": {"project_adam": 1214.6e6 / 201.3184e6, "backproject_sr": 527.7e6 / 201.3184e6,
+                "dequant_p_grouped": 48.7e6 / 201.3184e6},
 }
 
 
@@ -167,7 +181,9 @@ def oracle_sample(workload, steps, warmup):
         per_step += best * count
         elements += m * n * count
         detail.append(f"{m}x{n} r{r}: {best:.3f}s x{count}")
-    return elements / per_step, per_step, "one oracle step per distinct shape, extrapolated by shape counts (" + "; ".join(detail) + ")"
+    return (elements / per_step, per_step,
+            f"best of {steps} oracle steps (after {warmup} warm-up) on one matrix of each distinct shape, extrapolated by "
+            "shape counts (" + "; ".join(detail) + ")")
 
 
 def blas_threads():
@@ -341,18 +357,32 @@ def run_ours(args):
         t_c = flops / (peaks["bf16_tflops"] * 1e12)
         t_m = nbytes / (peaks["hbm_gbs"] * 1e9)
         sec = ms_per_step * 1e-3
-        # roofline of the dominant kernel (largest share of device time), from its live-measured duration
+        # roofline of every kernel from its live-measured duration: the bound is the slowest of the tensor
+        # pipe (sustained bf16 peak: the kernels are timed inside a long step), HBM (copy peak) and, for the
+        # requantizing epilogue, the plain ALUs (lanes x SMs x the maximum SM clock)
         names = ["dequant_p_grouped", "project_adam", "backproject_sr"]
         units = [dq_units, k1_units, k2_units]
+        peak_tf = peaks["bf16_tflops_sustained"]
+        sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+        alu_peak = torch.cuda.get_device_properties(device).multi_processor_count * ALU_LANES_PER_SM_CLOCK * sm_mhz * 1e6
+        per_kernel = {}
+        for k, nm in enumerate(names):
+            kf = sum(units[k](sp.m, sp.n, sp.r)[0] for sp in specs) * args.steps
+            kb = sum(units[k](sp.m, sp.n, sp.r)[1] for sp in specs) * args.steps
+            ko = sum(k2_alu_ops(sp.m, sp.n, sp.r) for sp in specs) * args.steps if nm == "backproject_sr" else 0.0
+            ksec = max(kms[k] * 1e-3, 1e-12)
+            cand = {"tensor": (kf / (peak_tf * 1e12), kf / ksec / 1e12, peak_tf, "TFLOP/s"),
+                    "hbm": (kb / (peaks["hbm_gbs"] * 1e9), kb / ksec / 1e9, peaks["hbm_gbs"], "GB/s"),
+                    "alu": (ko / alu_peak, ko / ksec / 1e12, alu_peak / 1e12, "Tlane-op/s")}
+            bound = max(cand, key=lambda c: cand[c][0])
+            per_kernel[nm] = {"bound": bound, "achieved": cand[bound][1], "peak": cand[bound][2], "unit": cand[bound][3],
+                              "frac": cand[bound][1] / cand[bound][2], "ms_per_step": kms[k] / args.steps,
+                              "bound_ms_per_step": {c: cand[c][0] * 1e3 / args.steps for c in cand},
+                              "flops": kf / args.steps, "bytes": kb / args.steps, "alu_ops": ko / args.steps}
         dom = max(range(3), key=lambda k: kms[k])
-        k_flops = sum(units[dom](sp.m, sp.n, sp.r)[0] for sp in specs) * args.steps
-        k_bytes = sum(units[dom](sp.m, sp.n, sp.r)[1] for sp in specs) * args.steps
-        k_sec = kms[dom] * 1e-3
-        peak_tf = peaks["bf16_tflops_sustained"]          # kernels timed inside a long step: the sustained figure
-        if k_flops / (peak_tf * 1e12) >= k_bytes / (peaks["hbm_gbs"] * 1e9):
-            roof = {"bound": "tensor", "achieved": k_flops / k_sec / 1e12, "peak": peak_tf, "unit": "TFLOP/s"}
-        else:
-            roof = {"bound": "hbm", "achieved": k_bytes / k_sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+        k_flops = per_kernel[names[dom]]["flops"] * args.steps
+        k_bytes = per_kernel[names[dom]]["bytes"] * args.steps
+        roof = {key: per_kernel[names[dom]][key] for key in ("bound", "achieved", "peak", "unit")}
         roof["frac"] = roof["achieved"] / roof["peak"]
         tpe = NCU_TRAFFIC_PER_ELEMENT.get(args.workload, {}).get(names[dom])
         roof["traffic"] = None if tpe is None else tpe * elements * args.steps / max(kcount[dom], 1)
@@ -361,7 +391,9 @@ def run_ours(args):
         roof["avg_launch_ms"] = kms[dom] / max(kcount[dom], 1)
         roof["algorithmic_bytes_per_launch"] = k_bytes / max(kcount[dom], 1)
         roof["algorithmic_flops_per_launch"] = k_flops / max(kcount[dom], 1)
-        roof["peak_source"] = peak_kind + (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy)")
+        roof["peak_source"] = {"tensor": peak_kind + " (sustained bf16)", "hbm": peak_kind + " (copy)",
+                               "alu": "derived: SMs x 128 lanes x maximum SM clock"}[roof["bound"]]
+        roof["per_kernel"] = per_kernel
         roof["timing"] = "separate pass of the same steps with a CUDA event pair around every launch"
         roof["kernel_ms_per_step"] = {nm: kms[k] / args.steps for k, nm in enumerate(names)}
         roof["kernel_share"] = {nm: kms[k] / max(sum(kms), 1e-12) for k, nm in enumerate(names)}
