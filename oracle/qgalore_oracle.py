@@ -196,14 +196,17 @@ def quantize_rtn(x, bits, group=GROUP):
     return QTensor(codes, scales, zeros, bits, group)
 
 
-def quantize_sr(x, seed, step, group=GROUP, return_scaled=False):
+def quantize_sr(x, seed, step, group=GROUP, return_scaled=False, col0=0):
     """INT8 block-wise quantization with stochastic rounding F_SR (Sec. 3.4).
 
     The scaled value t = x / s is rounded down with probability ceil(t) - t and up
     with probability t - floor(t); the draw is the element's 16-bit Philox lane h:
     round up iff frac(t) * 65536 > h.  Scale and zero point are recomputed from the
     updated group (Sec. 3.5: the weight update needs "an additional quantization step").
+    ``col0``: x is the column block [col0, col0 + cols) of a wider matrix (col0 a multiple of the
+    group size); it only shifts the column index that selects each element's Philox lane.
     """
+    assert col0 % group == 0
     x = np.ascontiguousarray(x, dtype=np.float32)
     rows, cols = x.shape
     sl = _group_slices(cols, group)
@@ -211,7 +214,7 @@ def quantize_sr(x, seed, step, group=GROUP, return_scaled=False):
     scales = np.empty((rows, len(sl)), dtype=np.float32)
     zeros = np.empty((rows, len(sl)), dtype=np.float32)
     scaled = np.empty((rows, cols), dtype=np.float32)
-    h = sr_uniform16(seed, step, rows, cols).astype(np.float32)
+    h = sr_uniform16(seed, step, rows, cols, col0=col0).astype(np.float32)
     for k, (a, b) in enumerate(sl):
         seg = x[:, a:b]
         s, inv, z = group_params(seg, 8)
@@ -274,7 +277,7 @@ class Hyper:
         return g(self.lr), g(self.alpha), g(self.beta1), g(self.beta2), g(self.eps), g(self.weight_decay)
 
 
-def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=None, N_b_override=None):
+def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=None, N_b_override=None, col0=0):
     """One Q-GaLore update of one weight matrix (Sec. 3.5, Fig. 4; GaLore projection as cited there).
 
     G_bits : uint16 [m, n] bfloat16 gradient.         P_q : INT4 m x r projection.
@@ -288,6 +291,9 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     direction N = M^ / (sqrt(V^) + eps) amplifies rounding differences of R without bound where
     sqrt(V^) is of the order of eps, so the weight update of another implementation is checked
     against steps 5-6 applied to that implementation's own direction.
+    ``col0``: G, W, M, V are the column block starting at column col0 (a multiple of the group
+    size) of a wider matrix; every column of the step depends on its own column of G, M, V, W only
+    (and on P), so the block's results are those of the full matrix.  col0 enters the Philox lanes.
     """
     lr, alpha, b1, b2, eps, wd = h.as_f32()
     t = int(h.step)
@@ -316,7 +322,7 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     W_hat = dequantize(W_q).astype(np.float64)
     W_pre = fl32(W_hat - (lr * alpha) * D - (lr * wd) * W_hat)
     # 6. requantize every group with stochastic rounding
-    W_new, T = quantize_sr(W_pre, h.seed, t, W_q.group, return_scaled=True)
+    W_new, T = quantize_sr(W_pre, h.seed, t, W_q.group, return_scaled=True, col0=col0)
     return dict(W=W_new, M=M_new, V=V_new, R32=R32, N=N32, N_b=N_b, W_pre=W_pre, T=T, P_tilde=Pt)
 
 

@@ -82,7 +82,7 @@ def check_direction(gpu, ref, hyp, name="N", tol=2e-3):
     return float(ill.mean())
 
 
-def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_frac=1e-3):
+def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_frac=1e-3, col0=0):
     """INT8 weights after one step against the oracle's (same direction N_b on both sides).
 
     Scales agree to 1e-5 relative and zero points exactly wherever the group's scaled minimum is
@@ -108,7 +108,7 @@ def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_fr
     assert frac_bad <= max_frac, f"{frac_bad:.2e} of the weight codes differ"
     if bad.any():
         T = out["T"].astype(np.float64)
-        h = O.sr_uniform16(seed, step, m, n).astype(np.float64)
+        h = O.sr_uniform16(seed, step, m, n, col0=col0).astype(np.float64)
         fr = (T - np.floor(T)) * 65536.0
         near_draw = np.abs(fr - h) <= 1e-3 * 65536 + 1
         near_int = (fr <= 1e-3 * 65536) | (fr >= (1 - 1e-3) * 65536)
@@ -198,3 +198,38 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
             assert float(base[:, n:].abs().max().item()) == 0.0, "padding of the moment rows was written"
     return {"mismatch": frac, "mismatch_unforced": frac_unforced, "ill": ill, "wpre_err_lsb": wpre_err,
             "W": gw, "M": dM.cpu().numpy(), "V": dV.cpu().numpy(), "ref": ref}
+
+
+def column_block(q: O.QTensor, a: int, b: int) -> O.QTensor:
+    """Columns [a, b) of a quantized matrix, a on a group boundary, b on one or at the end."""
+    g = q.group
+    assert a % g == 0 and (b % g == 0 or b == q.codes.shape[1])
+    return O.QTensor(q.codes[:, a:b].copy(), q.scales[:, a // g:(b + g - 1) // g].copy(),
+                     q.zeros[:, a // g:(b + g - 1) // g].copy(), q.bits, g)
+
+
+def check_step_on_column_blocks(blocks, gb, P, W, M, V, hyp, gpu, tol=2e-3):
+    """Parity of one step of a large matrix on a few column blocks the oracle can afford.
+
+    Column j of every result of the step depends on column j of G, M, V, W only (and on P), so the
+    oracle runs on the blocks alone.  ``gpu`` holds the library's results for the whole matrix:
+    M, V, R, N, W_pre (numpy) and W (oracle QTensor).  Same two stages and rules as run_and_check_step.
+    """
+    stats = []
+    for (a, b) in blocks:
+        Wb = column_block(W, a, b)
+        ref = O.project_step(gb[:, a:b], P, Wb, M[:, a:b], V[:, a:b], hyp, col0=a)
+        check_moments(gpu["M"][:, a:b], ref["M"], f"M[:, {a}:{b}]", tol)
+        check_moments(gpu["V"][:, a:b], ref["V"], f"V[:, {a}:{b}]", tol)
+        check_moments(gpu["R"][:, a:b], ref["R32"], f"R[:, {a}:{b}]", tol)
+        n_gpu = gpu["N"][:, a:b]
+        check_direction(n_gpu, ref, hyp, f"N[:, {a}:{b}]", tol)
+        forced = O.project_step(gb[:, a:b], P, Wb, M[:, a:b], V[:, a:b], hyp, N_b_override=O.bf16_round(n_gpu), col0=a)
+        lsb = np.repeat(forced["W"].scales, 256, axis=1)[:, :b - a]
+        wpre_err = float((np.abs(gpu["W_pre"][:, a:b] - forced["W_pre"]) / lsb).max())
+        assert wpre_err <= 1e-3, f"pre-rounding weight off by {wpre_err:.2e} LSB in columns {a}:{b}"
+        gw = column_block(gpu["W"], a, b)
+        frac = check_weight_codes(gw, forced, hyp.seed, hyp.step, col0=a)
+        check_weight_codes_unforced(gw, ref)
+        stats.append((a, b, frac, wpre_err))
+    return stats

@@ -8,7 +8,8 @@ import oracle as O
 from paper_2407_08296_b200 import binding as B
 from paper_2407_08296_b200 import synth
 
-from parity_utils import f32_to_device, from_device_q, g_to_device, run_and_check_step, to_device_q
+from parity_utils import (StepTaps, check_step_on_column_blocks, f32_to_device, from_device_q, g_to_device,
+                          run_and_check_step, to_device_q)
 
 pytestmark = pytest.mark.gpu
 
@@ -307,3 +308,53 @@ def test_cta_pair_kernels_equal_single_cta_kernels(mask):
         assert torch.equal(a["W"].codes, b["W"].codes)
         assert torch.equal(a["W"].scales, b["W"].scales) and torch.equal(a["W"].zeros, b["W"].zeros)
         assert torch.equal(a["M"], b["M"]) and torch.equal(a["V"], b["V"])
+
+
+# ----------------------------------------------------------------------------- full sizes, as the bench runs them
+def _full_size_case(shapes, blocks_of, seed):
+    """A plan over full-size matrices (the launch configuration bench.py times: grouped launches, CTA pairs,
+    host-made tile lists) against (a) per-matrix calls, bit for bit, and (b) the oracle on a few column blocks."""
+    step = 3
+    host, items, singles = [], [], []
+    rng = np.random.default_rng(seed)
+    for idx, (m, n, r) in enumerate(shapes):
+        gb = synth.GradientModel(m, n, seed=seed, matrix_index=idx).sample(step)
+        P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=seed, stream=idx), 4)
+        W = O.quantize_rtn(synth.initial_weight(m, n, seed, idx), 8)
+        M = rng.normal(0, 1e-3, (r, n)).astype(np.float32)
+        V = (rng.normal(0, 1e-3, (r, n)) ** 2).astype(np.float32)
+        sr = synth.matrix_seed(seed, idx)
+        host.append((gb, P, W, M, V, sr))
+        dG, dP = g_to_device(gb), to_device_q(P)
+        items.append({"G": dG, "P": dP, "W": to_device_q(W), "M": f32_to_device(M), "V": f32_to_device(V), "seed": sr})
+        dW1, dM1, dV1 = to_device_q(W), f32_to_device(M), f32_to_device(V)
+        taps = StepTaps(m, n, r, dW1.ld)
+        B.project_step(dG, dP, dW1, dM1, dV1, B.Hyper(step=step, seed=sr), debug=taps.as_dict())
+        singles.append((dW1, dM1, dV1, taps))
+    plan = B.StepPlan(items)
+    plan.step(B.Hyper(step=step))
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0
+    for (dW1, dM1, dV1, taps), it, (gb, P, W, M, V, sr), (m, n, r) in zip(singles, items, host, shapes):
+        assert torch.equal(dW1.codes, it["W"].codes)
+        assert torch.equal(dW1.scales, it["W"].scales) and torch.equal(dW1.zeros, it["W"].zeros)
+        assert torch.equal(dM1._base, it["M"]._base) and torch.equal(dV1._base, it["V"]._base)
+        gpu = {"M": it["M"].cpu().numpy(), "V": it["V"].cpu().numpy(), "R": taps.R.cpu().numpy(),
+               "N": taps.N.cpu().numpy(), "W_pre": taps.W_pre.cpu().numpy(), "W": from_device_q(it["W"])}
+        check_step_on_column_blocks(blocks_of(n), gb, P, W, M, V, O.Hyper(step=step, seed=sr), gpu)
+    plan.close()
+
+
+def test_plan_at_llama1b_sizes_on_sampled_column_blocks():
+    # the three LLaMA-1B shapes (r = 512) in one plan; first, a middle and the ragged last group of columns
+    def blocks(n):
+        last = (n - 1) // 256 * 256
+        return [(0, 256), (last // 2 // 256 * 256, last // 2 // 256 * 256 + 256), (last, n)]
+    _full_size_case([(2048, 2048, 512), (2048, 5461, 512), (5461, 2048, 512)], blocks, seed=21)
+
+
+def test_plan_at_llama7b_sizes_on_sampled_column_blocks():
+    # the three LLaMA-7B shapes (r = 1024) in one plan, two column groups each
+    def blocks(n):
+        return [(0, 256), (n - 256, n)]
+    _full_size_case([(4096, 4096, 1024), (4096, 11008, 1024), (11008, 4096, 1024)], blocks, seed=22)

@@ -472,3 +472,29 @@ def test_synthetic_gradient_recipe():
     assert sum(s.m * s.n for s in synth.stack_matrices("llama1b")) == 24 * (4 * 2048 * 2048 + 3 * 2048 * 5461)
     shapes = {(m, n, r): c for m, n, r, c in synth.distinct_shapes("llama1b")}
     assert shapes == {(2048, 2048, 512): 96, (2048, 5461, 512): 48, (5461, 2048, 512): 24}
+
+
+def test_step_of_a_column_block_equals_the_block_of_the_full_step():
+    # Sec. 3.5: R = P^T G, Adam, P N and the row-wise groups act on each column block on its own, so the
+    # oracle may be run on a few blocks of a matrix too large to run whole; col0 only moves the Philox lanes.
+    from paper_2407_08296_b200 import synth
+    m, n, r = 96, 256 * 2 + 85, 32
+    gb = synth.GradientModel(m, n, seed=3, matrix_index=0).sample(2)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=3), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 3), 8)
+    rng = np.random.default_rng(7)
+    M = rng.normal(0, 1e-3, (r, n)).astype(np.float32)
+    V = (rng.normal(0, 1e-3, (r, n)) ** 2).astype(np.float32)
+    hyp = O.Hyper(step=2, seed=11)
+    full = O.project_step(gb, P, W, M, V, hyp)
+    for (a, b) in [(0, 256), (256, 512), (512, n)]:
+        Wb = O.QTensor(W.codes[:, a:b], W.scales[:, a // 256:(b + 255) // 256], W.zeros[:, a // 256:(b + 255) // 256], 8)
+        blk = O.project_step(gb[:, a:b], P, Wb, M[:, a:b], V[:, a:b], hyp, col0=a)
+        assert np.array_equal(blk["W"].codes, full["W"].codes[:, a:b])
+        assert np.array_equal(blk["W"].scales, full["W"].scales[:, a // 256:(b + 255) // 256])
+        assert np.array_equal(blk["M"], full["M"][:, a:b]) and np.array_equal(blk["V"], full["V"][:, a:b])
+        assert np.array_equal(blk["W_pre"], full["W_pre"][:, a:b])
+    # without the offset the second block draws other uniforms
+    Wb = O.QTensor(W.codes[:, 256:512], W.scales[:, 1:2], W.zeros[:, 1:2], 8)
+    assert not np.array_equal(O.project_step(gb[:, 256:512], P, Wb, M[:, 256:512], V[:, 256:512], hyp)["W"].codes,
+                              full["W"].codes[:, 256:512])
