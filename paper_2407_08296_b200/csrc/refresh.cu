@@ -34,10 +34,13 @@ __device__ __forceinline__ float ld_as_float(const float* p, int64_t i) { return
 
 // C[M x N] = alpha * A * B + beta * C.  A(i, k) = A[i * sa_m + k * sa_k], B(k, j) = B[k * sb_k + j * sb_n],
 // C(i, j) = C[i * ldc + j].  TA is uint16_t (bfloat16 bits) or float; ACC/TC float or double.
+// With k_slice < K the grid's z index selects a slice of K, and slice z writes its bare partial sums to
+// part + z * M * N (row-major M x N) instead of C: products with a small result and a long K (the Gram
+// matrices and projection coefficients of the orthonormalisation) would otherwise keep a handful of SMs busy.
 template <class TA, class ACC, class TC>
 __global__ void __launch_bounds__(256)
 gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* __restrict__ B, int64_t sb_k, int64_t sb_n,
-            TC* __restrict__ C, int64_t ldc, int M, int N, int K, ACC alpha, ACC beta) {
+            TC* __restrict__ C, int64_t ldc, int M, int N, int K, ACC alpha, ACC beta, int k_slice, ACC* __restrict__ part) {
   __shared__ __align__(16) float As[kGK][kGT + 4];
   __shared__ __align__(16) float Bs[kGK][kGT + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -48,7 +51,9 @@ gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* _
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = (ACC)0;
   const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
-  for (int k0 = 0; k0 < K; k0 += kGK) {
+  const int k_begin = (int)blockIdx.z * k_slice;
+  if (k_slice < K) K = min(K, k_begin + k_slice);
+  for (int k0 = k_begin; k0 < K; k0 += kGK) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       int mm, kk;
@@ -81,6 +86,10 @@ gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* _
     for (int j = 0; j < 4; ++j) {
       const int64_t gn = n0 + tx * 4 + j;
       if (gn >= N) continue;
+      if (part != nullptr) {
+        part[((int64_t)blockIdx.z * M + gm) * N + gn] = acc[i][j];
+        continue;
+      }
       TC* c = C + gm * ldc + gn;
       const ACC v = alpha * acc[i][j] + (beta != (ACC)0 ? beta * (ACC)(*c) : (ACC)0);
       *c = (TC)v;
@@ -88,12 +97,59 @@ gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* _
   }
 }
 
+// C = alpha * (sum of the slices' partial sums, in slice order) + beta * C
+template <class ACC, class TC>
+__global__ void __launch_bounds__(256)
+gemm_reduce_kernel(const ACC* __restrict__ part, int slices, TC* __restrict__ C, int64_t ldc, int M, int N, ACC alpha, ACC beta) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)M * N) return;
+  ACC s = (ACC)0;
+  for (int z = 0; z < slices; ++z) s += part[(int64_t)z * M * N + idx];
+  TC* c = C + (idx / N) * ldc + idx % N;
+  *c = (TC)(alpha * s + (beta != (ACC)0 ? beta * (ACC)(*c) : (ACC)0));
+}
+
+int refresh_sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) sms = v;
+    else sms = 148;
+  }
+  return sms;
+}
+
+constexpr int kSplitTiles = 64;          // products with fewer output tiles than this split their K range
+constexpr int kSplitMinK = 256;          // ... into slices no shorter than this
+constexpr int64_t kSplitScratch = 8 << 20;   // bytes of partial sums a product may use
+
+// `part` (kSplitScratch bytes, or null) lets a product with few output tiles and a long K run as slices.
 template <class TA, class ACC, class TC>
 int gemm(const TA* A, int64_t sa_m, int64_t sa_k, const float* B, int64_t sb_k, int64_t sb_n, TC* C, int64_t ldc, int64_t M,
-         int64_t N, int64_t K, ACC alpha, ACC beta, cudaStream_t st) {
+         int64_t N, int64_t K, ACC alpha, ACC beta, cudaStream_t st, void* part = nullptr) {
   if (M <= 0 || N <= 0) return QG_OK;
   dim3 grid((unsigned)ceil_div(N, kGT), (unsigned)ceil_div(M, kGT));
-  gemm_kernel<TA, ACC, TC><<<grid, 256, 0, st>>>(A, sa_m, sa_k, B, sb_k, sb_n, C, ldc, (int)M, (int)N, (int)K, alpha, beta);
+  const int64_t tiles = (int64_t)grid.x * grid.y;
+  int64_t slices = 1;
+  if (part != nullptr && tiles < kSplitTiles && K >= 2 * kSplitMinK) {
+    slices = ceil_div(2 * (int64_t)refresh_sm_count(), tiles);
+    if (slices > K / kSplitMinK) slices = K / kSplitMinK;
+    const int64_t fit = kSplitScratch / (M * N * (int64_t)sizeof(ACC));
+    if (slices > fit) slices = fit;
+  }
+  if (slices <= 1) {
+    gemm_kernel<TA, ACC, TC><<<grid, 256, 0, st>>>(A, sa_m, sa_k, B, sb_k, sb_n, C, ldc, (int)M, (int)N, (int)K, alpha, beta,
+                                                   (int)K, nullptr);
+    QG_LAUNCH_CHECK();
+    return QG_OK;
+  }
+  const int64_t k_slice = round_up(ceil_div(K, slices), kGK);
+  grid.z = (unsigned)ceil_div(K, k_slice);
+  gemm_kernel<TA, ACC, TC><<<grid, 256, 0, st>>>(A, sa_m, sa_k, B, sb_k, sb_n, C, ldc, (int)M, (int)N, (int)K, alpha, beta,
+                                                 (int)k_slice, reinterpret_cast<ACC*>(part));
+  QG_LAUNCH_CHECK();
+  gemm_reduce_kernel<ACC, TC><<<(unsigned)ceil_div(M * N, 256), 256, 0, st>>>(reinterpret_cast<const ACC*>(part), (int)grid.z, C,
+                                                                              ldc, (int)M, (int)N, alpha, beta);
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
@@ -281,6 +337,7 @@ sign_fix_kernel(float* __restrict__ P, int64_t m, int r, float* __restrict__ P_o
 
 struct RefreshWs {
   float *Q, *Y, *Z, *Wp, *Cb, *S, *Linv, *Xsel, *P32;
+  void* part;      // partial sums of sliced products
   double *T, *XT, *lam, *off;
   int32_t* done;
 };
@@ -303,6 +360,7 @@ size_t carve_refresh(void* base, int64_t m, int64_t n, int64_t b, int64_t r, Ref
   t.Linv = (float*)take((size_t)kPanel * kPanel * 4);
   t.Xsel = (float*)take((size_t)b * r * 4);
   t.P32 = (float*)take((size_t)m * r * 4);
+  t.part = take((size_t)kSplitScratch);
   if (w) *w = t;
   return off;
 }
@@ -315,7 +373,7 @@ int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cu
     int rc;
     for (int pass = 0; pass < 2 && j0 > 0; ++pass) {
       // C = Q[:, :j0]^T Yj   (j0 x 64);   Yj -= Q[:, :j0] C
-      rc = gemm<float, float, float>(w.Q, 1, b, Yj, b, 1, w.Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st);
+      rc = gemm<float, float, float>(w.Q, 1, b, Yj, b, 1, w.Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st, w.part);
       if (rc != QG_OK) return rc;
       rc = gemm<float, float, float>(w.Q, b, 1, w.Cb, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st);
       if (rc != QG_OK) return rc;
@@ -324,7 +382,7 @@ int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cu
     const float* src = Yj; int64_t lds = b;
     float* dst = w.Wp; int64_t ldd = kPanel;
     for (int pass = 0; pass < 2; ++pass) {
-      rc = gemm<float, float, float>(src, 1, lds, src, lds, 1, w.S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st);
+      rc = gemm<float, float, float>(src, 1, lds, src, lds, 1, w.S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st, w.part);
       if (rc != QG_OK) return rc;
       chol64_inverse_kernel<<<1, 64, 0, st>>>(w.S, w.Linv, status);
       QG_LAUNCH_CHECK();
