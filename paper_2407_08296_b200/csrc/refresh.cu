@@ -11,7 +11,7 @@
 // Everything heavy is a GEMM (one generic fp32 kernel, fp64 accumulation for T).  orth() is block
 // Gram-Schmidt over panels of 64 columns, each projection done twice, the panel itself by two rounds of
 // Cholesky QR.  The eigenvectors of T come from a one-sided (Hestenes) Jacobi iteration in fp64 with a
-// round-robin pair ordering, one launch per round of b/2 disjoint column pairs.  Each column of P is then
+// round-robin pair ordering: all sweeps in one cooperative launch, a grid barrier between rounds of b/2 disjoint pairs.  Each column of P is then
 // given the sign that makes its largest entry positive, and P is quantized to INT4 (Quant_4).
 //
 // The arithmetic is plain fp32/fp64 on the CUDA cores: the singular values next to the r-th one sit in the
@@ -26,6 +26,7 @@ namespace qg {
 namespace {
 
 constexpr int kPanel = 64;    // columns orthonormalised together
+constexpr int kMaxSweeps = 32;
 constexpr int kGT = 64;       // GEMM tile (square), 16 x 16 threads, 4 x 4 outputs each
 constexpr int kGK = 16;
 
@@ -207,9 +208,10 @@ chol64_inverse_kernel(const float* __restrict__ S, float* __restrict__ Linv, int
   }
 }
 
-// ---- one-sided Jacobi on the rows of two b x b fp64 matrices (T symmetric, so its rows are its columns;
-// XT holds X transposed).  Round `rnd` of a sweep pairs the b indices by the round-robin tournament
-// schedule; block k rotates rows (p, q) of T and of XT so that the two rows of T become orthogonal.
+// ---- one-sided (Hestenes) Jacobi on the rows of the symmetric b x b fp64 matrix T: rows are rotated in
+// pairs until they are mutually orthogonal.  Then row j is lambda_j x_j^T (from T X = X Lambda), so the
+// eigenvectors are the normalised rows and no second matrix has to follow the rotations.  Round `rnd` of a
+// sweep pairs the b indices by the round-robin tournament schedule.
 __device__ __forceinline__ void tournament_pair(int nitems, int rnd, int k, int& p, int& q) {
   const int mod = nitems - 1;
   if (k == 0) { p = nitems - 1; q = rnd % mod; }
@@ -217,64 +219,126 @@ __device__ __forceinline__ void tournament_pair(int nitems, int rnd, int k, int&
   if (p > q) { const int t = p; p = q; q = t; }
 }
 
-__global__ void __launch_bounds__(128)
-jacobi_round_kernel(double* __restrict__ T, double* __restrict__ XT, int b, int rnd, double* __restrict__ off_max,
-                    const int32_t* __restrict__ done) {
-  if (*done) return;
-  int p, q;
-  tournament_pair(b, rnd, blockIdx.x, p, q);
-  double* tp = T + (int64_t)p * b;
-  double* tq = T + (int64_t)q * b;
-  double a = 0.0, c = 0.0, d = 0.0;
-  for (int i = threadIdx.x; i < b; i += blockDim.x) {
-    const double x = tp[i], y = tq[i];
-    a += x * x; d += y * y; c += x * y;
-  }
-  __shared__ double red[3][4];
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
-    d += __shfl_xor_sync(0xFFFFFFFFu, d, o);
-    c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-  }
-  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = a; red[1][threadIdx.x >> 5] = d; red[2][threadIdx.x >> 5] = c; }
+// Barrier across the CTAs of a cooperative launch (all resident at once): a counter that only grows and a
+// generation word.  The wait is bounded; when it runs out the caller flags the status word and every CTA
+// leaves.  `gen` counts the barriers this CTA has passed.
+constexpr uint32_t kGridWaitPolls = 1u << 24;
+__device__ __forceinline__ bool grid_barrier(unsigned int* count, unsigned int* generation, unsigned int& gen) {
   __syncthreads();
-  a = red[0][0] + red[0][1] + red[0][2] + red[0][3];
-  d = red[1][0] + red[1][1] + red[1][2] + red[1][3];
-  c = red[2][0] + red[2][1] + red[2][2] + red[2][3];
-  const double denom = sqrt(a * d);
-  const double rel = denom > 0.0 ? fabs(c) / denom : 0.0;
-  if (threadIdx.x == 0 && rel > 0.0) {
-    // off_max is only ever compared, so the monotone integer view of a non-negative double serves atomicMax
-    atomicMax(reinterpret_cast<unsigned long long*>(off_max), (unsigned long long)__double_as_longlong(rel));
+  int ok = 1;
+  ++gen;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(count, 1u) + 1u == gen * gridDim.x) {
+      __threadfence();
+      atomicExch(generation, gen);
+    } else {
+      uint32_t polls = 0;
+      while (*reinterpret_cast<volatile unsigned int*>(generation) < gen) {
+        if (++polls >= kGridWaitPolls) { ok = 0; break; }
+      }
+    }
+    __threadfence();
   }
-  if (rel < 1e-15) return;
-  const double zeta = (d - a) / (2.0 * c);
-  const double tt = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-  const double cs = 1.0 / sqrt(1.0 + tt * tt), sn = cs * tt;
-  double* xp = XT + (int64_t)p * b;
-  double* xq = XT + (int64_t)q * b;
-  for (int i = threadIdx.x; i < b; i += blockDim.x) {
-    const double x = tp[i], y = tq[i];
-    tp[i] = cs * x - sn * y;
-    tq[i] = sn * x + cs * y;
-    const double u = xp[i], v = xq[i];
-    xp[i] = cs * u - sn * v;
-    xq[i] = sn * u + cs * v;
-  }
+  return __syncthreads_and(ok) != 0;
 }
 
-__global__ void jacobi_sweep_end_kernel(double* off_max, int32_t* done, double tol, int last, int32_t* status) {
-  if (*done) return;
-  if (*off_max <= tol) *done = 1;
-  else if (last && status) atomicOr(status, QG_DEV_NOT_CONVERGED);
-  *off_max = 0.0;
+// All sweeps in one cooperative launch.  A team of 128 threads takes a pair of rows, NE elements of each row
+// per thread, kept in registers between the three inner products and the rotation; four teams per CTA move
+// in step.  A grid barrier follows every round (the next round pairs the rows differently).  Rows move
+// between SMs from round to round, so they are read and written through L2 (.cg).  The sweep's largest
+// normalised inner product is collected in off[sweep]; the iteration stops after the first sweep whose value
+// is <= tol and flags QG_DEV_NOT_CONVERGED if none is.
+constexpr int kTeam = 128, kTeamsPerCta = 4;
+template <int NE>
+__global__ void __launch_bounds__(kTeam * kTeamsPerCta, 1)
+jacobi_sweeps_kernel(double* __restrict__ T, int b, int sweeps, double tol, unsigned long long* __restrict__ off,
+                     unsigned int* __restrict__ sync_words, int32_t* __restrict__ status) {
+  __shared__ double red[kTeamsPerCta][3][kTeam / 32];
+  const int team = threadIdx.x / kTeam, tt = threadIdx.x % kTeam, tw = tt >> 5, lane = threadIdx.x & 31;
+  const int pairs = b / 2, batch = (int)gridDim.x * kTeamsPerCta;
+  unsigned int gen = 0;
+  bool converged = false;
+  for (int sw = 0; sw < sweeps && !converged; ++sw) {
+    double worst = 0.0;
+    for (int rnd = 0; rnd < b - 1; ++rnd) {
+      for (int k0 = 0; k0 < pairs; k0 += batch) {
+        const int k = k0 + (int)blockIdx.x * kTeamsPerCta + team;
+        const bool live = k < pairs;
+        int p = 0, q = 0;
+        if (live) tournament_pair(b, rnd, k, p, q);
+        double* tp = T + (int64_t)p * b;
+        double* tq = T + (int64_t)q * b;
+        double x[NE], y[NE];
+        double a = 0.0, c = 0.0, d = 0.0;
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+          const int i = tt + kTeam * e;
+          const bool in = live && i < b;
+          x[e] = in ? __ldcg(tp + i) : 0.0;
+          y[e] = in ? __ldcg(tq + i) : 0.0;
+        }
+#pragma unroll
+        for (int e = 0; e < NE; ++e) { a += x[e] * x[e]; d += y[e] * y[e]; c += x[e] * y[e]; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+          d += __shfl_xor_sync(0xFFFFFFFFu, d, o);
+          c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+        }
+        __syncthreads();                               // the previous batch has read `red`
+        if (lane == 0) { red[team][0][tw] = a; red[team][1][tw] = d; red[team][2][tw] = c; }
+        __syncthreads();
+        a = red[team][0][0] + red[team][0][1] + red[team][0][2] + red[team][0][3];
+        d = red[team][1][0] + red[team][1][1] + red[team][1][2] + red[team][1][3];
+        c = red[team][2][0] + red[team][2][1] + red[team][2][2] + red[team][2][3];
+        const double denom = sqrt(a * d);
+        const double rel = denom > 0.0 ? fabs(c) / denom : 0.0;
+        worst = fmax(worst, rel);
+        if (live && rel >= 1e-15) {
+          const double zeta = (d - a) / (2.0 * c);
+          const double tn = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
+          const double cs = 1.0 / sqrt(1.0 + tn * tn), sn = cs * tn;
+#pragma unroll
+          for (int e = 0; e < NE; ++e) {
+            const int i = tt + kTeam * e;
+            if (i < b) {
+              __stcg(tp + i, cs * x[e] - sn * y[e]);
+              __stcg(tq + i, sn * x[e] + cs * y[e]);
+            }
+          }
+        }
+      }
+      if (rnd == b - 2 && tt == 0 && worst > 0.0) {
+        // only ever compared, so the monotone integer view of a non-negative double serves atomicMax
+        atomicMax(off + sw, (unsigned long long)__double_as_longlong(worst));
+      }
+      if (!grid_barrier(sync_words, sync_words + 1, gen)) {
+        if (threadIdx.x == 0 && status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
+        return;
+      }
+    }
+    converged = __longlong_as_double((long long)__ldcg(off + sw)) <= tol;
+  }
+  if (!converged && blockIdx.x == 0 && threadIdx.x == 0 && status) atomicOr(status, QG_DEV_NOT_CONVERGED);
 }
 
-__global__ void __launch_bounds__(256)
-identity64_kernel(double* __restrict__ XT, int b) {
-  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx < (int64_t)b * b) XT[idx] = (idx / b == idx % b) ? 1.0 : 0.0;
+template <int NE>
+int launch_jacobi(double* T, int64_t b, int sweeps, double tol, unsigned long long* off, unsigned int* sync_words,
+                  int32_t* status, cudaStream_t st) {
+  // one cooperative launch, never more CTAs than are resident at once
+  int per_sm = 0;
+  QG_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_sweeps_kernel<NE>, kTeam * kTeamsPerCta, 0));
+  const int64_t resident = (int64_t)per_sm * refresh_sm_count();
+  if (resident < 1) { note_cuda_error(cudaErrorCooperativeLaunchTooLarge, "jacobi_sweeps_kernel occupancy"); return QG_CUDA_ERROR; }
+  int64_t grid = ceil_div(b / 2, kTeamsPerCta);
+  if (grid > resident) grid = resident;
+  int bi = (int)b;
+  void* args[] = {&T, &bi, &sweeps, &tol, &off, &sync_words, &status};
+  QG_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)jacobi_sweeps_kernel<NE>, dim3((unsigned)grid), dim3(kTeam * kTeamsPerCta),
+                                          args, 0, st));
+  count_launch();
+  return QG_OK;
 }
 
 // lambda_j = norm of row j of the rotated T (= |eigenvalue j|); rank_j = its position in descending order
@@ -291,9 +355,9 @@ row_norm_kernel(const double* __restrict__ T, int b, double* __restrict__ lam) {
   if (threadIdx.x == 0) lam[blockIdx.x] = sqrt(red[0] + red[1] + red[2] + red[3]);
 }
 
-// Xsel[i][rank_j] = X[i][j] = XT[j][i] for the r largest lambda_j
+// Xsel[i][rank_j] = X[i][j] = T[j][i] / lambda_j for the r largest lambda_j
 __global__ void __launch_bounds__(256)
-select_top_kernel(const double* __restrict__ XT, const double* __restrict__ lam, int b, int r, float* __restrict__ Xsel) {
+select_top_kernel(const double* __restrict__ T, const double* __restrict__ lam, int b, int r, float* __restrict__ Xsel) {
   const int j = blockIdx.x;
   const double lj = lam[j];
   __shared__ int s_rank;
@@ -308,7 +372,8 @@ select_top_kernel(const double* __restrict__ XT, const double* __restrict__ lam,
   __syncthreads();
   const int rank = s_rank;
   if (rank >= r) return;
-  for (int i = threadIdx.x; i < b; i += blockDim.x) Xsel[(int64_t)i * r + rank] = (float)XT[(int64_t)j * b + i];
+  const double inv = lj > 0.0 ? 1.0 / lj : 0.0;
+  for (int i = threadIdx.x; i < b; i += blockDim.x) Xsel[(int64_t)i * r + rank] = (float)(T[(int64_t)j * b + i] * inv);
 }
 
 // Each column of P gets the sign that makes its largest-magnitude entry positive; optional copy to P_out.
@@ -338,7 +403,7 @@ sign_fix_kernel(float* __restrict__ P, int64_t m, int r, float* __restrict__ P_o
 struct RefreshWs {
   float *Q, *Y, *Z, *Wp, *Cb, *S, *Linv, *Xsel, *P32;
   void* part;      // partial sums of sliced products
-  double *T, *XT, *lam, *off;
+  double *T, *lam, *off;
   int32_t* done;
 };
 
@@ -347,10 +412,9 @@ size_t carve_refresh(void* base, int64_t m, int64_t n, int64_t b, int64_t r, Ref
   auto take = [&](size_t bytes) { void* p = base ? (char*)base + off : nullptr; off += (size_t)round_up((int64_t)bytes, 256); return p; };
   RefreshWs t{};
   t.T = (double*)take((size_t)b * b * 8);
-  t.XT = (double*)take((size_t)b * b * 8);
   t.lam = (double*)take((size_t)b * 8);
-  t.off = (double*)take(8);
-  t.done = (int32_t*)take(4);
+  t.off = (double*)take(kMaxSweeps * 8);     // largest normalised inner product of each sweep
+  t.done = (int32_t*)take(8);               // the two words of the grid barrier
   t.Q = (float*)take((size_t)m * b * 4);
   t.Y = (float*)take((size_t)m * b * 4);
   t.Z = (float*)take((size_t)n * b * 4);
@@ -427,21 +491,20 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
   // Rayleigh-Ritz: T = Z^T Z in fp64, eigenvectors by one-sided Jacobi
   rc = gemm<float, double, double>(w.Z, 1, b, w.Z, b, 1, w.T, b, b, b, n, 1.0, 0.0, st);
   if (rc != QG_OK) return rc;
-  identity64_kernel<<<(unsigned)ceil_div(b * b, 256), 256, 0, st>>>(w.XT, (int)b);
-  QG_LAUNCH_CHECK();
-  QG_CUDA_TRY(cudaMemsetAsync(w.off, 0, 8, st));
-  QG_CUDA_TRY(cudaMemsetAsync(w.done, 0, 4, st));
-  for (int sw = 0; sw < sweeps; ++sw) {
-    for (int rnd = 0; rnd < (int)b - 1; ++rnd) {
-      jacobi_round_kernel<<<(unsigned)(b / 2), 128, 0, st>>>(w.T, w.XT, (int)b, rnd, w.off, w.done);
-      QG_LAUNCH_CHECK();
-    }
-    jacobi_sweep_end_kernel<<<1, 1, 0, st>>>(w.off, w.done, 1e-9, sw == sweeps - 1, status);
-    QG_LAUNCH_CHECK();
+  if (sweeps > kMaxSweeps) sweeps = kMaxSweeps;
+  QG_CUDA_TRY(cudaMemsetAsync(w.off, 0, kMaxSweeps * 8, st));
+  QG_CUDA_TRY(cudaMemsetAsync(w.done, 0, 8, st));
+  {
+    unsigned long long* off = reinterpret_cast<unsigned long long*>(w.off);
+    unsigned int* sync_words = reinterpret_cast<unsigned int*>(w.done);
+    if (b <= 8 * kTeam) rc = launch_jacobi<8>(w.T, b, sweeps, 1e-9, off, sync_words, status, st);
+    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(w.T, b, sweeps, 1e-9, off, sync_words, status, st);
+    else rc = launch_jacobi<32>(w.T, b, sweeps, 1e-9, off, sync_words, status, st);
+    if (rc != QG_OK) return rc;
   }
   row_norm_kernel<<<(unsigned)b, 128, 0, st>>>(w.T, (int)b, w.lam);
   QG_LAUNCH_CHECK();
-  select_top_kernel<<<(unsigned)b, 256, 0, st>>>(w.XT, w.lam, (int)b, (int)r, w.Xsel);
+  select_top_kernel<<<(unsigned)b, 256, 0, st>>>(w.T, w.lam, (int)b, (int)r, w.Xsel);
   QG_LAUNCH_CHECK();
   // P = Q Xsel
   rc = gemm<float, float, float>(w.Q, b, 1, w.Xsel, r, 1, w.P32, r, m, r, b, 1.f, 0.f, st);
