@@ -172,39 +172,58 @@ gaussian_kernel(float* __restrict__ Q, int64_t ld, int64_t rows, int64_t cols, u
   *reinterpret_cast<float4*>(Q + i * ld + 4 * jq) = make_float4(r0 * c0, r0 * s0, r1 * c1, r1 * s1);
 }
 
-// ---- Cholesky factor of a 64 x 64 Gram matrix and the inverse of the factor, one CTA of 64 threads, fp64.
+// ---- Cholesky factor of a 64 x 64 Gram matrix and the inverse of the factor, one CTA of 256 threads, fp64.
 // S (row-major fp32) = L L^T;  Linv = L^-1 (lower triangular, row-major fp32).  A non-positive pivot raises
 // QG_DEV_BAD_FACTOR and is replaced by a tiny positive number so that the run continues with finite values.
-__global__ void __launch_bounds__(64)
+// One shared array holds both triangles: L below and on the diagonal, the transpose of L^-1 above it
+// (A[j][i] = (L^-1)[i][j] for i > j); the diagonal of L^-1 is kept apart.
+__global__ void __launch_bounds__(256)
 chol64_inverse_kernel(const float* __restrict__ S, float* __restrict__ Linv, int32_t* __restrict__ status) {
-  __shared__ double L[kPanel][kPanel + 1];
+  __shared__ double A[kPanel][kPanel + 1];
+  __shared__ double xd[kPanel];
   const int t = threadIdx.x;
-  for (int i = 0; i < kPanel; ++i) L[i][t] = (double)S[i * kPanel + t];
+  for (int e = t; e < kPanel * kPanel; e += 256) A[e / kPanel][e % kPanel] = (double)S[e];
   __syncthreads();
-  for (int k = 0; k < kPanel; ++k) {
-    if (t == 0) {
-      double d = L[k][k];
-      if (!(d > 0.0)) { if (status) atomicOr(status, QG_DEV_BAD_FACTOR); d = 1e-30; }
-      L[k][k] = sqrt(d);
+  // right-looking factorisation: thread (i, g) owns the entries L[i][j] with j = k + 1 + g, k + 5 + g, ...
+  {
+    const int i = t & 63, g = t >> 6;
+    for (int k = 0; k < kPanel; ++k) {
+      double d = A[k][k];
+      if (!(d > 0.0)) { if (t == 0 && status) atomicOr(status, QG_DEV_BAD_FACTOR); d = 1e-30; }
+      const double dk = sqrt(d);
+      __syncthreads();                                 // everyone has read the pivot
+      if (g == 0) {
+        if (i == k) A[k][k] = dk;
+        else if (i > k) A[i][k] /= dk;
+      }
+      __syncthreads();
+      if (i > k) {
+        const double lik = A[i][k];
+        for (int j = k + 1 + g; j <= i; j += 4) A[i][j] -= lik * A[j][k];
+      }
+      __syncthreads();
     }
-    __syncthreads();
-    if (t > k) L[t][k] /= L[k][k];
-    __syncthreads();
-    if (t > k)
-      for (int j = k + 1; j <= t; ++j) L[t][j] -= L[t][k] * L[j][k];
-    __syncthreads();
   }
-  // column t of L^-1 by forward substitution (L x = e_t), kept by its thread
-  double x[kPanel];
-  for (int i = 0; i < kPanel; ++i) {
-    double v = 0.0;
-    if (i >= t) {
-      v = (i == t) ? 1.0 : 0.0;
-      for (int j = t; j < i; ++j) v -= L[i][j] * x[j];
-      v /= L[i][i];
+  // forward substitution, row by row: X[i][j] = -(sum_{k=j}^{i-1} L[i][k] X[k][j]) / L[i][i] for j < i.
+  // Four neighbouring lanes share a column j and split the sum.
+  {
+    const int j = t >> 2, part = t & 3;
+    if (t < kPanel) xd[t] = 1.0 / A[t][t];
+    __syncthreads();
+    for (int i = 1; i < kPanel; ++i) {
+      double sum = 0.0;
+      if (j < i) {
+        for (int k = j + part; k < i; k += 4) sum += A[i][k] * (k == j ? xd[j] : A[j][k]);
+      }
+      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
+      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
+      if (j < i && part == 0) A[j][i] = -sum * xd[i];   // column i of the upper triangle: read by later rows only
+      __syncthreads();
     }
-    x[i] = v;
-    Linv[i * kPanel + t] = (float)v;
+  }
+  for (int e = t; e < kPanel * kPanel; e += 256) {
+    const int i = e / kPanel, j = e % kPanel;
+    Linv[e] = (float)(i == j ? xd[i] : (i > j ? A[j][i] : 0.0));
   }
 }
 
@@ -448,7 +467,7 @@ int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cu
     for (int pass = 0; pass < 2; ++pass) {
       rc = gemm<float, float, float>(src, 1, lds, src, lds, 1, w.S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st, w.part);
       if (rc != QG_OK) return rc;
-      chol64_inverse_kernel<<<1, 64, 0, st>>>(w.S, w.Linv, status);
+      chol64_inverse_kernel<<<1, 256, 0, st>>>(w.S, w.Linv, status);
       QG_LAUNCH_CHECK();
       // dst = src * Linv^T:  B(k, j) = Linv[j][k]
       rc = gemm<float, float, float>(src, lds, 1, w.Linv, 1, kPanel, dst, ldd, m, kPanel, kPanel, 1.f, 0.f, st);
