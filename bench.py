@@ -249,6 +249,41 @@ def build_stack(workload, device, seed=0, layers=0):
     return specs, items
 
 
+def time_refresh(items, device):
+    """The occasional subspace refresh (Sec. 3.5), timed apart from the step: one matrix of each distinct
+    shape (12 subspace iterations on a block of 2r columns, Rayleigh-Ritz, INT4), CUDA events around the second
+    of two calls, extrapolated to the stack by the shape counts.  Also the similarity to the random projection
+    the stack was built with, as the gate would see it."""
+    import torch
+    from paper_2407_08296_b200 import binding as B
+    first, counts = {}, {}
+    for it in items:
+        sp = it["spec"]
+        key = (sp.m, sp.n, sp.r)
+        counts[key] = counts.get(key, 0) + 1
+        first.setdefault(key, it)
+    per_shape, total = [], 0.0
+    for (m, n, r), it in first.items():
+        block = min((2 * r + 63) // 64 * 64, min(m, n) // 64 * 64)
+        ws = torch.empty(B.workspace_bytes(B.QG_OP_REFRESH, m, n, block), dtype=torch.uint8, device=device)
+        sim = torch.zeros(1, dtype=torch.float32, device=device)
+        status = torch.zeros(1, dtype=torch.int32, device=device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        stream = torch.cuda.current_stream()
+        for rep in range(2):
+            e0.record(stream)
+            B.refresh_subspace(it["G"], r, iters=12, seed=1, P_prev=it["P"], sim=sim, workspace=ws, status=status)
+            e1.record(stream)
+            torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        per_shape.append({"shape": f"{m}x{n} r{r}", "count": counts[(m, n, r)], "ms": ms, "block": block,
+                          "similarity_to_previous": float(sim.item()), "device_status": int(status.item())})
+        total += ms * counts[(m, n, r)] * 1e-3
+        del ws
+    return {"iters": 12, "per_shape": per_shape, "stack_seconds": total,
+            "note": "not part of the timed step; one matrix per distinct shape, extrapolated by shape counts"}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -402,6 +437,7 @@ def run_ours(args):
                               "frac_of_nominal_roofline": t_roof_nom / sec,
                               "bound": "tensor" if t_c >= t_m else "hbm",
                               "achieved_tflops": flops / sec / 1e12, "achieved_gbs": nbytes / sec / 1e9}
+        refresh = None if args.no_refresh else time_refresh(items, device)
         cpu = None
         if not args.no_cpu_baseline:
             v, per_step, sample = oracle_sample(args.workload, 3, 1)
@@ -417,7 +453,7 @@ def run_ours(args):
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
                     "steps": e2e_steps},
-            "gpu_launches": launches, "clocks": clocks, "device_status": status,
+            "gpu_launches": launches, "clocks": clocks, "device_status": status, "refresh": refresh,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -430,6 +466,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama1b")
+    ap.add_argument("--no-refresh", action="store_true", help="skip the separate timing of the subspace refresh")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
