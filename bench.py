@@ -213,6 +213,19 @@ def run_reference(args):
 
 
 # --------------------------------------------------------------------------------------------- our arm
+def whole_job_throughput(ms_total, elements_per_rank, steps, world, device):
+    """Every rank steps its own replica of the stack (matrices are independent units: no collective on the
+    data path).  The job's time is the slowest rank's (MAX over ranks of the device-timed milliseconds), its
+    throughput the elements all ranks updated in that time.  Returns (ms_total of the job, elements/s)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms_total], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    return ms, elements_per_rank * world * steps / (ms * 1e-3)
+
+
 def build_stack(workload, device, seed=0, layers=0):
     """Device-resident synthetic state of the whole stack: bf16 gradients (rank-32 signal + noise),
     INT8 weights, INT4 projections, zero moments.  Generated with torch on the device (input
@@ -342,12 +355,8 @@ def run_ours(args):
     clocks = sampler.stop(t_wall0, t_wall1) if rank == 0 else None
     status = int(batch.status.item())
 
-    tms = torch.tensor([ms_total], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-    ms_total = float(tms.item())
+    ms_total, value = whole_job_throughput(ms_total, elements, args.steps, world, device)
     ms_per_step = ms_total / args.steps
-    value = elements * world * args.steps / (ms_total * 1e-3)
 
     # ---- end to end: gradients arrive from pinned host memory every step, the status word is read back
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -369,10 +378,7 @@ def run_ours(args):
         stream.synchronize()
     e1.record(stream)
     barrier()
-    e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=device)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = elements * world * e2e_steps / (float(e2e_ms.item()) * 1e-3)
+    _, e2e_value = whole_job_throughput(e0.elapsed_time(e1), elements, e2e_steps, world, device)
     del host_g
 
     # ---- per-kernel device time: a second pass of the same steps with an event pair around every launch
