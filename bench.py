@@ -318,7 +318,7 @@ def run_ours(args):
     specs, items = build_stack(args.workload, device, seed=rank, layers=args.layers)
     batch = B.StepPlan(items)
     elements = batch.elements
-    hyper = B.Hyper()
+    hyper = B.Hyper(rounding=B.QG_ROUND_NEAREST if args.rounding == "nearest" else B.QG_ROUND_STOCHASTIC)
     torch.cuda.synchronize()
 
     def barrier():
@@ -454,7 +454,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload + (f"[first {args.layers} layers]" if args.layers else ""), "matrices": len(specs), "elements_per_step": elements,
-                       "rank": specs[0].r, "group": 256, "l2": "inputs larger than L2 (whole stack streams each step)",
+                       "rank": specs[0].r, "group": 256, "rounding": args.rounding, "l2": "inputs larger than L2 (whole stack streams each step)",
                        "parallelism": f"replica per GPU x{world}, no collective"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
@@ -473,6 +473,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama1b")
     ap.add_argument("--no-refresh", action="store_true", help="skip the separate timing of the subspace refresh")
+    ap.add_argument("--rounding", choices=["stochastic", "nearest"], default="stochastic",
+                    help="requantization of the updated weight: the method's stochastic rounding, or the round-to-nearest ablation")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")

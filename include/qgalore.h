@@ -73,11 +73,17 @@ typedef struct {
 
 /* Hyper-parameters of one step.  alpha is GaLore's scale factor (0.25 in Sec. 4.1), the
  * Adam constants are Kingma & Ba's; step is t >= 1 and enters the bias corrections and the
- * random-number counter; seed keys the stochastic rounding of this matrix. */
+ * random-number counter; seed keys the stochastic rounding of this matrix.  rounding selects how
+ * the updated weight is requantized: QG_ROUND_STOCHASTIC (Sec. 3.4, the method) or QG_ROUND_NEAREST
+ * (the ablation of Sec. 4.4, Fig. 6: round to nearest, ties to even; seed and step do not enter the codes). */
+#define QG_ROUND_STOCHASTIC 0
+#define QG_ROUND_NEAREST 1
 typedef struct {
   float    lr, alpha, beta1, beta2, eps, weight_decay;
   int64_t  step;
   uint64_t seed;
+  int32_t  rounding;   /* QG_ROUND_*; anything else: QG_INVALID_ARGUMENT */
+  int32_t  reserved;   /* 0 */
 } qg_hyper;
 
 /* Optional taps for tests: any non-null pointer receives that intermediate (device, fp32). */

@@ -175,7 +175,7 @@ def _group_slices(cols, group):
     return [(c, min(c + group, cols)) for c in range(0, cols, group)]
 
 
-def quantize_rtn(x, bits, group=GROUP):
+def quantize_rtn(x, bits, group=GROUP, return_scaled=False):
     """Round-to-nearest block-wise uniform quantization Quant_n (Sec. 3.1)."""
     x = np.ascontiguousarray(x, dtype=np.float32)
     rows, cols = x.shape
@@ -183,6 +183,7 @@ def quantize_rtn(x, bits, group=GROUP):
     codes = np.empty((rows, cols), dtype=np.int8)
     scales = np.empty((rows, len(sl)), dtype=np.float32)
     zeros = np.empty((rows, len(sl)), dtype=np.float32)
+    scaled = np.empty((rows, cols), dtype=np.float32)
     qlo = np.float32(-(1 << (bits - 1)))
     qhi = np.float32((1 << (bits - 1)) - 1)
     for k, (a, b) in enumerate(sl):
@@ -193,7 +194,9 @@ def quantize_rtn(x, bits, group=GROUP):
         codes[:, a:b] = q.astype(np.int8)
         scales[:, k] = s
         zeros[:, k] = z
-    return QTensor(codes, scales, zeros, bits, group)
+        scaled[:, a:b] = t
+    qt = QTensor(codes, scales, zeros, bits, group)
+    return (qt, scaled) if return_scaled else qt
 
 
 def quantize_sr(x, seed, step, group=GROUP, return_scaled=False, col0=0):
@@ -270,6 +273,7 @@ class Hyper:
     weight_decay: float = 0.0
     step: int = 1            # t >= 1
     seed: int = 0
+    rounding: str = "sr"     # "sr": stochastic rounding F_SR (Sec. 3.4); "rtn": round to nearest (the Fig. 6 ablation)
 
     def as_f32(self):
         """The values as the C boundary carries them (binary32), widened back to Python floats."""
@@ -321,8 +325,11 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     D = Pt @ N_b.astype(np.float64)
     W_hat = dequantize(W_q).astype(np.float64)
     W_pre = fl32(W_hat - (lr * alpha) * D - (lr * wd) * W_hat)
-    # 6. requantize every group with stochastic rounding
-    W_new, T = quantize_sr(W_pre, h.seed, t, W_q.group, return_scaled=True, col0=col0)
+    # 6. requantize every group: stochastic rounding (Sec. 3.4), or round to nearest for the ablation of Fig. 6
+    if h.rounding == "rtn":
+        W_new, T = quantize_rtn(W_pre, 8, W_q.group, return_scaled=True)
+    else:
+        W_new, T = quantize_sr(W_pre, h.seed, t, W_q.group, return_scaled=True, col0=col0)
     return dict(W=W_new, M=M_new, V=V_new, R32=R32, N=N32, N_b=N_b, W_pre=W_pre, T=T, P_tilde=Pt)
 
 

@@ -37,9 +37,13 @@ class _CQTensor(C.Structure):
                 ("bits", C.c_int32), ("group", C.c_int32)]
 
 
+QG_ROUND_STOCHASTIC, QG_ROUND_NEAREST = 0, 1
+
+
 class _CHyper(C.Structure):
     _fields_ = [("lr", C.c_float), ("alpha", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
-                ("eps", C.c_float), ("weight_decay", C.c_float), ("step", C.c_int64), ("seed", C.c_uint64)]
+                ("eps", C.c_float), ("weight_decay", C.c_float), ("step", C.c_int64), ("seed", C.c_uint64),
+                ("rounding", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _CStepItem(C.Structure):
@@ -186,9 +190,11 @@ class Hyper:
     weight_decay: float = 0.0
     step: int = 1
     seed: int = 0
+    rounding: int = 0        # QG_ROUND_STOCHASTIC (Sec. 3.4) or QG_ROUND_NEAREST (the ablation of Fig. 6)
 
     def c_struct(self) -> _CHyper:
-        return _CHyper(self.lr, self.alpha, self.beta1, self.beta2, self.eps, self.weight_decay, self.step, self.seed)
+        return _CHyper(self.lr, self.alpha, self.beta1, self.beta2, self.eps, self.weight_decay, self.step, self.seed,
+                       self.rounding, 0)
 
 
 def workspace_bytes(op: int, m: int, n: int, r: int) -> int:

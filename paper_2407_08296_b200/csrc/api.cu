@@ -131,10 +131,12 @@ static void fill_scalars(const qg_hyper* h, uint64_t seed, StepScalars* sc) {
   sc->lr_wd = (float)((double)h->lr * (double)h->weight_decay);
   sc->seed_lo = (uint32_t)(seed & 0xFFFFFFFFull); sc->seed_hi = (uint32_t)(seed >> 32);
   sc->step_lo = (uint32_t)((uint64_t)h->step & 0xFFFFFFFFull); sc->step_hi = (uint32_t)((uint64_t)h->step >> 32);
+  sc->rounding = h->rounding;
 }
 
 static int check_hyper(const qg_hyper* h) {
   if (!h || h->step < 1) return QG_INVALID_ARGUMENT;
+  if (h->rounding != QG_ROUND_STOCHASTIC && h->rounding != QG_ROUND_NEAREST) return QG_INVALID_ARGUMENT;
   if (!std::isfinite(h->lr) || !(h->beta1 >= 0.f && h->beta1 < 1.f) || !(h->beta2 >= 0.f && h->beta2 < 1.f))
     return QG_INVALID_ARGUMENT;
   return QG_OK;

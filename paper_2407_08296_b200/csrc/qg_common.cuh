@@ -54,6 +54,7 @@ struct StepScalars {
   float lr_alpha;          // lr * alpha
   float lr_wd;             // lr * weight_decay
   uint32_t seed_lo, seed_hi, step_lo, step_hi;
+  int32_t rounding;        // QG_ROUND_STOCHASTIC or QG_ROUND_NEAREST
 };
 
 // ----------------------------------------------------------------------------- device helpers

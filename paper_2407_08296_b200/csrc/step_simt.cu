@@ -150,7 +150,7 @@ struct RequantEpilogue {
     float h[8], c[8];
     sr_lanes8(sc, (uint32_t)i, (uint32_t)(j0 >> 3), h);
 #pragma unroll
-    for (int t = 0; t < 8; ++t) c[t] = sr_code(w[t], gp, h[t]);
+    for (int t = 0; t < 8; ++t) c[t] = sc.rounding == QG_ROUND_NEAREST ? rtn_code<8>(w[t], gp) : sr_code(w[t], gp, h[t]);
     if (nvalid == 8) {
       *reinterpret_cast<uint2*>(codes) = pack_int8x8(c);
     } else {

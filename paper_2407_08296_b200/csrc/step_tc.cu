@@ -612,6 +612,31 @@ __device__ __forceinline__ uint4 philox_rounds(uint4 c, const uint32_t* kx, cons
   return c;
 }
 
+// Round to nearest (ties to even) of 16 consecutive weights to codes of the new grid: the ablation of
+// Sec. 4.4.  FAST: rint(t) is read off the low mantissa bits of t + 1.5 * 2^23 (an even constant, so ties
+// fall as in rint), the integer zero point is added to the bits, the pack saturates.
+template <bool FAST>
+__device__ __forceinline__ uint4 rtn_codes16(const float* w, const GroupParams& gp) {
+  int code[16];
+  if (FAST) {
+    const float2 inv2 = make_float2(gp.inv, gp.inv), magic2 = make_float2(kMagic, kMagic);
+    const int cz = (int)gp.z - 0x4B400000;
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+      const float2 y = add2(mul2(make_float2(w[j], w[j + 1]), inv2), magic2);
+      code[j] = __float_as_int(y.x) + cz;                   // may leave [-128, 127]: the pack saturates
+      code[j + 1] = __float_as_int(y.y) + cz;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) code[j] = (int)rtn_code<8>(w[j], gp);
+  }
+  uint32_t o[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) o[k] = pack_sat_s8x4(code[4 * k], code[4 * k + 1], code[4 * k + 2], code[4 * k + 3]);
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 template <bool FAST>
 __device__ __forceinline__ uint4 sr_codes16(const float* w, const GroupParams& gp, const uint32_t h[8]) {
   int code[16];
@@ -791,6 +816,7 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
     const bool elected = (threadIdx.x == 64 + grp * S::kGroupThreads);
     const int bar_id = 1 + grp;
     const bool no_wd = (sc.lr_wd == 0.0f);
+    const bool nearest = (sc.rounding == QG_ROUND_NEAREST);
     float2* gpart = part + grp * 2 * kTileM;
     uint8_t* cbuf = code_base + grp * S::kCodeBytes;   // the group's own buffer for the INT8 codes of its tile
     // the codes of a tile are fetched by the group itself: the first tile here, each later one as soon as
@@ -902,10 +928,15 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
       auto pass2_piece = [&](int pc, const uint32_t* wbits) {
         const int col = n0 + myc0 + 16 * pc;
         const float* w = reinterpret_cast<const float*>(wbits);
-        const uint4 x0 = philox_rounds(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
-        const uint4 x1 = philox_rounds(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
-        const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-        const uint4 out = fast_sr ? sr_codes16<true>(w, gp, h) : sr_codes16<false>(w, gp, h);
+        uint4 out;
+        if (nearest) {
+          out = fast_sr ? rtn_codes16<true>(w, gp) : rtn_codes16<false>(w, gp);
+        } else {
+          const uint4 x0 = philox_rounds(make_uint4((uint32_t)(col >> 3), (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
+          const uint4 x1 = philox_rounds(make_uint4((uint32_t)(col >> 3) + 1u, (uint32_t)gi, sc.step_lo, sc.step_hi), kx, ky);
+          const uint32_t h[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+          out = fast_sr ? sr_codes16<true>(w, gp, h) : sr_codes16<false>(w, gp, h);
+        }
         // sixteen new codes of this row, straight to global memory (the two halves of a 32-byte sector are
         // written by consecutive pieces and merge in L2); the ragged end of a row byte by byte
         if (row_ok && col + 16 <= pn) {

@@ -82,7 +82,7 @@ def check_direction(gpu, ref, hyp, name="N", tol=2e-3):
     return float(ill.mean())
 
 
-def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_frac=1e-3, col0=0):
+def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_frac=1e-3, col0=0, rounding="sr"):
     """INT8 weights after one step against the oracle's (same direction N_b on both sides).
 
     Scales agree to 1e-5 relative and zero points exactly wherever the group's scaled minimum is
@@ -108,9 +108,12 @@ def check_weight_codes(gpu_w: O.QTensor, out: dict, seed: int, step: int, max_fr
     assert frac_bad <= max_frac, f"{frac_bad:.2e} of the weight codes differ"
     if bad.any():
         T = out["T"].astype(np.float64)
-        h = O.sr_uniform16(seed, step, m, n, col0=col0).astype(np.float64)
         fr = (T - np.floor(T)) * 65536.0
-        near_draw = np.abs(fr - h) <= 1e-3 * 65536 + 1
+        if rounding == "rtn":                                  # the boundary of round-to-nearest is the half
+            near_draw = np.abs(fr - 32768.0) <= 1e-3 * 65536
+        else:
+            h = O.sr_uniform16(seed, step, m, n, col0=col0).astype(np.float64)
+            near_draw = np.abs(fr - h) <= 1e-3 * 65536 + 1
         near_int = (fr <= 1e-3 * 65536) | (fr >= (1 - 1e-3) * 65536)
         zeros_el = ref_w.zeros[:, gcols]
         lvl = np.floor(T) + zeros_el
@@ -168,7 +171,8 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
     try:
         B.project_step(dG, dP, dW, dM, dV,
                        B.Hyper(lr=hyp.lr, alpha=hyp.alpha, beta1=hyp.beta1, beta2=hyp.beta2, eps=hyp.eps,
-                               weight_decay=hyp.weight_decay, step=hyp.step, seed=hyp.seed),
+                               weight_decay=hyp.weight_decay, step=hyp.step, seed=hyp.seed,
+                               rounding=B.QG_ROUND_NEAREST if hyp.rounding == "rtn" else B.QG_ROUND_STOCHASTIC),
                        status=status, debug=taps.as_dict())
         torch.cuda.synchronize()
     finally:
@@ -187,7 +191,7 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
     wpre_err = float((np.abs(taps.W_pre.cpu().numpy() - forced["W_pre"]) / lsb).max())
     assert wpre_err <= 1e-3, f"pre-rounding weight off by {wpre_err:.2e} LSB"
     gw = from_device_q(dW)
-    frac = check_weight_codes(gw, forced, hyp.seed, hyp.step)
+    frac = check_weight_codes(gw, forced, hyp.seed, hyp.step, rounding=hyp.rounding)
     frac_unforced = check_weight_codes_unforced(gw, ref)
     # padding of the rows is never written
     if dW.ld > n:

@@ -358,3 +358,37 @@ def test_plan_at_llama7b_sizes_on_sampled_column_blocks():
     def blocks(n):
         return [(0, 256), (n - 256, n)]
     _full_size_case([(4096, 4096, 1024), (4096, 11008, 1024), (11008, 4096, 1024)], blocks, seed=22)
+
+
+# ----------------------------------------------------------------------------- round to nearest (Sec. 4.4 ablation)
+@pytest.mark.parametrize("shape", [(512, 1376, 128), (300, 777, 96), (2048, 2048, 512)])
+@pytest.mark.parametrize("impl", [None, 1])
+def test_step_with_round_to_nearest(shape, impl):
+    m, n, r = shape
+    if impl == 1 and m > 1024:
+        pytest.skip("the CUDA-core cross-check is run on the small shapes")
+    gm = synth.GradientModel(m, n, seed=9, matrix_index=0)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=9), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 9), 8)
+    M = np.zeros((r, n), np.float32)
+    V = np.zeros((r, n), np.float32)
+    o = O.project_step(gm.sample(1), P, W, M, V, O.Hyper(step=1, seed=2, rounding="rtn"))
+    stats = run_and_check_step(gm.sample(2), P, o["W"], o["M"], o["V"], O.Hyper(step=2, seed=2, rounding="rtn"), impl=impl)
+    assert stats["mismatch"] <= 1e-3
+
+
+def test_round_to_nearest_ignores_the_seed_and_a_bad_mode_is_refused():
+    m, n, r = 256, 512, 64
+    gb = synth.GradientModel(m, n, seed=4, matrix_index=0).sample(1)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=4), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 4), 8)
+    z = np.zeros((r, n), np.float32)
+    outs = []
+    for seed in (5, 6):
+        dW, dM, dV = to_device_q(W), f32_to_device(z), f32_to_device(z)
+        B.project_step(g_to_device(gb), to_device_q(P), dW, dM, dV, B.Hyper(step=3, seed=seed, rounding=B.QG_ROUND_NEAREST))
+        outs.append(dW.codes.cpu().numpy().copy())
+    assert np.array_equal(outs[0], outs[1])
+    with pytest.raises(B.QgError):
+        B.project_step(g_to_device(gb), to_device_q(P), to_device_q(W), f32_to_device(z), f32_to_device(z),
+                       B.Hyper(step=1, rounding=7))

@@ -498,3 +498,29 @@ def test_step_of_a_column_block_equals_the_block_of_the_full_step():
     Wb = O.QTensor(W.codes[:, 256:512], W.scales[:, 1:2], W.zeros[:, 1:2], 8)
     assert not np.array_equal(O.project_step(gb[:, 256:512], P, Wb, M[:, 256:512], V[:, 256:512], hyp)["W"].codes,
                               full["W"].codes[:, 256:512])
+
+
+def test_round_to_nearest_step_is_the_same_step_with_quant8_at_the_end():
+    # Sec. 4.4 (Fig. 6) ablates stochastic rounding against round to nearest: everything before the last
+    # quantization is untouched by the choice, the nearest codes are Quant_8 of the pre-rounding weight, no
+    # code is further than one level from the stochastic one, and the seed no longer matters.
+    from paper_2407_08296_b200 import synth
+    m, n, r = 64, 256 + 85, 32
+    gb = synth.GradientModel(m, n, seed=5, matrix_index=0).sample(1)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=5), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 5), 8)
+    z = np.zeros((r, n), np.float32)
+    sr = O.project_step(gb, P, W, z, z, O.Hyper(step=1, seed=3))
+    rtn = O.project_step(gb, P, W, z, z, O.Hyper(step=1, seed=3, rounding="rtn"))
+    rtn2 = O.project_step(gb, P, W, z, z, O.Hyper(step=1, seed=4, rounding="rtn"))
+    sr2 = O.project_step(gb, P, W, z, z, O.Hyper(step=1, seed=4))
+    assert np.array_equal(sr["W_pre"], rtn["W_pre"]) and np.array_equal(sr["M"], rtn["M"]) and np.array_equal(sr["V"], rtn["V"])
+    assert np.array_equal(sr["W"].scales, rtn["W"].scales) and np.array_equal(sr["W"].zeros, rtn["W"].zeros)
+    q8 = O.quantize_rtn(rtn["W_pre"], 8)
+    assert np.array_equal(rtn["W"].codes, q8.codes)
+    d = np.abs(rtn["W"].codes.astype(np.int32) - sr["W"].codes.astype(np.int32))
+    assert d.max() == 1 and 0.2 < (d != 0).mean() < 0.8          # a coin per element, never two levels
+    assert np.array_equal(rtn["W"].codes, rtn2["W"].codes) and not np.array_equal(sr["W"].codes, sr2["W"].codes)
+    # nearest: the dequantized result is within half a level of the pre-rounding weight inside the clamp range
+    lsb = np.repeat(rtn["W"].scales, 256, axis=1)[:, :n]
+    assert np.all(np.abs(O.dequantize(rtn["W"]) - rtn["W_pre"]) <= 0.5 * lsb * (1 + 1e-5) + 1e-12)
