@@ -1188,13 +1188,8 @@ struct DequantItem {
 // nibble (code + 8) is dropped into the mantissa of 2^23 and (2^23 + 8 + z) subtracted, which gives q - z
 // exactly without an integer-to-float conversion.
 __global__ void __launch_bounds__(256)
-dequant_p_grouped_kernel(const DequantItem* __restrict__ items, int nitems) {
-  int lo = 0, hi = nitems - 1;
-  while (lo < hi) {                                  // last item whose block0 <= blockIdx.x
-    const int mid = (lo + hi + 1) >> 1;
-    if (items[mid].block0 <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
-  }
-  const DequantItem& it = items[lo];
+dequant_p_grouped_kernel(const DequantItem* __restrict__ items, const int32_t* __restrict__ block_item) {
+  const DequantItem& it = items[__ldg(block_item + blockIdx.x)];   // host-made map: block -> matrix of the chunk
   const uint32_t cols = (uint32_t)it.P.cols, rows = (uint32_t)it.P.rows;
   const uint32_t per_row = cols / 32, ngroups = (cols + kGroup - 1) / kGroup;
   const uint32_t idx = (blockIdx.x - (uint32_t)it.block0) * blockDim.x + threadIdx.x;
@@ -1256,6 +1251,7 @@ struct PlanChunk {
   int dq_blocks;
   int k1_grid, k2_grid, pairs, k1_pairs, k1p_tiles;
   size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
+  size_t dq_map_off;                                                // same: block -> item map of the dequantize launch
 };
 
 struct Plan {
@@ -1310,6 +1306,7 @@ size_t plan_table_bytes(const StepArgs* items, int32_t count) {
     const int64_t k1 = ceil_div(items[i].r, kTileM) * ceil_div(items[i].n, 128);
     const int64_t k2 = ceil_div(items[i].m, kTileM) * ceil_div(items[i].n, K2Smem::kBN);
     sched += (size_t)(2 * (k1 + k2)) + 2 * (size_t)(sm_count() + 3);
+    sched += (size_t)ceil_div(items[i].m * (items[i].r / 32), 256) + 2;      // block -> matrix map of the dequantize launch
   }
   return (size_t)round_up((int64_t)count * sizeof(TcProblem), 256) + (size_t)round_up((int64_t)count * sizeof(DequantItem), 256) +
          sched * sizeof(int32_t) + 256;
@@ -1349,6 +1346,7 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     size_t off = 0;
     std::vector<int2> t1, t2;
     std::vector<float> c1, c2;
+    std::vector<int32_t> dq_map;
     for (int k = i; k < j; ++k) {
       const StepArgs& a = items[k];
       const TcScratch w = carve(reinterpret_cast<char*>(workspace) + off, a.m, a.n, a.r);
@@ -1368,6 +1366,7 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       dq[k].block0 = ch.dq_blocks;
       dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 32), 256);
       ch.dq_blocks += dq[k].nblocks;
+      for (int32_t blk = 0; blk < dq[k].nblocks; ++blk) dq_map.push_back(k - i);
     }
     if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
     else ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
@@ -1377,6 +1376,9 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     schedule_tiles(t1, c1, ch.k1_pairs ? ch.k1_grid / 2 : ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);
     if (sched.size() & 1) sched.push_back(0);
     schedule_tiles(t2, c2, ch.pairs ? ch.k2_grid / 2 : ch.k2_grid, sched, &ch.k2_start_off, &ch.k2_items_off);
+    if (sched.size() & 1) sched.push_back(0);
+    ch.dq_map_off = sched.size();
+    sched.insert(sched.end(), dq_map.begin(), dq_map.end());
     if (sched.size() & 1) sched.push_back(0);
     plan->chunks.push_back(ch);
     i = j;
@@ -1410,7 +1412,7 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
   size_t c = 0;
   for (const PlanChunk& ch : plan->chunks) {
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 0], st));
-    dequant_p_grouped_kernel<<<ch.dq_blocks, 256, 0, st>>>(plan->dq_dev + ch.first, ch.count);
+    dequant_p_grouped_kernel<<<ch.dq_blocks, 256, 0, st>>>(plan->dq_dev + ch.first, plan->sched_dev + ch.dq_map_off);
     QG_LAUNCH_CHECK();
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 1], st));
     const TcProblem* tab = plan->table_dev + ch.first;
