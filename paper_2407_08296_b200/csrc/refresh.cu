@@ -120,9 +120,9 @@ int refresh_sm_count() {
   return sms;
 }
 
-constexpr int kSplitTiles = 64;          // products with fewer output tiles than this split their K range
-constexpr int kSplitMinK = 256;          // ... into slices no shorter than this
-constexpr int64_t kSplitScratch = 8 << 20;   // bytes of partial sums a product may use
+constexpr int kSplitTiles = 160;         // products with fewer output tiles than this split their K range
+constexpr int kSplitMinK = 128;          // ... into slices no shorter than this
+constexpr int64_t kSplitScratch = 32 << 20;  // bytes of partial sums a product may use
 
 // `part` (kSplitScratch bytes, or null) lets a product with few output tiles and a long K run as slices.
 template <class TA, class ACC, class TC>
@@ -458,7 +458,7 @@ int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cu
       // C = Q[:, :j0]^T Yj   (j0 x 64);   Yj -= Q[:, :j0] C
       rc = gemm<float, float, float>(w.Q, 1, b, Yj, b, 1, w.Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st, w.part);
       if (rc != QG_OK) return rc;
-      rc = gemm<float, float, float>(w.Q, b, 1, w.Cb, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st);
+      rc = gemm<float, float, float>(w.Q, b, 1, w.Cb, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st, w.part);
       if (rc != QG_OK) return rc;
     }
     // two rounds of Cholesky QR on the panel: Yj -> Wp -> Qj
@@ -516,9 +516,11 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
   {
     unsigned long long* off = reinterpret_cast<unsigned long long*>(w.off);
     unsigned int* sync_words = reinterpret_cast<unsigned int*>(w.done);
-    if (b <= 8 * kTeam) rc = launch_jacobi<8>(w.T, b, sweeps, 1e-9, off, sync_words, status, st);
-    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(w.T, b, sweeps, 1e-9, off, sync_words, status, st);
-    else rc = launch_jacobi<32>(w.T, b, sweeps, 1e-9, off, sync_words, status, st);
+    // the iteration converges quadratically at the end: a sweep that met nothing above 1e-5 leaves ~1e-10
+    constexpr double kTol = 1e-5;
+    if (b <= 8 * kTeam) rc = launch_jacobi<8>(w.T, b, sweeps, kTol, off, sync_words, status, st);
+    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(w.T, b, sweeps, kTol, off, sync_words, status, st);
+    else rc = launch_jacobi<32>(w.T, b, sweeps, kTol, off, sync_words, status, st);
     if (rc != QG_OK) return rc;
   }
   row_norm_kernel<<<(unsigned)b, 128, 0, st>>>(w.T, (int)b, w.lam);
