@@ -19,13 +19,15 @@
  *     during the call.
  *   - Matrices are row-major with a row pitch ("ld") in ELEMENTS.  Base pointers must be
  *     16-byte aligned and every row pitch a multiple of 16 bytes, i.e. ld % 8 == 0 for bf16,
- *     ld % 4 == 0 for fp32, ld % 16 == 0 for INT8 codes, ld % 32 == 0 for INT4 codes.
+ *     ld % 4 == 0 for fp32, ld % 16 == 0 for INT8 codes, ld % 32 == 0 for INT4, ld % 64 == 0 for INT2 codes.
  *     Elements between cols and ld are padding: never read as data, never written.
  *   - Quantization groups (Sec. 3.1, "block-wise", block 256) are runs of `group` consecutive
  *     elements along a row and restart at every row; a row whose length is not a multiple of
  *     `group` ends in one shorter group.  scales/zeros are dense [rows][ceil(cols/group)] fp32.
  *   - INT4 codes are packed two per byte: byte k of a row holds column 2k in its low nibble
  *     and column 2k+1 in its high nibble, each stored as code + 8 (codes lie in [-8, 7]).
+ *     INT2 codes (the 2-bit projection of the ablation in Sec. 4.4) are packed four per byte:
+ *     column 4k + i of a row sits in bits 2i, 2i + 1 of byte k, stored as code + 2 (codes in [-2, 1]).
  *   - A device status word (int32, optional, may be NULL) is OR-ed with QG_DEV_* flags when a
  *     kernel gives up a bounded wait or an iteration does not converge; it is never cleared
  *     by the library.
@@ -63,11 +65,11 @@ typedef enum {
 
 /* A block-wise quantized matrix (Sec. 3.1; App. A: W = (codes - zeros) * scales). */
 typedef struct {
-  void*   codes;   /* device; bits == 8: int8 [rows][ld]; bits == 4: uint8 [rows][ld / 2]  */
+  void*   codes;   /* device; bits == 8: int8 [rows][ld]; 4: uint8 [rows][ld / 2]; 2: uint8 [rows][ld / 4] */
   float*  scales;  /* device; [rows][ceil(cols / group)]                                    */
   float*  zeros;   /* device; same shape, integer valued                                    */
   int64_t rows, cols, ld;
-  int32_t bits;    /* 4 or 8                                                                */
+  int32_t bits;    /* 8 (weights, projection), 4 (projection, the method), 2 (projection)   */
   int32_t group;   /* 256                                                                   */
 } qg_qtensor;
 
@@ -98,8 +100,11 @@ typedef struct {
  * ld_src).  Per group: s = (max - min) / (2^bits - 1), z = -2^(bits-1) - rint(min / s),
  * code = clamp(rint(x / s) + z); x / s is evaluated as x * (1 / s) in binary32, ties to even.
  * A constant group takes z = 0, s = |max| (1 if that is 0).  dst->rows/cols must equal
- * rows/cols, dst->bits must be 4 (resp. 8).  Bit-exact against the CPU oracle. */
+ * rows/cols, dst->bits must be 4 (resp. 8, 2).  Bit-exact against the CPU oracle.
+ * qgalore_quantize_int2 is Quant_2, for the 2-bit projection of the ablation in Sec. 4.4 (Fig. 3). */
 QG_API int qgalore_quantize_int4(const float* src, int64_t rows, int64_t cols, int64_t ld_src,
+                          const qg_qtensor* dst, void* stream);
+QG_API int qgalore_quantize_int2(const float* src, int64_t rows, int64_t cols, int64_t ld_src,
                           const qg_qtensor* dst, void* stream);
 QG_API int qgalore_quantize_int8(const float* src, int64_t rows, int64_t cols, int64_t ld_src,
                           const qg_qtensor* dst, void* stream);
@@ -109,7 +114,7 @@ QG_API int qgalore_dequantize(const qg_qtensor* src, float* dst, int64_t ld_dst,
 
 /* --- Sec. 3.5 (with Sec. 3.4 for the write-back): one optimizer step of one matrix ------
  * G       bf16 bit patterns, m x n, pitch ldg                        (read)
- * P       INT4, m x r                                                (read)
+ * P       INT4 (the method; INT2 or INT8 for the ablation of Sec. 4.4), m x r   (read)
  * W       INT8, m x n: codes, scales and zeros are replaced          (read + write)
  * M, V    fp32, r x n, pitch ldmv                                    (read + write)
  * h       host; step >= 1

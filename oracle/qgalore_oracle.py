@@ -36,7 +36,7 @@ import scipy.linalg
 __all__ = [
     "GROUP", "fl32", "bf16_round", "bf16_bits_to_f32", "f32_to_bf16_bits",
     "philox4x32_10", "sr_uniform16", "group_params", "quantize_rtn", "quantize_sr",
-    "dequantize", "pack_int4", "unpack_int4", "QTensor", "Hyper", "project_step",
+    "dequantize", "pack_int4", "unpack_int4", "pack_int2", "unpack_int2", "QTensor", "Hyper", "project_step",
     "refresh_subspace", "subspace_similarity", "GateState", "gate_update",
     "principal_angle",
 ]
@@ -262,6 +262,24 @@ def unpack_int4(packed, cols):
     return (out[:, :cols] - 8).astype(np.int8)
 
 
+def pack_int2(codes):
+    """Four INT2 codes per byte: column 4k + i of a row in bits 2i, 2i + 1 of byte k, stored as q + 2."""
+    rows, cols = codes.shape
+    u = (codes.astype(np.int16) + 2).astype(np.uint8)
+    pad = (-cols) % 4
+    if pad:
+        u = np.concatenate([u, np.full((rows, pad), 2, dtype=np.uint8)], axis=1)
+    return (u[:, 0::4] | (u[:, 1::4] << np.uint8(2)) | (u[:, 2::4] << np.uint8(4)) | (u[:, 3::4] << np.uint8(6))).astype(np.uint8)
+
+
+def unpack_int2(packed, cols):
+    packed = np.asarray(packed, dtype=np.uint8)
+    out = np.empty((packed.shape[0], packed.shape[1] * 4), dtype=np.int16)
+    for i in range(4):
+        out[:, i::4] = (packed >> np.uint8(2 * i)) & np.uint8(3)
+    return (out[:, :cols] - 2).astype(np.int8)
+
+
 # --------------------------------------------------------------------------- the step (Sec. 3.5)
 @dataclass
 class Hyper:
@@ -334,12 +352,12 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
 
 
 # --------------------------------------------------------------------------- refresh (Sec. 3.5, Sec. 1)
-def refresh_subspace(G_bits, r, group=GROUP):
+def refresh_subspace(G_bits, r, group=GROUP, bits=4):
     """Projection matrix from the SVD of the gradient: the top-r left singular vectors.
 
     Exact LAPACK SVD (gesdd) of the gradient widened to fp64.  Each column's sign is
     fixed so that its largest-magnitude entry is positive.  Returns (P float32 m x r,
-    its INT4 quantization, singular values).
+    its quantization (INT4 is the method, Sec. 3.3; 2 and 8 bits are the ablation of Sec. 4.4), singular values).
     """
     G = bf16_bits_to_f32(G_bits).astype(np.float64)
     U, S, _ = scipy.linalg.svd(G, full_matrices=False, lapack_driver="gesdd")
@@ -348,7 +366,7 @@ def refresh_subspace(G_bits, r, group=GROUP):
     sgn = np.sign(P[piv, np.arange(P.shape[1])])
     sgn[sgn == 0] = 1.0
     P = fl32(P * sgn[None, :])
-    return P, quantize_rtn(P, 4, group), S
+    return P, quantize_rtn(P, bits, group), S
 
 
 def principal_angle(P_ref, P_test):

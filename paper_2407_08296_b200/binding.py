@@ -72,6 +72,7 @@ def lib() -> C.CDLL:
         qp = C.POINTER(_CQTensor)
         L.qgalore_quantize_int4.argtypes = [vp, i64, i64, i64, qp, vp]
         L.qgalore_quantize_int8.argtypes = [vp, i64, i64, i64, qp, vp]
+        L.qgalore_quantize_int2.argtypes = [vp, i64, i64, i64, qp, vp]
         L.qgalore_dequantize.argtypes = [qp, vp, i64, vp]
         L.qgalore_project_step.argtypes = [vp, i64, i64, i64, i64, qp, qp, vp, vp, i64, C.POINTER(_CHyper),
                                            vp, sz, vp, C.POINTER(_CDebug), vp]
@@ -147,8 +148,8 @@ def _matrix_ld(t: torch.Tensor, what: str) -> int:
 class QTensor:
     """A block-wise quantized matrix on the device (Sec. 3.1): codes, per-group scales and zeros.
 
-    ``codes`` is int8 [rows, cols] (a view with pitch ld) for bits == 8, and uint8 [rows, ld // 2]
-    holding two codes per byte for bits == 4.
+    ``codes`` is int8 [rows, cols] (a view with pitch ld) for bits == 8, uint8 [rows, ld // 2]
+    holding two codes per byte for bits == 4, uint8 [rows, ld // 4] holding four per byte for bits == 2.
     """
     codes: torch.Tensor
     scales: torch.Tensor
@@ -166,8 +167,10 @@ class QTensor:
             codes = torch.zeros((rows, ld), dtype=torch.int8, device=device)
         elif bits == 4:
             codes = torch.full((rows, ld // 2), 0x88, dtype=torch.uint8, device=device)
+        elif bits == 2:
+            codes = torch.full((rows, ld // 4), 0xAA, dtype=torch.uint8, device=device)
         else:
-            raise ValueError("bits must be 4 or 8")
+            raise ValueError("bits must be 2, 4 or 8")
         return QTensor(codes, torch.zeros((rows, ng), dtype=torch.float32, device=device),
                        torch.zeros((rows, ng), dtype=torch.float32, device=device), rows, cols, ld, bits)
 
@@ -223,6 +226,10 @@ def quantize_int4(src: torch.Tensor, out: QTensor | None = None, stream=None) ->
 
 def quantize_int8(src: torch.Tensor, out: QTensor | None = None, stream=None) -> QTensor:
     return _quantize("qgalore_quantize_int8", 8, src, out, stream)
+
+
+def quantize_int2(src: torch.Tensor, out: QTensor | None = None, stream=None) -> QTensor:
+    return _quantize("qgalore_quantize_int2", 2, src, out, stream)
 
 
 def dequantize(q: QTensor, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:

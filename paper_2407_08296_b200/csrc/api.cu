@@ -48,7 +48,7 @@ static int check_qtensor(const qg_qtensor* t, int bits) {
   if (!aligned16(t->codes) || (reinterpret_cast<uintptr_t>(t->scales) & 3u) ||
       (reinterpret_cast<uintptr_t>(t->zeros) & 3u))
     return QG_MISALIGNED;
-  if (t->ld % (bits == 8 ? 16 : 32) != 0) return QG_MISALIGNED;
+  if (t->ld % (128 / bits) != 0) return QG_MISALIGNED;      // a row of codes is a multiple of 16 bytes
   return QG_OK;
 }
 
@@ -89,6 +89,11 @@ int qgalore_quantize_int4(const float* src, int64_t rows, int64_t cols, int64_t 
   return quantize_common(4, src, rows, cols, ld_src, dst, stream);
 }
 
+int qgalore_quantize_int2(const float* src, int64_t rows, int64_t cols, int64_t ld_src, const qg_qtensor* dst,
+                          void* stream) {
+  return quantize_common(2, src, rows, cols, ld_src, dst, stream);
+}
+
 int qgalore_quantize_int8(const float* src, int64_t rows, int64_t cols, int64_t ld_src, const qg_qtensor* dst,
                           void* stream) {
   return quantize_common(8, src, rows, cols, ld_src, dst, stream);
@@ -96,7 +101,8 @@ int qgalore_quantize_int8(const float* src, int64_t rows, int64_t cols, int64_t 
 
 int qgalore_dequantize(const qg_qtensor* src, float* dst, int64_t ld_dst, void* stream) {
   if (!src || !dst) return QG_INVALID_ARGUMENT;
-  int rc = check_qtensor(src, src->bits == 4 ? 4 : 8);
+  if (src->bits != 2 && src->bits != 4 && src->bits != 8) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(src, src->bits);
   if (rc != QG_OK) return rc;
   if (ld_dst < src->cols) return QG_INVALID_ARGUMENT;
   if (!aligned16(dst) || ld_dst % 4 != 0) return QG_MISALIGNED;
@@ -147,7 +153,8 @@ static int check_matrix(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, in
                         const qg_qtensor* W, float* M, float* V, int64_t ldmv, StepArgs* a) {
   if (!G || !M || !V) return QG_INVALID_ARGUMENT;
   if (m <= 0 || n <= 0 || r <= 0 || ldg < n || ldmv < n) return QG_INVALID_ARGUMENT;
-  int rc = check_qtensor(P, 4);
+  if (!P || (P->bits != 2 && P->bits != 4 && P->bits != 8)) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(P, P->bits);
   if (rc != QG_OK) return rc;
   rc = check_qtensor(W, 8);
   if (rc != QG_OK) return rc;
@@ -287,11 +294,13 @@ int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
                              size_t workspace_bytes, int32_t* status_dev, void* stream) {
   if (!G || !workspace || m <= 0 || n <= 0 || r <= 0 || ldg < n || iters < 0 || oversample_cols < 0)
     return QG_INVALID_ARGUMENT;
-  int rc = check_qtensor(P_new, 4);
+  if (!P_new || (P_new->bits != 2 && P_new->bits != 4 && P_new->bits != 8)) return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(P_new, P_new->bits);
   if (rc != QG_OK) return rc;
   if (P_new->rows != m || P_new->cols != r || P_new->ld != r) return QG_INVALID_ARGUMENT;
   if (P_prev) {
-    rc = check_qtensor(P_prev, 4);
+    if (P_prev->bits != 2 && P_prev->bits != 4 && P_prev->bits != 8) return QG_INVALID_ARGUMENT;
+    rc = check_qtensor(P_prev, P_prev->bits);
     if (rc != QG_OK) return rc;
     if (P_prev->rows != m || P_prev->cols != r) return QG_INVALID_ARGUMENT;
   }
@@ -318,9 +327,11 @@ int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
 int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,
                                 void* workspace, size_t workspace_bytes, void* stream) {
   if (!sim_dev || !workspace) return QG_INVALID_ARGUMENT;
-  int rc = check_qtensor(A, 4);
+  if (!A || !B || (A->bits != 2 && A->bits != 4 && A->bits != 8) || (B->bits != 2 && B->bits != 4 && B->bits != 8))
+    return QG_INVALID_ARGUMENT;
+  int rc = check_qtensor(A, A->bits);
   if (rc != QG_OK) return rc;
-  rc = check_qtensor(B, 4);
+  rc = check_qtensor(B, B->bits);
   if (rc != QG_OK) return rc;
   if (A->rows != B->rows || A->cols != B->cols) return QG_INVALID_ARGUMENT;
   const int32_t c = (sim_cols <= 0 || sim_cols > A->cols) ? (int32_t)A->cols : sim_cols;

@@ -159,6 +159,47 @@ __device__ __forceinline__ void unpack_int4x8(uint32_t w, float q[8]) {
   for (int i = 0; i < 8; ++i) q[i] = (float)((int)((w >> (4 * i)) & 0xFu) - 8);
 }
 
+// Eight INT2 codes (one uint16, stored as code + 2, column 8k + i in bits 2i, 2i + 1) -> floats in [-2, 1].
+__device__ __forceinline__ void unpack_int2x8(uint32_t w, float q[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) q[i] = (float)((int)((w >> (2 * i)) & 0x3u) - 2);
+}
+
+// Bytes per row of codes and per eight codes, for the three widths the projection may take (Sec. 4.4, Fig. 3).
+__device__ __forceinline__ int64_t code_row_bytes(const qg_qtensor& T) { return T.bits == 8 ? T.ld : (T.bits == 4 ? T.ld / 2 : T.ld / 4); }
+
+// Codes of columns c0 .. c0 + 7 (c0 a multiple of 8) of a row as floats; the first nvalid are real.
+__device__ __forceinline__ void load_codes8(const qg_qtensor& T, int64_t row, int64_t c0, int nvalid, float q[8]) {
+  const uint8_t* base = (const uint8_t*)T.codes + row * code_row_bytes(T);
+  if (T.bits == 8) {
+    const uint8_t* p = base + c0;
+    if (nvalid == 8) {
+      unpack_int8x8(__ldg(reinterpret_cast<const uint2*>(p)), q);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) q[i] = (i < nvalid) ? (float)(int8_t)p[i] : 0.0f;
+    }
+  } else if (T.bits == 4) {
+    const uint8_t* p = base + (c0 >> 1);
+    uint32_t w = 0;
+    if (nvalid == 8) {
+      w = __ldg(reinterpret_cast<const uint32_t*>(p));
+    } else {
+      for (int i = 0; i < (nvalid + 1) / 2; ++i) w |= (uint32_t)p[i] << (8 * i);
+    }
+    unpack_int4x8(w, q);
+  } else {
+    const uint8_t* p = base + (c0 >> 2);
+    uint32_t w = 0;
+    if (nvalid == 8) {
+      w = __ldg(reinterpret_cast<const uint16_t*>(p));
+    } else {
+      for (int i = 0; i < (nvalid + 3) / 4; ++i) w |= (uint32_t)p[i] << (8 * i);
+    }
+    unpack_int2x8(w, q);
+  }
+}
+
 #endif  // __CUDACC__
 
 // ----------------------------------------------------------------------------- kernel launchers

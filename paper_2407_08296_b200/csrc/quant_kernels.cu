@@ -60,7 +60,7 @@ quantize_rtn_kernel(const float* __restrict__ src, int64_t ld_src, int64_t rows,
     } else {
       for (int i = 0; i < nvalid; ++i) out[i] = (uint8_t)(q[i] & 0xFF);
     }
-  } else {
+  } else if (BITS == 4) {
     uint8_t* out = codes + row * ld_code_bytes + (c0 >> 1);
     uint32_t w = 0;
 #pragma unroll
@@ -69,6 +69,16 @@ quantize_rtn_kernel(const float* __restrict__ src, int64_t ld_src, int64_t rows,
       *reinterpret_cast<uint32_t*>(out) = w;
     } else {
       for (int i = 0; i < (nvalid + 1) / 2; ++i) out[i] = (uint8_t)((w >> (8 * i)) & 0xFF);
+    }
+  } else {
+    uint8_t* out = codes + row * ld_code_bytes + (c0 >> 2);
+    uint32_t w = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) w |= (uint32_t)(((i < nvalid ? q[i] : 0) + 2) & 0x3) << (2 * i);   // padding holds code 0
+    if (nvalid == 8) {
+      *reinterpret_cast<uint16_t*>(out) = (uint16_t)w;
+    } else {
+      for (int i = 0; i < (nvalid + 3) / 4; ++i) out[i] = (uint8_t)((w >> (8 * i)) & 0xFF);
     }
   }
 }
@@ -82,46 +92,30 @@ int launch_quantize_rtn(int bits, const float* src, int64_t rows, int64_t cols, 
   if (bits == 8) {
     quantize_rtn_kernel<8><<<(unsigned)blocks, 256, 0, st>>>(src, ld_src, rows, cols, (uint8_t*)dst->codes, dst->ld,
                                                              dst->scales, dst->zeros, ngroups);
-  } else {
+  } else if (bits == 4) {
     quantize_rtn_kernel<4><<<(unsigned)blocks, 256, 0, st>>>(src, ld_src, rows, cols, (uint8_t*)dst->codes,
                                                              dst->ld / 2, dst->scales, dst->zeros, ngroups);
+  } else {
+    quantize_rtn_kernel<2><<<(unsigned)blocks, 256, 0, st>>>(src, ld_src, rows, cols, (uint8_t*)dst->codes,
+                                                             dst->ld / 4, dst->scales, dst->zeros, ngroups);
   }
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
 
 // ------------------------------------------------------------------------ dequantize
-template <int BITS>
 __global__ void __launch_bounds__(256)
-dequantize_kernel(const uint8_t* __restrict__ codes, int64_t ld_code_bytes, const float* __restrict__ scales,
-                  const float* __restrict__ zeros, int ngroups, int64_t rows, int64_t cols,
-                  float* __restrict__ dst, int64_t ld_dst) {
-  const int64_t chunks_per_row = ceil_div(cols, 8);
+dequantize_kernel(qg_qtensor T, int ngroups, float* __restrict__ dst, int64_t ld_dst) {
+  const int64_t chunks_per_row = ceil_div(T.cols, 8);
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= rows * chunks_per_row) return;
+  if (idx >= T.rows * chunks_per_row) return;
   const int64_t row = idx / chunks_per_row;
   const int64_t c0 = (idx % chunks_per_row) * 8;
-  const int nvalid = (int)min((int64_t)8, cols - c0);
+  const int nvalid = (int)min((int64_t)8, T.cols - c0);
   const int g = (int)(c0 / kGroup);
-  const float s = __ldg(scales + row * ngroups + g), z = __ldg(zeros + row * ngroups + g);
+  const float s = __ldg(T.scales + row * ngroups + g), z = __ldg(T.zeros + row * ngroups + g);
   float q[8];
-  if (BITS == 8) {
-    const uint8_t* p = codes + row * ld_code_bytes + c0;
-    if (nvalid == 8) {
-      unpack_int8x8(__ldg(reinterpret_cast<const uint2*>(p)), q);
-    } else {
-      for (int i = 0; i < 8; ++i) q[i] = (i < nvalid) ? (float)(int8_t)p[i] : 0.0f;
-    }
-  } else {
-    const uint8_t* p = codes + row * ld_code_bytes + (c0 >> 1);
-    uint32_t w = 0;
-    if (nvalid == 8) {
-      w = __ldg(reinterpret_cast<const uint32_t*>(p));
-    } else {
-      for (int i = 0; i < (nvalid + 1) / 2; ++i) w |= (uint32_t)p[i] << (8 * i);
-    }
-    unpack_int4x8(w, q);
-  }
+  load_codes8(T, row, c0, nvalid, q);
   float* out = dst + row * ld_dst + c0;
 #pragma unroll
   for (int i = 0; i < 8; ++i)
@@ -133,13 +127,7 @@ int launch_dequantize(const qg_qtensor* src, float* dst, int64_t ld_dst, cudaStr
   const int64_t threads = src->rows * ceil_div(src->cols, 8);
   const int64_t blocks = ceil_div(threads, 256);
   if (blocks > 0x7FFFFFFFll) return QG_UNSUPPORTED_SHAPE;
-  if (src->bits == 8) {
-    dequantize_kernel<8><<<(unsigned)blocks, 256, 0, st>>>((const uint8_t*)src->codes, src->ld, src->scales,
-                                                           src->zeros, ngroups, src->rows, src->cols, dst, ld_dst);
-  } else {
-    dequantize_kernel<4><<<(unsigned)blocks, 256, 0, st>>>((const uint8_t*)src->codes, src->ld / 2, src->scales,
-                                                           src->zeros, ngroups, src->rows, src->cols, dst, ld_dst);
-  }
+  dequantize_kernel<<<(unsigned)blocks, 256, 0, st>>>(*src, ngroups, dst, ld_dst);
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
@@ -153,18 +141,10 @@ constexpr int kSimRows = 32;
 
 __device__ __forceinline__ void load_p8(const qg_qtensor& T, int64_t row, int64_t c0, int ngroups, int nvalid,
                                         float v[8]) {
-  const uint8_t* p = (const uint8_t*)T.codes + row * (T.ld / 2) + (c0 >> 1);
-  uint32_t w = 0x88888888u;
-  if (nvalid == 8) {
-    w = __ldg(reinterpret_cast<const uint32_t*>(p));
-  } else {
-    w = 0;
-    for (int i = 0; i < (nvalid + 1) / 2; ++i) w |= (uint32_t)p[i] << (8 * i);
-  }
   const int g = (int)(c0 / kGroup);
   const float s = __ldg(T.scales + row * ngroups + g), z = __ldg(T.zeros + row * ngroups + g);
   float q[8];
-  unpack_int4x8(w, q);
+  load_codes8(T, row, c0, nvalid, q);
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = (i < nvalid) ? __fmul_rn(__fsub_rn(q[i], z), s) : 0.0f;
 }
@@ -275,8 +255,8 @@ extern "C" QG_API int qgalore_subspace_similarity_static(const qg_qtensor* A, co
   if (!A || !B || !sim_dev) return QG_INVALID_ARGUMENT;
   for (const qg_qtensor* t : {A, B}) {
     if (!t->codes || !t->scales || !t->zeros || t->rows <= 0 || t->cols <= 0 || t->ld < t->cols) return QG_INVALID_ARGUMENT;
-    if (t->bits != 4 || t->group != kGroup) return QG_INVALID_ARGUMENT;
-    if (!aligned16(t->codes) || t->ld % 32 != 0) return QG_MISALIGNED;
+    if ((t->bits != 2 && t->bits != 4 && t->bits != 8) || t->group != kGroup) return QG_INVALID_ARGUMENT;
+    if (!aligned16(t->codes) || t->ld % (128 / t->bits) != 0) return QG_MISALIGNED;
   }
   if (A->rows != B->rows || A->cols != B->cols) return QG_INVALID_ARGUMENT;
   if (A->cols > 16384) return QG_UNSUPPORTED_SHAPE;

@@ -532,7 +532,7 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
   if (rc != QG_OK) return rc;
   sign_fix_kernel<<<(unsigned)r, 256, 0, st>>>(w.P32, m, (int)r, P_fp32);
   QG_LAUNCH_CHECK();
-  return launch_quantize_rtn(4, w.P32, m, r, r, P_new, st);
+  return launch_quantize_rtn(P_new->bits, w.P32, m, r, r, P_new, st);
 }
 
 }  // namespace qg

@@ -20,11 +20,10 @@ dequant_p_bf16_kernel(qg_qtensor P, uint16_t* __restrict__ out, int64_t ld_out) 
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= P.rows * chunks) return;
   const int64_t row = idx / chunks, c0 = (idx % chunks) * 8;
-  const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>((const uint8_t*)P.codes + row * (P.ld / 2) + (c0 >> 1)));
   const int g = (int)(c0 / kGroup);
   const float s = __ldg(P.scales + row * ngroups + g), z = __ldg(P.zeros + row * ngroups + g);
   float q[8], v[8];
-  unpack_int4x8(w, q);
+  load_codes8(P, row, c0, 8, q);                     // 2-, 4- or 8-bit codes
 #pragma unroll
   for (int i = 0; i < 8; ++i) v[i] = __fmul_rn(__fsub_rn(q[i], z), s);
   *reinterpret_cast<uint4*>(out + row * ld_out + c0) = pack_bf16x8(v);

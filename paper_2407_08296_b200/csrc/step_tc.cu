@@ -1195,9 +1195,21 @@ dequant_p_grouped_kernel(const DequantItem* __restrict__ items, const int32_t* _
   const uint32_t idx = (blockIdx.x - (uint32_t)it.block0) * blockDim.x + threadIdx.x;
   if (idx >= rows * per_row) return;
   const uint32_t row = idx / per_row, c0 = (idx - row * per_row) * 32;
-  const uint4 w4 = __ldg(reinterpret_cast<const uint4*>((const uint8_t*)it.P.codes + (size_t)row * (it.P.ld / 2) + (c0 >> 1)));
   const uint32_t g = c0 / kGroup;
   const float s = __ldg(it.P.scales + (size_t)row * ngroups + g), z = __ldg(it.P.zeros + (size_t)row * ngroups + g);
+  if (it.P.bits != 4) {                              // the 2- and 8-bit projections of the ablation: plain conversion
+    uint4* o = reinterpret_cast<uint4*>(it.out + (size_t)row * cols + c0);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float q[8], v[8];
+      load_codes8(it.P, row, c0 + 8 * k, 8, q);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) v[e] = __fmul_rn(__fsub_rn(q[e], z), s);
+      o[k] = pack_bf16x8(v);
+    }
+    return;
+  }
+  const uint4 w4 = __ldg(reinterpret_cast<const uint4*>((const uint8_t*)it.P.codes + (size_t)row * (it.P.ld / 2) + (c0 >> 1)));
   const float c = 8388616.0f + z;                    // 2^23 + 8 + z, exact for |z| < 2^22
   const bool fast = fabsf(z) < 4.0e6f;
   const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};

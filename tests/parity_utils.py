@@ -13,7 +13,7 @@ def to_device_q(q: O.QTensor, device="cuda") -> B.QTensor:
     if q.bits == 8:
         out.codes[:, :cols] = torch.from_numpy(q.codes).to(device)
     else:
-        packed = O.pack_int4(q.codes)
+        packed = O.pack_int4(q.codes) if q.bits == 4 else O.pack_int2(q.codes)
         out.codes[:, :packed.shape[1]] = torch.from_numpy(packed).to(device)
     out.scales.copy_(torch.from_numpy(q.scales))
     out.zeros.copy_(torch.from_numpy(q.zeros))
@@ -23,8 +23,10 @@ def to_device_q(q: O.QTensor, device="cuda") -> B.QTensor:
 def from_device_q(q: B.QTensor) -> O.QTensor:
     if q.bits == 8:
         codes = q.codes[:, :q.cols].cpu().numpy().astype(np.int8)
-    else:
+    elif q.bits == 4:
         codes = O.unpack_int4(q.codes.cpu().numpy(), q.cols)
+    else:
+        codes = O.unpack_int2(q.codes.cpu().numpy(), q.cols)
     return O.QTensor(codes, q.scales.cpu().numpy(), q.zeros.cpu().numpy(), q.bits)
 
 

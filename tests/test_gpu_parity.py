@@ -392,3 +392,74 @@ def test_round_to_nearest_ignores_the_seed_and_a_bad_mode_is_refused():
     with pytest.raises(B.QgError):
         B.project_step(g_to_device(gb), to_device_q(P), to_device_q(W), f32_to_device(z), f32_to_device(z),
                        B.Hyper(step=1, rounding=7))
+
+
+# ----------------------------------------------------------------------------- projection bit width (Sec. 4.4, Fig. 3)
+@pytest.mark.parametrize("shape", [(64, 256), (33, 777), (512, 128)])
+def test_int2_quantizer_is_bit_exact(shape):
+    rows, cols = shape
+    x = np.random.default_rng(rows + cols).normal(0, 0.05, (rows, cols)).astype(np.float32)
+    x[0, :] = 0.25                                    # a constant group
+    ref = O.quantize_rtn(x, 2)
+    q = B.quantize_int2(f32_to_device(x))
+    got = from_device_q(q)
+    assert np.array_equal(got.codes, ref.codes) and np.array_equal(got.scales, ref.scales) and np.array_equal(got.zeros, ref.zeros)
+    assert np.array_equal(B.dequantize(q).cpu().numpy(), O.dequantize(ref))
+    assert np.array_equal(B.dequantize(to_device_q(ref)).cpu().numpy(), O.dequantize(ref))
+
+
+@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("impl", [None, 1])
+def test_step_with_a_2_or_8_bit_projection(bits, impl):
+    m, n, r = 512, 1376, 128
+    gm = synth.GradientModel(m, n, seed=12, matrix_index=0)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=12), bits)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 12), 8)
+    z = np.zeros((r, n), np.float32)
+    o = O.project_step(gm.sample(1), P, W, z, z, O.Hyper(step=1, seed=8))
+    stats = run_and_check_step(gm.sample(2), P, o["W"], o["M"], o["V"], O.Hyper(step=2, seed=8), impl=impl)
+    assert stats["mismatch"] <= 1e-3
+
+
+def test_plan_mixes_projection_bit_widths_and_similarity_takes_them():
+    shapes = [(256, 512, 64), (512, 1376, 128), (768, 768, 256)]
+    step = 2
+    single, items = [], []
+    for idx, ((m, n, r), bits) in enumerate(zip(shapes, (2, 8, 4))):
+        gm = synth.GradientModel(m, n, seed=13, matrix_index=idx)
+        P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=13, stream=idx), bits)
+        W = O.quantize_rtn(synth.initial_weight(m, n, 13, idx), 8)
+        M = np.zeros((r, n), np.float32)
+        V = np.zeros((r, n), np.float32)
+        gb = gm.sample(step)
+        dG, dP = g_to_device(gb), to_device_q(P)
+        dW1, dM1, dV1 = to_device_q(W), f32_to_device(M), f32_to_device(V)
+        B.project_step(dG, dP, dW1, dM1, dV1, B.Hyper(step=step, seed=idx))
+        single.append((dW1, dM1, dV1))
+        items.append({"G": dG, "P": dP, "W": to_device_q(W), "M": f32_to_device(M), "V": f32_to_device(V), "seed": idx})
+        # similarity of the projection with a perturbed copy of itself, both at this bit width
+        P2 = O.quantize_rtn(O.dequantize(P) + np.random.default_rng(idx).normal(0, 0.01, (m, r)).astype(np.float32), bits)
+        sim = B.subspace_similarity(dP, to_device_q(P2))
+        assert abs(float(sim.item()) - O.subspace_similarity(P, P2)) <= 1e-5
+    plan = B.StepPlan(items)
+    plan.step(B.Hyper(step=step))
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0
+    for (dW1, dM1, dV1), it in zip(single, items):
+        assert torch.equal(dW1.codes, it["W"].codes) and torch.equal(dM1._base, it["M"]._base) and torch.equal(dV1._base, it["V"]._base)
+    plan.close()
+
+
+def test_refresh_writes_an_8_bit_projection_when_asked():
+    m, n, r = 512, 1376, 128
+    gb = synth.GradientModel(m, n, seed=14, matrix_index=0).sample(1)
+    P32 = torch.zeros((m, r), dtype=torch.float32, device="cuda")
+    P8 = B.QTensor(torch.zeros((m, r), dtype=torch.int8, device="cuda"), torch.zeros((m, 1), dtype=torch.float32, device="cuda"),
+                   torch.zeros((m, 1), dtype=torch.float32, device="cuda"), m, r, r, 8)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.refresh_subspace(g_to_device(gb), r, P_new=P8, P_fp32=P32, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref = O.quantize_rtn(P32.cpu().numpy(), 8)
+    got = from_device_q(P8)
+    assert np.array_equal(got.codes, ref.codes) and np.array_equal(got.scales, ref.scales)

@@ -524,3 +524,37 @@ def test_round_to_nearest_step_is_the_same_step_with_quant8_at_the_end():
     # nearest: the dequantized result is within half a level of the pre-rounding weight inside the clamp range
     lsb = np.repeat(rtn["W"].scales, 256, axis=1)[:, :n]
     assert np.all(np.abs(O.dequantize(rtn["W"]) - rtn["W_pre"]) <= 0.5 * lsb * (1 + 1e-5) + 1e-12)
+
+
+def test_int2_quantizer_levels_bound_and_packing():
+    # Quant_n of Sec. 3.1 with n = 2 (the 2-bit projection of Sec. 4.4): four levels per group, the group's
+    # minimum and maximum take the end codes, every value lands within half a step, packing round-trips.
+    rng = np.random.default_rng(3)
+    x = rng.normal(0, 0.03, (16, 256 * 2 + 40)).astype(np.float32)
+    q = O.quantize_rtn(x, 2)
+    assert q.codes.min() == -2 and q.codes.max() == 1
+    xh = O.dequantize(q)
+    step = np.repeat(q.scales, 256, axis=1)[:, :x.shape[1]]
+    assert np.all(np.abs(xh - x) <= 0.5 * step * (1 + 1e-5) + 1e-12)
+    for g, (a, b) in enumerate([(0, 256), (256, 512), (512, 552)]):
+        seg, codes = x[:, a:b], q.codes[:, a:b]
+        rows = np.arange(16)
+        assert np.all(codes[rows, seg.argmin(axis=1)] == -2) and np.all(codes[rows, seg.argmax(axis=1)] == 1)
+        assert np.allclose(q.scales[:, g], (seg.max(axis=1) - seg.min(axis=1)) / 3.0, rtol=1e-6)
+    packed = O.pack_int2(q.codes)
+    assert packed.shape == (16, (552 + 3) // 4)
+    assert np.array_equal(O.unpack_int2(packed, 552), q.codes)
+    # byte layout: column 4k + i in bits 2i, 2i + 1, stored as code + 2
+    c = np.array([[-2, -1, 0, 1, 1, 0, -1, -2]], dtype=np.int8)
+    assert O.pack_int2(c).tolist() == [[0b11100100, 0b00011011]]
+
+
+def test_coarser_projection_loses_more_of_the_subspace():
+    # Sec. 3.3 / Fig. 3: the projection tolerates 4 bits; fewer bits reproduce the orthonormal basis worse.
+    from paper_2407_08296_b200 import synth
+    P = synth.random_orthonormal(512, 128, seed=1)
+    err = {}
+    for bits in (2, 4, 8):
+        Ph = O.dequantize(O.quantize_rtn(P, bits)).astype(np.float64)
+        err[bits] = np.linalg.norm(Ph.T @ Ph - np.eye(128)) / np.sqrt(128)
+    assert err[8] < err[4] < err[2] and err[8] < 1e-2 and err[2] > 0.1
