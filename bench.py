@@ -293,8 +293,50 @@ def time_refresh(items, device):
                           "similarity_to_previous": float(sim.item()), "device_status": int(status.item())})
         total += ms * counts[(m, n, r)] * 1e-3
         del ws
-    return {"iters": 12, "per_shape": per_shape, "stack_seconds": total,
-            "note": "not part of the timed step; one matrix per distinct shape, extrapolated by shape counts"}
+    out = {"iters": 12, "per_shape": per_shape, "stack_seconds": total,
+           "note": "not part of the timed step; one matrix per distinct shape, extrapolated by shape counts"}
+    # several matrices at once on several streams (each with its own scratch): the refresh is a long chain of
+    # small kernels, so independent matrices fill each other's gaps.  The first `batch` matrices of the stack,
+    # timed once one after the other and once round-robin over `streams` streams; the ratio scales the figure above.
+    streams, batch = 4, min(8, len(items))
+    some = items[:batch]
+    side = [torch.cuda.Stream(device=device) for _ in range(streams)]
+    wss, outs = [], []
+    for k in range(streams):
+        need = max(B.workspace_bytes(B.QG_OP_REFRESH, it["spec"].m, it["spec"].n,
+                                     min((2 * it["spec"].r + 63) // 64 * 64, min(it["spec"].m, it["spec"].n) // 64 * 64))
+                   for it in some)
+        wss.append(torch.empty(need, dtype=torch.uint8, device=device))
+    for it in some:
+        sp = it["spec"]
+        ng = (sp.r + 255) // 256
+        outs.append(B.QTensor(torch.full((sp.m, sp.r // 2), 0x88, dtype=torch.uint8, device=device),
+                              torch.zeros((sp.m, ng), dtype=torch.float32, device=device),
+                              torch.zeros((sp.m, ng), dtype=torch.float32, device=device), sp.m, sp.r, sp.r, 4))
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    main = torch.cuda.current_stream()
+    times = []
+    for concurrent in (False, True):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(main)
+        for k, (it, pq) in enumerate(zip(some, outs)):
+            s = side[k % streams] if concurrent else main
+            if concurrent:
+                s.wait_stream(main)
+            with torch.cuda.stream(s):
+                B.refresh_subspace(it["G"], it["spec"].r, iters=12, seed=1, P_new=pq, workspace=wss[k % streams], status=status,
+                                   stream=s)
+        if concurrent:
+            for s in side:
+                main.wait_stream(s)
+        e1.record(main)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    out["concurrent"] = {"streams": streams, "matrices": batch, "sequential_ms": times[0], "concurrent_ms": times[1],
+                         "device_status": int(status.item())}
+    out["stack_seconds_concurrent"] = total * times[1] / max(times[0], 1e-9)
+    return out
 
 
 def run_ours(args):
@@ -446,7 +488,7 @@ def run_ours(args):
         refresh = None if args.no_refresh else time_refresh(items, device)
         if refresh is not None:
             # the step and the refresh blended at the base interval of Sec. 4.1 (a refresh every 200 steps)
-            refresh["blended_ms_per_step_at_interval_200"] = ms_per_step + refresh["stack_seconds"] * 1e3 / 200.0
+            refresh["blended_ms_per_step_at_interval_200"] = ms_per_step + refresh["stack_seconds_concurrent"] * 1e3 / 200.0
         cpu = None
         if not args.no_cpu_baseline:
             v, per_step, sample = oracle_sample(args.workload, 3, 1)

@@ -18,12 +18,17 @@
 // noise bulk of the gradient with relative gaps of 1e-4..1e-3, and resolving that subspace to 1e-2 rad
 // needs fp32-faithful products (bf16 tensor-core products do not get there).
 #include <cmath>
+#include <mutex>
 
 #include "qg_common.cuh"
 
 namespace qg {
 
 namespace {
+
+constexpr int kCoopDevices = 64;
+std::mutex g_coop_mutex;
+cudaEvent_t g_coop_done[kCoopDevices] = {};   // completion of the last cooperative launch, per device ordinal
 
 constexpr int kPanel = 64;    // columns orthonormalised together
 constexpr int kMaxSweeps = 32;
@@ -518,10 +523,24 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
     unsigned int* sync_words = reinterpret_cast<unsigned int*>(w.done);
     // the iteration converges quadratically at the end: a sweep that met nothing above 1e-5 leaves ~1e-10
     constexpr double kTol = 1e-5;
+    // Refreshes of several matrices may run on several streams at once (their many small kernels overlap
+    // well), but two grids whose CTAs wait for one another must never be half resident together: each
+    // cooperative launch waits for the previous one of this process on the device, whatever its stream.
+    std::lock_guard<std::mutex> lock(g_coop_mutex);
+    int dev = 0;
+    QG_CUDA_TRY(cudaGetDevice(&dev));
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    QG_CUDA_TRY(cudaStreamIsCapturing(st, &cap));
+    const bool chain = cap == cudaStreamCaptureStatusNone && dev >= 0 && dev < kCoopDevices;
+    if (chain) {
+      if (!g_coop_done[dev]) QG_CUDA_TRY(cudaEventCreateWithFlags(&g_coop_done[dev], cudaEventDisableTiming));
+      else QG_CUDA_TRY(cudaStreamWaitEvent(st, g_coop_done[dev], 0));
+    }
     if (b <= 8 * kTeam) rc = launch_jacobi<8>(w.T, b, sweeps, kTol, off, sync_words, status, st);
     else if (b <= 16 * kTeam) rc = launch_jacobi<16>(w.T, b, sweeps, kTol, off, sync_words, status, st);
     else rc = launch_jacobi<32>(w.T, b, sweeps, kTol, off, sync_words, status, st);
     if (rc != QG_OK) return rc;
+    if (chain) QG_CUDA_TRY(cudaEventRecord(g_coop_done[dev], st));
   }
   row_norm_kernel<<<(unsigned)b, 128, 0, st>>>(w.T, (int)b, w.lam);
   QG_LAUNCH_CHECK();
