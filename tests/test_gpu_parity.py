@@ -463,3 +463,69 @@ def test_refresh_writes_an_8_bit_projection_when_asked():
     ref = O.quantize_rtn(P32.cpu().numpy(), 8)
     got = from_device_q(P8)
     assert np.array_equal(got.codes, ref.codes) and np.array_equal(got.scales, ref.scales)
+
+
+# ----------------------------------------------------------------------------- degenerate and limiting cases
+def test_zero_gradient_and_constant_groups_are_bit_exact():
+    # G = 0 at t = 1: R = M' = V' = 0 and N = 0 / (0 + eps) = 0 exactly, so W' is the dequantized weight and every
+    # bit of the requantization is decided by identical inputs; one row of W is constant (a degenerate group:
+    # z = 0, s = |max|), one is all zero.
+    m, n, r = 128, 256 + 85, 32
+    gb = np.zeros((m, n), np.uint16)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=2), 4)
+    w = synth.initial_weight(m, n, 2).copy()
+    w[3, :] = 0.0125
+    w[5, :] = 0.0
+    W = O.quantize_rtn(w, 8)
+    z = np.zeros((r, n), np.float32)
+    hyp = O.Hyper(step=1, seed=77)
+    ref = O.project_step(gb, P, W, z, z, hyp)
+    dW, dM, dV = to_device_q(W), f32_to_device(z), f32_to_device(z)
+    taps = StepTaps(m, n, r, dW.ld)
+    B.project_step(g_to_device(gb), to_device_q(P), dW, dM, dV, B.Hyper(step=1, seed=77), debug=taps.as_dict())
+    torch.cuda.synchronize()
+    assert float(dM.abs().max().item()) == 0.0 and float(dV.abs().max().item()) == 0.0
+    assert float(taps.N.abs().max().item()) == 0.0 and float(taps.R.abs().max().item()) == 0.0
+    got = from_device_q(dW)
+    assert np.array_equal(taps.W_pre.cpu().numpy(), ref["W_pre"])
+    assert np.array_equal(got.codes, ref["W"].codes)
+    assert np.array_equal(got.scales, ref["W"].scales) and np.array_equal(got.zeros, ref["W"].zeros)
+
+
+def test_step_at_the_largest_rank():
+    # r = 2048 is the limit of the step (r <= m, r % 32 == 0)
+    run_step_case(2048, 600, 2048, seed=6, step=1)
+
+
+def test_step_refuses_empty_oversized_and_misshapen_problems():
+    m, n, r = 128, 256, 32
+    gb = synth.GradientModel(m, n, seed=1, matrix_index=0).sample(1)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=1), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 1), 8)
+    z = np.zeros((r, n), np.float32)
+    dG, dP, dW, dM, dV = g_to_device(gb), to_device_q(P), to_device_q(W), f32_to_device(z), f32_to_device(z)
+    L, C = B.lib(), B.C
+    ws = torch.empty(B.workspace_bytes(B.QG_OP_PROJECT_STEP, m, n, r), dtype=torch.uint8, device="cuda")
+    h = B.Hyper().c_struct()
+    pc, wc = dP.c_struct(), dW.c_struct()
+
+    def call(mm, nn, rr, hyper=h, ws_bytes=ws.numel()):
+        return L.qgalore_project_step(dG.data_ptr(), dG.stride(0), mm, nn, rr, C.byref(pc), C.byref(wc), dM.data_ptr(),
+                                      dV.data_ptr(), dM.stride(0), C.byref(hyper), ws.data_ptr(), ws_bytes, None, None, None)
+
+    before = dW.codes.clone()
+    assert call(0, n, r) == B.QG_INVALID_ARGUMENT           # empty
+    assert call(m, 0, r) == B.QG_INVALID_ARGUMENT
+    assert call(m, n, 0) == B.QG_INVALID_ARGUMENT
+    assert call(m, n, 64) == B.QG_INVALID_ARGUMENT          # P is m x 32
+    assert call(m, n, r, ws_bytes=16) == B.QG_WORKSPACE_TOO_SMALL
+    bad = B.Hyper(step=0).c_struct()
+    assert call(m, n, r, hyper=bad) == B.QG_INVALID_ARGUMENT
+    torch.cuda.synchronize()
+    assert torch.equal(before, dW.codes)                    # nothing was enqueued
+    # rank limits are shape errors
+    big = B.QTensor.empty(4096, 4096, 4)
+    bc = big.c_struct()
+    assert L.qgalore_project_step(dG.data_ptr(), 4096, 4096, 256, 4096, C.byref(bc), C.byref(wc), dM.data_ptr(), dV.data_ptr(),
+                                  256, C.byref(h), ws.data_ptr(), ws.numel(), None, None, None) in (B.QG_UNSUPPORTED_SHAPE,
+                                                                                                    B.QG_INVALID_ARGUMENT)
