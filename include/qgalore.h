@@ -130,6 +130,20 @@ QG_API int qgalore_project_step(const uint16_t* G, int64_t ldg, int64_t m, int64
                          void* workspace, size_t workspace_bytes,
                          int32_t* status_dev, const qg_debug* dbg, void* stream);
 
+/* --- Sec. 3.5 with the projection on the right (the paper takes GaLore's projection, which projects
+ * on the side of the shorter dimension): R = G Q with Q n x r, Adam on the m x r state, D = N Q^T.
+ * Q       INT4 (or INT2 / INT8), n x r                                (read)
+ * Mt, Vt  fp32, the m x r moments stored TRANSPOSED: r x m, pitch ldmv >= m   (read + write)
+ * dbg->R, dbg->N (if given) are r x m too.  Everything else as in qgalore_project_step; r <= n.
+ * In a plan or a batched call an item selects this form with side = QG_SIDE_RIGHT. */
+#define QG_SIDE_LEFT 0
+#define QG_SIDE_RIGHT 1
+QG_API int qgalore_project_step_right(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r,
+                               const qg_qtensor* Q, const qg_qtensor* W,
+                               float* Mt, float* Vt, int64_t ldmv, const qg_hyper* h,
+                               void* workspace, size_t workspace_bytes,
+                               int32_t* status_dev, const qg_debug* dbg, void* stream);
+
 /* --- Sec. 3.5, the same step for several matrices (a layer, or a whole stack) in one call ----
  * Every item is one independent matrix with its own buffers and its own stochastic-rounding
  * seed; lr, alpha, the Adam constants and the step index come from h (h->seed is ignored).
@@ -141,6 +155,8 @@ typedef struct {
   qg_qtensor P, W;
   float* M; float* V; int64_t ldmv;
   uint64_t seed;
+  int32_t side;       /* QG_SIDE_LEFT (0) or QG_SIDE_RIGHT: see qgalore_project_step_right */
+  int32_t reserved;   /* 0 */
 } qg_step_item;
 
 QG_API int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const qg_hyper* h,

@@ -299,7 +299,8 @@ class Hyper:
         return g(self.lr), g(self.alpha), g(self.beta1), g(self.beta2), g(self.eps), g(self.weight_decay)
 
 
-def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=None, N_b_override=None, col0=0):
+def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=None, N_b_override=None, col0=0,
+                 side="left"):
     """One Q-GaLore update of one weight matrix (Sec. 3.5, Fig. 4; GaLore projection as cited there).
 
     G_bits : uint16 [m, n] bfloat16 gradient.         P_q : INT4 m x r projection.
@@ -316,7 +317,14 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     ``col0``: G, W, M, V are the column block starting at column col0 (a multiple of the group
     size) of a wider matrix; every column of the step depends on its own column of G, M, V, W only
     (and on P), so the block's results are those of the full matrix.  col0 enters the Philox lanes.
+    ``side``: "left" is R = P^T G with P m x r and the moments r x n (what the rest of this docstring
+    describes).  "right" is GaLore's other form, R = G Q with Q = P_q of shape n x r: the low-rank state is
+    m x r, and M, V, R32, N, N_b are kept and returned TRANSPOSED (r x m, row-major) so that both forms
+    hand the same kind of array around; the update is D = N Q^T.  (col0 is for the left form only.)
     """
+    if side == "right":
+        assert col0 == 0
+        return _project_step_right(G_bits, P_q, W_q, M, V, h, N_b_override)
     lr, alpha, b1, b2, eps, wd = h.as_f32()
     t = int(h.step)
     G = bf16_bits_to_f32(G_bits).astype(np.float64)
@@ -349,6 +357,34 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     else:
         W_new, T = quantize_sr(W_pre, h.seed, t, W_q.group, return_scaled=True, col0=col0)
     return dict(W=W_new, M=M_new, V=V_new, R32=R32, N=N32, N_b=N_b, W_pre=W_pre, T=T, P_tilde=Pt)
+
+
+def _project_step_right(G_bits, Q_q: QTensor, W_q: QTensor, Mt, Vt, h: Hyper, N_b_override=None):
+    """The step with the projection on the right (Sec. 3.5 defers the choice of side to GaLore):
+    R = G Q~ (m x r), Adam on the m x r state, D = N_b Q~^T.  Mt, Vt and every returned low-rank array are
+    the transposes (r x m)."""
+    lr, alpha, b1, b2, eps, wd = h.as_f32()
+    t = int(h.step)
+    G = bf16_bits_to_f32(G_bits).astype(np.float64)
+    Qt = bf16_round(dequantize(Q_q)).astype(np.float64)              # n x r, enters the contraction as bfloat16
+    R32 = fl32((G @ Qt).T)                                            # r x m
+    R = R32.astype(np.float64)
+    M_new = fl32(b1 * Mt.astype(np.float64) + (1.0 - b1) * R)
+    V_new = fl32(b2 * Vt.astype(np.float64) + (1.0 - b2) * R * R)
+    m_hat = M_new.astype(np.float64) / (1.0 - b1 ** t)
+    v_hat = V_new.astype(np.float64) / (1.0 - b2 ** t)
+    N32 = fl32(m_hat / (np.sqrt(v_hat) + eps))
+    N_b = bf16_round(N32)
+    if N_b_override is not None:
+        N_b = np.asarray(N_b_override, dtype=np.float32)
+    D = N_b.astype(np.float64).T @ Qt.T                               # m x n
+    W_hat = dequantize(W_q).astype(np.float64)
+    W_pre = fl32(W_hat - (lr * alpha) * D - (lr * wd) * W_hat)
+    if h.rounding == "rtn":
+        W_new, T = quantize_rtn(W_pre, 8, W_q.group, return_scaled=True)
+    else:
+        W_new, T = quantize_sr(W_pre, h.seed, t, W_q.group, return_scaled=True)
+    return dict(W=W_new, M=M_new, V=V_new, R32=R32, N=N32, N_b=N_b, W_pre=W_pre, T=T, P_tilde=Qt)
 
 
 # --------------------------------------------------------------------------- refresh (Sec. 3.5, Sec. 1)

@@ -38,6 +38,7 @@ class _CQTensor(C.Structure):
 
 
 QG_ROUND_STOCHASTIC, QG_ROUND_NEAREST = 0, 1
+QG_SIDE_LEFT, QG_SIDE_RIGHT = 0, 1
 
 
 class _CHyper(C.Structure):
@@ -49,7 +50,7 @@ class _CHyper(C.Structure):
 class _CStepItem(C.Structure):
     _fields_ = [("G", C.c_void_p), ("ldg", C.c_int64), ("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int64),
                 ("P", _CQTensor), ("W", _CQTensor), ("M", C.c_void_p), ("V", C.c_void_p), ("ldmv", C.c_int64),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("side", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _CDebug(C.Structure):
@@ -76,6 +77,7 @@ def lib() -> C.CDLL:
         L.qgalore_dequantize.argtypes = [qp, vp, i64, vp]
         L.qgalore_project_step.argtypes = [vp, i64, i64, i64, i64, qp, qp, vp, vp, i64, C.POINTER(_CHyper),
                                            vp, sz, vp, C.POINTER(_CDebug), vp]
+        L.qgalore_project_step_right.argtypes = L.qgalore_project_step.argtypes
         L.qgalore_project_step_batched.argtypes = [C.POINTER(_CStepItem), i32, C.POINTER(_CHyper), vp, sz, vp, vp]
         L.qgalore_workspace_bytes_batched.argtypes = [C.POINTER(_CStepItem), i32]
         L.qgalore_workspace_bytes_batched.restype = sz
@@ -243,16 +245,18 @@ def dequantize(q: QTensor, out: torch.Tensor | None = None, stream=None) -> torc
 
 def project_step(G: torch.Tensor, P: QTensor, W: QTensor, M: torch.Tensor, V: torch.Tensor, hyper: Hyper,
                  workspace: torch.Tensor | None = None, status: torch.Tensor | None = None,
-                 debug: dict | None = None, stream=None) -> None:
-    """One Q-GaLore step of one matrix (Sec. 3.5): W, M and V are updated in place."""
+                 debug: dict | None = None, stream=None, side: str = "left") -> None:
+    """One Q-GaLore step of one matrix (Sec. 3.5): W, M and V are updated in place.  ``side`` = "right" takes
+    P as the n x r right-hand projection and M, V as the transposed (r x m) moments."""
     m, n = G.shape
     r = P.cols
+    right = side == "right"
     if G.dtype not in (torch.bfloat16, torch.int16, torch.uint16):
         raise ValueError("G must hold bfloat16 values (bfloat16 / int16 / uint16 storage)")
     if M.dtype != torch.float32 or V.dtype != torch.float32:
         raise ValueError("M and V must be float32")
-    if tuple(M.shape) != (r, n) or tuple(V.shape) != (r, n):
-        raise ValueError("M and V must be r x n")
+    if tuple(M.shape) != (r, m if right else n) or tuple(V.shape) != (r, m if right else n):
+        raise ValueError("M and V must be r x n (r x m for the right-hand projection)")
     ldmv = _matrix_ld(M, "M")
     if _matrix_ld(V, "V") != ldmv:
         raise ValueError("M and V must share their row pitch")
@@ -262,10 +266,11 @@ def project_step(G: torch.Tensor, P: QTensor, W: QTensor, M: torch.Tensor, V: to
     if debug:
         dbg = _CDebug(_ptr(debug.get("R")), _ptr(debug.get("N")), _ptr(debug.get("W_pre")))
     pc, wc, hc = P.c_struct(), W.c_struct(), hyper.c_struct()
-    _check(lib().qgalore_project_step(_ptr(G), _matrix_ld(G, "G"), m, n, r, C.byref(pc), C.byref(wc), _ptr(M), _ptr(V),
-                                      ldmv, C.byref(hc), _ptr(workspace), workspace.numel() * workspace.element_size(),
-                                      _ptr(status), C.byref(dbg) if dbg is not None else None, _stream_ptr(stream)),
-           "qgalore_project_step")
+    fn = lib().qgalore_project_step_right if right else lib().qgalore_project_step
+    _check(fn(_ptr(G), _matrix_ld(G, "G"), m, n, r, C.byref(pc), C.byref(wc), _ptr(M), _ptr(V),
+              ldmv, C.byref(hc), _ptr(workspace), workspace.numel() * workspace.element_size(),
+              _ptr(status), C.byref(dbg) if dbg is not None else None, _stream_ptr(stream)),
+           "qgalore_project_step_right" if right else "qgalore_project_step")
 
 
 class StepBatch:
@@ -284,7 +289,8 @@ class StepBatch:
             G, P, W, M, V = it["G"], it["P"], it["W"], it["M"], it["V"]
             m, ncol = G.shape
             self._table[k] = _CStepItem(_ptr(G), _matrix_ld(G, "G"), m, ncol, P.cols, P.c_struct(), W.c_struct(),
-                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)))
+                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)),
+                                        QG_SIDE_RIGHT if it.get("side", "left") == "right" else QG_SIDE_LEFT, 0)
         dev = device if device is not None else items[0]["G"].device
         nbytes = int(lib().qgalore_workspace_bytes_batched(self._table, n))
         self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
@@ -315,7 +321,8 @@ class StepPlan:
             G, P, W, M, V = it["G"], it["P"], it["W"], it["M"], it["V"]
             m, ncol = G.shape
             self._table[k] = _CStepItem(_ptr(G), _matrix_ld(G, "G"), m, ncol, P.cols, P.c_struct(), W.c_struct(),
-                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)))
+                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)),
+                                        QG_SIDE_RIGHT if it.get("side", "left") == "right" else QG_SIDE_LEFT, 0)
         dev = device if device is not None else items[0]["G"].device
         L = lib()
         need = int(L.qgalore_workspace_bytes_batched(self._table, n))

@@ -114,8 +114,9 @@ size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r) {
   switch (op) {
     case QG_OP_PROJECT_STEP: {
       if (n <= 0) return 0;
-      const size_t a = simt_workspace_bytes(m, n, r), b = tc_workspace_bytes(m, n, r);
-      return a > b ? a : b;
+      // either projection side: the scratch holds P~ (rows of the projection x r) and N_b (r x columns of the state)
+      const size_t a = simt_workspace_bytes(m, n, r), b = tc_workspace_bytes(m, n, r), c = tc_workspace_bytes(n, m, r);
+      return a > b ? (a > c ? a : c) : (b > c ? b : c);
     }
     case QG_OP_REFRESH: {
       if (n <= 0) return 0;
@@ -150,33 +151,37 @@ static int check_hyper(const qg_hyper* h) {
 
 // Shape, pointer and alignment rules of one matrix of the step; fills everything of `a` but the scalars.
 static int check_matrix(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
-                        const qg_qtensor* W, float* M, float* V, int64_t ldmv, StepArgs* a) {
+                        const qg_qtensor* W, float* M, float* V, int64_t ldmv, int side, StepArgs* a) {
   if (!G || !M || !V) return QG_INVALID_ARGUMENT;
-  if (m <= 0 || n <= 0 || r <= 0 || ldg < n || ldmv < n) return QG_INVALID_ARGUMENT;
+  if (side != QG_SIDE_LEFT && side != QG_SIDE_RIGHT) return QG_INVALID_ARGUMENT;
+  const bool right = side == QG_SIDE_RIGHT;
+  const int64_t prow = right ? n : m, scol = right ? m : n;     // rows of the projection, columns of the moments
+  if (m <= 0 || n <= 0 || r <= 0 || ldg < n || ldmv < scol) return QG_INVALID_ARGUMENT;
   if (!P || (P->bits != 2 && P->bits != 4 && P->bits != 8)) return QG_INVALID_ARGUMENT;
   int rc = check_qtensor(P, P->bits);
   if (rc != QG_OK) return rc;
   rc = check_qtensor(W, 8);
   if (rc != QG_OK) return rc;
-  if (P->rows != m || P->cols != r || W->rows != m || W->cols != n) return QG_INVALID_ARGUMENT;
-  if (r % 32 != 0 || r < 32 || r > 2048 || r > m) return QG_UNSUPPORTED_SHAPE;
+  if (P->rows != prow || P->cols != r || W->rows != m || W->cols != n) return QG_INVALID_ARGUMENT;
+  if (r % 32 != 0 || r < 32 || r > 2048 || r > prow) return QG_UNSUPPORTED_SHAPE;
   if (m > (1ll << 31) - 1 || n > (1ll << 31) - 1) return QG_UNSUPPORTED_SHAPE;
   if (!aligned16(G) || !aligned16(M) || !aligned16(V) || ldg % 8 != 0 || ldmv % 4 != 0) return QG_MISALIGNED;
   memset(a, 0, sizeof(*a));
   a->G = G; a->ldg = ldg; a->m = m; a->n = n; a->r = r;
   a->P = *P; a->W = *W; a->M = M; a->V = V; a->ldmv = ldmv;
+  a->right = right ? 1 : 0;
   return QG_OK;
 }
 
 static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
                              const qg_qtensor* W, float* M, float* V, int64_t ldmv, const qg_hyper* h,
                              void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
-                             void* stream, bool validate_only) {
+                             void* stream, bool validate_only, int side = QG_SIDE_LEFT) {
   if (!workspace) return QG_INVALID_ARGUMENT;
   int rc = check_hyper(h);
   if (rc != QG_OK) return rc;
   StepArgs a;
-  rc = check_matrix(G, ldg, m, n, r, P, W, M, V, ldmv, &a);
+  rc = check_matrix(G, ldg, m, n, r, P, W, M, V, ldmv, side, &a);
   if (rc != QG_OK) return rc;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QG_MISALIGNED;
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
@@ -185,7 +190,10 @@ static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
   a.ws = workspace; a.ws_bytes = workspace_bytes; a.status = status_dev;
   if (dbg) a.dbg = *dbg;
   fill_scalars(h, h->seed, &a.sc);
-  if (g_step_impl == 1) return launch_project_step_simt(a, (cudaStream_t)stream);
+  if (g_step_impl == 1) {
+    if (a.right) return QG_UNSUPPORTED_SHAPE;       // the CUDA-core cross-check knows the left form only
+    return launch_project_step_simt(a, (cudaStream_t)stream);
+  }
   return launch_project_step_tc(a, (cudaStream_t)stream);
 }
 
@@ -195,6 +203,14 @@ int qgalore_project_step(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, i
                          void* stream) {
   return project_step_impl(G, ldg, m, n, r, P, W, M, V, ldmv, h, workspace, workspace_bytes, status_dev, dbg, stream,
                            false);
+}
+
+int qgalore_project_step_right(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* Q,
+                               const qg_qtensor* W, float* Mt, float* Vt, int64_t ldmv, const qg_hyper* h,
+                               void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
+                               void* stream) {
+  return project_step_impl(G, ldg, m, n, r, Q, W, Mt, Vt, ldmv, h, workspace, workspace_bytes, status_dev, dbg, stream,
+                           false, QG_SIDE_RIGHT);
 }
 
 size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t count) {
@@ -217,7 +233,7 @@ int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const
       qg_hyper hi = *h;
       hi.seed = it.seed;
       const int rc = project_step_impl(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &hi,
-                                       workspace, workspace_bytes, status_dev, nullptr, stream, pass == 0);
+                                       workspace, workspace_bytes, status_dev, nullptr, stream, pass == 0, it.side);
       if (rc != QG_OK) return rc;
     }
   }
@@ -232,7 +248,7 @@ static int plan_args(const qg_step_item* items, int32_t count, std::vector<StepA
   args->resize((size_t)count);
   for (int32_t i = 0; i < count; ++i) {
     const qg_step_item& it = items[i];
-    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &(*args)[i]);
+    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, it.side, &(*args)[i]);
     if (rc != QG_OK) return rc;
     (*args)[i].sc.seed_lo = (uint32_t)(it.seed & 0xFFFFFFFFull);
     (*args)[i].sc.seed_hi = (uint32_t)(it.seed >> 32);

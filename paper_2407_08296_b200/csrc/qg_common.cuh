@@ -220,6 +220,7 @@ struct StepArgs {
   void* ws; size_t ws_bytes;
   int32_t* status;
   qg_debug dbg;
+  int32_t right;           // 0: R = P^T G, P m x r, moments r x n;  1: R = G Q, Q n x r, moments kept as r x m
 };
 // P~ = bf16((q - z) * s) of an INT4 matrix whose column count is a multiple of 32 (row pitch ld_out elements)
 int launch_dequant_p(const qg_qtensor& P, uint16_t* out, int64_t ld_out, cudaStream_t st);

@@ -58,6 +58,7 @@ constexpr int kChunk = 32;              // accumulator columns per tcgen05.ld
 // matrix.
 struct alignas(64) TcProblem {
   CUtensorMap mapP, mapG, mapP3, mapG3, mapG3h, mapN3, mapN3h, mapPk, mapW, mapM, mapV;
+  CUtensorMap mapGk, mapQk;            // right projection: G and Q~ as K-major B operands (see below)
   float* w_scales;
   float* w_zeros;
   float* dbgR;
@@ -69,6 +70,12 @@ struct alignas(64) TcProblem {
   uint16_t* nb;                        // N_b, bf16 r x ldn (scratch)
   int64_t ldmv, ldw, ldn;
   int32_t m, n, r, ngroups;
+  // The projection kernel sees a K extent and a column extent: (m, n) for R = P~^T G, and (n, m) for the
+  // right-hand form R^T = Q~^T G^T, where the same kernel runs on the transposed gradient: G itself (m x n,
+  // row-major) is then the B operand with K contiguous (mapGk, box 64 x 128 rows), the moments and N_b are
+  // r x m, and the back-projection D = N_b^T Q~^T takes N_b as an MN-major A (mapN3h) and Q~ (n x r) as a
+  // K-major B (mapQk, box 64 x 256 rows).
+  int32_t right, k1_k, k1_n;
   int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles;
@@ -233,14 +240,15 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         const int local = item.y, rblocks = CTAS == 2 ? p->k1_rpairs : p->k1_rblocks;
         const int r0 = (local % rblocks) * (CTAS * kTileM) + (int)rank * kTileM;
         const int n0 = (local / rblocks) * BN + (int)rank * BNC;      // first column this CTA stages
-        const int kblocks = (p->m + kBK - 1) / kBK;
+        const int kblocks = (p->k1_k + kBK - 1) / kBK;
+        const bool right = p->right != 0;
         const CUtensorMap* mapP = &p->mapP;
         const CUtensorMap* mapG = &p->mapG;
         const CUtensorMap* mapP3 = &p->mapP3;
         const CUtensorMap* mapG3 = CTAS == 2 ? &p->mapG3h : &p->mapG3;
         // whole-chunk tiles take one 3-D copy per operand; chunks past the end of a 3-D view read as zero
         const bool a3 = (p->r_whole == p->r) || (r0 + kTileM <= p->r_whole);
-        const bool b3 = (p->n_whole == p->n) || (n0 + BNC <= p->n_whole);
+        const bool b3 = (p->n_whole == p->k1_n) || (n0 + BNC <= p->n_whole);
         // (An L2 prefetch of G a few K blocks ahead was tried and removed: the extra TMA instruction per K
         // block cost the single producer thread more than the hidden latency was worth.)
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -259,7 +267,9 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
 #pragma unroll
               for (int h = 0; h < 2; ++h) tma_load_2d_pair(sA + h * kBoxBytes, mapP, lead_full, r0 + 64 * h, kb * kBK);
             }
-            if (b3) {
+            if (right) {                               // G rows n0.. as a K-major tile of 128 rows
+              tma_load_2d_pair(sB, &p->mapGk, lead_full, kb * kBK, n0);
+            } else if (b3) {
               tma_load_3d_pair(sB, mapG3, lead_full, 0, kb * kBK, n0 / 64);
             } else {
 #pragma unroll
@@ -273,7 +283,10 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
 #pragma unroll
               for (int h = 0; h < 2; ++h) tma_load_2d(sA + h * kBoxBytes, mapP, &full[s], r0 + 64 * h, kb * kBK);
             }
-            if (b3) {
+            if (right) {
+#pragma unroll
+              for (int h = 0; h < BN / 128; ++h) tma_load_2d(sB + h * 2 * kBoxBytes, &p->mapGk, &full[s], kb * kBK, n0 + 128 * h);
+            } else if (b3) {
               tma_load_3d(sB, mapG3, &full[s], 0, kb * kBK, n0 / 64);
             } else {
 #pragma unroll
@@ -287,14 +300,19 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(CTAS * kTileM, BN, true, true);
+      constexpr uint32_t idesc_left = umma_idesc_bf16(CTAS * kTileM, BN, true, true);
+      constexpr uint32_t idesc_right = umma_idesc_bf16(CTAS * kTileM, BN, true, false);   // B with K contiguous
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), kBoxBytes, 1024);
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
+      const uint64_t desc_bk0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, 16, 1024);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
         const TcProblem* p = probs + tw.cur().x;
-        const int kblocks = (p->m + kBK - 1) / kBK;
+        const int kblocks = (p->k1_k + kBK - 1) / kBK;
+        const bool right = p->right != 0;
+        const uint32_t idesc = right ? idesc_right : idesc_left;
+        const uint64_t bstep = right ? (32 >> 4) : (2048 >> 4);   // 16 K indices further along B
         const uint32_t ab = tcount & 1;
         if (!(CTAS == 2 ? mbar_wait_cluster(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)
                         : mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1))) { ok = false; break; }
@@ -310,11 +328,11 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
           // both operands are MN-major: 16 K indices = two 8-index groups of 1024 bytes each; the start
           // address field counts 16-byte units, so a stage or K step is an add on the descriptor
           const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
-          const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
+          const uint64_t db = (right ? desc_bk0 : desc_b0) + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
-            if (CTAS == 2) umma_bf16_pair(d_tmem, da + k * (2048 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
-            else umma_bf16(d_tmem, da + k * (2048 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
+            if (CTAS == 2) umma_bf16_pair(d_tmem, da + k * (2048 >> 4), db + k * bstep, idesc, (kb | k) != 0);
+            else umma_bf16(d_tmem, da + k * (2048 >> 4), db + k * bstep, idesc, (kb | k) != 0);
           }
           if (CTAS == 2) umma_commit_pair(&empty[s]); else umma_commit(&empty[s]);
         }
@@ -362,7 +380,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       const int rblocks = CTAS == 2 ? cu.p->k1_rpairs : cu.p->k1_rblocks;
       cu.y0 = (item.y % rblocks) * (CTAS * kTileM) + (int)rank * kTileM + wrow;
       cu.x0 = (item.y / rblocks) * BN;
-      cu.nch = min(BN / kChunk, (cu.p->n - cu.x0 + kChunk - 1) / kChunk);
+      cu.nch = min(BN / kChunk, (cu.p->k1_n - cu.x0 + kChunk - 1) / kChunk);
       cu.c = 0;
     };
     auto next_chunk = [&](Cursor& cu) {
@@ -392,7 +410,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       const TcProblem* p = probs + item.x;
       const int local = item.y, rblocks = CTAS == 2 ? p->k1_rpairs : p->k1_rblocks;
       const int r0 = (local % rblocks) * (CTAS * kTileM) + (int)rank * kTileM, n0 = (local / rblocks) * BN;
-      const int pn = p->n;
+      const int pn = p->k1_n;
       const int nch = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
       const int cmax = pn - n0 - lcol;               // offset `off` (from n0 + lcol) is a valid column iff off < cmax
       const int64_t ldmv = p->ldmv, ldn = p->ldn;
@@ -754,6 +772,12 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
             const uint32_t lead_full = mapa_u32(smem_u32(&full[s]), 0);
             tma_load_2d_pair(sA, mapPk, lead_full, kb * kBK, m0);
             tma_load_3d_pair(sB, mapN3, lead_full, 0, kb * kBK, n0 / 64 + 2 * (int)rank);
+          } else if (p->right) {
+            // D = N_b^T Q~^T: rows m0.. of N_b^T are columns of N_b (an MN-major A tile, two 64-row chunks),
+            // columns n0.. of Q~^T are rows of Q~ (a K-major B tile of 256 rows)
+            mbar_arrive_expect_tx(&full[s], S::kStageBytes);
+            tma_load_3d(sA, &p->mapN3h, &full[s], 0, kb * kBK, m0 / 64);
+            tma_load_2d(sB, &p->mapQk, &full[s], kb * kBK, n0);
           } else {
             mbar_arrive_expect_tx(&full[s], S::kStageBytes);
             tma_load_2d(sA, mapPk, &full[s], kb * kBK, m0);
@@ -766,14 +790,21 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(CTAS * kTileM, S::kBN, false, true);
+      constexpr uint32_t idesc_left = umma_idesc_bf16(CTAS * kTileM, S::kBN, false, true);
+      constexpr uint32_t idesc_right = umma_idesc_bf16(CTAS * kTileM, S::kBN, true, false);
       const uint64_t desc_a0 = umma_smem_desc_sw128(smem_u32(stage_base), 16, 1024);
       const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kBoxBytes, 1024);
+      // right projection: A is MN-major (64-row chunks of 8 KB), B is K-major
+      const uint64_t desc_am0 = umma_smem_desc_sw128(smem_u32(stage_base), kBoxBytes, 1024);
+      const uint64_t desc_bk0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, 16, 1024);
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (TileWalk<SINGLE> tw(sched, total_tiles); ok && tw.valid(); tw.advance(), ++tcount) {
         const TcProblem* p = probs + tw.cur().x;
         const int kblocks = (p->r + kBK - 1) / kBK;
+        const bool right = p->right != 0;
+        const uint32_t idesc = right ? idesc_right : idesc_left;
+        const uint64_t astep = right ? (2048 >> 4) : (32 >> 4), bstep = right ? (32 >> 4) : (2048 >> 4);
         const uint32_t ab = tcount & 1;
         if (!(CTAS == 2 ? mbar_wait_cluster(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)
                         : mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1))) { ok = false; break; }
@@ -788,12 +819,12 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
           tc_fence_after_sync();
           // A is K-major (rows of 128 bytes, 16 K indices = 32 bytes further along the row),
           // B is MN-major (16 K indices = two 8-index groups of 1024 bytes)
-          const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
-          const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
+          const uint64_t da = (right ? desc_am0 : desc_a0) + (uint64_t)((s * S::kStageBytes) >> 4);
+          const uint64_t db = (right ? desc_bk0 : desc_b0) + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k) {
-            if (CTAS == 2) umma_bf16_pair(d_tmem, da + k * (32 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
-            else umma_bf16(d_tmem, da + k * (32 >> 4), db + k * (2048 >> 4), idesc, (kb | k) != 0);
+            if (CTAS == 2) umma_bf16_pair(d_tmem, da + k * astep, db + k * bstep, idesc, (kb | k) != 0);
+            else umma_bf16(d_tmem, da + k * astep, db + k * bstep, idesc, (kb | k) != 0);
           }
           if (CTAS == 2) umma_commit_pair(&empty[s]); else umma_commit(&empty[s]);
         }
@@ -1058,24 +1089,33 @@ TcScratch carve(void* base, int64_t m, int64_t n, int64_t r) {
   return w;
 }
 
+// Extents as the projection kernel sees them: rows of the projection matrix (its K extent) and columns of the
+// low-rank state.  Left: (m, n).  Right: (n, m).
+inline int64_t proj_rows(const StepArgs& a) { return a.right ? a.n : a.m; }
+inline int64_t state_cols(const StepArgs& a) { return a.right ? a.m : a.n; }
+
 int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   memset(p, 0, sizeof(*p));
   bool ok = true;
-  ok &= make_map(&p->mapP, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, a.m, a.r, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
+  const int64_t prow = proj_rows(a), scol = state_cols(a);
+  ok &= make_map(&p->mapP, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, prow, a.r, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
   ok &= make_map(&p->mapG, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.G, a.n, a.m, a.ldg, 64, kBK, CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapPk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, a.m, a.r, 64, kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapPk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, prow, a.r, 64, kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
   const int64_t r_whole = a.r & ~int64_t(63), n_whole = a.n & ~int64_t(63);
-  ok &= make_map_chunked(&p->mapP3, w.Pt, a.m, r_whole > 0 ? r_whole / 64 : 1, a.r, kBK, 2);
+  ok &= make_map_chunked(&p->mapP3, w.Pt, prow, r_whole > 0 ? r_whole / 64 : 1, a.r, kBK, 2);
   ok &= make_map_chunked(&p->mapG3, a.G, a.m, n_whole > 0 ? n_whole / 64 : 1, a.ldg, kBK, bn / 64);
   ok &= make_map_chunked(&p->mapG3h, a.G, a.m, n_whole > 0 ? n_whole / 64 : 1, a.ldg, kBK, 2);
   ok &= make_map_chunked(&p->mapN3, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 4);
   ok &= make_map_chunked(&p->mapN3h, w.Nb, a.r, w.ldn / 64, w.ldn, kBK, 2);
+  // right projection: G (inner n = K, outer m) in boxes of 64 x 128 rows, Q~ (inner r = K, outer n) in 64 x 256
+  ok &= make_map(&p->mapGk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.G, a.n, a.m, a.ldg, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapQk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, prow, a.r, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
   p->r_whole = (int32_t)r_whole;
   p->n_whole = (int32_t)n_whole;
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, a.n, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, a.n, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+  ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
   if (!ok) {
     note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
     return QG_CUDA_ERROR;
@@ -1087,12 +1127,13 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->nb = w.Nb;
   p->ldmv = a.ldmv; p->ldw = a.W.ld; p->ldn = w.ldn;
   p->m = (int32_t)a.m; p->n = (int32_t)a.n; p->r = (int32_t)a.r;
+  p->right = a.right ? 1 : 0; p->k1_k = (int32_t)prow; p->k1_n = (int32_t)scol;
   p->ngroups = (int32_t)ceil_div(a.n, kGroup);
   p->seed_lo = a.sc.seed_lo; p->seed_hi = a.sc.seed_hi;
   p->k1_rblocks = (int32_t)ceil_div(a.r, kTileM);
-  p->k1_tiles = p->k1_rblocks * (int32_t)ceil_div(a.n, bn);
+  p->k1_tiles = p->k1_rblocks * (int32_t)ceil_div(scol, bn);
   p->k1_rpairs = (p->k1_rblocks + 1) / 2;
-  p->k1p_tiles = p->k1_rpairs * (int32_t)ceil_div(a.n, 256);
+  p->k1p_tiles = p->k1_rpairs * (int32_t)ceil_div(scol, 256);
   p->k2_mblocks = (int32_t)ceil_div(a.m, kTileM);
   p->k2_tiles = p->k2_mblocks * (int32_t)ceil_div(a.n, K2Smem::kBN);
   p->k2_mpairs = (p->k2_mblocks + 1) / 2;
@@ -1237,13 +1278,15 @@ dequant_p_grouped_kernel(const DequantItem* __restrict__ items, const int32_t* _
 
 }  // namespace
 
+// (m, n) here are the projection's row count and the state's column count: (m, n) of the matrix for the left
+// form, (n, m) for the right one
 size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r) { return scratch_pt_bytes(m, r) + scratch_nb_bytes(n, r); }
 
 int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
-  const TcScratch w = carve(a.ws, a.m, a.n, a.r);
+  const TcScratch w = carve(a.ws, proj_rows(a), state_cols(a), a.r);
   int rc = launch_dequant_p(a.P, w.Pt, a.r, st);
   if (rc != QG_OK) return rc;
-  const int bn = choose_bn(ceil_div(a.r, kTileM) * ceil_div(a.n, 256));
+  const int bn = choose_bn(ceil_div(a.r, kTileM) * ceil_div(state_cols(a), 256));
   TcProblem prob;
   rc = fill_problem(a, w, &prob, bn);
   if (rc != QG_OK) return rc;
@@ -1315,10 +1358,10 @@ size_t g_chunk_budget = 256ull << 20;
 size_t plan_table_bytes(const StepArgs* items, int32_t count) {
   size_t sched = 0;                                           // int32 words: pairs of every tile + starts per chunk
   for (int32_t i = 0; i < count; ++i) {
-    const int64_t k1 = ceil_div(items[i].r, kTileM) * ceil_div(items[i].n, 128);
+    const int64_t k1 = ceil_div(items[i].r, kTileM) * ceil_div(state_cols(items[i]), 128);
     const int64_t k2 = ceil_div(items[i].m, kTileM) * ceil_div(items[i].n, K2Smem::kBN);
     sched += (size_t)(2 * (k1 + k2)) + 2 * (size_t)(sm_count() + 3);
-    sched += (size_t)ceil_div(items[i].m * (items[i].r / 32), 256) + 2;      // block -> matrix map of the dequantize launch
+    sched += (size_t)ceil_div(proj_rows(items[i]) * (items[i].r / 32), 256) + 2;   // block -> matrix map of the dequantize launch
   }
   return (size_t)round_up((int64_t)count * sizeof(TcProblem), 256) + (size_t)round_up((int64_t)count * sizeof(DequantItem), 256) +
          sched * sizeof(int32_t) + 256;
@@ -1340,11 +1383,11 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     int j = i;
     int64_t tiles256 = 0;
     while (j < count) {
-      const size_t need = tc_workspace_bytes(items[j].m, items[j].n, items[j].r);
+      const size_t need = tc_workspace_bytes(proj_rows(items[j]), state_cols(items[j]), items[j].r);
       if (need > workspace_bytes) { delete plan; return QG_WORKSPACE_TOO_SMALL; }
       if (j > i && used + need > budget) break;
       used += need;
-      tiles256 += ceil_div(items[j].r, kTileM) * ceil_div(items[j].n, 256);
+      tiles256 += ceil_div(items[j].r, kTileM) * ceil_div(state_cols(items[j]), 256);
       ++j;
     }
     PlanChunk ch{};
@@ -1361,28 +1404,30 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     std::vector<int32_t> dq_map;
     for (int k = i; k < j; ++k) {
       const StepArgs& a = items[k];
-      const TcScratch w = carve(reinterpret_cast<char*>(workspace) + off, a.m, a.n, a.r);
-      off += tc_workspace_bytes(a.m, a.n, a.r);
+      const TcScratch w = carve(reinterpret_cast<char*>(workspace) + off, proj_rows(a), state_cols(a), a.r);
+      off += tc_workspace_bytes(proj_rows(a), state_cols(a), a.r);
       const int rc = fill_problem(a, w, &probs[k], ch.bn);
       if (rc != QG_OK) { delete plan; return rc; }
       ch.k1_tiles += probs[k].k1_tiles;
       ch.k2_tiles += probs[k].k2_tiles;
       // cost of a tile in K blocks of its main loop, plus a constant for its epilogue and hand-over
       const int k1n = ch.k1_pairs ? probs[k].k1p_tiles : probs[k].k1_tiles;
-      for (int t = 0; t < k1n; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(a.m, kBK) + 6.f); }
+      for (int t = 0; t < k1n; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(proj_rows(a), kBK) + 6.f); }
       ch.k1p_tiles += probs[k].k1p_tiles;
       const int k2n = (g_pair_mode & 1) ? probs[k].k2p_tiles : probs[k].k2_tiles;
       for (int t = 0; t < k2n; ++t) { t2.push_back(make_int2(k - i, t)); c2.push_back((float)ceil_div(a.r, kBK) + 6.f); }
       ch.k2p_tiles += probs[k].k2p_tiles;
       dq[k].P = a.P; dq[k].out = w.Pt;
       dq[k].block0 = ch.dq_blocks;
-      dq[k].nblocks = (int32_t)ceil_div(a.m * (a.r / 32), 256);
+      dq[k].nblocks = (int32_t)ceil_div(proj_rows(a) * (a.r / 32), 256);
       ch.dq_blocks += dq[k].nblocks;
       for (int32_t blk = 0; blk < dq[k].nblocks; ++blk) dq_map.push_back(k - i);
     }
     if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
     else ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
     ch.pairs = g_pair_mode & 1;
+    for (int k = i; k < j; ++k)
+      if (items[k].right) ch.pairs = 0;              // the paired back-projection knows the left form only
     if (ch.pairs) ch.k2_grid = 2 * (ch.k2p_tiles < sm_count() / 2 ? ch.k2p_tiles : sm_count() / 2);   // CTA pairs
     else ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
     schedule_tiles(t1, c1, ch.k1_pairs ? ch.k1_grid / 2 : ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);

@@ -144,16 +144,17 @@ def check_weight_codes_unforced(gpu_w: O.QTensor, ref: dict, max_frac=5e-3):
 class StepTaps:
     """Device buffers for the optional intermediates of qgalore_project_step."""
 
-    def __init__(self, m, n, r, w_ld):
-        self.R = B.zeros_matrix(r, n, torch.float32)
-        self.N = B.zeros_matrix(r, n, torch.float32)
+    def __init__(self, m, n, r, w_ld, side="left"):
+        sc = m if side == "right" else n                # columns of the low-rank state
+        self.R = B.zeros_matrix(r, sc, torch.float32)
+        self.N = B.zeros_matrix(r, sc, torch.float32)
         self.W_pre = torch.zeros((m, w_ld), dtype=torch.float32, device="cuda")[:, :n]
 
     def as_dict(self):
         return {"R": self.R, "N": self.N, "W_pre": self.W_pre}
 
 
-def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2e-3, impl=None):
+def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2e-3, impl=None, side="left"):
     """Teacher-forced single-step parity of qgalore_project_step against the oracle.
 
     Stage 1 (steps 1-4): M', V', R and the direction N against the oracle's own.
@@ -163,10 +164,10 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
     """
     m, n = gb.shape
     r = P.codes.shape[1]
-    ref = O.project_step(gb, P, W, M, V, hyp)
+    ref = O.project_step(gb, P, W, M, V, hyp, side=side)
     dG, dP, dW = g_to_device(gb), to_device_q(P), to_device_q(W)
     dM, dV = f32_to_device(M), f32_to_device(V)
-    taps = StepTaps(m, n, r, dW.ld)
+    taps = StepTaps(m, n, r, dW.ld, side)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     if impl is not None:
         B.debug_set_step_impl(impl)
@@ -175,7 +176,7 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
                        B.Hyper(lr=hyp.lr, alpha=hyp.alpha, beta1=hyp.beta1, beta2=hyp.beta2, eps=hyp.eps,
                                weight_decay=hyp.weight_decay, step=hyp.step, seed=hyp.seed,
                                rounding=B.QG_ROUND_NEAREST if hyp.rounding == "rtn" else B.QG_ROUND_STOCHASTIC),
-                       status=status, debug=taps.as_dict())
+                       status=status, debug=taps.as_dict(), side=side)
         torch.cuda.synchronize()
     finally:
         if impl is not None:
@@ -188,7 +189,7 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
     n_gpu = taps.N.cpu().numpy()
     ill = check_direction(n_gpu, ref, hyp, "N", tol)
     # stage 2: same direction on both sides
-    forced = O.project_step(gb, P, W, M, V, hyp, N_b_override=O.bf16_round(n_gpu))
+    forced = O.project_step(gb, P, W, M, V, hyp, N_b_override=O.bf16_round(n_gpu), side=side)
     lsb = np.repeat(forced["W"].scales, 256, axis=1)[:, :n]
     wpre_err = float((np.abs(taps.W_pre.cpu().numpy() - forced["W_pre"]) / lsb).max())
     assert wpre_err <= 1e-3, f"pre-rounding weight off by {wpre_err:.2e} LSB"
@@ -200,8 +201,9 @@ def run_and_check_step(gb, P: O.QTensor, W: O.QTensor, M, V, hyp: O.Hyper, tol=2
         assert int(dW.codes[:, n:].abs().max().item()) == 0, "padding of the code rows was written"
     for t in (dM, dV):
         base = t._base
-        if base is not None and base.shape[1] > n:
-            assert float(base[:, n:].abs().max().item()) == 0.0, "padding of the moment rows was written"
+        sc = m if side == "right" else n
+        if base is not None and base.shape[1] > sc:
+            assert float(base[:, sc:].abs().max().item()) == 0.0, "padding of the moment rows was written"
     return {"mismatch": frac, "mismatch_unforced": frac_unforced, "ill": ill, "wpre_err_lsb": wpre_err,
             "W": gw, "M": dM.cpu().numpy(), "V": dV.cpu().numpy(), "ref": ref}
 

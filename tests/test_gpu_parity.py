@@ -529,3 +529,66 @@ def test_step_refuses_empty_oversized_and_misshapen_problems():
     assert L.qgalore_project_step(dG.data_ptr(), 4096, 4096, 256, 4096, C.byref(bc), C.byref(wc), dM.data_ptr(), dV.data_ptr(),
                                   256, C.byref(h), ws.data_ptr(), ws.numel(), None, None, None) in (B.QG_UNSUPPORTED_SHAPE,
                                                                                                     B.QG_INVALID_ARGUMENT)
+
+
+# ----------------------------------------------------------------------------- projection on the right (GaLore's other side)
+def _right_case(m, n, r, seed, step=2):
+    gm = synth.GradientModel(m, n, seed=seed, matrix_index=0)
+    Q = O.quantize_rtn(synth.random_orthonormal(n, r, seed=seed), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, seed), 8)
+    Mt = np.zeros((r, m), np.float32)
+    Vt = np.zeros((r, m), np.float32)
+    for t in range(1, step):
+        o = O.project_step(gm.sample(t), Q, W, Mt, Vt, O.Hyper(step=t, seed=seed), side="right")
+        W, Mt, Vt = o["W"], o["M"], o["V"]
+    return gm.sample(step), Q, W, Mt, Vt
+
+
+@pytest.mark.parametrize("m,n,r", [(512, 256, 64), (777, 300, 96), (1376, 512, 128), (85, 1000, 32), (2736, 1024, 256)])
+def test_step_with_the_projection_on_the_right(m, n, r):
+    gb, Q, W, Mt, Vt = _right_case(m, n, r, seed=m + n)
+    stats = run_and_check_step(gb, Q, W, Mt, Vt, O.Hyper(step=2, seed=m + n), side="right")
+    assert stats["mismatch"] <= 1e-3
+
+
+def test_right_projection_at_a_llama1b_size():
+    m, n, r = 5461, 2048, 512                            # the down projection: m > n
+    gb, Q, W, Mt, Vt = _right_case(m, n, r, seed=31)
+    run_and_check_step(gb, Q, W, Mt, Vt, O.Hyper(step=2, seed=31), side="right")
+
+
+def test_plan_mixes_projection_sides():
+    cases = [((512, 256, 64), "right"), ((256, 512, 64), "left"), ((1376, 512, 256), "right"), ((768, 768, 256), "left"),
+             ((2048, 1024, 512), "right")]
+    step = 2
+    single, items = [], []
+    for idx, ((m, n, r), side) in enumerate(cases):
+        right = side == "right"
+        gb = synth.GradientModel(m, n, seed=17, matrix_index=idx).sample(step)
+        P = O.quantize_rtn(synth.random_orthonormal(n if right else m, r, seed=17, stream=idx), 4)
+        W = O.quantize_rtn(synth.initial_weight(m, n, 17, idx), 8)
+        rng = np.random.default_rng(idx)
+        sc = m if right else n
+        M = rng.normal(0, 1e-3, (r, sc)).astype(np.float32)
+        V = (rng.normal(0, 1e-3, (r, sc)) ** 2).astype(np.float32)
+        dG, dP = g_to_device(gb), to_device_q(P)
+        dW1, dM1, dV1 = to_device_q(W), f32_to_device(M), f32_to_device(V)
+        B.project_step(dG, dP, dW1, dM1, dV1, B.Hyper(step=step, seed=idx), side=side)
+        single.append((dW1, dM1, dV1))
+        items.append({"G": dG, "P": dP, "W": to_device_q(W), "M": f32_to_device(M), "V": f32_to_device(V), "seed": idx,
+                      "side": side})
+    for pair_mode in (2, 0):
+        B.lib().qgalore_debug_set_pair_mode(pair_mode)
+        try:
+            fresh = [{**it, "W": it["W"].clone(), "M": it["M"]._base.clone()[:, :it["M"].shape[1]],
+                      "V": it["V"]._base.clone()[:, :it["V"].shape[1]]} for it in items]
+            plan = B.StepPlan(fresh)
+            plan.step(B.Hyper(step=step))
+            torch.cuda.synchronize()
+            assert int(plan.status.item()) == 0
+            for (dW1, dM1, dV1), it in zip(single, fresh):
+                assert torch.equal(dW1.codes, it["W"].codes)
+                assert torch.equal(dM1._base, it["M"]._base) and torch.equal(dV1._base, it["V"]._base)
+            plan.close()
+        finally:
+            B.lib().qgalore_debug_set_pair_mode(2)

@@ -558,3 +558,36 @@ def test_coarser_projection_loses_more_of_the_subspace():
         Ph = O.dequantize(O.quantize_rtn(P, bits)).astype(np.float64)
         err[bits] = np.linalg.norm(Ph.T @ Ph - np.eye(128)) / np.sqrt(128)
     assert err[8] < err[4] < err[2] and err[8] < 1e-2 and err[2] > 0.1
+
+
+def test_right_projection_is_the_left_projection_of_the_transposed_gradient():
+    # GaLore projects on the side of the shorter dimension; R = G Q is (Q^T G^T)^T, so the low-rank state of the
+    # right form on G is that of the left form on G^T, and the two updates are transposes of each other.  The
+    # weights differ (quantization groups run along the rows of W either way), so they are compared through D.
+    from paper_2407_08296_b200 import synth
+    m, n, r = 300, 128, 32
+    gb = synth.GradientModel(m, n, seed=8, matrix_index=0).sample(1)
+    Q = O.quantize_rtn(synth.random_orthonormal(n, r, seed=8), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 8), 8)
+    Wt = O.quantize_rtn(synth.initial_weight(n, m, 8), 8)
+    rng = np.random.default_rng(8)
+    Mt = rng.normal(0, 1e-3, (r, m)).astype(np.float32)
+    Vt = (rng.normal(0, 1e-3, (r, m)) ** 2).astype(np.float32)
+    hyp = O.Hyper(step=3, seed=1)
+    right = O.project_step(gb, Q, W, Mt, Vt, hyp, side="right")
+    left = O.project_step(np.ascontiguousarray(gb.T), Q, Wt, Mt, Vt, hyp)
+    assert right["M"].shape == (r, m)
+    for k in ("R32", "M", "V"):
+        assert np.allclose(right[k], left[k], rtol=1e-6, atol=1e-12), k
+    good = np.sqrt(left["V"].astype(np.float64) / (1 - 0.999 ** 3)) > 1e-5
+    assert np.allclose(right["N"][good], left["N"][good], rtol=1e-4)
+    # with the same direction on both sides the two updates are transposes
+    right_f = O.project_step(gb, Q, W, Mt, Vt, hyp, side="right", N_b_override=left["N_b"])
+    d_right = (O.dequantize(W).astype(np.float64) - right_f["W_pre"]) / (0.004 * 0.25)
+    d_left = (O.dequantize(Wt).astype(np.float64) - left["W_pre"]) / (0.004 * 0.25)
+    scale = np.abs(d_left).max()
+    assert np.abs(d_right - d_left.T).max() <= 1e-3 * scale       # fp32 rounding of W' on either side
+    # and the definition itself on a tiny case: R = G Q~
+    Qt = O.bf16_round(O.dequantize(Q)).astype(np.float64)
+    G = O.bf16_bits_to_f32(gb).astype(np.float64)
+    assert np.allclose(right["R32"], (G @ Qt).T.astype(np.float32), rtol=1e-6, atol=1e-12)
