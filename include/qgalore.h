@@ -213,6 +213,15 @@ QG_API int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, i
                              const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev,
                              void* workspace, size_t workspace_bytes,
                              int32_t* status_dev, void* stream);
+/* The same for the right-hand projection: the top-r RIGHT singular vectors of G, i.e. the left ones of G^T
+ * (G is read with its strides swapped, nothing is transposed in memory).  Q_new, Q_prev, Q_fp32 are n x r;
+ * workspace qgalore_workspace_bytes(QG_OP_REFRESH, n, m, b). */
+QG_API int qgalore_refresh_subspace_right(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r,
+                                   int32_t iters, int32_t oversample_cols, uint64_t seed,
+                                   const qg_qtensor* Q_new, float* Q_fp32,
+                                   const qg_qtensor* Q_prev, int32_t sim_cols, float* sim_dev,
+                                   void* workspace, size_t workspace_bytes,
+                                   int32_t* status_dev, void* stream);
 
 /* --- Sec. 3.2: cosine similarity between adjacent projection matrices -------------------
  * *sim_dev = sum_{j < c} |<a_j, b_j>| / (||A[:, :c]||_F ||B[:, :c]||_F), c = sim_cols

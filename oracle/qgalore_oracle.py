@@ -388,7 +388,7 @@ def _project_step_right(G_bits, Q_q: QTensor, W_q: QTensor, Mt, Vt, h: Hyper, N_
 
 
 # --------------------------------------------------------------------------- refresh (Sec. 3.5, Sec. 1)
-def refresh_subspace(G_bits, r, group=GROUP, bits=4):
+def refresh_subspace(G_bits, r, group=GROUP, bits=4, side="left"):
     """Projection matrix from the SVD of the gradient: the top-r left singular vectors.
 
     Exact LAPACK SVD (gesdd) of the gradient widened to fp64.  Each column's sign is
@@ -396,6 +396,8 @@ def refresh_subspace(G_bits, r, group=GROUP, bits=4):
     its quantization (INT4 is the method, Sec. 3.3; 2 and 8 bits are the ablation of Sec. 4.4), singular values).
     """
     G = bf16_bits_to_f32(G_bits).astype(np.float64)
+    if side == "right":          # the right singular vectors of G are the left ones of its transpose
+        G = np.ascontiguousarray(G.T)
     U, S, _ = scipy.linalg.svd(G, full_matrices=False, lapack_driver="gesdd")
     P = U[:, :r].copy()
     piv = np.argmax(np.abs(P), axis=0)

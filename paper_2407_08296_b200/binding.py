@@ -90,6 +90,7 @@ def lib() -> C.CDLL:
         L.qgalore_plan_destroy.restype = None
         L.qgalore_refresh_subspace.argtypes = [vp, i64, i64, i64, i64, i32, i32, C.c_uint64, qp, vp, qp, i32, vp,
                                                vp, sz, vp, vp]
+        L.qgalore_refresh_subspace_right.argtypes = L.qgalore_refresh_subspace.argtypes
         L.qgalore_subspace_similarity.argtypes = [qp, qp, i32, vp, vp, sz, vp]
         L.qgalore_subspace_similarity_static.argtypes = [qp, qp, i32, vp, vp]
         L.qgalore_subspace_similarity_static_max_bytes.restype = sz
@@ -367,29 +368,33 @@ class StepPlan:
 def refresh_subspace(G: torch.Tensor, r: int, iters: int = 12, oversample_cols: int | None = None, seed: int = 0,
                      P_new: QTensor | None = None, P_fp32: torch.Tensor | None = None, P_prev: QTensor | None = None,
                      sim_cols: int = 0, sim: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
-                     status: torch.Tensor | None = None, stream=None) -> QTensor:
-    """New INT4 projection matrix from the top-r left singular subspace of G (Sec. 3.5, Sec. 3.3)."""
+                     status: torch.Tensor | None = None, stream=None, side: str = "left") -> QTensor:
+    """New INT4 projection matrix from the top-r left singular subspace of G (Sec. 3.5, Sec. 3.3); with
+    ``side`` = "right" from its right singular subspace (an n x r matrix, for the right-hand projection)."""
     m, n = G.shape
+    right = side == "right"
+    pm, pn_ = (n, m) if right else (m, n)
     if oversample_cols is None:     # block of 2 r columns, in whole panels of 64, never wider than the matrix
         block = min((2 * r + 63) // 64 * 64, min(m, n) // 64 * 64)
         oversample_cols = max(block - r, 0)
     if P_new is None:
-        P_new = QTensor.empty(m, r, 4, G.device)
+        P_new = QTensor.empty(pm, r, 4, G.device)
         if P_new.ld != r:               # the refresh writes a densely packed P (ld == r)
             ng = (r + GROUP - 1) // GROUP
-            P_new = QTensor(torch.full((m, r // 2), 0x88, dtype=torch.uint8, device=G.device),
-                            torch.zeros((m, ng), dtype=torch.float32, device=G.device),
-                            torch.zeros((m, ng), dtype=torch.float32, device=G.device), m, r, r, 4)
+            P_new = QTensor(torch.full((pm, r // 2), 0x88, dtype=torch.uint8, device=G.device),
+                            torch.zeros((pm, ng), dtype=torch.float32, device=G.device),
+                            torch.zeros((pm, ng), dtype=torch.float32, device=G.device), pm, r, r, 4)
     if workspace is None:
-        workspace = torch.empty(workspace_bytes(QG_OP_REFRESH, m, n, r + oversample_cols), dtype=torch.uint8,
+        workspace = torch.empty(workspace_bytes(QG_OP_REFRESH, pm, pn_, r + oversample_cols), dtype=torch.uint8,
                                 device=G.device)
     pn = P_new.c_struct()
     pp = P_prev.c_struct() if P_prev is not None else None
-    _check(lib().qgalore_refresh_subspace(_ptr(G), _matrix_ld(G, "G"), m, n, r, iters, oversample_cols, seed,
-                                          C.byref(pn), _ptr(P_fp32), C.byref(pp) if pp is not None else None,
-                                          sim_cols, _ptr(sim), _ptr(workspace),
-                                          workspace.numel() * workspace.element_size(), _ptr(status),
-                                          _stream_ptr(stream)), "qgalore_refresh_subspace")
+    fn = lib().qgalore_refresh_subspace_right if right else lib().qgalore_refresh_subspace
+    _check(fn(_ptr(G), _matrix_ld(G, "G"), m, n, r, iters, oversample_cols, seed,
+              C.byref(pn), _ptr(P_fp32), C.byref(pp) if pp is not None else None,
+              sim_cols, _ptr(sim), _ptr(workspace),
+              workspace.numel() * workspace.element_size(), _ptr(status),
+              _stream_ptr(stream)), "qgalore_refresh_subspace_right" if right else "qgalore_refresh_subspace")
     return P_new
 
 

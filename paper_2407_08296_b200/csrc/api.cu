@@ -25,7 +25,7 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st);
 size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r);
 int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
                    uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
-                   cudaStream_t st);
+                   cudaStream_t st, bool transposed);
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b);
 struct Plan;
 size_t plan_table_bytes(const StepArgs* items, int32_t count);
@@ -304,21 +304,23 @@ void qgalore_plan_destroy(qg_plan* plan) {
   delete plan;
 }
 
-int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
-                             int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
-                             const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
-                             size_t workspace_bytes, int32_t* status_dev, void* stream) {
+static int refresh_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
+                        int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
+                        const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
+                        size_t workspace_bytes, int32_t* status_dev, void* stream, bool right) {
   if (!G || !workspace || m <= 0 || n <= 0 || r <= 0 || ldg < n || iters < 0 || oversample_cols < 0)
     return QG_INVALID_ARGUMENT;
+  // the matrix whose LEFT singular vectors are wanted: G, or G^T for the right-hand projection
+  const int64_t pm = right ? n : m, pn = right ? m : n;
   if (!P_new || (P_new->bits != 2 && P_new->bits != 4 && P_new->bits != 8)) return QG_INVALID_ARGUMENT;
   int rc = check_qtensor(P_new, P_new->bits);
   if (rc != QG_OK) return rc;
-  if (P_new->rows != m || P_new->cols != r || P_new->ld != r) return QG_INVALID_ARGUMENT;
+  if (P_new->rows != pm || P_new->cols != r || P_new->ld != r) return QG_INVALID_ARGUMENT;
   if (P_prev) {
     if (P_prev->bits != 2 && P_prev->bits != 4 && P_prev->bits != 8) return QG_INVALID_ARGUMENT;
     rc = check_qtensor(P_prev, P_prev->bits);
     if (rc != QG_OK) return rc;
-    if (P_prev->rows != m || P_prev->cols != r) return QG_INVALID_ARGUMENT;
+    if (P_prev->rows != pm || P_prev->cols != r) return QG_INVALID_ARGUMENT;
   }
   const int64_t b = r + oversample_cols;
   // the block is handled in panels of 64 columns and cannot be wider than the matrix is tall or wide
@@ -327,10 +329,10 @@ int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
   if (!aligned16(G) || ldg % 8 != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return QG_MISALIGNED;
   if (P_fp32 && !aligned16(P_fp32)) return QG_MISALIGNED;
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
-  if (workspace_bytes < qgalore_workspace_bytes(QG_OP_REFRESH, m, n, b)) return QG_WORKSPACE_TOO_SMALL;
+  if (workspace_bytes < qgalore_workspace_bytes(QG_OP_REFRESH, pm, pn, b)) return QG_WORKSPACE_TOO_SMALL;
   constexpr int kJacobiSweeps = 12;
-  rc = launch_refresh(G, ldg, m, n, r, b, iters, kJacobiSweeps, seed, P_new, P_fp32, workspace, workspace_bytes,
-                      status_dev, (cudaStream_t)stream);
+  rc = launch_refresh(G, ldg, pm, pn, r, b, iters, kJacobiSweeps, seed, P_new, P_fp32, workspace, workspace_bytes,
+                      status_dev, (cudaStream_t)stream, right);
   if (rc != QG_OK) return rc;
   if (P_prev && sim_dev) {
     const int32_t c = (sim_cols <= 0 || sim_cols > r) ? (int32_t)r : sim_cols;
@@ -338,6 +340,22 @@ int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
     return launch_similarity(P_prev, P_new, c, sim_dev, workspace, (cudaStream_t)stream);
   }
   return QG_OK;
+}
+
+int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
+                             int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
+                             const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
+                             size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  return refresh_impl(G, ldg, m, n, r, iters, oversample_cols, seed, P_new, P_fp32, P_prev, sim_cols, sim_dev, workspace,
+                      workspace_bytes, status_dev, stream, false);
+}
+
+int qgalore_refresh_subspace_right(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
+                                   int32_t oversample_cols, uint64_t seed, const qg_qtensor* Q_new, float* Q_fp32,
+                                   const qg_qtensor* Q_prev, int32_t sim_cols, float* sim_dev, void* workspace,
+                                   size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  return refresh_impl(G, ldg, m, n, r, iters, oversample_cols, seed, Q_new, Q_fp32, Q_prev, sim_cols, sim_dev, workspace,
+                      workspace_bytes, status_dev, stream, true);
 }
 
 int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,

@@ -487,9 +487,12 @@ int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cu
 
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b) { return carve_refresh(nullptr, m, n, b, b, nullptr); }
 
+// `transposed`: the singular vectors wanted are the RIGHT ones of G, i.e. the left ones of G^T; G is then read
+// with its two strides swapped and (m, n) below are the extents of G^T.
 int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
                    uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
-                   cudaStream_t st) {
+                   cudaStream_t st, bool transposed) {
+  const int64_t rs = transposed ? 1 : ldg, cs = transposed ? ldg : 1;   // strides between rows / columns of the matrix
   RefreshWs w;
   if (carve_refresh(ws, m, n, b, r, &w) > ws_bytes) return QG_WORKSPACE_TOO_SMALL;
   int rc;
@@ -503,11 +506,11 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
   }
   for (int it = 0; it <= iters; ++it) {
     // Z = G^T Q
-    rc = gemm<uint16_t, float, float>(G, 1, ldg, w.Q, b, 1, w.Z, b, n, b, m, 1.f, 0.f, st);
+    rc = gemm<uint16_t, float, float>(G, cs, rs, w.Q, b, 1, w.Z, b, n, b, m, 1.f, 0.f, st);
     if (rc != QG_OK) return rc;
     if (it == iters) break;
     // Y = G Z
-    rc = gemm<uint16_t, float, float>(G, ldg, 1, w.Z, b, 1, w.Y, b, m, b, n, 1.f, 0.f, st);
+    rc = gemm<uint16_t, float, float>(G, rs, cs, w.Z, b, 1, w.Y, b, m, b, n, 1.f, 0.f, st);
     if (rc != QG_OK) return rc;
     rc = orthonormalize(w, m, b, status, st);
     if (rc != QG_OK) return rc;

@@ -592,3 +592,20 @@ def test_plan_mixes_projection_sides():
             plan.close()
         finally:
             B.lib().qgalore_debug_set_pair_mode(2)
+
+
+@pytest.mark.parametrize("m,n,r", [(320, 256, 64), (1376, 512, 128)])
+def test_refresh_of_the_right_singular_subspace(m, n, r):
+    gb = synth.GradientModel(m, n, seed=5, matrix_index=2).sample(1)
+    Q_ref, _, _ = O.refresh_subspace(gb, r, side="right")
+    Q32 = torch.zeros((n, r), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Qq = B.refresh_subspace(g_to_device(gb), r, P_fp32=Q32, status=status, side="right")
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and (Qq.rows, Qq.cols) == (n, r)
+    q = Q32.cpu().numpy()
+    assert O.principal_angle(Q_ref, q) < 1e-2
+    assert np.abs(q.T.astype(np.float64) @ q - np.eye(r)).max() < 1e-4
+    ref_q = O.quantize_rtn(q, 4)
+    got = from_device_q(Qq)
+    assert np.array_equal(got.codes, ref_q.codes) and np.array_equal(got.scales, ref_q.scales)
