@@ -38,7 +38,7 @@ __all__ = [
     "philox4x32_10", "sr_uniform16", "group_params", "quantize_rtn", "quantize_sr",
     "dequantize", "pack_int4", "unpack_int4", "pack_int2", "unpack_int2", "QTensor", "Hyper", "project_step",
     "refresh_subspace", "subspace_similarity", "GateState", "gate_update",
-    "principal_angle",
+    "principal_angle", "STATE_BLOCK", "Moments8", "quantize_m8", "quantize_v8", "dequantize_m8", "dequantize_v8",
 ]
 
 GROUP = 256  # Sec. 3.1: block size 256 in all implementations
@@ -280,6 +280,83 @@ def unpack_int2(packed, cols):
     return (out[:, :cols] - 2).astype(np.int8)
 
 
+# --------------------------------------------------------------------------- 8-bit moments (Sec. 3.5 "8-bit Adam")
+# The paper keeps the Adam states of the low-rank subspace in 8 bits and cites block-wise 8-bit optimizers
+# for it without giving a format.  The format here is this build's own: blocks of STATE_BLOCK consecutive
+# elements along a row (restarting at every row, a shorter block at a ragged end), one binary32 scale per block.
+#   first moment  (signed):   s = max |x|;  code = rint(x * (1 / (s / 127))) in [-127, 127];  x^ = code * (s / 127)
+#   second moment (>= 0):     s = max x;    code = rint(255 * sqrt(x * (1 / s))) in [0, 255];  x^ = (code / 255)^2 * s
+# (the square-root law gives small second moments the relative precision a linear code would not).  Every
+# operation is a single binary32 operation in the order written; an all-zero block has scale 0 and codes 0.
+STATE_BLOCK = 32
+
+
+@dataclass
+class Moments8:
+    codes: np.ndarray    # int8 (first moment) or uint8 (second moment) [rows, cols]
+    scales: np.ndarray   # float32 [rows, ceil(cols / STATE_BLOCK)]
+
+
+def _state_blocks(cols):
+    return [(a, min(a + STATE_BLOCK, cols)) for a in range(0, cols, STATE_BLOCK)]
+
+
+def quantize_m8(x):
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    rows, cols = x.shape
+    bl = _state_blocks(cols)
+    codes = np.zeros((rows, cols), np.int8)
+    scales = np.zeros((rows, len(bl)), np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        for k, (a, b) in enumerate(bl):
+            seg = x[:, a:b]
+            s = np.abs(seg).max(axis=1).astype(np.float32)
+            step = (s / np.float32(127.0)).astype(np.float32)
+            inv = np.where(step > 0, np.float32(1.0) / step, np.float32(0.0)).astype(np.float32)
+            q = np.rint((seg * inv[:, None]).astype(np.float32))
+            codes[:, a:b] = np.clip(q, -127, 127).astype(np.int8)
+            scales[:, k] = s
+    return Moments8(codes, scales)
+
+
+def dequantize_m8(q: Moments8):
+    rows, cols = q.codes.shape
+    out = np.empty((rows, cols), np.float32)
+    for k, (a, b) in enumerate(_state_blocks(cols)):
+        step = (q.scales[:, k] / np.float32(127.0)).astype(np.float32)
+        out[:, a:b] = (q.codes[:, a:b].astype(np.float32) * step[:, None]).astype(np.float32)
+    return out
+
+
+def quantize_v8(x):
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    rows, cols = x.shape
+    bl = _state_blocks(cols)
+    codes = np.zeros((rows, cols), np.uint8)
+    scales = np.zeros((rows, len(bl)), np.float32)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        for k, (a, b) in enumerate(bl):
+            seg = x[:, a:b]
+            s = seg.max(axis=1).astype(np.float32)
+            inv = np.where(s > 0, np.float32(1.0) / s, np.float32(0.0)).astype(np.float32)
+            t = (seg * inv[:, None]).astype(np.float32)
+            u = np.sqrt(np.maximum(t, np.float32(0.0))).astype(np.float32)
+            q = np.rint((u * np.float32(255.0)).astype(np.float32))
+            codes[:, a:b] = np.clip(q, 0, 255).astype(np.uint8)
+            scales[:, k] = s
+    return Moments8(codes, scales)
+
+
+def dequantize_v8(q: Moments8):
+    rows, cols = q.codes.shape
+    out = np.empty((rows, cols), np.float32)
+    c = np.float32(1.0) / np.float32(255.0)
+    for k, (a, b) in enumerate(_state_blocks(cols)):
+        w = (q.codes[:, a:b].astype(np.float32) * c).astype(np.float32)
+        out[:, a:b] = ((w * w).astype(np.float32) * q.scales[:, k:k + 1]).astype(np.float32)
+    return out
+
+
 # --------------------------------------------------------------------------- the step (Sec. 3.5)
 @dataclass
 class Hyper:
@@ -321,10 +398,24 @@ def project_step(G_bits, P_q: QTensor, W_q: QTensor, M, V, h: Hyper, P_override=
     describes).  "right" is GaLore's other form, R = G Q with Q = P_q of shape n x r: the low-rank state is
     m x r, and M, V, R32, N, N_b are kept and returned TRANSPOSED (r x m, row-major) so that both forms
     hand the same kind of array around; the update is D = N Q^T.  (col0 is for the left form only.)
+    M and V may also be Moments8 (the 8-bit block-wise storage defined above): they are dequantized on the
+    way in, the step runs on binary32 moments as written, the direction N is taken from the binary32 M', V',
+    and the result also carries their 8-bit form as "M8", "V8" ("M", "V" stay the binary32 values before storage).
     """
+    state8 = isinstance(M, Moments8)
+    if state8:
+        M, V = dequantize_m8(M), dequantize_v8(V)
     if side == "right":
         assert col0 == 0
-        return _project_step_right(G_bits, P_q, W_q, M, V, h, N_b_override)
+        out = _project_step_right(G_bits, P_q, W_q, M, V, h, N_b_override)
+    else:
+        out = _project_step_left(G_bits, P_q, W_q, M, V, h, P_override, N_b_override, col0)
+    if state8:
+        out["M8"], out["V8"] = quantize_m8(out["M"]), quantize_v8(out["V"])
+    return out
+
+
+def _project_step_left(G_bits, P_q, W_q, M, V, h, P_override, N_b_override, col0):
     lr, alpha, b1, b2, eps, wd = h.as_f32()
     t = int(h.step)
     G = bf16_bits_to_f32(G_bits).astype(np.float64)

@@ -591,3 +591,64 @@ def test_right_projection_is_the_left_projection_of_the_transposed_gradient():
     Qt = O.bf16_round(O.dequantize(Q)).astype(np.float64)
     G = O.bf16_bits_to_f32(gb).astype(np.float64)
     assert np.allclose(right["R32"], (G @ Qt).T.astype(np.float32), rtol=1e-6, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- 8-bit moments (format of this build)
+def test_8bit_moment_formats_bounds_idempotence_and_zero_blocks():
+    # Sec. 3.5 keeps the Adam states in 8 bits without giving a format; the one built here is pinned by what it
+    # promises: the first moment is off by at most half a step s/127, the square root of the second by at most
+    # half of sqrt(s)/255 (the square-root law), the largest element of a block is exact, storing a stored
+    # value again changes nothing, codes are monotone, zero blocks stay zero, ragged rows end in a short block.
+    rng = np.random.default_rng(11)
+    rows, cols = 9, 3 * 32 + 7
+    x = (rng.normal(0, 1e-3, (rows, cols)) * rng.lognormal(0, 2, (rows, 1))).astype(np.float32)
+    x[2, 32:64] = 0.0
+    q = O.quantize_m8(x)
+    assert q.scales.shape == (rows, 4) and q.codes.dtype == np.int8 and np.abs(q.codes.astype(int)).max() == 127
+    xh = O.dequantize_m8(q)
+    step = np.repeat(q.scales / 127.0, 32, axis=1)[:, :cols]
+    assert np.all(np.abs(xh - x) <= 0.5 * step * (1 + 1e-5))
+    assert np.all(q.codes[2, 32:64] == 0) and q.scales[2, 1] == 0.0 and np.all(xh[2, 32:64] == 0.0)
+    for k, (a, b) in enumerate([(0, 32), (32, 64), (64, 96), (96, cols)]):
+        top = np.abs(x[:, a:b]).argmax(axis=1)
+        assert np.array_equal(np.abs(xh[np.arange(rows), a + top]), q.scales[:, k])       # the block maximum is exact
+    again = O.quantize_m8(xh)
+    assert np.array_equal(again.codes, q.codes) and np.allclose(again.scales, q.scales, rtol=2e-7)
+    order = np.argsort(x[0, :32])
+    assert np.all(np.diff(q.codes[0, :32][order].astype(int)) >= 0)                        # monotone
+
+    v = (x.astype(np.float64) ** 2).astype(np.float32)
+    qv = O.quantize_v8(v)
+    assert qv.codes.dtype == np.uint8 and qv.codes.max() == 255
+    vh = O.dequantize_v8(qv)
+    root = np.repeat(np.sqrt(qv.scales.astype(np.float64)) / 255.0, 32, axis=1)[:, :cols]
+    assert np.all(np.abs(np.sqrt(vh.astype(np.float64)) - np.sqrt(v.astype(np.float64))) <= 0.5 * root * (1 + 1e-4))
+    assert np.all(qv.codes[2, 32:64] == 0) and np.all(vh[2, 32:64] == 0.0)
+    assert np.array_equal(O.quantize_v8(vh).codes, qv.codes)
+    # the square-root law: an element 10^4 times smaller than the block maximum still has a code
+    t = np.full((1, 32), 1e-12, np.float32)
+    t[0, 0] = 1e-8
+    assert O.quantize_v8(t).codes[0, 1] >= 2 and O.dequantize_v8(O.quantize_v8(t))[0, 1] > 0
+
+
+def test_step_on_8bit_moments_is_the_step_on_their_values_and_tracks_the_fp32_run():
+    from paper_2407_08296_b200 import synth
+    m, n, r = 96, 2 * 32 + 20, 32
+    gm = synth.GradientModel(m, n, seed=6, matrix_index=0)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=6), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 6), 8)
+    z = np.zeros((r, n), np.float32)
+    M8, V8 = O.quantize_m8(z), O.quantize_v8(z)
+    Mf, Vf, Wf, W8 = z, z, W, W
+    for t in range(1, 6):
+        hyp = O.Hyper(step=t, seed=2)
+        a = O.project_step(gm.sample(t), P, W8, M8, V8, hyp)
+        b = O.project_step(gm.sample(t), P, W8, O.dequantize_m8(M8), O.dequantize_v8(V8), hyp)
+        assert np.array_equal(a["M"], b["M"]) and np.array_equal(a["W"].codes, b["W"].codes)      # same step
+        assert np.array_equal(a["M8"].codes, O.quantize_m8(a["M"]).codes)
+        f = O.project_step(gm.sample(t), P, Wf, Mf, Vf, hyp)
+        M8, V8, W8 = a["M8"], a["V8"], a["W"]
+        Mf, Vf, Wf = f["M"], f["V"], f["W"]
+    # five steps on: the stored moments stay close to the binary32 ones (no drift from the rounding of the state)
+    assert np.linalg.norm(O.dequantize_m8(M8) - Mf) <= 0.02 * np.linalg.norm(Mf)
+    assert np.linalg.norm(np.sqrt(O.dequantize_v8(V8)) - np.sqrt(Vf)) <= 0.02 * np.linalg.norm(np.sqrt(Vf))
