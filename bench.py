@@ -42,12 +42,16 @@ def matrix_flops(m, n, r):
     return 4.0 * m * n * r                      # two dense contractions of 2 m n r each
 
 
+MOMENT_BYTES = 16.0      # M, V read + written per element of the low-rank state: 4 x 4 bytes in fp32,
+                         # 4 x 1 byte + 4 scale words per 32 elements = 4.5 with --moments 8
+
+
 def matrix_bytes(m, n, r):
     """Algorithmic HBM bytes of one step of one matrix: G (bf16), W codes read+write, W scale/zero
     read+write, P codes + scale/zero, M and V fp32 read+write."""
     ng_n = (n + 255) // 256
     ng_r = (r + 255) // 256
-    return 2 * m * n + 2 * m * n + 16 * m * ng_n + m * r // 2 + 8 * m * ng_r + 16 * r * n
+    return 2 * m * n + 2 * m * n + 16 * m * ng_n + m * r // 2 + 8 * m * ng_r + MOMENT_BYTES * r * n
 
 
 # Algorithmic units of each kernel of the step, per matrix (what the method has to move or compute, not what
@@ -55,7 +59,7 @@ def matrix_bytes(m, n, r):
 # the back-projection reads+writes the INT8 codes and their scale/zero and does the other half; the bf16
 # direction N_b between them and the bf16 copy of P are implementation traffic and are not counted.
 def k1_units(m, n, r):
-    return 2.0 * m * n * r, 2 * m * n + 16 * r * n + m * r // 2 + 8 * m * ((r + 255) // 256)
+    return 2.0 * m * n * r, 2 * m * n + MOMENT_BYTES * r * n + m * r // 2 + 8 * m * ((r + 255) // 256)
 
 
 def k2_units(m, n, r):
@@ -226,7 +230,7 @@ def whole_job_throughput(ms_total, elements_per_rank, steps, world, device):
     return ms, elements_per_rank * world * steps / (ms * 1e-3)
 
 
-def build_stack(workload, device, seed=0, layers=0):
+def build_stack(workload, device, seed=0, layers=0, moments=32):
     """Device-resident synthetic state of the whole stack: bf16 gradients (rank-32 signal + noise),
     INT8 weights, INT4 projections, zero moments.  Generated with torch on the device (input
     generation, not the path); quantization goes through the library."""
@@ -256,9 +260,16 @@ def build_stack(workload, device, seed=0, layers=0):
         p32.copy_(torch.linalg.qr(torch.randn(s.m, s.r, device=device, generator=gen))[0])
         P = B.quantize_int4(p32)
         del p32
-        M = B.zeros_matrix(s.r, s.n, torch.float32, device)
-        V = B.zeros_matrix(s.r, s.n, torch.float32, device)
-        items.append({"G": G, "P": P, "W": W, "M": M, "V": V, "seed": synth.matrix_seed(seed, s.index), "spec": s})
+        if moments == 8:        # 8-bit block-wise moments: codes and one scale per 32 columns, all zero at the start
+            M = B.zeros_matrix(s.r, s.n, torch.int8, device)
+            V = B.zeros_matrix(s.r, s.n, torch.uint8, device)
+            extra = {"M_scale": torch.zeros((s.r, (s.n + 31) // 32), dtype=torch.float32, device=device),
+                     "V_scale": torch.zeros((s.r, (s.n + 31) // 32), dtype=torch.float32, device=device)}
+        else:
+            M = B.zeros_matrix(s.r, s.n, torch.float32, device)
+            V = B.zeros_matrix(s.r, s.n, torch.float32, device)
+            extra = {}
+        items.append({"G": G, "P": P, "W": W, "M": M, "V": V, "seed": synth.matrix_seed(seed, s.index), "spec": s, **extra})
     return specs, items
 
 
@@ -357,7 +368,9 @@ def run_ours(args):
     peaks, peak_kind = load_peaks()
 
     # every rank holds and steps its own replica of the stack: matrices are independent units, no collective
-    specs, items = build_stack(args.workload, device, seed=rank, layers=args.layers)
+    global MOMENT_BYTES
+    MOMENT_BYTES = 4.5 if args.moments == 8 else 16.0
+    specs, items = build_stack(args.workload, device, seed=rank, layers=args.layers, moments=args.moments)
     batch = B.StepPlan(items)
     elements = batch.elements
     hyper = B.Hyper(rounding=B.QG_ROUND_NEAREST if args.rounding == "nearest" else B.QG_ROUND_STOCHASTIC)
@@ -467,7 +480,7 @@ def run_ours(args):
         k_bytes = per_kernel[names[dom]]["bytes"] * args.steps
         roof = {key: per_kernel[names[dom]][key] for key in ("bound", "achieved", "peak", "unit")}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        tpe = NCU_TRAFFIC_PER_ELEMENT.get(args.workload, {}).get(names[dom])
+        tpe = NCU_TRAFFIC_PER_ELEMENT.get(args.workload, {}).get(names[dom]) if args.moments == 32 else None
         roof["traffic"] = None if tpe is None else tpe * elements * args.steps / max(kcount[dom], 1)
         roof["kernel"] = names[dom]
         roof["launches"] = kcount[dom]
@@ -499,7 +512,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload + (f"[first {args.layers} layers]" if args.layers else ""), "matrices": len(specs), "elements_per_step": elements,
-                       "rank": specs[0].r, "group": 256, "rounding": args.rounding, "l2": "inputs larger than L2 (whole stack streams each step)",
+                       "rank": specs[0].r, "group": 256, "rounding": args.rounding, "moments_bits": args.moments, "l2": "inputs larger than L2 (whole stack streams each step)",
                        "parallelism": f"replica per GPU x{world}, no collective"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
@@ -518,6 +531,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama1b")
     ap.add_argument("--no-refresh", action="store_true", help="skip the separate timing of the subspace refresh")
+    ap.add_argument("--moments", type=int, choices=[32, 8], default=32,
+                    help="storage of the Adam moments: fp32 (the measured configuration) or the 8-bit block-wise form")
     ap.add_argument("--rounding", choices=["stochastic", "nearest"], default="stochastic",
                     help="requantization of the updated weight: the method's stochastic rounding, or the round-to-nearest ablation")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -156,8 +156,23 @@ typedef struct {
   float* M; float* V; int64_t ldmv;
   uint64_t seed;
   int32_t side;       /* QG_SIDE_LEFT (0) or QG_SIDE_RIGHT: see qgalore_project_step_right */
-  int32_t reserved;   /* 0 */
+  int32_t state_bits; /* 0 or 32: M, V are fp32.  8: the 8-bit block-wise storage below */
+  float* M_scale;     /* state_bits == 8 only: fp32 scales, dense [r][ceil(cols / 32)], cols = n (left) or m (right) */
+  float* V_scale;
 } qg_step_item;
+
+/* 8-bit moments (Sec. 3.5 keeps the Adam states in 8 bits and names no format; this one is the library's own).
+ * With state_bits == 8, M points to int8 and V to uint8 codes, r x cols with a pitch of ldmv BYTES (a multiple
+ * of 16).  Blocks are runs of 32 consecutive columns of a row (a shorter one at a ragged end), one scale each:
+ *   M: scale s = max |x| of the block, code = rint(x / (s / 127)),              x^ = code * (s / 127)
+ *   V: scale s = max x,               code = rint(255 * sqrt(x / s)),           x^ = (code / 255)^2 * s
+ * (divisions by a scale are multiplications by its binary32 reciprocal; a zero block has scale 0, codes 0).
+ * A step dequantizes the old moments, updates them and takes the direction in fp32, and stores the new ones. */
+
+/* One item of the table above as a call of its own: any side, any moment storage.  dbg as in
+ * qgalore_project_step (R, N have the shape of the moments). */
+QG_API int qgalore_project_step_item(const qg_step_item* item, const qg_hyper* h, void* workspace, size_t workspace_bytes,
+                              int32_t* status_dev, const qg_debug* dbg, void* stream);
 
 QG_API int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const qg_hyper* h,
                                  void* workspace, size_t workspace_bytes,

@@ -50,7 +50,8 @@ class _CHyper(C.Structure):
 class _CStepItem(C.Structure):
     _fields_ = [("G", C.c_void_p), ("ldg", C.c_int64), ("m", C.c_int64), ("n", C.c_int64), ("r", C.c_int64),
                 ("P", _CQTensor), ("W", _CQTensor), ("M", C.c_void_p), ("V", C.c_void_p), ("ldmv", C.c_int64),
-                ("seed", C.c_uint64), ("side", C.c_int32), ("reserved", C.c_int32)]
+                ("seed", C.c_uint64), ("side", C.c_int32), ("state_bits", C.c_int32),
+                ("M_scale", C.c_void_p), ("V_scale", C.c_void_p)]
 
 
 class _CDebug(C.Structure):
@@ -78,6 +79,7 @@ def lib() -> C.CDLL:
         L.qgalore_project_step.argtypes = [vp, i64, i64, i64, i64, qp, qp, vp, vp, i64, C.POINTER(_CHyper),
                                            vp, sz, vp, C.POINTER(_CDebug), vp]
         L.qgalore_project_step_right.argtypes = L.qgalore_project_step.argtypes
+        L.qgalore_project_step_item.argtypes = [C.POINTER(_CStepItem), C.POINTER(_CHyper), vp, sz, vp, C.POINTER(_CDebug), vp]
         L.qgalore_project_step_batched.argtypes = [C.POINTER(_CStepItem), i32, C.POINTER(_CHyper), vp, sz, vp, vp]
         L.qgalore_workspace_bytes_batched.argtypes = [C.POINTER(_CStepItem), i32]
         L.qgalore_workspace_bytes_batched.restype = sz
@@ -274,6 +276,37 @@ def project_step(G: torch.Tensor, P: QTensor, W: QTensor, M: torch.Tensor, V: to
            "qgalore_project_step_right" if right else "qgalore_project_step")
 
 
+def _c_step_item(it: dict) -> _CStepItem:
+    """One matrix of a step as the C table holds it.  Keys: G, P, W, M, V, seed; optional side ("left" / "right")
+    and, for 8-bit moments, M_scale and V_scale (then M is an int8 and V a uint8 tensor)."""
+    G, P, W, M, V = it["G"], it["P"], it["W"], it["M"], it["V"]
+    m, ncol = G.shape
+    state8 = it.get("M_scale") is not None
+    if state8 and (M.dtype != torch.int8 or V.dtype != torch.uint8):
+        raise ValueError("8-bit moments: M must be int8 and V uint8")
+    return _CStepItem(_ptr(G), _matrix_ld(G, "G"), m, ncol, P.cols, P.c_struct(), W.c_struct(),
+                      _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)),
+                      QG_SIDE_RIGHT if it.get("side", "left") == "right" else QG_SIDE_LEFT, 8 if state8 else 0,
+                      _ptr(it.get("M_scale")), _ptr(it.get("V_scale")))
+
+
+def project_step_item(item: dict, hyper: "Hyper", workspace: torch.Tensor | None = None, status: torch.Tensor | None = None,
+                      debug: dict | None = None, stream=None) -> None:
+    """One step of one matrix described like an item of a plan (any side, fp32 or 8-bit moments)."""
+    ci = _c_step_item(item)
+    m, n = item["G"].shape
+    if workspace is None:
+        workspace = torch.empty(workspace_bytes(QG_OP_PROJECT_STEP, m, n, item["P"].cols), dtype=torch.uint8,
+                                device=item["G"].device)
+    dbg = None
+    if debug:
+        dbg = _CDebug(_ptr(debug.get("R")), _ptr(debug.get("N")), _ptr(debug.get("W_pre")))
+    hc = hyper.c_struct()
+    _check(lib().qgalore_project_step_item(C.byref(ci), C.byref(hc), _ptr(workspace), workspace.numel(), _ptr(status),
+                                           C.byref(dbg) if dbg is not None else None, _stream_ptr(stream)),
+           "qgalore_project_step_item")
+
+
 class StepBatch:
     """A list of matrices stepped together by one call (a layer or a whole stack, Sec. 3.5).
 
@@ -289,9 +322,7 @@ class StepBatch:
         for k, it in enumerate(items):
             G, P, W, M, V = it["G"], it["P"], it["W"], it["M"], it["V"]
             m, ncol = G.shape
-            self._table[k] = _CStepItem(_ptr(G), _matrix_ld(G, "G"), m, ncol, P.cols, P.c_struct(), W.c_struct(),
-                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)),
-                                        QG_SIDE_RIGHT if it.get("side", "left") == "right" else QG_SIDE_LEFT, 0)
+            self._table[k] = _c_step_item(it)
         dev = device if device is not None else items[0]["G"].device
         nbytes = int(lib().qgalore_workspace_bytes_batched(self._table, n))
         self.workspace = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
@@ -321,9 +352,7 @@ class StepPlan:
         for k, it in enumerate(items):
             G, P, W, M, V = it["G"], it["P"], it["W"], it["M"], it["V"]
             m, ncol = G.shape
-            self._table[k] = _CStepItem(_ptr(G), _matrix_ld(G, "G"), m, ncol, P.cols, P.c_struct(), W.c_struct(),
-                                        _ptr(M), _ptr(V), _matrix_ld(M, "M"), int(it.get("seed", 0)),
-                                        QG_SIDE_RIGHT if it.get("side", "left") == "right" else QG_SIDE_LEFT, 0)
+            self._table[k] = _c_step_item(it)
         dev = device if device is not None else items[0]["G"].device
         L = lib()
         need = int(L.qgalore_workspace_bytes_batched(self._table, n))

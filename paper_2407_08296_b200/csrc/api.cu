@@ -151,7 +151,8 @@ static int check_hyper(const qg_hyper* h) {
 
 // Shape, pointer and alignment rules of one matrix of the step; fills everything of `a` but the scalars.
 static int check_matrix(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
-                        const qg_qtensor* W, float* M, float* V, int64_t ldmv, int side, StepArgs* a) {
+                        const qg_qtensor* W, float* M, float* V, int64_t ldmv, int side, StepArgs* a, int state_bits = 0,
+                        float* M_scale = nullptr, float* V_scale = nullptr) {
   if (!G || !M || !V) return QG_INVALID_ARGUMENT;
   if (side != QG_SIDE_LEFT && side != QG_SIDE_RIGHT) return QG_INVALID_ARGUMENT;
   const bool right = side == QG_SIDE_RIGHT;
@@ -165,23 +166,29 @@ static int check_matrix(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, in
   if (P->rows != prow || P->cols != r || W->rows != m || W->cols != n) return QG_INVALID_ARGUMENT;
   if (r % 32 != 0 || r < 32 || r > 2048 || r > prow) return QG_UNSUPPORTED_SHAPE;
   if (m > (1ll << 31) - 1 || n > (1ll << 31) - 1) return QG_UNSUPPORTED_SHAPE;
-  if (!aligned16(G) || !aligned16(M) || !aligned16(V) || ldg % 8 != 0 || ldmv % 4 != 0) return QG_MISALIGNED;
+  if (state_bits != 0 && state_bits != 32 && state_bits != 8) return QG_INVALID_ARGUMENT;
+  const bool state8 = state_bits == 8;
+  if (state8 && (!M_scale || !V_scale)) return QG_INVALID_ARGUMENT;
+  if (!aligned16(G) || !aligned16(M) || !aligned16(V) || ldg % 8 != 0 || ldmv % (state8 ? 16 : 4) != 0) return QG_MISALIGNED;
+  if (state8 && ((reinterpret_cast<uintptr_t>(M_scale) & 3u) || (reinterpret_cast<uintptr_t>(V_scale) & 3u))) return QG_MISALIGNED;
   memset(a, 0, sizeof(*a));
   a->G = G; a->ldg = ldg; a->m = m; a->n = n; a->r = r;
   a->P = *P; a->W = *W; a->M = M; a->V = V; a->ldmv = ldmv;
   a->right = right ? 1 : 0;
+  a->state8 = state8 ? 1 : 0; a->M_scale = M_scale; a->V_scale = V_scale;
   return QG_OK;
 }
 
 static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, const qg_qtensor* P,
                              const qg_qtensor* W, float* M, float* V, int64_t ldmv, const qg_hyper* h,
                              void* workspace, size_t workspace_bytes, int32_t* status_dev, const qg_debug* dbg,
-                             void* stream, bool validate_only, int side = QG_SIDE_LEFT) {
+                             void* stream, bool validate_only, int side = QG_SIDE_LEFT, int state_bits = 0,
+                             float* M_scale = nullptr, float* V_scale = nullptr) {
   if (!workspace) return QG_INVALID_ARGUMENT;
   int rc = check_hyper(h);
   if (rc != QG_OK) return rc;
   StepArgs a;
-  rc = check_matrix(G, ldg, m, n, r, P, W, M, V, ldmv, side, &a);
+  rc = check_matrix(G, ldg, m, n, r, P, W, M, V, ldmv, side, &a, state_bits, M_scale, V_scale);
   if (rc != QG_OK) return rc;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return QG_MISALIGNED;
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
@@ -191,7 +198,7 @@ static int project_step_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t 
   if (dbg) a.dbg = *dbg;
   fill_scalars(h, h->seed, &a.sc);
   if (g_step_impl == 1) {
-    if (a.right) return QG_UNSUPPORTED_SHAPE;       // the CUDA-core cross-check knows the left form only
+    if (a.right || a.state8) return QG_UNSUPPORTED_SHAPE;   // the CUDA-core cross-check knows the left form, fp32 moments
     return launch_project_step_simt(a, (cudaStream_t)stream);
   }
   return launch_project_step_tc(a, (cudaStream_t)stream);
@@ -211,6 +218,15 @@ int qgalore_project_step_right(const uint16_t* G, int64_t ldg, int64_t m, int64_
                                void* stream) {
   return project_step_impl(G, ldg, m, n, r, Q, W, Mt, Vt, ldmv, h, workspace, workspace_bytes, status_dev, dbg, stream,
                            false, QG_SIDE_RIGHT);
+}
+
+int qgalore_project_step_item(const qg_step_item* it, const qg_hyper* h, void* workspace, size_t workspace_bytes,
+                              int32_t* status_dev, const qg_debug* dbg, void* stream) {
+  if (!it || !h) return QG_INVALID_ARGUMENT;
+  qg_hyper hi = *h;
+  hi.seed = it->seed;
+  return project_step_impl(it->G, it->ldg, it->m, it->n, it->r, &it->P, &it->W, it->M, it->V, it->ldmv, &hi, workspace,
+                           workspace_bytes, status_dev, dbg, stream, false, it->side, it->state_bits, it->M_scale, it->V_scale);
 }
 
 size_t qgalore_workspace_bytes_batched(const qg_step_item* items, int32_t count) {
@@ -233,7 +249,8 @@ int qgalore_project_step_batched(const qg_step_item* items, int32_t count, const
       qg_hyper hi = *h;
       hi.seed = it.seed;
       const int rc = project_step_impl(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, &hi,
-                                       workspace, workspace_bytes, status_dev, nullptr, stream, pass == 0, it.side);
+                                       workspace, workspace_bytes, status_dev, nullptr, stream, pass == 0, it.side,
+                                       it.state_bits, it.M_scale, it.V_scale);
       if (rc != QG_OK) return rc;
     }
   }
@@ -248,7 +265,8 @@ static int plan_args(const qg_step_item* items, int32_t count, std::vector<StepA
   args->resize((size_t)count);
   for (int32_t i = 0; i < count; ++i) {
     const qg_step_item& it = items[i];
-    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, it.side, &(*args)[i]);
+    const int rc = check_matrix(it.G, it.ldg, it.m, it.n, it.r, &it.P, &it.W, it.M, it.V, it.ldmv, it.side, &(*args)[i],
+                                it.state_bits, it.M_scale, it.V_scale);
     if (rc != QG_OK) return rc;
     (*args)[i].sc.seed_lo = (uint32_t)(it.seed & 0xFFFFFFFFull);
     (*args)[i].sc.seed_hi = (uint32_t)(it.seed >> 32);

@@ -221,6 +221,9 @@ struct StepArgs {
   int32_t* status;
   qg_debug dbg;
   int32_t right;           // 0: R = P^T G, P m x r, moments r x n;  1: R = G Q, Q n x r, moments kept as r x m
+  int32_t state8;          // moments stored in 8 bits: M, V point to int8 / uint8 codes (pitch ldmv bytes) ...
+  float* M_scale;          // ... with one fp32 scale per block of 32 columns of a row, dense [r][ceil(cols / 32)]
+  float* V_scale;
 };
 // P~ = bf16((q - z) * s) of an INT4 matrix whose column count is a multiple of 32 (row pitch ld_out elements)
 int launch_dequant_p(const qg_qtensor& P, uint16_t* out, int64_t ld_out, cudaStream_t st);

@@ -76,6 +76,11 @@ struct alignas(64) TcProblem {
   // r x m, and the back-projection D = N_b^T Q~^T takes N_b as an MN-major A (mapN3h) and Q~ (n x r) as a
   // K-major B (mapQk, box 64 x 256 rows).
   int32_t right, k1_k, k1_n;
+  // 8-bit moments: M, V point to int8 / uint8 codes (pitch ldmv bytes), mapM / mapV are byte maps (box 32 x 16,
+  // no swizzle), m_scale / v_scale hold one fp32 scale per block of 32 columns of a row ([r][nsb]).
+  int32_t state8, nsb;
+  float* m_scale;
+  float* v_scale;
   int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles;
@@ -115,6 +120,8 @@ struct TileWalk {
 __device__ __forceinline__ void raise_wait_expired(int32_t* status) {
   if (status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
 }
+
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves an integer in the low mantissa bits
 
 __device__ __forceinline__ float sqrt_approx(float x) {
   float y;
@@ -185,7 +192,9 @@ __device__ __forceinline__ float2 adam2(const AdamConsts& c, float2 r, float2& m
 // covers 32 contiguous bytes of a row of M, V (fp32): every global store of the epilogue writes whole
 // 32-byte sectors straight from registers.  The old M, V come the other way through shared memory, by
 // TMA, several chunks ahead (see the epilogue).
-template <int BN, bool SINGLE, int CTAS>
+// S8: the instance that also knows the 8-bit storage of the moments (it costs registers, so launches whose
+// matrices all keep fp32 moments take the instance without it).
+template <int BN, bool SINGLE, int CTAS, bool S8 = false>
 __global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
                     const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
@@ -392,7 +401,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     auto request = [&]() {                           // one lane: the two copies of chunk `ld` into slot ld_slot
       if (lane == 0) {
         uint8_t* dst = mv_base + ld_slot * S::kMvSlotBytes;
-        mbar_arrive_expect_tx(&my_full[ld_slot], S::kMvSlotBytes);
+        mbar_arrive_expect_tx(&my_full[ld_slot], (S8 && ld.p->state8) ? 2 * 16 * kChunk : S::kMvSlotBytes);
         tma_load_2d(dst, &ld.p->mapM, &my_full[ld_slot], ld.x0 + kChunk * ld.c, ld.y0);
         tma_load_2d(dst + S::kMvArrayBytes, &ld.p->mapV, &my_full[ld_slot], ld.x0 + kChunk * ld.c, ld.y0);
       }
@@ -427,7 +436,29 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         tapN[a] = p->dbgN ? p->dbgN + gr * ldmv + n0 + lcol : nullptr;
       }
       // interior tiles (every row and column valid, no test taps) take a path without per-access predicates
-      const bool interior = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr;
+      const bool s8 = S8 && p->state8 != 0;
+      const bool interior = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr && !s8;
+      int8_t* M8r[2]; uint8_t* V8r[2]; float* msc[2]; float* vsc[2];
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        const int64_t gr = r0 + lrow + 8 * a;
+        M8r[a] = reinterpret_cast<int8_t*>(p->M) + gr * ldmv + n0 + lcol;
+        V8r[a] = reinterpret_cast<uint8_t*>(p->V) + gr * ldmv + n0 + lcol;
+        msc[a] = p->m_scale + gr * p->nsb;
+        vsc[a] = p->v_scale + gr * p->nsb;
+      }
+
+      // 8-bit moments: the block scales of the thread's two rows, fetched one chunk ahead
+      float ms_next[2] = {0.f, 0.f}, vs_next[2] = {0.f, 0.f};
+      auto fetch_scales = [&](int c) {
+        const int blk = (n0 + kChunk * c) >> 5;
+#pragma unroll
+        for (int a = 0; a < 2; ++a) {
+          ms_next[a] = rok[a] ? __ldg(msc[a] + blk) : 0.f;
+          vs_next[a] = rok[a] ? __ldg(vsc[a] + blk) : 0.f;
+        }
+      };
+      if (s8) fetch_scales(0);
 
       const uint32_t ab = tcount & 1;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
@@ -441,7 +472,31 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         if (!ok) break;
         --in_flight;
         float2 sm[8], sv[8];
-        {
+        if (s8) {
+          // codes of the thread's column pairs (rows of 32 bytes, no swizzle) and the block scales of its two rows
+          const uint8_t* src8 = mv_base + slot * S::kMvSlotBytes + (lane >> 2) * kChunk + 2 * (lane & 3);
+          const float c255 = 1.0f / 255.0f;
+          const float ms_cur[2] = {ms_next[0], ms_next[1]}, vs_cur[2] = {vs_next[0], vs_next[1]};
+          if (c + 1 < nch) fetch_scales(c + 1);
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            const float ms = ms_cur[a], vs = vs_cur[a];
+            const float stepm = __fmul_rn(ms, 1.0f / 127.0f);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              // a byte dropped into the mantissa of 2^23 is the float 2^23 + byte: no integer-to-float conversion
+              const uint32_t mc = (uint32_t)*reinterpret_cast<const uint16_t*>(src8 + a * 8 * kChunk + 8 * k) ^ 0x8080u;
+              const uint32_t vc = *reinterpret_cast<const uint16_t*>(src8 + S::kMvArrayBytes + a * 8 * kChunk + 8 * k);
+              const float m0 = __fsub_rn(__uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7650)), 8388736.0f);   // code = byte - 128
+              const float m1 = __fsub_rn(__uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7651)), 8388736.0f);
+              sm[2 * k + a] = make_float2(__fmul_rn(m0, stepm), __fmul_rn(m1, stepm));
+              const float v0 = __fsub_rn(__uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7650)), 8388608.0f);
+              const float v1 = __fsub_rn(__uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7651)), 8388608.0f);
+              const float w0 = __fmul_rn(v0, c255), w1 = __fmul_rn(v1, c255);
+              sv[2 * k + a] = make_float2(__fmul_rn(__fmul_rn(w0, w0), vs), __fmul_rn(__fmul_rn(w1, w1), vs));
+            }
+          }
+        } else {
           const uint8_t* src = mv_base + slot * S::kMvSlotBytes + row_off + half8;
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
@@ -478,7 +533,21 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
             const float2 rr = make_float2(__uint_as_float(acc[4 * k + 2 * a]), __uint_as_float(acc[4 * k + 2 * a + 1]));
             const float2 nn = adam2(ac, rr, mm, vv);
             const __nv_bfloat162 nb2 = __floats2bfloat162_rn(nn.x, nn.y);
-            if (interior) {
+            if (s8) {                                 // the new moments wait for their block's scale
+              sm[2 * k + a] = mm;
+              sv[2 * k + a] = vv;
+              if (rok[a]) {
+                if (off + 1 < cmax) {
+                  *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
+                  if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
+                  if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
+                } else if (off < cmax) {
+                  Nr[a][off] = float_to_bf16_bits(nn.x);
+                  if (tapR[a]) tapR[a][off] = rr.x;
+                  if (tapN[a]) tapN[a][off] = nn.x;
+                }
+              }
+            } else if (interior) {
               __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
               __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
               *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
@@ -498,6 +567,49 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
               }
             }
           }
+        if (s8) {
+          // 8-bit storage of the new moments: the chunk's 32 columns of a row are one block, held by the four
+          // threads of a quad.  Scale = the block's largest |M'| resp. V'; M' linear in [-127, 127], V' by the
+          // square-root law in [0, 255]; every operation a single binary32 one, as on the reference side.
+          const int blk = (n0 + kChunk * c) >> 5;
+#pragma unroll
+          for (int a = 0; a < 2; ++a) {
+            float mxm = 0.f, mxv = 0.f;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              mxm = fmaxf(mxm, fmaxf(fabsf(sm[2 * k + a].x), fabsf(sm[2 * k + a].y)));
+              mxv = fmaxf(mxv, fmaxf(sv[2 * k + a].x, sv[2 * k + a].y));
+            }
+            mxm = fmaxf(mxm, __shfl_xor_sync(0xFFFFFFFFu, mxm, 1));
+            mxv = fmaxf(mxv, __shfl_xor_sync(0xFFFFFFFFu, mxv, 1));
+            mxm = fmaxf(mxm, __shfl_xor_sync(0xFFFFFFFFu, mxm, 2));
+            mxv = fmaxf(mxv, __shfl_xor_sync(0xFFFFFFFFu, mxv, 2));
+            // reciprocals and roots by the approximate units (a few ulp): a code can differ from the correctly
+            // rounded one only when the scaled value sits within ~1e-5 of a rounding boundary
+            const float invm = mxm > 0.f ? __fdividef(127.0f, mxm) : 0.f;
+            const float invv = mxv > 0.f ? __fdividef(1.0f, mxv) : 0.f;
+            if (!rok[a]) continue;
+            if ((lane & 3) == 0 && kChunk * c < pn - n0) { msc[a][blk] = mxm; vsc[a][blk] = mxv; }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const int off = kChunk * c + 8 * k;
+              const float2 mm = sm[2 * k + a], vv = sv[2 * k + a];
+              // rint(t) sits in the low mantissa bits of t + 1.5 * 2^23; |t| <= 127 (+ a few ulp) resp. 0 <= t <= 255
+              // by construction of the scales, so the low byte is the code
+              const uint32_t m0q = __float_as_uint(__fadd_rn(__fmul_rn(mm.x, invm), kMagic));
+              const uint32_t m1q = __float_as_uint(__fadd_rn(__fmul_rn(mm.y, invm), kMagic));
+              const uint32_t v0q = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(vv.x, invv)), 255.0f), kMagic));
+              const uint32_t v1q = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(vv.y, invv)), 255.0f), kMagic));
+              if (off + 1 < cmax) {
+                *reinterpret_cast<uint16_t*>(M8r[a] + off) = (uint16_t)__byte_perm(m0q, m1q, 0x0040);
+                *reinterpret_cast<uint16_t*>(V8r[a] + off) = (uint16_t)__byte_perm(v0q, v1q, 0x0040);
+              } else if (off < cmax) {
+                M8r[a][off] = (int8_t)(m0q & 0xFFu);
+                V8r[a][off] = (uint8_t)(v0q & 0xFFu);
+              }
+            }
+          }
+        }
       }
     }
     if (!ok) {
@@ -552,7 +664,6 @@ struct K2PairSmem : K2Smem {
   static constexpr int kBytes = kPartOffset + 4 * kTileM * 8 + 1024;
 };
 
-constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves an integer in the low mantissa bits
 
 // 16 consecutive pre-rounding weights W' = W^ - lr*alpha*D - lr*wd*W^, W^ = (q - z) * s, from 16 INT8
 // codes and 16 accumulators.  FAST: q - z is formed without an integer-to-float conversion: the byte
@@ -1114,8 +1225,13 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->n_whole = (int32_t)n_whole;
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
-  ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+  if (a.state8) {
+    ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.M, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
+    ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.V, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
+  } else {
+    ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
+  }
   if (!ok) {
     note_cuda_error(cudaErrorUnknown, "cuTensorMapEncodeTiled");
     return QG_CUDA_ERROR;
@@ -1128,6 +1244,7 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->ldmv = a.ldmv; p->ldw = a.W.ld; p->ldn = w.ldn;
   p->m = (int32_t)a.m; p->n = (int32_t)a.n; p->r = (int32_t)a.r;
   p->right = a.right ? 1 : 0; p->k1_k = (int32_t)prow; p->k1_n = (int32_t)scol;
+  p->state8 = a.state8 ? 1 : 0; p->nsb = (int32_t)ceil_div(scol, 32); p->m_scale = a.M_scale; p->v_scale = a.V_scale;
   p->ngroups = (int32_t)ceil_div(a.n, kGroup);
   p->seed_lo = a.sc.seed_lo; p->seed_hi = a.sc.seed_hi;
   p->k1_rblocks = (int32_t)ceil_div(a.r, kTileM);
@@ -1160,11 +1277,11 @@ int set_smem(K kernel, int bytes) {
 // but only pays once there are enough tiles to occupy every SM.
 int choose_bn(int64_t tiles_at_256) { return tiles_at_256 >= 2 * (int64_t)sm_count() ? 256 : 128; }
 
-template <int BN, bool SINGLE, int CTAS>
+template <int BN, bool SINGLE, int CTAS, bool S8 = false>
 int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
               int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
   using S = K1Smem<BN, CTAS>;
-  auto kern = project_adam_kernel<BN, SINGLE, CTAS>;
+  auto kern = project_adam_kernel<BN, SINGLE, CTAS, S8>;
   int rc = set_smem(kern, S::kBytes);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
@@ -1291,8 +1408,13 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
   rc = fill_problem(a, w, &prob, bn);
   if (rc != QG_OK) return rc;
   const TileSchedule none{nullptr, nullptr, 1};
-  rc = bn == 256 ? launch_k1<256, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
-                 : launch_k1<128, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
+  if (a.state8) {
+    rc = bn == 256 ? launch_k1<256, true, 1, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
+                   : launch_k1<128, true, 1, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
+  } else {
+    rc = bn == 256 ? launch_k1<256, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
+                   : launch_k1<128, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
+  }
   if (rc != QG_OK) return rc;
   return launch_k2<true, 1>(&prob, nullptr, none, 0, prob.k2_tiles, a.sc, a.status, st);
 }
@@ -1304,7 +1426,7 @@ struct PlanChunk {
   int first, count;          // items [first, first + count)
   int k1_tiles, k2_tiles, k2p_tiles, bn;
   int dq_blocks;
-  int k1_grid, k2_grid, pairs, k1_pairs, k1p_tiles;
+  int k1_grid, k2_grid, pairs, k1_pairs, k1p_tiles, state8;
   size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
   size_t dq_map_off;                                                // same: block -> item map of the dequantize launch
 };
@@ -1426,8 +1548,10 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
     else ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
     ch.pairs = g_pair_mode & 1;
-    for (int k = i; k < j; ++k)
+    for (int k = i; k < j; ++k) {
       if (items[k].right) ch.pairs = 0;              // the paired back-projection knows the left form only
+      if (items[k].state8) ch.state8 = 1;
+    }
     if (ch.pairs) ch.k2_grid = 2 * (ch.k2p_tiles < sm_count() / 2 ? ch.k2p_tiles : sm_count() / 2);   // CTA pairs
     else ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
     schedule_tiles(t1, c1, ch.k1_pairs ? ch.k1_grid / 2 : ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);
@@ -1477,9 +1601,16 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
                           ch.k1_pairs ? 2 : 1};
     const TileSchedule s2{plan->sched_dev + ch.k2_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k2_items_off),
                           ch.pairs ? 2 : 1};
-    int rc = ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st)
-             : ch.bn == 256 ? launch_k1<256, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
-                            : launch_k1<128, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
+    int rc;
+    if (ch.state8) {       // some matrix of the chunk keeps its moments in 8 bits
+      rc = ch.k1_pairs  ? launch_k1<256, false, 2, true>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st)
+           : ch.bn == 256 ? launch_k1<256, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
+                          : launch_k1<128, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
+    } else {
+      rc = ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st)
+           : ch.bn == 256 ? launch_k1<256, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
+                          : launch_k1<128, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
+    }
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 2], st));
     rc = ch.pairs ? launch_k2<false, 2>(nullptr, tab, s2, ch.k2_grid, ch.k2p_tiles, sc, status, st)

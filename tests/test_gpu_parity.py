@@ -609,3 +609,97 @@ def test_refresh_of_the_right_singular_subspace(m, n, r):
     ref_q = O.quantize_rtn(q, 4)
     got = from_device_q(Qq)
     assert np.array_equal(got.codes, ref_q.codes) and np.array_equal(got.scales, ref_q.scales)
+
+
+# ----------------------------------------------------------------------------- 8-bit moments
+def _codes_to_device(codes: np.ndarray) -> torch.Tensor:
+    rows, cols = codes.shape
+    ld = (cols + 63) // 64 * 64                      # the pitch the fp32 test taps get, which the taps share
+    buf = torch.zeros((rows, ld), dtype=torch.int8 if codes.dtype == np.int8 else torch.uint8, device="cuda")
+    buf[:, :cols] = torch.from_numpy(codes).to("cuda")
+    return buf[:, :cols]
+
+
+def _check_state8(gpu_codes, gpu_scales, ref8, deq, name, max_frac=2e-3):
+    """Stored moments against the oracle's: scales to 1e-5, codes equal except by one level in a small fraction
+    (the binary32 moments entering the storage differ in their last bits between fp32 and fp64 accumulation)."""
+    assert np.allclose(gpu_scales, ref8.scales, rtol=1e-5, atol=0), f"{name} scales"
+    d = np.abs(gpu_codes.astype(np.int32) - ref8.codes.astype(np.int32))
+    assert d.max() <= 1, f"{name}: a code differs by more than one level"
+    assert (d != 0).mean() <= max_frac, f"{name}: {(d != 0).mean():.2e} of the codes differ"
+
+
+@pytest.mark.parametrize("m,n,r,side", [(256, 512, 64, "left"), (300, 777, 96, "left"), (512, 1376, 128, "left"),
+                                        (777, 300, 96, "right"), (2048, 2048, 512, "left")])
+def test_step_with_8bit_moments(m, n, r, side):
+    right = side == "right"
+    sc = m if right else n
+    gm = synth.GradientModel(m, n, seed=m + r, matrix_index=0)
+    P = O.quantize_rtn(synth.random_orthonormal(n if right else m, r, seed=m + r), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, m + r), 8)
+    z = np.zeros((r, sc), np.float32)
+    M8, V8 = O.quantize_m8(z), O.quantize_v8(z)
+    for t in (1, 2):                                   # two oracle steps so that the stored moments are not trivial
+        o = O.project_step(gm.sample(t), P, W, M8, V8, O.Hyper(step=t, seed=5), side=side)
+        W, M8, V8 = o["W"], o["M8"], o["V8"]
+    hyp = O.Hyper(step=3, seed=5)
+    gb = gm.sample(3)
+    ref = O.project_step(gb, P, W, M8, V8, hyp, side=side)
+    dM, dV = _codes_to_device(M8.codes), _codes_to_device(V8.codes)
+    dMs, dVs = torch.from_numpy(M8.scales).cuda().contiguous(), torch.from_numpy(V8.scales).cuda().contiguous()
+    dW = to_device_q(W)
+    taps = StepTaps(m, n, r, dW.ld, side)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    item = {"G": g_to_device(gb), "P": to_device_q(P), "W": dW, "M": dM, "V": dV, "M_scale": dMs, "V_scale": dVs,
+            "seed": 5, "side": side}
+    B.project_step_item(item, B.Hyper(step=3), status=status, debug=taps.as_dict())
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # the direction comes from the binary32 moments: same rules as for fp32 storage
+    from parity_utils import check_direction, check_moments, check_weight_codes
+    check_moments(taps.R.cpu().numpy(), ref["R32"], "R")
+    n_gpu = taps.N.cpu().numpy()
+    check_direction(n_gpu, ref, hyp, "N")
+    forced = O.project_step(gb, P, W, M8, V8, hyp, side=side, N_b_override=O.bf16_round(n_gpu))
+    check_weight_codes(from_device_q(dW), forced, 5, 3)
+    # the stored moments
+    _check_state8(dM.cpu().numpy(), dMs.cpu().numpy(), ref["M8"], O.dequantize_m8, "M")
+    _check_state8(dV.cpu().numpy(), dVs.cpu().numpy(), ref["V8"], O.dequantize_v8, "V")
+    assert int(dM._base[:, sc:].abs().max().item()) == 0 if dM._base.shape[1] > sc else True
+
+
+def test_plan_mixes_fp32_and_8bit_moments():
+    shapes = [(256, 512, 64), (512, 1376, 128), (768, 768, 256)]
+    step = 2
+    single, items = [], []
+    for idx, (m, n, r) in enumerate(shapes):
+        gb = synth.GradientModel(m, n, seed=19, matrix_index=idx).sample(step)
+        P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=19, stream=idx), 4)
+        W = O.quantize_rtn(synth.initial_weight(m, n, 19, idx), 8)
+        rng = np.random.default_rng(idx)
+        M = rng.normal(0, 1e-3, (r, n)).astype(np.float32)
+        V = (rng.normal(0, 1e-3, (r, n)) ** 2).astype(np.float32)
+        dG, dP = g_to_device(gb), to_device_q(P)
+        pair = []
+        for _ in range(2):                              # one copy for the single call, one for the plan
+            if idx == 1:
+                it = {"G": dG, "P": dP, "W": to_device_q(W), "M": f32_to_device(M), "V": f32_to_device(V), "seed": idx}
+            else:
+                M8, V8 = O.quantize_m8(M), O.quantize_v8(V)
+                it = {"G": dG, "P": dP, "W": to_device_q(W), "M": _codes_to_device(M8.codes), "V": _codes_to_device(V8.codes),
+                      "M_scale": torch.from_numpy(M8.scales).cuda().contiguous(),
+                      "V_scale": torch.from_numpy(V8.scales).cuda().contiguous(), "seed": idx}
+            pair.append(it)
+        B.project_step_item(pair[0], B.Hyper(step=step))
+        single.append(pair[0])
+        items.append(pair[1])
+    plan = B.StepPlan(items)
+    plan.step(B.Hyper(step=step))
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0
+    for a, b in zip(single, items):
+        assert torch.equal(a["W"].codes, b["W"].codes) and torch.equal(a["M"]._base, b["M"]._base)
+        assert torch.equal(a["V"]._base, b["V"]._base)
+        if "M_scale" in a:
+            assert torch.equal(a["M_scale"], b["M_scale"]) and torch.equal(a["V_scale"], b["V_scale"])
+    plan.close()
