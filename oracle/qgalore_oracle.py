@@ -13,8 +13,12 @@ E[W_q] = W for stochastic rounding, reduction to dense Adam at full rank, a
 hand-written Jacobi eigen-solver on 8x8 inputs, closed forms of the similarity
 statistic and scripted gate sequences.
 
-Parity unpinned: nothing (8-bit moment storage and right-hand projection are
-not implemented here).
+Parity unpinned: the 8-bit storage of the Adam moments (``Moments8``,
+``quantize_m8``, ``quantize_v8`` and their inverses): the paper names 8-bit Adam
+without a format, so the format is a choice and only its own promises are pinned.
+The right-hand projection is pinned against the left-hand form on the
+transposed gradient; the 2-bit quantizer and the round-to-nearest step by the
+same bounds as the 4- and 8-bit quantizers.
 
 Conventions
 -----------
@@ -282,8 +286,10 @@ def unpack_int2(packed, cols):
 
 # --------------------------------------------------------------------------- 8-bit moments (Sec. 3.5 "8-bit Adam")
 # The paper keeps the Adam states of the low-rank subspace in 8 bits and cites block-wise 8-bit optimizers
-# for it without giving a format.  The format here is this build's own: blocks of STATE_BLOCK consecutive
-# elements along a row (restarting at every row, a shorter block at a ragged end), one binary32 scale per block.
+# for it without giving a format.  PARITY UNPINNED: there is no definition in the paper to check this against;
+# the format below is a choice (pinned only by what it promises: error bounds, exact block maximum, idempotence).
+# Blocks of STATE_BLOCK consecutive elements along a row (restarting at every row, a shorter block at a ragged
+# end), one binary32 scale per block.
 #   first moment  (signed):   s = max |x|;  code = rint(x * (1 / (s / 127))) in [-127, 127];  x^ = code * (s / 127)
 #   second moment (>= 0):     s = max x;    code = rint(255 * sqrt(x * (1 / s))) in [0, 255];  x^ = (code / 255)^2 * s
 # (the square-root law gives small second moments the relative precision a linear code would not).  Every
