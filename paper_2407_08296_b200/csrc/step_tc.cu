@@ -437,7 +437,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       }
       // interior tiles (every row and column valid, no test taps) take a path without per-access predicates
       const bool s8 = S8 && p->state8 != 0;
-      const bool interior = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr && !s8;
+      const bool whole = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr;
+      const bool interior = whole && !s8;
       int8_t* M8r[2]; uint8_t* V8r[2]; float* msc[2]; float* vsc[2];
 #pragma unroll
       for (int a = 0; a < 2; ++a) {
@@ -475,25 +476,27 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         if (s8) {
           // codes of the thread's column pairs (rows of 32 bytes, no swizzle) and the block scales of its two rows
           const uint8_t* src8 = mv_base + slot * S::kMvSlotBytes + (lane >> 2) * kChunk + 2 * (lane & 3);
-          const float c255 = 1.0f / 255.0f;
           const float ms_cur[2] = {ms_next[0], ms_next[1]}, vs_cur[2] = {vs_next[0], vs_next[1]};
           if (c + 1 < nch) fetch_scales(c + 1);
 #pragma unroll
           for (int a = 0; a < 2; ++a) {
             const float ms = ms_cur[a], vs = vs_cur[a];
             const float stepm = __fmul_rn(ms, 1.0f / 127.0f);
+            const float2 stepm2 = make_float2(stepm, stepm), vs2 = make_float2(vs, vs);
+            const float2 c255 = make_float2(1.0f / 255.0f, 1.0f / 255.0f);
+            const float2 bias_m = make_float2(-8388736.0f, -8388736.0f), bias_v = make_float2(-8388608.0f, -8388608.0f);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               // a byte dropped into the mantissa of 2^23 is the float 2^23 + byte: no integer-to-float conversion
               const uint32_t mc = (uint32_t)*reinterpret_cast<const uint16_t*>(src8 + a * 8 * kChunk + 8 * k) ^ 0x8080u;
               const uint32_t vc = *reinterpret_cast<const uint16_t*>(src8 + S::kMvArrayBytes + a * 8 * kChunk + 8 * k);
-              const float m0 = __fsub_rn(__uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7650)), 8388736.0f);   // code = byte - 128
-              const float m1 = __fsub_rn(__uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7651)), 8388736.0f);
-              sm[2 * k + a] = make_float2(__fmul_rn(m0, stepm), __fmul_rn(m1, stepm));
-              const float v0 = __fsub_rn(__uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7650)), 8388608.0f);
-              const float v1 = __fsub_rn(__uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7651)), 8388608.0f);
-              const float w0 = __fmul_rn(v0, c255), w1 = __fmul_rn(v1, c255);
-              sv[2 * k + a] = make_float2(__fmul_rn(__fmul_rn(w0, w0), vs), __fmul_rn(__fmul_rn(w1, w1), vs));
+              const float2 mq = make_float2(__uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7650)),
+                                            __uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7651)));
+              sm[2 * k + a] = mul2(add2(mq, bias_m), stepm2);                         // code = byte - 128
+              const float2 vq = make_float2(__uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7650)),
+                                            __uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7651)));
+              const float2 w = mul2(add2(vq, bias_v), c255);
+              sv[2 * k + a] = mul2(mul2(w, w), vs2);
             }
           }
         } else {
@@ -536,7 +539,9 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
             if (s8) {                                 // the new moments wait for their block's scale
               sm[2 * k + a] = mm;
               sv[2 * k + a] = vv;
-              if (rok[a]) {
+              if (whole) {
+                *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
+              } else if (rok[a]) {
                 if (off + 1 < cmax) {
                   *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
                   if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
@@ -600,7 +605,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
               const uint32_t m1q = __float_as_uint(__fadd_rn(__fmul_rn(mm.y, invm), kMagic));
               const uint32_t v0q = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(vv.x, invv)), 255.0f), kMagic));
               const uint32_t v1q = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(vv.y, invv)), 255.0f), kMagic));
-              if (off + 1 < cmax) {
+              if (whole || off + 1 < cmax) {
                 *reinterpret_cast<uint16_t*>(M8r[a] + off) = (uint16_t)__byte_perm(m0q, m1q, 0x0040);
                 *reinterpret_cast<uint16_t*>(V8r[a] + off) = (uint16_t)__byte_perm(v0q, v1q, 0x0040);
               } else if (off < cmax) {
