@@ -108,7 +108,8 @@ def run_refresh_case(m, n, r, seed=0, iters=12):
     return angle, P_new
 
 
-@pytest.mark.parametrize("m,n,r", [(256, 320, 64), (320, 256, 64), (512, 1376, 128), (768, 768, 256), (2048, 2048, 512)])
+@pytest.mark.parametrize("m,n,r", [(256, 320, 64), (320, 256, 64), (512, 1376, 128), (768, 768, 256), (2048, 2048, 512),
+                                   (4096, 4096, 1024)])
 def test_refresh_subspace_matches_exact_svd(m, n, r):
     run_refresh_case(m, n, r, seed=m + r)
 
