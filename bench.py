@@ -87,9 +87,9 @@ def k2_alu_ops(m, n, r):
 # the captured launch, so that it scales to the launches timed here.  None = no valid capture for the
 # kernels as they stand.
 NCU_TRAFFIC_PER_ELEMENT = {
-    # profiles/project_adam_and_backproject_sr_llama1b_4layers.md: 1214.0, 527.0 and 48.9 MB over 201.3 M elements
-    "llama1b": {"project_adam": 1214.0e6 / 201.3184e6, "backproject_sr": 527.0e6 / 201.3184e6,
-                "dequant_p_grouped": 48.9e6 / 201.3184e6},
+    # profiles/project_adam_and_backproject_sr_llama1b_4layers.md: 1215.4, 526.7 and 51.3 MB over 201.3 M elements
+    "llama1b": {"project_adam": 1215.4e6 / 201.3184e6, "backproject_sr": 526.7e6 / 201.3184e6,
+                "dequant_p_grouped": 51.3e6 / 201.3184e6},
 }
 
 
