@@ -420,21 +420,40 @@ def run_ours(args):
     for hg, it in zip(host_g, items):
         hg.copy_(it["G"])
     host_status = torch.zeros(1, dtype=torch.int32).pin_memory()
+    # two sets of device gradient buffers and a plan over each (same weights, moments, projections): the copy of
+    # the next step's gradients runs on a second stream while this step computes, as a training loop whose
+    # gradients arrive from the host would arrange it.  Every step still pays its whole copy and its read-back.
+    alt_g = [B.empty_matrix(it["G"].shape[0], it["G"].shape[1], torch.bfloat16, device) for it in items]
+    plan_alt = B.StepPlan([{**it, "G": g} for it, g in zip(items, alt_g)])
+    plans, gsets = [batch, plan_alt], [[it["G"] for it in items], alt_g]
+    copy_stream = torch.cuda.Stream(device=device)
+    copied = [torch.cuda.Event(), torch.cuda.Event()]
+    done = [torch.cuda.Event(), torch.cuda.Event()]
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for _ in range(e2e_steps):
+    copy_stream.wait_event(e0)
+    for k in range(e2e_steps):
         step_no += 1
         hyper.step = step_no
-        for hg, it in zip(host_g, items):
-            it["G"].copy_(hg, non_blocking=True)
-        batch.step(hyper)
-        host_status.copy_(batch.status, non_blocking=True)
-        stream.synchronize()
+        b = k & 1
+        with torch.cuda.stream(copy_stream):
+            if k >= 2:
+                copy_stream.wait_event(done[b])            # the step that read this set has finished
+            for hg, g in zip(host_g, gsets[b]):
+                g.copy_(hg, non_blocking=True)
+            copied[b].record(copy_stream)
+        stream.wait_event(copied[b])
+        plans[b].step(hyper)
+        host_status.copy_(plans[b].status, non_blocking=True)
+        done[b].record(stream)
     e1.record(stream)
+    stream.synchronize()
     barrier()
     _, e2e_value = whole_job_throughput(e0.elapsed_time(e1), elements, e2e_steps, world, device)
-    del host_g
+    status |= int(plan_alt.status.item())
+    plan_alt.close()
+    del host_g, alt_g, plan_alt, plans, gsets
 
     # ---- per-kernel device time: a second pass of the same steps with an event pair around every launch
     kms = [0.0, 0.0, 0.0]
@@ -536,7 +555,7 @@ def main():
     ap.add_argument("--rounding", choices=["stochastic", "nearest"], default="stochastic",
                     help="requantization of the updated weight: the method's stochastic rounding, or the round-to-nearest ablation")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0,
                     help="keep only the first L layers of the stack (small cases for profiler captures); 0 = all")
