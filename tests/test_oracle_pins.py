@@ -593,7 +593,7 @@ def test_right_projection_is_the_left_projection_of_the_transposed_gradient():
     assert np.allclose(right["R32"], (G @ Qt).T.astype(np.float32), rtol=1e-6, atol=1e-12)
 
 
-# ----------------------------------------------------------------------------- 8-bit moments (format of this build)
+# ----------------------------------------------------------------------------- 8-bit moments (a format of the library)
 def test_8bit_moment_formats_bounds_idempotence_and_zero_blocks():
     # Sec. 3.5 keeps the Adam states in 8 bits without giving a format; the one built here is pinned by what it
     # promises: the first moment is off by at most half a step s/127, the square root of the second by at most
