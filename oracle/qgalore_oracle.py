@@ -11,7 +11,8 @@ Pinned by tests/test_oracle_*.py against facts that do not come from this file:
 published Philox known answers, the half-step error bound of the quantizer,
 E[W_q] = W for stochastic rounding, reduction to dense Adam at full rank, a
 hand-written Jacobi eigen-solver on 8x8 inputs, closed forms of the similarity
-statistic and scripted gate sequences.
+statistic and scripted gate sequences; the INT8 linear layer of App. A by index
+loops on a tiny case, a permutation weight, the adjoint identity and autograd.
 
 Parity unpinned: the 8-bit storage of the Adam moments (``Moments8``,
 ``quantize_m8``, ``quantize_v8`` and their inverses): the paper names 8-bit Adam
@@ -42,7 +43,7 @@ __all__ = [
     "philox4x32_10", "sr_uniform16", "group_params", "quantize_rtn", "quantize_sr",
     "dequantize", "pack_int4", "unpack_int4", "pack_int2", "unpack_int2", "QTensor", "Hyper", "project_step",
     "refresh_subspace", "subspace_similarity", "GateState", "gate_update",
-    "principal_angle", "STATE_BLOCK", "Moments8", "quantize_m8", "quantize_v8", "dequantize_m8", "dequantize_v8",
+    "principal_angle", "int8_linear_forward", "int8_linear_backward", "STATE_BLOCK", "Moments8", "quantize_m8", "quantize_v8", "dequantize_m8", "dequantize_v8",
 ]
 
 GROUP = 256  # Sec. 3.1: block size 256 in all implementations
@@ -553,3 +554,29 @@ def gate_update(state: GateState, sim, threshold=0.4, k=1):
         state.history = []
         return True
     return False
+
+
+# --------------------------------------------------------------------------- App. A: the INT8 linear layer
+def _weight_operand(W_q: QTensor):
+    """The weight as the products see it: dequantized in binary32 (App. A, the dequantization line), then
+    rounded once to the activations' type, bfloat16.  Returned in float64."""
+    return bf16_bits_to_f32(f32_to_bf16_bits(dequantize(W_q))).astype(np.float64)
+
+
+def int8_linear_forward(X_bits, W_q: QTensor):
+    """App. A, forward: Y = X W^T with W dequantized on the fly.  X is T x n (bfloat16 bit patterns), W is
+    m x n, Y is T x m.  No bias (the listing names one without defining it; the LLaMA layers have none).
+    Returns (Y exact in float64, Y rounded to bfloat16 bit patterns)."""
+    X = bf16_bits_to_f32(X_bits).astype(np.float64)
+    Y = X @ _weight_operand(W_q).T
+    return Y, f32_to_bf16_bits(fl32(Y))
+
+
+def int8_linear_backward(dY_bits, X_bits, W_q: QTensor):
+    """App. A, backward: grad_input = dY W (T x n) and grad_W = dY^T X (m x n), the latter being the gradient
+    G the optimizer step consumes.  Returns (dX exact, dX bf16 bits, G exact, G bf16 bits)."""
+    dY = bf16_bits_to_f32(dY_bits).astype(np.float64)
+    X = bf16_bits_to_f32(X_bits).astype(np.float64)
+    dX = dY @ _weight_operand(W_q)
+    G = dY.T @ X
+    return dX, f32_to_bf16_bits(fl32(dX)), G, f32_to_bf16_bits(fl32(G))

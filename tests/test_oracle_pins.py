@@ -652,3 +652,85 @@ def test_step_on_8bit_moments_is_the_step_on_their_values_and_tracks_the_fp32_ru
     # five steps on: the stored moments stay close to the binary32 ones (no drift from the rounding of the state)
     assert np.linalg.norm(O.dequantize_m8(M8) - Mf) <= 0.02 * np.linalg.norm(Mf)
     assert np.linalg.norm(np.sqrt(O.dequantize_v8(V8)) - np.sqrt(Vf)) <= 0.02 * np.linalg.norm(np.sqrt(Vf))
+
+
+# ----------------------------------------------------------------------------- App. A: the INT8 linear layer
+def _small_linear_case(T=5, m=3, n=260, seed=3):
+    rng = np.random.default_rng(seed)
+    W = rng.standard_normal((m, n)).astype(np.float32) * 0.05
+    W_q = O.quantize_rtn(W, 8)
+    X_bits = O.f32_to_bf16_bits(rng.standard_normal((T, n)).astype(np.float32))
+    dY_bits = O.f32_to_bf16_bits(rng.standard_normal((T, m)).astype(np.float32))
+    return W_q, X_bits, dY_bits
+
+
+def test_int8_linear_matches_index_loops_on_a_tiny_case():
+    """App. A written out index by index in Python floats: y[t][i] = sum_j x[t][j] w[i][j],
+    dx[t][j] = sum_i dy[t][i] w[i][j], g[i][j] = sum_t dy[t][i] x[t][j], with w the INT8 weight
+    dequantized per group of 256 and rounded to bfloat16."""
+    T, m, n = 5, 3, 260                     # two groups per row, the second one 4 wide
+    W_q, X_bits, dY_bits = _small_linear_case(T, m, n)
+    x = O.bf16_bits_to_f32(X_bits).tolist()
+    dy = O.bf16_bits_to_f32(dY_bits).tolist()
+    w = [[0.0] * n for _ in range(m)]
+    for i in range(m):
+        for j in range(n):
+            g = j // 256
+            v = np.float32(np.float32(float(W_q.codes[i, j]) - float(W_q.zeros[i, g])) * W_q.scales[i, g])
+            w[i][j] = float(O.bf16_bits_to_f32(O.f32_to_bf16_bits(np.array([v], np.float32)))[0])
+    Y, Yb = O.int8_linear_forward(X_bits, W_q)
+    dX, dXb, G, Gb = O.int8_linear_backward(dY_bits, X_bits, W_q)
+    assert Y.shape == (T, m) and dX.shape == (T, n) and G.shape == (m, n)
+    for t in range(T):
+        for i in range(m):
+            assert Y[t, i] == pytest.approx(math.fsum(x[t][j] * w[i][j] for j in range(n)), rel=1e-12, abs=1e-14)
+        for j in range(0, n, 37):
+            assert dX[t, j] == pytest.approx(math.fsum(dy[t][i] * w[i][j] for i in range(m)), rel=1e-12, abs=1e-14)
+    for i in range(m):
+        for j in range(0, n, 37):
+            assert G[i, j] == pytest.approx(math.fsum(dy[t][i] * x[t][j] for t in range(T)), rel=1e-12, abs=1e-14)
+    # the bfloat16 outputs are the exact ones rounded once
+    np.testing.assert_array_equal(Yb, O.f32_to_bf16_bits(Y.astype(np.float32)))
+    np.testing.assert_array_equal(Gb, O.f32_to_bf16_bits(G.astype(np.float32)))
+
+
+def test_int8_linear_with_a_permutation_weight_moves_columns():
+    """A weight whose dequantized value is exactly a permutation matrix (Quant_8 of a 0/1 row represents 0
+    and 1 exactly): the forward pass permutes the columns of X one way, the input gradient permutes dY the
+    other way.  A transposed operand in either product fails this."""
+    n = 256
+    perm = np.roll(np.arange(n), 5)                  # not an involution
+    Wm = np.zeros((n, n), np.float32)
+    Wm[np.arange(n), perm] = 1.0                     # row i has its one in column perm[i]
+    W_q = O.quantize_rtn(Wm, 8)
+    np.testing.assert_array_equal(O.dequantize(W_q), Wm)
+    rng = np.random.default_rng(0)
+    X_bits = O.f32_to_bf16_bits(rng.standard_normal((4, n)).astype(np.float32))
+    dY_bits = O.f32_to_bf16_bits(rng.standard_normal((4, n)).astype(np.float32))
+    Y, Yb = O.int8_linear_forward(X_bits, W_q)
+    dX, dXb, G, _ = O.int8_linear_backward(dY_bits, X_bits, W_q)
+    np.testing.assert_array_equal(Yb, X_bits[:, perm])               # y[:, i] = x[:, perm[i]]
+    inv = np.argsort(perm)
+    np.testing.assert_array_equal(dXb, dY_bits[:, inv])              # dx[:, perm[i]] = dy[:, i]
+    assert not np.array_equal(Yb, X_bits[:, inv])
+
+
+def test_int8_linear_adjoint_identity_and_autograd():
+    """<dY, X W^T> = <dY W, X> = <dY^T X, W> (the three products are one trilinear form), and torch's
+    autograd on y = x @ w.t() returns the same two gradients."""
+    torch = pytest.importorskip("torch")
+    W_q, X_bits, dY_bits = _small_linear_case(T=7, m=6, n=300, seed=11)
+    Y, _ = O.int8_linear_forward(X_bits, W_q)
+    dX, _, G, _ = O.int8_linear_backward(dY_bits, X_bits, W_q)
+    X = O.bf16_bits_to_f32(X_bits).astype(np.float64)
+    dY = O.bf16_bits_to_f32(dY_bits).astype(np.float64)
+    Wt = O.bf16_bits_to_f32(O.f32_to_bf16_bits(O.dequantize(W_q))).astype(np.float64)
+    a, b, c = np.sum(dY * Y), np.sum(dX * X), np.sum(G * Wt)
+    assert a == pytest.approx(b, rel=1e-12) and a == pytest.approx(c, rel=1e-12)
+    xt = torch.tensor(X, requires_grad=True)
+    wt = torch.tensor(Wt, requires_grad=True)
+    y = xt @ wt.t()
+    y.backward(torch.tensor(dY))
+    np.testing.assert_allclose(y.detach().numpy(), Y, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(xt.grad.numpy(), dX, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(wt.grad.numpy(), G, rtol=1e-12, atol=1e-14)
