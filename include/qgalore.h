@@ -274,6 +274,28 @@ QG_API size_t qgalore_subspace_similarity_static_max_bytes(void);
 QG_API int qgalore_gate_update(float sim, float threshold, int32_t k, int32_t* interval,
                         float* history, int32_t* count);
 
+/* --- App. A: the INT8 linear layer (the products either side of the optimizer step) ------
+ * W~ = bfloat16((codes - zeros) * scales): the INT8 weight (m x n, groups of 256 along a row) dequantized in
+ * binary32 and rounded once to bfloat16 while its tiles enter the GEMM; it is never written to global memory.
+ * All matrices are bfloat16 bit patterns, row-major, DEVICE memory; base pointers 16-byte aligned, row
+ * pitches multiples of 8 elements; accumulation is binary32, the result is rounded once to bfloat16.
+ * The listing's bias term is left out (the LLaMA layers have none).  W is only read.
+ *   forward          Y  (T x m, pitch ldy)  = X  (T x n, pitch ldx)  * W~^T
+ *   backward_input   dX (T x n, pitch lddx) = dY (T x m, pitch lddy) * W~
+ *   backward_weight  G  (m x n, pitch ldg)  = dY^T * X     - the gradient qgalore_project_step consumes; no
+ *                    quantized operand.  dY and X are read in whole 64-column slabs: lddy >= m and ldx >= n
+ *                    rounded up to multiples of 64 (what lies in the padding does not matter), else
+ *                    QG_UNSUPPORTED_SHAPE.
+ * status (device int32, may be null) receives QG_DEV_WAIT_EXPIRED if a bounded wait ran out.  Extents up to
+ * 2^30.  No workspace. */
+QG_API int qgalore_int8_linear_forward(const uint16_t* X, int64_t T, int64_t ldx, const qg_qtensor* W,
+                                uint16_t* Y, int64_t ldy, int32_t* status, void* stream);
+QG_API int qgalore_int8_linear_backward_input(const uint16_t* dY, int64_t T, int64_t lddy, const qg_qtensor* W,
+                                       uint16_t* dX, int64_t lddx, int32_t* status, void* stream);
+QG_API int qgalore_int8_linear_backward_weight(const uint16_t* dY, int64_t T, int64_t lddy, const uint16_t* X,
+                                        int64_t ldx, int64_t m, int64_t n, uint16_t* G, int64_t ldg,
+                                        int32_t* status, void* stream);
+
 enum { QG_OP_PROJECT_STEP = 1, QG_OP_REFRESH = 2, QG_OP_SIMILARITY = 3 };
 
 /* Scratch bytes the given operation needs for an m x n matrix at rank r (host, pure).

@@ -76,6 +76,9 @@ def lib() -> C.CDLL:
         L.qgalore_quantize_int8.argtypes = [vp, i64, i64, i64, qp, vp]
         L.qgalore_quantize_int2.argtypes = [vp, i64, i64, i64, qp, vp]
         L.qgalore_dequantize.argtypes = [qp, vp, i64, vp]
+        L.qgalore_int8_linear_forward.argtypes = [vp, i64, i64, qp, vp, i64, vp, vp]
+        L.qgalore_int8_linear_backward_input.argtypes = [vp, i64, i64, qp, vp, i64, vp, vp]
+        L.qgalore_int8_linear_backward_weight.argtypes = [vp, i64, i64, vp, i64, i64, i64, vp, i64, vp, vp]
         L.qgalore_project_step.argtypes = [vp, i64, i64, i64, i64, qp, qp, vp, vp, i64, C.POINTER(_CHyper),
                                            vp, sz, vp, C.POINTER(_CDebug), vp]
         L.qgalore_project_step_right.argtypes = L.qgalore_project_step.argtypes
@@ -243,6 +246,59 @@ def dequantize(q: QTensor, out: torch.Tensor | None = None, stream=None) -> torc
     cs = q.c_struct()
     _check(lib().qgalore_dequantize(C.byref(cs), _ptr(out), _matrix_ld(out, "out"), _stream_ptr(stream)),
            "qgalore_dequantize")
+    return out
+
+
+def _bf16_arg(t: torch.Tensor, what: str) -> torch.Tensor:
+    if t.dtype not in (torch.bfloat16, torch.int16, torch.uint16):
+        raise ValueError(f"{what} must hold bfloat16 values (bfloat16 / int16 / uint16 storage)")
+    return t
+
+
+def int8_linear_forward(X: torch.Tensor, W: QTensor, out: torch.Tensor | None = None,
+                        status: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """App. A, forward: Y (T x m) = X (T x n) W~^T with the INT8 weight dequantized inside the GEMM."""
+    T = X.shape[0]
+    if out is None:
+        out = empty_matrix(T, W.rows, torch.bfloat16, X.device, 64)
+    cs = W.c_struct()
+    _check(lib().qgalore_int8_linear_forward(_ptr(_bf16_arg(X, "X")), T, _matrix_ld(X, "X"), C.byref(cs),
+                                             _ptr(_bf16_arg(out, "out")), _matrix_ld(out, "out"),
+                                             _ptr(status), _stream_ptr(stream)),
+           "qgalore_int8_linear_forward")
+    return out
+
+
+def int8_linear_backward_input(dY: torch.Tensor, W: QTensor, out: torch.Tensor | None = None,
+                               status: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """App. A, backward: grad_input (T x n) = dY (T x m) W~."""
+    T = dY.shape[0]
+    if out is None:
+        out = empty_matrix(T, W.cols, torch.bfloat16, dY.device, 64)
+    cs = W.c_struct()
+    _check(lib().qgalore_int8_linear_backward_input(_ptr(_bf16_arg(dY, "dY")), T, _matrix_ld(dY, "dY"), C.byref(cs),
+                                                    _ptr(_bf16_arg(out, "out")), _matrix_ld(out, "out"),
+                                                    _ptr(status),
+                                                    _stream_ptr(stream)),
+           "qgalore_int8_linear_backward_input")
+    return out
+
+
+def int8_linear_backward_weight(dY: torch.Tensor, X: torch.Tensor, out: torch.Tensor | None = None,
+                                status: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """App. A, backward: grad_W (m x n) = dY^T (T x m) X (T x n): the gradient G of the optimizer step."""
+    T, m = dY.shape
+    n = X.shape[1]
+    if X.shape[0] != T:
+        raise ValueError("dY and X must have the same number of rows")
+    if out is None:
+        out = empty_matrix(m, n, torch.bfloat16, dY.device, 64)
+    _check(lib().qgalore_int8_linear_backward_weight(_ptr(_bf16_arg(dY, "dY")), T, _matrix_ld(dY, "dY"),
+                                                     _ptr(_bf16_arg(X, "X")), _matrix_ld(X, "X"), m, n,
+                                                     _ptr(_bf16_arg(out, "out")), _matrix_ld(out, "out"),
+                                                     _ptr(status),
+                                                     _stream_ptr(stream)),
+           "qgalore_int8_linear_backward_weight")
     return out
 
 

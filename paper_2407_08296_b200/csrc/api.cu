@@ -109,6 +109,47 @@ int qgalore_dequantize(const qg_qtensor* src, float* dst, int64_t ld_dst, void* 
   return launch_dequantize(src, dst, ld_dst, (cudaStream_t)stream);
 }
 
+// --- App. A: the INT8 linear layer ------------------------------------------------------------
+static int check_bf16_matrix(const uint16_t* p, int64_t rows, int64_t cols, int64_t ld) {
+  if (!p || rows <= 0 || cols <= 0 || ld < cols) return QG_INVALID_ARGUMENT;
+  if (!aligned16(p) || ld % 8 != 0) return QG_MISALIGNED;
+  return QG_OK;
+}
+static bool linear_extent_ok(int64_t v) { return v > 0 && v <= (int64_t)1 << 30; }
+
+int qgalore_int8_linear_forward(const uint16_t* X, int64_t T, int64_t ldx, const qg_qtensor* W, uint16_t* Y,
+                                int64_t ldy, int32_t* status, void* stream) {
+  int rc = check_qtensor(W, 8);
+  if (rc != QG_OK) return rc;
+  if (!linear_extent_ok(T) || !linear_extent_ok(W->rows) || !linear_extent_ok(W->cols)) return QG_UNSUPPORTED_SHAPE;
+  if ((rc = check_bf16_matrix(X, T, W->cols, ldx)) != QG_OK) return rc;
+  if ((rc = check_bf16_matrix(Y, T, W->rows, ldy)) != QG_OK) return rc;
+  return launch_int8_linear(0, X, ldx, nullptr, 0, W, T, W->rows, W->cols, Y, ldy, status, (cudaStream_t)stream);
+}
+
+int qgalore_int8_linear_backward_input(const uint16_t* dY, int64_t T, int64_t lddy, const qg_qtensor* W,
+                                       uint16_t* dX, int64_t lddx, int32_t* status, void* stream) {
+  int rc = check_qtensor(W, 8);
+  if (rc != QG_OK) return rc;
+  if (!linear_extent_ok(T) || !linear_extent_ok(W->rows) || !linear_extent_ok(W->cols)) return QG_UNSUPPORTED_SHAPE;
+  if ((rc = check_bf16_matrix(dY, T, W->rows, lddy)) != QG_OK) return rc;
+  if ((rc = check_bf16_matrix(dX, T, W->cols, lddx)) != QG_OK) return rc;
+  return launch_int8_linear(1, dY, lddy, nullptr, 0, W, T, W->rows, W->cols, dX, lddx, status, (cudaStream_t)stream);
+}
+
+int qgalore_int8_linear_backward_weight(const uint16_t* dY, int64_t T, int64_t lddy, const uint16_t* X, int64_t ldx,
+                                        int64_t m, int64_t n, uint16_t* G, int64_t ldg, int32_t* status,
+                                        void* stream) {
+  if (!linear_extent_ok(T) || !linear_extent_ok(m) || !linear_extent_ok(n)) return QG_UNSUPPORTED_SHAPE;
+  int rc;
+  if ((rc = check_bf16_matrix(dY, T, m, lddy)) != QG_OK) return rc;
+  if ((rc = check_bf16_matrix(X, T, n, ldx)) != QG_OK) return rc;
+  if ((rc = check_bf16_matrix(G, m, n, ldg)) != QG_OK) return rc;
+  // both operands are read in whole 64-column slabs: the row pitch has to cover the last one
+  if (lddy < (m + 63) / 64 * 64 || ldx < (n + 63) / 64 * 64) return QG_UNSUPPORTED_SHAPE;
+  return launch_int8_linear(2, dY, lddy, X, ldx, nullptr, T, m, n, G, ldg, status, (cudaStream_t)stream);
+}
+
 size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r) {
   if (m <= 0 || r <= 0) return 0;
   switch (op) {

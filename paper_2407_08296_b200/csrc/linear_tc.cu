@@ -1,0 +1,387 @@
+// The INT8 linear layer of App. A as tcgen05 GEMMs that take the INT8 weight as it is stored:
+//
+//   forward          Y  = X W~^T        (T x m)    A = X   K-major,   B = W~^T  K-major  (K = n)
+//   input gradient   dX = dY W~         (T x n)    A = dY  K-major,   B = W~    MN-major (K = m)
+//   weight gradient  G  = dY^T X        (m x n)    A = dY^T MN-major, B = X     MN-major (K = T)
+//
+// with W~ = bf16((q - z) * s), the weight dequantized in binary32 per group of 256 (Sec. 3.1) and rounded once
+// to the activations' type.  W~ never exists in global memory: the INT8 codes of a B tile arrive in shared
+// memory by TMA, eight converter warps dequantize them straight into the 128-byte-swizzled operand layout the
+// MMA reads, and the accumulator (fp32, tensor memory) leaves as bfloat16.  The weight gradient has no
+// quantized operand: both tiles come by TMA in MN-major form, and its output is the matrix G the optimizer
+// step reads.
+//
+// One persistent CTA per SM, tiles of 128 x 256, two accumulators in tensor memory so that the epilogue of a
+// tile overlaps the main loop of the next.  Warp roles: 0 TMA producer (A, and B of the weight gradient),
+// 1 MMA issuer and tensor-memory owner, 2 TMA producer of the INT8 tiles, 4-7 epilogue, 8-15 converters.
+// Every barrier wait is bounded; a wait that runs out raises QG_DEV_WAIT_EXPIRED and the role stops.
+#include <cstring>
+
+#include "qg_common.cuh"
+#include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace qg {
+
+using namespace ptx;
+
+namespace {
+
+constexpr int kBK = 64;        // K extent of a pipeline stage
+constexpr int kTileM = 128;    // accumulator rows (TMEM lanes)
+constexpr int kTileN = 256;    // accumulator columns; a multiple of the quantization group along n
+constexpr int kSlab = 64 * kBK * 2;   // one 64-wide MN-major slab of a stage: 64 K rows of 128 bytes
+
+enum : int { kForward = 0, kInputGrad = 1, kWeightGrad = 2 };
+
+struct LinArgs {
+  CUtensorMap mapA;            // bf16 activations: K-major 2-D (forward, input gradient) or chunked 3-D
+  CUtensorMap mapB;            // INT8 codes of W (2-D, bytes) or, for the weight gradient, X chunked 3-D
+  const float* scales;         // of W: [w_rows][ngroups]
+  const float* zeros;
+  int32_t ngroups, w_rows;
+  uint16_t* D;                 // bf16 output, row-major
+  int64_t ldd;
+  int32_t rows, cols, K;       // output extents and contraction length
+  int32_t mblocks, nblocks;
+};
+
+template <int MODE>
+struct LinSmem {
+  static constexpr bool kConvert = MODE != kWeightGrad;
+  static constexpr int kABytes = kTileM * kBK * 2;             // 16 KB
+  static constexpr int kBBytes = kTileN * kBK * 2;             // 32 KB
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kStages = kConvert ? 3 : 4;
+  static constexpr int kRawBytes = kTileN * kBK;               // one INT8 tile: 16 KB
+  static constexpr int kRawStages = kConvert ? 3 : 0;
+  static constexpr int kBarOffset = kStages * kStageBytes + kRawStages * kRawBytes;
+  static constexpr int kBytes = kBarOffset + 256 + 1024;       // barriers + slack for 1024-byte alignment
+  static constexpr int kEpiWarps = 4, kConvWarps = 8;
+  static constexpr int kThreads = (4 + kEpiWarps + kConvWarps) * 32;
+  static_assert(kBytes <= 227 * 1024, "shared memory budget");
+};
+
+__device__ __forceinline__ void raise_expired(int32_t* status) {
+  if (status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
+}
+
+// Sixteen INT8 codes (one 16-byte word) -> sixteen bfloat16 of (q - z) * s, as two 16-byte words.
+// bias = 2^23 + 128 + z: the code byte with its sign bit flipped is q + 128, placed in the low mantissa
+// byte of 2^23 it reads as the float 2^23 + 128 + q, and subtracting bias leaves q - z exactly; one
+// binary32 multiplication and one rounding to bfloat16 follow, the same two roundings as the definition.
+__device__ __forceinline__ void dequant16(const uint4 codes, float bias, float s, uint4& lo, uint4& hi) {
+  const uint32_t w[4] = {codes.x ^ 0x80808080u, codes.y ^ 0x80808080u, codes.z ^ 0x80808080u, codes.w ^ 0x80808080u};
+  const float2 nb = make_float2(-bias, -bias), s2 = make_float2(s, s);
+  uint32_t out[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 a = make_float2(__uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7440)),
+                                 __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7441)));
+    const float2 b = make_float2(__uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7442)),
+                                 __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7443)));
+    const float2 va = mul2(add2(a, nb), s2), vb = mul2(add2(b, nb), s2);
+    __nv_bfloat162 pa = __floats2bfloat162_rn(va.x, va.y), pb = __floats2bfloat162_rn(vb.x, vb.y);
+    out[2 * i] = *reinterpret_cast<uint32_t*>(&pa);
+    out[2 * i + 1] = *reinterpret_cast<uint32_t*>(&pb);
+  }
+  lo = make_uint4(out[0], out[1], out[2], out[3]);
+  hi = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(LinSmem<MODE>::kThreads, 1)
+int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ status) {
+  using S = LinSmem<MODE>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* stage_base = smem;
+  uint8_t* raw_base = smem + S::kStages * S::kStageBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::kBarOffset);
+  uint64_t* full = bars;
+  uint64_t* empty = full + S::kStages;
+  uint64_t* raw_full = empty + S::kStages;
+  uint64_t* raw_empty = raw_full + 4;
+  uint64_t* acc_full = raw_empty + 4;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < S::kStages; ++i) {
+      mbar_init(&full[i], S::kConvert ? 1 + S::kConvWarps : 1);   // the TMA producer, and each converter warp
+      mbar_init(&empty[i], 1);
+    }
+    for (int i = 0; i < S::kRawStages; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], S::kConvWarps); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], S::kEpiWarps); }
+    fence_mbar_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // tile t -> (m block, n block): consecutive tiles (concurrent CTAs) share the n block, i.e. the same
+  // columns of B, which for two of the three products is the weight
+  const int total = a.mblocks * a.nblocks;
+  const int kblocks = (a.K + kBK - 1) / kBK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer of A (and bf16 B)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
+        const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % S::kStages;
+          if (!mbar_wait(&empty[s], ((it / S::kStages) & 1) ^ 1)) { ok = false; break; }
+          uint8_t* sA = stage_base + s * S::kStageBytes;
+          if (MODE == kWeightGrad) {
+            mbar_arrive_expect_tx(&full[s], S::kStageBytes);
+            tma_load_3d(sA, &a.mapA, &full[s], 0, kb * kBK, m0 / 64);
+            tma_load_3d(sA + S::kABytes, &a.mapB, &full[s], 0, kb * kBK, n0 / 64);
+          } else {
+            mbar_arrive_expect_tx(&full[s], S::kABytes);
+            tma_load_2d(sA, &a.mapA, &full[s], kb * kBK, m0);
+          }
+        }
+      }
+      if (!ok) raise_expired(status);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kTileN, MODE == kWeightGrad, MODE != kForward);
+      // K-major: rows of 128 bytes, 8-row groups 1024 bytes apart, 16 K indices = 32 bytes along the row.
+      // MN-major: 64-wide slabs of kSlab bytes, 8 K indices = 1024 bytes, 16 K indices = 2048 bytes.
+      const uint64_t desc_a0 = MODE == kWeightGrad ? umma_smem_desc_sw128(smem_u32(stage_base), kSlab, 1024)
+                                                   : umma_smem_desc_sw128(smem_u32(stage_base), 16, 1024);
+      const uint64_t desc_b0 = MODE == kForward ? umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, 16, 1024)
+                                                : umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kSlab, 1024);
+      constexpr uint64_t astep = MODE == kWeightGrad ? (2048 >> 4) : (32 >> 4);
+      constexpr uint64_t bstep = MODE == kForward ? (32 >> 4) : (2048 >> 4);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
+        const uint32_t ab = tcount & 1;
+        if (!mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + ab * kTileN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % S::kStages;
+          if (!mbar_wait(&full[s], (it / S::kStages) & 1)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
+          const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, da + k * astep, db + k * bstep, idesc, (kb | k) != 0);
+          umma_commit(&empty[s]);
+        }
+        if (ok) umma_commit(&acc_full[ab]);
+      }
+      if (!ok) raise_expired(status);
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ TMA producer of the INT8 tiles
+    if (S::kConvert && lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
+        const int n0 = (t / a.mblocks) * kTileN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int rs = it % 3;
+          if (!mbar_wait(&raw_empty[rs], ((it / 3) & 1) ^ 1)) { ok = false; break; }
+          mbar_arrive_expect_tx(&raw_full[rs], S::kRawBytes);
+          // forward: 256 rows of W (the tile's N) x 64 bytes along n (its K), 64-byte swizzle;
+          // input gradient: 64 rows of W (its K) x 256 bytes along n (the tile's N), no swizzle
+          if (MODE == kForward) tma_load_2d(raw_base + rs * S::kRawBytes, &a.mapB, &raw_full[rs], kb * kBK, n0);
+          else tma_load_2d(raw_base + rs * S::kRawBytes, &a.mapB, &raw_full[rs], n0, kb * kBK);
+        }
+      }
+      if (!ok) raise_expired(status);
+    }
+  } else if (warp >= 4 && warp < 4 + S::kEpiWarps) {
+    // ------------------------------------------------------------------ epilogue: fp32 accumulator -> bf16
+    const int q = warp & 3;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
+      const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
+      const uint32_t ab = tcount & 1;
+      if (!mbar_wait(&acc_full[ab], (tcount >> 1) & 1)) { ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + ab * kTileN;
+      const int row = m0 + q * 32 + lane;
+      uint16_t* drow = a.D + (int64_t)row * a.ldd;
+#pragma unroll 1
+      for (int c = 0; c < kTileN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(tacc + 32 * c, v);
+        tmem_ld_wait();
+        if (c == kTileN / 32 - 1) {                    // every read of this accumulator has landed
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&acc_empty[ab]);
+        }
+        const int col = n0 + 32 * c;
+        if (row < a.rows && col < a.cols) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+            pk[i] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          if (col + 32 <= a.cols) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              *reinterpret_cast<uint4*>(drow + col + 8 * i) = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col + i < a.cols) drow[col + i] = (uint16_t)((i & 1) ? (pk[i >> 1] >> 16) : (pk[i >> 1] & 0xFFFFu));
+          }
+        }
+      }
+    }
+    if (!ok && lane == 0) raise_expired(status);
+  } else if (S::kConvert && warp >= 8) {
+    // ------------------------------------------------------------------ converters: INT8 tile -> bf16 operand
+    const int ct = threadIdx.x - 256;                  // 0..255
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
+      const int n0 = (t / a.mblocks) * kTileN;
+      // forward: this thread owns row n0 + ct of W and its scale changes every four K blocks (256 columns);
+      // input gradient: it owns row 64 kb + ct / 4 of W, a new one (with its scale of group n0 / 256) per K block
+      float s_cur = 0.f, z_cur = 0.f, s_nxt = 0.f, z_nxt = 0.f;
+      auto fetch = [&](int kb, float& s, float& z) {
+        int64_t idx;
+        bool valid;
+        if (MODE == kForward) { const int wr = n0 + ct; valid = wr < a.w_rows; idx = (int64_t)wr * a.ngroups + (kb >> 2); }
+        else { const int wr = kb * kBK + (ct >> 2); valid = wr < a.w_rows; idx = (int64_t)wr * a.ngroups + n0 / kGroup; }
+        s = valid ? __ldg(a.scales + idx) : 0.f;
+        z = valid ? __ldg(a.zeros + idx) : 0.f;
+      };
+      fetch(0, s_nxt, z_nxt);
+      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        const bool renew = MODE == kForward ? (kb & 3) == 0 : true;
+        if (renew) {
+          s_cur = s_nxt; z_cur = z_nxt;
+          const int nk = MODE == kForward ? kb + 4 : kb + 1;
+          if (nk < kblocks) fetch(nk, s_nxt, z_nxt);
+        }
+        const int rs = it % 3, s = it % S::kStages;
+        if (!mbar_wait(&raw_full[rs], (it / 3) & 1) || !mbar_wait(&empty[s], ((it / S::kStages) & 1) ^ 1)) { ok = false; break; }
+        const float bias = 8388736.0f + z_cur;         // 2^23 + 128 + z
+        const uint8_t* raw = raw_base + rs * S::kRawBytes;
+        uint8_t* sB = stage_base + s * S::kStageBytes + S::kABytes;
+        if (MODE == kForward) {
+          // raw: [256 rows][64 bytes], 16-byte piece c of row r stored at c ^ ((r >> 1) & 3);
+          // operand (K-major): row r = 128 bytes, 16-byte piece j stored at j ^ (r & 7)
+          const uint8_t* rrow = raw + ct * 64;
+          uint8_t* orow = sB + ct * 128;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const uint4 codes = *reinterpret_cast<const uint4*>(rrow + ((c ^ ((ct >> 1) & 3)) << 4));
+            uint4 lo, hi;
+            dequant16(codes, bias, s_cur, lo, hi);
+            *reinterpret_cast<uint4*>(orow + (((2 * c) ^ (ct & 7)) << 4)) = lo;
+            *reinterpret_cast<uint4*>(orow + (((2 * c + 1) ^ (ct & 7)) << 4)) = hi;
+          }
+        } else {
+          // raw: [64 rows][256 bytes]; operand (MN-major): slab i holds columns 64 i .. 64 i + 63 as
+          // [64 K rows][128 bytes], 16-byte piece j of row k stored at j ^ (k & 7)
+          const int k = ct >> 2, q4 = ct & 3;
+          const uint8_t* rrow = raw + k * 256 + q4 * 16;
+          uint8_t* orow = sB + k * 128;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4 codes = *reinterpret_cast<const uint4*>(rrow + i * 64);
+            uint4 lo, hi;
+            dequant16(codes, bias, s_cur, lo, hi);
+            *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4) ^ (k & 7)) << 4)) = lo;
+            *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4 + 1) ^ (k & 7)) << 4)) = hi;
+          }
+        }
+        fence_proxy_async_smem();                      // the MMA reads these stores through the async proxy
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(&full[s]); mbar_arrive(&raw_empty[rs]); }
+      }
+    }
+    if (!ok && lane == 0) raise_expired(status);
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+int device_sms() {
+  static int n = [] {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) v = 0;
+    (void)cudaGetLastError();
+    return v;
+  }();
+  return n > 0 ? n : 148;
+}
+
+template <int MODE>
+int launch_mode(const LinArgs& args, int32_t* status, cudaStream_t st) {
+  using S = LinSmem<MODE>;
+  auto kern = int8_linear_kernel<MODE>;
+  QG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
+  const int total = args.mblocks * args.nblocks;
+  const int sms = device_sms();
+  kern<<<total < sms ? total : sms, S::kThreads, S::kBytes, st>>>(args, status);
+  QG_LAUNCH_CHECK();
+  return QG_OK;
+}
+
+}  // namespace
+
+int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint16_t* act2, int64_t ld_act2,
+                       const qg_qtensor* W, int64_t T, int64_t m, int64_t n, uint16_t* D, int64_t ldd,
+                       int32_t* status, cudaStream_t st) {
+  LinArgs a;
+  memset(&a, 0, sizeof(a));
+  a.D = D;
+  a.ldd = ldd;
+  bool ok = true;
+  if (mode == kWeightGrad) {
+    // act = dY (T x m), act2 = X (T x n); both enter as 64-wide column slabs, K = T runs down the rows
+    ok &= make_map_chunked(&a.mapA, act, T, (m + 63) / 64, ld_act, kBK, 2);
+    ok &= make_map_chunked(&a.mapB, act2, T, (n + 63) / 64, ld_act2, kBK, 4);
+    a.rows = (int32_t)m; a.cols = (int32_t)n; a.K = (int32_t)T;
+  } else {
+    const int64_t kdim = mode == kForward ? n : m;     // act = X (T x n) or dY (T x m)
+    ok &= make_map(&a.mapA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, kdim, T, ld_act, kBK, kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (mode == kForward)
+      ok &= make_map(&a.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kBK, kTileN, CU_TENSOR_MAP_SWIZZLE_64B);
+    else
+      ok &= make_map(&a.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kTileN, kBK, CU_TENSOR_MAP_SWIZZLE_NONE);
+    a.scales = W->scales;
+    a.zeros = W->zeros;
+    a.ngroups = (int32_t)((n + kGroup - 1) / kGroup);
+    a.w_rows = (int32_t)m;
+    a.rows = (int32_t)T;
+    a.cols = (int32_t)(mode == kForward ? m : n);
+    a.K = (int32_t)kdim;
+  }
+  if (!ok) return QG_CUDA_ERROR;
+  a.mblocks = (a.rows + kTileM - 1) / kTileM;
+  a.nblocks = (a.cols + kTileN - 1) / kTileN;
+  switch (mode) {
+    case kForward: return launch_mode<kForward>(a, status, st);
+    case kInputGrad: return launch_mode<kInputGrad>(a, status, st);
+    default: return launch_mode<kWeightGrad>(a, status, st);
+  }
+}
+
+}  // namespace qg

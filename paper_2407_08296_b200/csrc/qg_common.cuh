@@ -228,4 +228,11 @@ struct StepArgs {
 // P~ = bf16((q - z) * s) of an INT4 matrix whose column count is a multiple of 32 (row pitch ld_out elements)
 int launch_dequant_p(const qg_qtensor& P, uint16_t* out, int64_t ld_out, cudaStream_t st);
 
+
+// linear_tc.cu: the INT8 linear layer of App. A.  mode 0: D (T x m) = act (X, T x n) W~^T; mode 1: D (T x n) =
+// act (dY, T x m) W~; mode 2: D (m x n) = act^T (dY, T x m) act2 (X, T x n), W unused.  All bf16, row-major.
+int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint16_t* act2, int64_t ld_act2,
+                       const qg_qtensor* W, int64_t T, int64_t m, int64_t n, uint16_t* D, int64_t ldd,
+                       int32_t* status, cudaStream_t st);
+
 }  // namespace qg

@@ -27,6 +27,7 @@
 #include <vector>
 
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 #include "step_epilogue.cuh"
 
 namespace qg {
@@ -153,25 +154,6 @@ struct K1Smem {
 
 // The Adam update of Sec. 3.5: M <- b1 M + (1-b1) R, V <- b2 V + (1-b2) R^2,
 // N = (M / (1 - b1^t)) / (sqrt(V / (1 - b2^t)) + eps)   (Kingma & Ba; eps outside the root).
-// Packed fp32 pairs (one instruction for two lanes of a float2).
-__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
-  float2 d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(*reinterpret_cast<uint64_t*>(&d)) : "l"(*reinterpret_cast<uint64_t*>(&a)), "l"(*reinterpret_cast<uint64_t*>(&b)));
-  return d;
-}
-__device__ __forceinline__ float2 add2(float2 a, float2 b) {
-  float2 d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(*reinterpret_cast<uint64_t*>(&d)) : "l"(*reinterpret_cast<uint64_t*>(&a)), "l"(*reinterpret_cast<uint64_t*>(&b)));
-  return d;
-}
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
-  float2 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;"
-      : "=l"(*reinterpret_cast<uint64_t*>(&d))
-      : "l"(*reinterpret_cast<uint64_t*>(&a)), "l"(*reinterpret_cast<uint64_t*>(&b)), "l"(*reinterpret_cast<uint64_t*>(&c)));
-  return d;
-}
-
 // Constants of the Adam update in the form the epilogue uses them: with k_v = bias1^2 / bias2 and
 // eps_b = eps * bias1,  N = (M / bias1) / (sqrt(V / bias2) + eps) = M / (sqrt(V * k_v) + eps_b).
 struct AdamConsts {
@@ -1140,53 +1122,6 @@ backproject_sr_kernel(const __grid_constant__ TcProblem single, const TcProblem*
 // ============================================================================================
 // host side
 // ============================================================================================
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    (void)cudaGetLastError();
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// Row-major 2-D tensor [outer][pitch], `inner` valid elements per row; out-of-range elements read as zero
-// and are not written.
-bool make_map(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, int64_t inner, int64_t outer,
-              int64_t pitch_elems, int box_inner, int box_outer, CUtensorMapSwizzle sw) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
-  const cuuint64_t gstr[1] = {(cuuint64_t)pitch_elems * elem_bytes};
-  const cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, dt, 2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// A row-major bf16 matrix [rows][pitch] seen as (64 columns, rows, chunks): element (x, y, z) is column
-// 64 z + x of row y.  A box 64 x box_rows x box_chunks lands in shared memory as box_chunks consecutive
-// [box_rows][64] slabs, i.e. the MN-major 128-byte-swizzled operand layout.
-bool make_map_chunked(CUtensorMap* map, const void* base, int64_t rows, int64_t chunks, int64_t pitch_elems, int box_rows,
-                      int box_chunks) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)chunks};
-  const cuuint64_t gstr[2] = {(cuuint64_t)pitch_elems * 2, 128};
-  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_chunks};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // Scratch of one matrix: P~ (bf16, m x r, pitch r) then N_b (bf16, r x ldn).
 struct TcScratch {
   uint16_t* Pt;

@@ -704,3 +704,64 @@ def test_plan_mixes_fp32_and_8bit_moments():
         if "M_scale" in a:
             assert torch.equal(a["M_scale"], b["M_scale"]) and torch.equal(a["V_scale"], b["V_scale"])
     plan.close()
+
+
+# ----------------------------------------------------------------------------- App. A: the INT8 linear layer
+def _linear_case(T, m, n, seed):
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((m, n)) * 0.02).astype(np.float32)
+    W[:, : min(n, 256)] += 0.5                    # a group far from zero: large zero points
+    W_q = O.quantize_rtn(W, 8)
+    X_bits = O.f32_to_bf16_bits(rng.standard_normal((T, n)).astype(np.float32))
+    dY_bits = O.f32_to_bf16_bits((rng.standard_normal((T, m)) * 0.1).astype(np.float32))
+    return W_q, X_bits, dY_bits
+
+
+def _check_product(got: torch.Tensor, exact: np.ndarray, ref_bits: np.ndarray, abs_sum: np.ndarray, K: int, name: str):
+    """bf16 operands are exact on both sides, so the only differences are the binary32 accumulation of the
+    tensor core (each of the K / 16 instructions adds its products to the accumulator with an error of at most
+    one unit in the last place of the running sum: (K / 16 + 1) * 2^-22 of the sum of magnitudes bounds it with a
+    factor two to spare) and the final rounding to bfloat16 (half a unit in the last place, 2^-9 relative; 2^-8
+    allows the rounding to fall the other way)."""
+    got_bits = got.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert got_bits.shape == ref_bits.shape, name
+    val = O.bf16_bits_to_f32(got_bits).astype(np.float64)
+    tol = 2.0 ** -8 * np.abs(exact) + (K / 16 + 1) * 2.0 ** -22 * abs_sum + 1e-30
+    bad = np.abs(val - exact) > tol
+    assert not bad.any(), f"{name}: {int(bad.sum())} of {bad.size} outside the tolerance"
+    same = np.mean(got_bits == ref_bits)
+    assert same >= 0.98, f"{name}: only {same:.4f} of the outputs round to the same bfloat16"
+
+
+@pytest.mark.parametrize("shape", [(300, 520, 1376), (1, 256, 256), (130, 300, 5461), (1000, 2048, 2048), (257, 64, 200)])
+def test_int8_linear_forward_and_backward(shape):
+    T, m, n = shape
+    W_q, X_bits, dY_bits = _linear_case(T, m, n, seed=T + 3 * m + 7 * n)
+    Wd, Xd, dYd = to_device_q(W_q), g_to_device(X_bits), g_to_device(dY_bits)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    w_before = Wd.codes.clone()
+    Y = B.int8_linear_forward(Xd, Wd, status=status)
+    dX = B.int8_linear_backward_input(dYd, Wd, status=status)
+    G = B.int8_linear_backward_weight(dYd, Xd, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(w_before, Wd.codes)          # the weight is only read
+
+    Y_ref, Y_bits = O.int8_linear_forward(X_bits, W_q)
+    dX_ref, dX_bits, G_ref, G_bits = O.int8_linear_backward(dY_bits, X_bits, W_q)
+    X = np.abs(O.bf16_bits_to_f32(X_bits).astype(np.float64))
+    dY = np.abs(O.bf16_bits_to_f32(dY_bits).astype(np.float64))
+    Wt = np.abs(O.bf16_bits_to_f32(O.f32_to_bf16_bits(O.dequantize(W_q))).astype(np.float64))
+    _check_product(Y, Y_ref, Y_bits, X @ Wt.T, n, "Y")
+    _check_product(dX, dX_ref, dX_bits, dY @ Wt, m, "dX")
+    _check_product(G, G_ref, G_bits, dY.T @ X, T, "G")
+
+
+def test_int8_linear_refusals():
+    W_q, X_bits, dY_bits = _linear_case(8, 64, 256, seed=0)
+    Wd, Xd, dYd = to_device_q(W_q), g_to_device(X_bits), g_to_device(dY_bits)
+    with pytest.raises(B.QgError):                   # X with the wrong inner extent for W: pitch shorter than n
+        B.int8_linear_forward(Xd[:, :64].contiguous(), Wd)
+    narrow = torch.zeros((8, 72), dtype=torch.int16, device="cuda")[:, :70]
+    with pytest.raises(B.QgError):                   # the pitch (72) does not cover the last 64-column slab of 70 columns
+        B.int8_linear_backward_weight(narrow, Xd)
