@@ -109,10 +109,10 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int i = 0; i < S::kStages; ++i) {
-      mbar_init(&full[i], S::kConvert ? 1 + S::kConvWarps : 1);   // the TMA producer, and each converter warp
+      mbar_init(&full[i], S::kConvert ? 1 + S::kConvWarps / 2 : 1);   // the TMA producer, and the converter warps of one group
       mbar_init(&empty[i], 1);
     }
-    for (int i = 0; i < S::kRawStages; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], S::kConvWarps); }
+    for (int i = 0; i < S::kRawStages; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], S::kConvWarps / 2); }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], S::kEpiWarps); }
     fence_mbar_init();
     fence_proxy_async_smem();
@@ -249,61 +249,60 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
     if (!ok && lane == 0) raise_expired(status);
   } else if (S::kConvert && warp >= 8) {
     // ------------------------------------------------------------------ converters: INT8 tile -> bf16 operand
-    const int ct = threadIdx.x - 256;                  // 0..255
+    // Two groups of four warps take alternate K blocks, so that the chain of one block (wait, load, convert,
+    // store, fence, arrive) overlaps that of the next; a thread converts two rows of the tile.
+    const int grp = (warp - 8) >> 2, lt = (threadIdx.x - 256) & 127;
     uint32_t it = 0;
     bool ok = true;
     for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
       const int n0 = (t / a.mblocks) * kTileN;
-      // forward: this thread owns row n0 + ct of W and its scale changes every four K blocks (256 columns);
-      // input gradient: it owns row 64 kb + ct / 4 of W, a new one (with its scale of group n0 / 256) per K block
-      float s_cur = 0.f, z_cur = 0.f, s_nxt = 0.f, z_nxt = 0.f;
-      auto fetch = [&](int kb, float& s, float& z) {
-        int64_t idx;
-        bool valid;
-        if (MODE == kForward) { const int wr = n0 + ct; valid = wr < a.w_rows; idx = (int64_t)wr * a.ngroups + (kb >> 2); }
-        else { const int wr = kb * kBK + (ct >> 2); valid = wr < a.w_rows; idx = (int64_t)wr * a.ngroups + n0 / kGroup; }
-        s = valid ? __ldg(a.scales + idx) : 0.f;
-        z = valid ? __ldg(a.zeros + idx) : 0.f;
-      };
-      fetch(0, s_nxt, z_nxt);
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
-        const bool renew = MODE == kForward ? (kb & 3) == 0 : true;
-        if (renew) {
-          s_cur = s_nxt; z_cur = z_nxt;
-          const int nk = MODE == kForward ? kb + 4 : kb + 1;
-          if (nk < kblocks) fetch(nk, s_nxt, z_nxt);
+        if ((int)(it & 1) != grp) continue;
+        // forward: rows n0 + lt and n0 + lt + 128 of W, scale of the 256-column group of this K block;
+        // input gradient: rows 64 kb + lt / 4 and + 32 of W, scale of group n0 / 256
+        float sc[2], bias[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int wr = MODE == kForward ? n0 + lt + 128 * h : kb * kBK + (lt >> 2) + 32 * h;
+          const int64_t idx = (int64_t)wr * a.ngroups + (MODE == kForward ? (kb >> 2) : n0 / kGroup);
+          const bool valid = wr < a.w_rows;
+          sc[h] = valid ? __ldg(a.scales + idx) : 0.f;
+          bias[h] = 8388736.0f + (valid ? __ldg(a.zeros + idx) : 0.f);     // 2^23 + 128 + z
         }
         const int rs = it % 3, s = it % S::kStages;
         if (!mbar_wait(&raw_full[rs], (it / 3) & 1) || !mbar_wait(&empty[s], ((it / S::kStages) & 1) ^ 1)) { ok = false; break; }
-        const float bias = 8388736.0f + z_cur;         // 2^23 + 128 + z
         const uint8_t* raw = raw_base + rs * S::kRawBytes;
         uint8_t* sB = stage_base + s * S::kStageBytes + S::kABytes;
-        if (MODE == kForward) {
-          // raw: [256 rows][64 bytes], 16-byte piece c of row r stored at c ^ ((r >> 1) & 3);
-          // operand (K-major): row r = 128 bytes, 16-byte piece j stored at j ^ (r & 7)
-          const uint8_t* rrow = raw + ct * 64;
-          uint8_t* orow = sB + ct * 128;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const uint4 codes = *reinterpret_cast<const uint4*>(rrow + ((c ^ ((ct >> 1) & 3)) << 4));
-            uint4 lo, hi;
-            dequant16(codes, bias, s_cur, lo, hi);
-            *reinterpret_cast<uint4*>(orow + (((2 * c) ^ (ct & 7)) << 4)) = lo;
-            *reinterpret_cast<uint4*>(orow + (((2 * c + 1) ^ (ct & 7)) << 4)) = hi;
-          }
-        } else {
-          // raw: [64 rows][256 bytes]; operand (MN-major): slab i holds columns 64 i .. 64 i + 63 as
-          // [64 K rows][128 bytes], 16-byte piece j of row k stored at j ^ (k & 7)
-          const int k = ct >> 2, q4 = ct & 3;
-          const uint8_t* rrow = raw + k * 256 + q4 * 16;
-          uint8_t* orow = sB + k * 128;
+        for (int h = 0; h < 2; ++h) {
+          if (MODE == kForward) {
+            // raw: [256 rows][64 bytes], 16-byte piece c of row r stored at c ^ ((r >> 1) & 3);
+            // operand (K-major): row r = 128 bytes, 16-byte piece j stored at j ^ (r & 7)
+            const int r = lt + 128 * h;
+            const uint8_t* rrow = raw + r * 64;
+            uint8_t* orow = sB + r * 128;
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint4 codes = *reinterpret_cast<const uint4*>(rrow + i * 64);
-            uint4 lo, hi;
-            dequant16(codes, bias, s_cur, lo, hi);
-            *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4) ^ (k & 7)) << 4)) = lo;
-            *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4 + 1) ^ (k & 7)) << 4)) = hi;
+            for (int c = 0; c < 4; ++c) {
+              const uint4 codes = *reinterpret_cast<const uint4*>(rrow + ((c ^ ((r >> 1) & 3)) << 4));
+              uint4 lo, hi;
+              dequant16(codes, bias[h], sc[h], lo, hi);
+              *reinterpret_cast<uint4*>(orow + (((2 * c) ^ (r & 7)) << 4)) = lo;
+              *reinterpret_cast<uint4*>(orow + (((2 * c + 1) ^ (r & 7)) << 4)) = hi;
+            }
+          } else {
+            // raw: [64 rows][256 bytes]; operand (MN-major): slab i holds columns 64 i .. 64 i + 63 as
+            // [64 K rows][128 bytes], 16-byte piece j of row k stored at j ^ (k & 7)
+            const int k = (lt >> 2) + 32 * h, q4 = lt & 3;
+            const uint8_t* rrow = raw + k * 256 + q4 * 16;
+            uint8_t* orow = sB + k * 128;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint4 codes = *reinterpret_cast<const uint4*>(rrow + i * 64);
+              uint4 lo, hi;
+              dequant16(codes, bias[h], sc[h], lo, hi);
+              *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4) ^ (k & 7)) << 4)) = lo;
+              *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4 + 1) ^ (k & 7)) << 4)) = hi;
+            }
           }
         }
         fence_proxy_async_smem();                      // the MMA reads these stores through the async proxy
