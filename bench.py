@@ -273,6 +273,50 @@ def build_stack(workload, device, seed=0, layers=0, moments=32):
     return specs, items
 
 
+def time_linear(items, device, tokens, peak_tflops):
+    """The INT8 linear layer either side of the step (App. A), timed apart from it: forward, input gradient and
+    weight gradient of one matrix of each distinct shape on `tokens` rows of synthetic activations, CUDA events
+    around 10 calls after 3 warm-up calls.  TFLOP/s against the burst bf16 peak (each product is timed alone)."""
+    import torch
+    from paper_2407_08296_b200 import binding as B
+    seen, out = set(), []
+    status = torch.zeros(1, dtype=torch.int32, device=device)
+    stream = torch.cuda.current_stream()
+    for it in items:
+        sp = it["spec"]
+        if (sp.m, sp.n) in seen:
+            continue
+        seen.add((sp.m, sp.n))
+        gen = torch.Generator(device=device).manual_seed(sp.m * 31 + sp.n)
+        X = B.zeros_matrix(tokens, sp.n, torch.bfloat16, device)
+        X.copy_(torch.randn((tokens, sp.n), device=device, generator=gen))
+        dY = B.zeros_matrix(tokens, sp.m, torch.bfloat16, device)
+        dY.copy_(torch.randn((tokens, sp.m), device=device, generator=gen) * 0.1)
+        Y = B.empty_matrix(tokens, sp.m, torch.bfloat16, device)
+        dX = B.empty_matrix(tokens, sp.n, torch.bfloat16, device)
+        G = B.empty_matrix(sp.m, sp.n, torch.bfloat16, device)
+        calls = {"forward": lambda: B.int8_linear_forward(X, it["W"], out=Y, status=status),
+                 "backward_input": lambda: B.int8_linear_backward_input(dY, it["W"], out=dX, status=status),
+                 "backward_weight": lambda: B.int8_linear_backward_weight(dY, X, out=G, status=status)}
+        row = {"shape": f"{sp.m}x{sp.n}"}
+        flops = 2.0 * tokens * sp.m * sp.n
+        for name, fn in calls.items():
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(10):
+                fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 10
+            row[name] = {"ms": ms, "tflops": flops / ms / 1e9, "frac_of_peak": flops / ms / 1e9 / peak_tflops}
+        out.append(row)
+        del X, dY, Y, dX, G
+    return {"tokens": tokens, "peak_tflops": peak_tflops, "per_shape": out, "device_status": int(status.item()),
+            "note": "not part of the timed step; forward and backward_input dequantize the INT8 weight inside the GEMM"}
+
+
 def time_refresh(items, device):
     """The occasional subspace refresh (Sec. 3.5), timed apart from the step: one matrix of each distinct
     shape (12 subspace iterations on a block of 2r columns, Rayleigh-Ritz, INT4), CUDA events around the second
@@ -521,6 +565,7 @@ def run_ours(args):
         if refresh is not None:
             # the step and the refresh blended at the base interval of Sec. 4.1 (a refresh every 200 steps)
             refresh["blended_ms_per_step_at_interval_200"] = ms_per_step + refresh["stack_seconds_concurrent"] * 1e3 / 200.0
+        linear = time_linear(items, device, args.linear_tokens, peaks["bf16_tflops"]) if args.linear_tokens > 0 else None
         cpu = None
         if not args.no_cpu_baseline:
             v, per_step, sample = oracle_sample(args.workload, 3, 1)
@@ -537,6 +582,7 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
                     "steps": e2e_steps},
             "gpu_launches": launches, "clocks": clocks, "device_status": status, "refresh": refresh,
+            "int8_linear": linear,
         }
         print(json.dumps(line), flush=True)
     if world > 1:
@@ -550,6 +596,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="llama1b")
     ap.add_argument("--no-refresh", action="store_true", help="skip the separate timing of the subspace refresh")
+    ap.add_argument("--linear-tokens", type=int, default=8192,
+                    help="rows of activations for the separate timing of the INT8 linear layer's GEMMs (0: skip)")
     ap.add_argument("--moments", type=int, choices=[32, 8], default=32,
                     help="storage of the Adam moments: fp32 (the measured configuration) or the 8-bit block-wise form")
     ap.add_argument("--rounding", choices=["stochastic", "nearest"], default="stochastic",
