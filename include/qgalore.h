@@ -287,7 +287,7 @@ QG_API int qgalore_gate_update(float sim, float threshold, int32_t k, int32_t* i
  *                    rounded up to multiples of 64 (what lies in the padding does not matter), else
  *                    QG_UNSUPPORTED_SHAPE.
  * status (device int32, may be null) receives QG_DEV_WAIT_EXPIRED if a bounded wait ran out.  Extents up to
- * 2^30.  No workspace. */
+ * 2^30 and at most 2^30 output tiles of 128 x 256, else QG_UNSUPPORTED_SHAPE.  No workspace. */
 QG_API int qgalore_int8_linear_forward(const uint16_t* X, int64_t T, int64_t ldx, const qg_qtensor* W,
                                 uint16_t* Y, int64_t ldy, int32_t* status, void* stream);
 QG_API int qgalore_int8_linear_backward_input(const uint16_t* dY, int64_t T, int64_t lddy, const qg_qtensor* W,

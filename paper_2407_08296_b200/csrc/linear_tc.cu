@@ -376,6 +376,7 @@ int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint
   if (!ok) return QG_CUDA_ERROR;
   a.mblocks = (a.rows + kTileM - 1) / kTileM;
   a.nblocks = (a.cols + kTileN - 1) / kTileN;
+  if ((int64_t)a.mblocks * a.nblocks > (int64_t)1 << 30) return QG_UNSUPPORTED_SHAPE;   // the tile index is an int
   switch (mode) {
     case kForward: return launch_mode<kForward>(a, status, st);
     case kInputGrad: return launch_mode<kInputGrad>(a, status, st);
