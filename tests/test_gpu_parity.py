@@ -128,6 +128,34 @@ def test_refresh_reports_similarity_with_previous_projection():
     assert float(sim.item()) > 0.9                         # the leading planted directions persist
 
 
+def test_refresh_replayed_from_a_cuda_graph_gives_the_same_codes():
+    """Nothing in the refresh decides on the host: a captured refresh (a few thousand launches, one of them
+    cooperative) replays to the codes of the direct call, also on another gradient placed in the same buffer."""
+    m, n, r = 512, 768, 128
+    gm = synth.GradientModel(m, n, seed=4, matrix_index=0)
+    dG = g_to_device(gm.sample(1))
+    block = 2 * r
+    ws = torch.empty(B.workspace_bytes(B.QG_OP_REFRESH, m, n, block), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    direct = B.refresh_subspace(dG, r, seed=3, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    P_new = B.QTensor.empty(m, r, 4, "cuda")
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.graph(graph, stream=side):
+        B.refresh_subspace(dG, r, seed=3, P_new=P_new, workspace=ws, status=status, stream=torch.cuda.current_stream())
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(P_new.codes, direct.codes) and torch.equal(P_new.scales, direct.scales)
+    g2 = g_to_device(gm.sample(2))
+    want = B.refresh_subspace(g2, r, seed=3, workspace=ws, status=status)
+    torch.cuda.synchronize()
+    dG.copy_(g2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(P_new.codes, want.codes) and torch.equal(P_new.zeros, want.zeros)
+
+
 def test_refresh_rejects_bad_block_widths():
     dG = torch.zeros((128, 256), dtype=torch.int16, device="cuda")
     with pytest.raises(B.QgError) as e:
