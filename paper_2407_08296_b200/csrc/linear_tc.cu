@@ -321,6 +321,211 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
   }
 }
 
+// ----------------------------------------------------------------------------------------------------------
+// The forward product with the converted weight handed to the MMA through TENSOR memory instead of shared
+// memory.  The product is computed transposed, Y^T = W~ X^T: the accumulator's 128 rows are rows of W, its 256
+// columns are rows of X (tokens); operand A is a 128 x 64 tile of W~ that a converter thread per row writes with
+// one tcgen05.st (64 bf16 = 32 packed registers), operand B is a K-major tile of X by TMA.  Per K block the
+// shared memory then carries 80 KB (32 KB of X written and read, 8 KB of codes written and read) instead of the
+// 128 KB of the layout above.  Tensor memory: columns 0..255 the accumulator, 256..511 eight A stages of 32
+// columns, so the epilogue of a tile does not overlap the next main loop (the operand pipelines keep filling).
+// Warp roles: 0 TMA producer (X tiles and codes), 1 MMA issuer and tensor-memory owner, 4-7 and 12-15 two
+// converter groups that take alternate K blocks (a warp reaches the lane quarter warp % 4), 8-11 epilogue.
+struct FwdSmem {
+  static constexpr int kBBytes = kTileN * kBK * 2;             // 32 KB of X
+  static constexpr int kStages = 5;
+  static constexpr int kRawBytes = kTileM * kBK;               // 8 KB of codes
+  static constexpr int kRawStages = 4;
+  static constexpr int kAStages = 8, kACols = kBK / 2;         // tensor-memory stages of A, 32 columns each
+  // per epilogue warp: a 32 x 32 bf16 block on its way to being stored transposed; rows of 80 bytes keep the
+  // 16-byte reads of eight lanes in different banks
+  static constexpr int kTransRow = 80, kTransBytes = 32 * kTransRow;
+  static constexpr int kTransOffset = kStages * kBBytes + kRawStages * kRawBytes;
+  static constexpr int kBarOffset = kTransOffset + 4 * kTransBytes;
+  static constexpr int kBytes = kBarOffset + 512 + 1024;
+  static constexpr int kThreads = 512;
+};
+
+__global__ void __launch_bounds__(FwdSmem::kThreads, 1)
+int8_linear_forward_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ status) {
+  using S = FwdSmem;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* b_base = smem;
+  uint8_t* raw_base = smem + S::kStages * S::kBBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + S::kBarOffset);
+  uint64_t* b_full = bars;
+  uint64_t* b_empty = b_full + S::kStages;
+  uint64_t* raw_full = b_empty + S::kStages;
+  uint64_t* raw_empty = raw_full + S::kRawStages;
+  uint64_t* a_full = raw_empty + S::kRawStages;
+  uint64_t* a_empty = a_full + S::kAStages;
+  uint64_t* acc_full = a_empty + S::kAStages;
+  uint64_t* acc_empty = acc_full + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < S::kStages; ++i) { mbar_init(&b_full[i], 1); mbar_init(&b_empty[i], 1); }
+    for (int i = 0; i < S::kRawStages; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], 4); }
+    for (int i = 0; i < S::kAStages; ++i) { mbar_init(&a_full[i], 4); mbar_init(&a_empty[i], 1); }
+    mbar_init(acc_full, 1);
+    mbar_init(acc_empty, 4);
+    fence_mbar_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_a = tmem_base + kTileN;
+
+  // here a.rows / a.mblocks count rows of W (the accumulator's rows), a.cols / a.nblocks rows of X (its columns);
+  // consecutive tiles (concurrent CTAs) share the block of X
+  const int total = a.mblocks * a.nblocks;
+  const int kblocks = (a.K + kBK - 1) / kBK;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer: X tile and codes
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
+        const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int rs = it % S::kRawStages, s = it % S::kStages;
+          if (!mbar_wait(&raw_empty[rs], ((it / S::kRawStages) & 1) ^ 1)) { ok = false; break; }
+          mbar_arrive_expect_tx(&raw_full[rs], S::kRawBytes);
+          tma_load_2d(raw_base + rs * S::kRawBytes, &a.mapB, &raw_full[rs], kb * kBK, m0);
+          if (!mbar_wait(&b_empty[s], ((it / S::kStages) & 1) ^ 1)) { ok = false; break; }
+          mbar_arrive_expect_tx(&b_full[s], S::kBBytes);
+          tma_load_2d(b_base + s * S::kBBytes, &a.mapA, &b_full[s], kb * kBK, n0);
+        }
+      }
+      if (!ok) raise_expired(status);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kTileN, false, false);
+      const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(b_base), 16, 1024);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
+        if (!mbar_wait(acc_empty, (tcount & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after_sync();
+        for (int kb = 0; kb < kblocks; ++kb, ++it) {
+          const int s = it % S::kStages, as = it % S::kAStages;
+          if (!mbar_wait(&b_full[s], (it / S::kStages) & 1) || !mbar_wait(&a_full[as], (it / S::kAStages) & 1)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint64_t db = desc_b0 + (uint64_t)((s * S::kBBytes) >> 4);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)
+            umma_bf16_tmem_a(tmem_base, tmem_a + as * S::kACols + k * 8, db + k * (32 >> 4), idesc, (kb | k) != 0);
+          umma_commit(&b_empty[s]);
+          umma_commit(&a_empty[as]);
+        }
+        if (ok) umma_commit(acc_full);
+      }
+      if (!ok) raise_expired(status);
+    }
+  } else if (warp >= 8 && warp < 12) {
+    // ------------------------------------------------------------------ epilogue: row i of the tile is row m0 + i of W,
+    // column c is row n0 + c of X.  A thread holds one row of the tile; each 32 x 32 block goes through shared
+    // memory so that a thread stores 64 contiguous bytes of one row of Y (2-byte stores, 256 per thread and
+    // tile, took longer than the main loop of a short K)
+    const int q = warp & 3;
+    uint8_t* trans = smem + S::kTransOffset + q * S::kTransBytes;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
+      const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
+      if (!mbar_wait(acc_full, tcount & 1)) { ok = false; break; }
+      tc_fence_after_sync();
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < kTileN / 32; ++c) {
+        uint32_t v[32];
+        tmem_ld_32x32(tacc + 32 * c, v);
+        tmem_ld_wait();
+        if (c == kTileN / 32 - 1) {
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty);
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {                   // block[j][lane] = D[lane][j]
+          const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(v[j]));
+          *reinterpret_cast<uint16_t*>(trans + j * S::kTransRow + lane * 2) = *reinterpret_cast<const uint16_t*>(&h);
+        }
+        __syncwarp();
+        const int tok = n0 + 32 * c + lane, w0 = m0 + q * 32;   // this lane now owns one row of Y: 32 values from w0 on
+        if (tok < a.cols) {
+          uint16_t* yrow = a.D + (int64_t)tok * a.ldd + w0;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint4 val = *reinterpret_cast<const uint4*>(trans + lane * S::kTransRow + 16 * i);
+            if (w0 + 8 * i + 8 <= a.rows) {
+              *reinterpret_cast<uint4*>(yrow + 8 * i) = val;
+            } else {
+              const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+              for (int e = 0; e < 8; ++e)
+                if (w0 + 8 * i + e < a.rows) yrow[8 * i + e] = (uint16_t)((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu));
+            }
+          }
+        }
+        __syncwarp();
+      }
+    }
+    if (!ok && lane == 0) raise_expired(status);
+  } else if ((warp >= 4 && warp < 8) || warp >= 12) {
+    // ------------------------------------------------------------------ converters: codes -> bf16 rows of A in tensor memory
+    const int grp = warp >= 12 ? 1 : 0, q = warp & 3;
+    const int row = q * 32 + lane;                       // row of the tile = lane of tensor memory
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
+      const int wr = (t % a.mblocks) * kTileM + row;
+      const bool valid = wr < a.w_rows;
+      for (int kb = 0; kb < kblocks; ++kb, ++it) {
+        if ((int)(it & 1) != grp) continue;
+        const int64_t idx = (int64_t)wr * a.ngroups + (kb >> 2);
+        const float sc = valid ? __ldg(a.scales + idx) : 0.f;
+        const float bias = 8388736.0f + (valid ? __ldg(a.zeros + idx) : 0.f);      // 2^23 + 128 + z
+        const int rs = it % S::kRawStages, as = it % S::kAStages;
+        if (!mbar_wait(&raw_full[rs], (it / S::kRawStages) & 1) || !mbar_wait(&a_empty[as], ((it / S::kAStages) & 1) ^ 1)) { ok = false; break; }
+        tc_fence_after_sync();
+        // codes: [128 rows][64 bytes], 16-byte piece c of row r stored at c ^ ((r >> 1) & 3)
+        const uint8_t* rrow = raw_base + rs * S::kRawBytes + row * 64;
+        uint32_t packed[32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint4 codes = *reinterpret_cast<const uint4*>(rrow + ((c ^ ((row >> 1) & 3)) << 4));
+          uint4 lo, hi;
+          dequant16(codes, bias, sc, lo, hi);
+          packed[8 * c + 0] = lo.x; packed[8 * c + 1] = lo.y; packed[8 * c + 2] = lo.z; packed[8 * c + 3] = lo.w;
+          packed[8 * c + 4] = hi.x; packed[8 * c + 5] = hi.y; packed[8 * c + 6] = hi.z; packed[8 * c + 7] = hi.w;
+        }
+        tmem_st_32x32(tmem_a + ((uint32_t)(q * 32) << 16) + as * S::kACols, packed);
+        tmem_st_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(&a_full[as]); mbar_arrive(&raw_empty[rs]); }
+      }
+    }
+    if (!ok && lane == 0) raise_expired(status);
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
 int device_sms() {
   static int n = [] {
     int dev = 0, v = 0;
@@ -377,6 +582,22 @@ int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint
   a.mblocks = (a.rows + kTileM - 1) / kTileM;
   a.nblocks = (a.cols + kTileN - 1) / kTileN;
   if ((int64_t)a.mblocks * a.nblocks > (int64_t)1 << 30) return QG_UNSUPPORTED_SHAPE;   // the tile index is an int
+  if (mode == kForward) {
+    // transposed product: rows of the accumulator are rows of W, its columns rows of X
+    LinArgs f = a;
+    bool ok2 = make_map(&f.mapA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, n, T, ld_act, kBK, kTileN, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok2 &= make_map(&f.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kBK, kTileM, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (!ok2) return QG_CUDA_ERROR;
+    f.rows = (int32_t)m; f.cols = (int32_t)T;
+    f.mblocks = (f.rows + kTileM - 1) / kTileM;
+    f.nblocks = (f.cols + kTileN - 1) / kTileN;
+    if ((int64_t)f.mblocks * f.nblocks > (int64_t)1 << 30) return QG_UNSUPPORTED_SHAPE;
+    QG_CUDA_TRY(cudaFuncSetAttribute(int8_linear_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem::kBytes));
+    const int total = f.mblocks * f.nblocks, sms = device_sms();
+    int8_linear_forward_kernel<<<total < sms ? total : sms, FwdSmem::kThreads, FwdSmem::kBytes, st>>>(f, status);
+    QG_LAUNCH_CHECK();
+    return QG_OK;
+  }
   switch (mode) {
     case kForward: return launch_mode<kForward>(a, status, st);
     case kInputGrad: return launch_mode<kInputGrad>(a, status, st);
