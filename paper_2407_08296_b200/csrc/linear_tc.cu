@@ -1,19 +1,20 @@
 // The INT8 linear layer of App. A as tcgen05 GEMMs that take the INT8 weight as it is stored:
 //
-//   forward          Y  = X W~^T        (T x m)    A = X   K-major,   B = W~^T  K-major  (K = n)
-//   input gradient   dX = dY W~         (T x n)    A = dY  K-major,   B = W~    MN-major (K = m)
-//   weight gradient  G  = dY^T X        (m x n)    A = dY^T MN-major, B = X     MN-major (K = T)
+//   forward          Y^T = W~ X^T       (m x T)    A = W~  from tensor memory, B = X K-major    (K = n)
+//   input gradient   dX  = dY W~        (T x n)    A = dY  K-major,   B = W~    MN-major        (K = m)
+//   weight gradient  G   = dY^T X       (m x n)    A = dY^T MN-major, B = X     MN-major        (K = T)
 //
 // with W~ = bf16((q - z) * s), the weight dequantized in binary32 per group of 256 (Sec. 3.1) and rounded once
-// to the activations' type.  W~ never exists in global memory: the INT8 codes of a B tile arrive in shared
-// memory by TMA, eight converter warps dequantize them straight into the 128-byte-swizzled operand layout the
-// MMA reads, and the accumulator (fp32, tensor memory) leaves as bfloat16.  The weight gradient has no
-// quantized operand: both tiles come by TMA in MN-major form, and its output is the matrix G the optimizer
-// step reads.
+// to the activations' type.  W~ never exists in global memory: the INT8 codes of a tile arrive in shared memory
+// by TMA and converter warps dequantize them straight into the operand the MMA reads - tensor memory for the
+// forward product (second kernel below), the 128-byte-swizzled shared-memory layout for the input gradient.
+// The accumulator (fp32, tensor memory) leaves as bfloat16.  The weight gradient has no quantized operand: both
+// tiles come by TMA in MN-major form, and its output is the matrix G the optimizer step reads.
 //
-// One persistent CTA per SM, tiles of 128 x 256, two accumulators in tensor memory so that the epilogue of a
-// tile overlaps the main loop of the next.  Warp roles: 0 TMA producer (A, and B of the weight gradient),
-// 1 MMA issuer and tensor-memory owner, 2 TMA producer of the INT8 tiles, 4-7 epilogue, 8-15 converters.
+// One persistent CTA per SM, tiles of 128 x 256.  The first kernel (input and weight gradient) keeps two
+// accumulators in tensor memory so that the epilogue of a tile overlaps the main loop of the next; warp roles:
+// 0 TMA producer (A, and B of the weight gradient), 1 MMA issuer and tensor-memory owner, 2 TMA producer of the
+// INT8 tiles, 4-7 epilogue, 8-15 converters.
 // Every barrier wait is bounded; a wait that runs out raises QG_DEV_WAIT_EXPIRED and the role stops.
 #include <cstring>
 
@@ -35,14 +36,15 @@ constexpr int kSlab = 64 * kBK * 2;   // one 64-wide MN-major slab of a stage: 6
 enum : int { kForward = 0, kInputGrad = 1, kWeightGrad = 2 };
 
 struct LinArgs {
-  CUtensorMap mapA;            // bf16 activations: K-major 2-D (forward, input gradient) or chunked 3-D
+  CUtensorMap mapA;            // bf16 activations: K-major 2-D (X of the forward product, where it is the MMA's B
+                               // operand; dY of the input gradient) or chunked 3-D (dY of the weight gradient)
   CUtensorMap mapB;            // INT8 codes of W (2-D, bytes) or, for the weight gradient, X chunked 3-D
   const float* scales;         // of W: [w_rows][ngroups]
   const float* zeros;
   int32_t ngroups, w_rows;
   uint16_t* D;                 // bf16 output, row-major
   int64_t ldd;
-  int32_t rows, cols, K;       // output extents and contraction length
+  int32_t rows, cols, K;       // accumulator extents (forward: rows of W x rows of X) and contraction length
   int32_t mblocks, nblocks;
 };
 
@@ -154,15 +156,14 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kTileN, MODE == kWeightGrad, MODE != kForward);
+      constexpr uint32_t idesc = umma_idesc_bf16(kTileM, kTileN, MODE == kWeightGrad, true);
       // K-major: rows of 128 bytes, 8-row groups 1024 bytes apart, 16 K indices = 32 bytes along the row.
       // MN-major: 64-wide slabs of kSlab bytes, 8 K indices = 1024 bytes, 16 K indices = 2048 bytes.
       const uint64_t desc_a0 = MODE == kWeightGrad ? umma_smem_desc_sw128(smem_u32(stage_base), kSlab, 1024)
                                                    : umma_smem_desc_sw128(smem_u32(stage_base), 16, 1024);
-      const uint64_t desc_b0 = MODE == kForward ? umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, 16, 1024)
-                                                : umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kSlab, 1024);
+      const uint64_t desc_b0 = umma_smem_desc_sw128(smem_u32(stage_base) + S::kABytes, kSlab, 1024);
       constexpr uint64_t astep = MODE == kWeightGrad ? (2048 >> 4) : (32 >> 4);
-      constexpr uint64_t bstep = MODE == kForward ? (32 >> 4) : (2048 >> 4);
+      constexpr uint64_t bstep = 2048 >> 4;
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
@@ -195,10 +196,8 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
           const int rs = it % 3;
           if (!mbar_wait(&raw_empty[rs], ((it / 3) & 1) ^ 1)) { ok = false; break; }
           mbar_arrive_expect_tx(&raw_full[rs], S::kRawBytes);
-          // forward: 256 rows of W (the tile's N) x 64 bytes along n (its K), 64-byte swizzle;
-          // input gradient: 64 rows of W (its K) x 256 bytes along n (the tile's N), no swizzle
-          if (MODE == kForward) tma_load_2d(raw_base + rs * S::kRawBytes, &a.mapB, &raw_full[rs], kb * kBK, n0);
-          else tma_load_2d(raw_base + rs * S::kRawBytes, &a.mapB, &raw_full[rs], n0, kb * kBK);
+          // 64 rows of W (the tile's K) x 256 bytes along n (its N), no swizzle
+          tma_load_2d(raw_base + rs * S::kRawBytes, &a.mapB, &raw_full[rs], n0, kb * kBK);
         }
       }
       if (!ok) raise_expired(status);
@@ -258,13 +257,12 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
       const int n0 = (t / a.mblocks) * kTileN;
       for (int kb = 0; kb < kblocks; ++kb, ++it) {
         if ((int)(it & 1) != grp) continue;
-        // forward: rows n0 + lt and n0 + lt + 128 of W, scale of the 256-column group of this K block;
-        // input gradient: rows 64 kb + lt / 4 and + 32 of W, scale of group n0 / 256
+        // rows 64 kb + lt / 4 and + 32 of W, scale of group n0 / 256
         float sc[2], bias[2];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          const int wr = MODE == kForward ? n0 + lt + 128 * h : kb * kBK + (lt >> 2) + 32 * h;
-          const int64_t idx = (int64_t)wr * a.ngroups + (MODE == kForward ? (kb >> 2) : n0 / kGroup);
+          const int wr = kb * kBK + (lt >> 2) + 32 * h;
+          const int64_t idx = (int64_t)wr * a.ngroups + n0 / kGroup;
           const bool valid = wr < a.w_rows;
           sc[h] = valid ? __ldg(a.scales + idx) : 0.f;
           bias[h] = 8388736.0f + (valid ? __ldg(a.zeros + idx) : 0.f);     // 2^23 + 128 + z
@@ -275,34 +273,18 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
         uint8_t* sB = stage_base + s * S::kStageBytes + S::kABytes;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-          if (MODE == kForward) {
-            // raw: [256 rows][64 bytes], 16-byte piece c of row r stored at c ^ ((r >> 1) & 3);
-            // operand (K-major): row r = 128 bytes, 16-byte piece j stored at j ^ (r & 7)
-            const int r = lt + 128 * h;
-            const uint8_t* rrow = raw + r * 64;
-            uint8_t* orow = sB + r * 128;
+          // raw: [64 rows][256 bytes]; operand (MN-major): slab i holds columns 64 i .. 64 i + 63 as
+          // [64 K rows][128 bytes], 16-byte piece j of row k stored at j ^ (k & 7)
+          const int k = (lt >> 2) + 32 * h, q4 = lt & 3;
+          const uint8_t* rrow = raw + k * 256 + q4 * 16;
+          uint8_t* orow = sB + k * 128;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const uint4 codes = *reinterpret_cast<const uint4*>(rrow + ((c ^ ((r >> 1) & 3)) << 4));
-              uint4 lo, hi;
-              dequant16(codes, bias[h], sc[h], lo, hi);
-              *reinterpret_cast<uint4*>(orow + (((2 * c) ^ (r & 7)) << 4)) = lo;
-              *reinterpret_cast<uint4*>(orow + (((2 * c + 1) ^ (r & 7)) << 4)) = hi;
-            }
-          } else {
-            // raw: [64 rows][256 bytes]; operand (MN-major): slab i holds columns 64 i .. 64 i + 63 as
-            // [64 K rows][128 bytes], 16-byte piece j of row k stored at j ^ (k & 7)
-            const int k = (lt >> 2) + 32 * h, q4 = lt & 3;
-            const uint8_t* rrow = raw + k * 256 + q4 * 16;
-            uint8_t* orow = sB + k * 128;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint4 codes = *reinterpret_cast<const uint4*>(rrow + i * 64);
-              uint4 lo, hi;
-              dequant16(codes, bias[h], sc[h], lo, hi);
-              *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4) ^ (k & 7)) << 4)) = lo;
-              *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4 + 1) ^ (k & 7)) << 4)) = hi;
-            }
+          for (int i = 0; i < 4; ++i) {
+            const uint4 codes = *reinterpret_cast<const uint4*>(rrow + i * 64);
+            uint4 lo, hi;
+            dequant16(codes, bias[h], sc[h], lo, hi);
+            *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4) ^ (k & 7)) << 4)) = lo;
+            *reinterpret_cast<uint4*>(orow + i * kSlab + (((2 * q4 + 1) ^ (k & 7)) << 4)) = hi;
           }
         }
         fence_proxy_async_smem();                      // the MMA reads these stores through the async proxy
@@ -564,45 +546,34 @@ int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint
     ok &= make_map_chunked(&a.mapB, act2, T, (n + 63) / 64, ld_act2, kBK, 4);
     a.rows = (int32_t)m; a.cols = (int32_t)n; a.K = (int32_t)T;
   } else {
-    const int64_t kdim = mode == kForward ? n : m;     // act = X (T x n) or dY (T x m)
-    ok &= make_map(&a.mapA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, kdim, T, ld_act, kBK, kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
-    if (mode == kForward)
-      ok &= make_map(&a.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kBK, kTileN, CU_TENSOR_MAP_SWIZZLE_64B);
-    else
-      ok &= make_map(&a.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kTileN, kBK, CU_TENSOR_MAP_SWIZZLE_NONE);
     a.scales = W->scales;
     a.zeros = W->zeros;
     a.ngroups = (int32_t)((n + kGroup - 1) / kGroup);
     a.w_rows = (int32_t)m;
-    a.rows = (int32_t)T;
-    a.cols = (int32_t)(mode == kForward ? m : n);
-    a.K = (int32_t)kdim;
+    if (mode == kForward) {
+      // the product is computed transposed: rows of the accumulator are rows of W, its columns rows of X
+      ok &= make_map(&a.mapA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, n, T, ld_act, kBK, kTileN, CU_TENSOR_MAP_SWIZZLE_128B);
+      ok &= make_map(&a.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kBK, kTileM, CU_TENSOR_MAP_SWIZZLE_64B);
+      a.rows = (int32_t)m; a.cols = (int32_t)T; a.K = (int32_t)n;
+    } else {
+      // act = dY (T x m)
+      ok &= make_map(&a.mapA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, m, T, ld_act, kBK, kTileM, CU_TENSOR_MAP_SWIZZLE_128B);
+      ok &= make_map(&a.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kTileN, kBK, CU_TENSOR_MAP_SWIZZLE_NONE);
+      a.rows = (int32_t)T; a.cols = (int32_t)n; a.K = (int32_t)m;
+    }
   }
   if (!ok) return QG_CUDA_ERROR;
   a.mblocks = (a.rows + kTileM - 1) / kTileM;
   a.nblocks = (a.cols + kTileN - 1) / kTileN;
   if ((int64_t)a.mblocks * a.nblocks > (int64_t)1 << 30) return QG_UNSUPPORTED_SHAPE;   // the tile index is an int
   if (mode == kForward) {
-    // transposed product: rows of the accumulator are rows of W, its columns rows of X
-    LinArgs f = a;
-    bool ok2 = make_map(&f.mapA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, act, n, T, ld_act, kBK, kTileN, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok2 &= make_map(&f.mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, W->codes, n, m, W->ld, kBK, kTileM, CU_TENSOR_MAP_SWIZZLE_64B);
-    if (!ok2) return QG_CUDA_ERROR;
-    f.rows = (int32_t)m; f.cols = (int32_t)T;
-    f.mblocks = (f.rows + kTileM - 1) / kTileM;
-    f.nblocks = (f.cols + kTileN - 1) / kTileN;
-    if ((int64_t)f.mblocks * f.nblocks > (int64_t)1 << 30) return QG_UNSUPPORTED_SHAPE;
     QG_CUDA_TRY(cudaFuncSetAttribute(int8_linear_forward_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem::kBytes));
-    const int total = f.mblocks * f.nblocks, sms = device_sms();
-    int8_linear_forward_kernel<<<total < sms ? total : sms, FwdSmem::kThreads, FwdSmem::kBytes, st>>>(f, status);
+    const int total = a.mblocks * a.nblocks, sms = device_sms();
+    int8_linear_forward_kernel<<<total < sms ? total : sms, FwdSmem::kThreads, FwdSmem::kBytes, st>>>(a, status);
     QG_LAUNCH_CHECK();
     return QG_OK;
   }
-  switch (mode) {
-    case kForward: return launch_mode<kForward>(a, status, st);
-    case kInputGrad: return launch_mode<kInputGrad>(a, status, st);
-    default: return launch_mode<kWeightGrad>(a, status, st);
-  }
+  return mode == kInputGrad ? launch_mode<kInputGrad>(a, status, st) : launch_mode<kWeightGrad>(a, status, st);
 }
 
 }  // namespace qg
