@@ -785,6 +785,38 @@ def test_int8_linear_forward_and_backward(shape):
     _check_product(G, G_ref, G_bits, dY.T @ X, T, "G")
 
 
+def test_int8_linear_backward_feeds_the_optimizer_step():
+    """One training step of one layer on the device, no host copy in between: the weight gradient the layer's
+    backward pass writes is the G the optimizer step reads (same buffer, same pitch).  The oracle runs the same
+    chain on its own: its G differs from the device's in the last bfloat16 bit of a few entries, which the
+    moments see as noise far below their tolerance; the stochastic rounding of the weights is compared in
+    bulk only (a changed G moves some elements across a rounding boundary)."""
+    from parity_utils import check_moments
+    T, m, n, r = 640, 256, 768, 64
+    W_q, X_bits, dY_bits = _linear_case(T, m, n, seed=21)
+    rng = np.random.default_rng(2)
+    P = O.quantize_rtn(np.linalg.qr(rng.standard_normal((m, r)))[0].astype(np.float32), 4)
+    M0 = (rng.standard_normal((r, n)) * 1e-3).astype(np.float32)
+    V0 = (rng.random((r, n)) * 1e-6).astype(np.float32)
+    hyp = O.Hyper(lr=1e-3, step=3, seed=77)
+    _, _, _, G_bits = O.int8_linear_backward(dY_bits, X_bits, W_q)
+    ref = O.project_step(G_bits, P, W_q, M0, V0, hyp)
+
+    Wd, Xd, dYd, Pd = to_device_q(W_q), g_to_device(X_bits), g_to_device(dY_bits), to_device_q(P)
+    Md, Vd = f32_to_device(M0), f32_to_device(V0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    G = B.int8_linear_backward_weight(dYd, Xd, status=status)
+    B.project_step(G, Pd, Wd, Md, Vd, B.Hyper(lr=hyp.lr, step=hyp.step, seed=hyp.seed), status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    check_moments(Md.cpu().numpy(), ref["M"], "M", MOMENT_TOL)
+    check_moments(Vd.cpu().numpy(), ref["V"], "V", MOMENT_TOL)
+    got = from_device_q(Wd)
+    diff = np.abs(got.codes.astype(np.int32) - ref["W"].codes.astype(np.int32))
+    assert diff.max() <= 1 and np.mean(diff != 0) <= 0.02
+    np.testing.assert_allclose(got.scales, ref["W"].scales, rtol=1e-4)
+
+
 def test_int8_linear_refusals():
     W_q, X_bits, dY_bits = _linear_case(8, 64, 256, seed=0)
     Wd, Xd, dYd = to_device_q(W_q), g_to_device(X_bits), g_to_device(dY_bits)
