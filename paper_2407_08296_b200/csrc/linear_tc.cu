@@ -319,9 +319,8 @@ struct FwdSmem {
   static constexpr int kRawBytes = kTileM * kBK;               // 8 KB of codes
   static constexpr int kRawStages = 4;
   static constexpr int kAStages = 8, kACols = kBK / 2;         // tensor-memory stages of A, 32 columns each
-  // per epilogue warp: a 32 x 32 bf16 block on its way to being stored transposed; rows of 80 bytes keep the
-  // 16-byte reads of eight lanes in different banks
-  static constexpr int kTransRow = 80, kTransBytes = 32 * kTransRow;
+  // per epilogue warp: a 32 x 32 bf16 block on its way to being stored transposed (rows of 64 bytes)
+  static constexpr int kTransRow = 64, kTransBytes = 32 * kTransRow;
   static constexpr int kTransOffset = kStages * kBBytes + kRawStages * kRawBytes;
   static constexpr int kBarOffset = kTransOffset + 4 * kTransBytes;
   static constexpr int kBytes = kBarOffset + 512 + 1024;
@@ -415,8 +414,9 @@ int8_linear_forward_kernel(const __grid_constant__ LinArgs a, int32_t* __restric
   } else if (warp >= 8 && warp < 12) {
     // ------------------------------------------------------------------ epilogue: row i of the tile is row m0 + i of W,
     // column c is row n0 + c of X.  A thread holds one row of the tile; each 32 x 32 block goes through shared
-    // memory so that a thread stores 64 contiguous bytes of one row of Y (2-byte stores, 256 per thread and
-    // tile, took longer than the main loop of a short K)
+    // memory so that four lanes together store the 64 contiguous bytes it holds of one row of Y (2-byte stores,
+    // 256 per thread and tile, took longer than the main loop of a short K; 16-byte stores to 32 different rows
+    // per instruction flooded L2 with half-sector writes)
     const int q = warp & 3;
     uint8_t* trans = smem + S::kTransOffset + q * S::kTransBytes;
     uint32_t tcount = 0;
@@ -426,39 +426,48 @@ int8_linear_forward_kernel(const __grid_constant__ LinArgs a, int32_t* __restric
       if (!mbar_wait(acc_full, tcount & 1)) { ok = false; break; }
       tc_fence_after_sync();
       const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < kTileN / 32; ++c) {
-        uint32_t v[32];
-        tmem_ld_32x32(tacc + 32 * c, v);
-        tmem_ld_wait();
-        if (c == kTileN / 32 - 1) {
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty);
-        }
+      auto emit = [&](int c, const uint32_t* v) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) {                   // block[j][lane] = D[lane][j]
           const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(v[j]));
           *reinterpret_cast<uint16_t*>(trans + j * S::kTransRow + lane * 2) = *reinterpret_cast<const uint16_t*>(&h);
         }
         __syncwarp();
-        const int tok = n0 + 32 * c + lane, w0 = m0 + q * 32;   // this lane now owns one row of Y: 32 values from w0 on
-        if (tok < a.cols) {
-          uint16_t* yrow = a.D + (int64_t)tok * a.ldd + w0;
+        const int piece = lane & 3, w0 = m0 + q * 32 + 8 * piece;   // this lane's 8 values of a row of Y start at w0
 #pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint4 val = *reinterpret_cast<const uint4*>(trans + lane * S::kTransRow + 16 * i);
-            if (w0 + 8 * i + 8 <= a.rows) {
-              *reinterpret_cast<uint4*>(yrow + 8 * i) = val;
-            } else {
-              const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+        for (int i = 0; i < 4; ++i) {
+          const int j = (lane >> 2) + 8 * i, tok = n0 + 32 * c + j;
+          if (tok >= a.cols) continue;
+          const uint4 val = *reinterpret_cast<const uint4*>(trans + j * S::kTransRow + 16 * piece);
+          uint16_t* y = a.D + (int64_t)tok * a.ldd + w0;
+          if (w0 + 8 <= a.rows) {
+            *reinterpret_cast<uint4*>(y) = val;
+          } else {
+            const uint32_t w[4] = {val.x, val.y, val.z, val.w};
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
-                if (w0 + 8 * i + e < a.rows) yrow[8 * i + e] = (uint16_t)((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu));
-            }
+            for (int e = 0; e < 8; ++e)
+              if (w0 + e < a.rows) y[e] = (uint16_t)((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu));
           }
         }
         __syncwarp();
+      };
+      // the load of the next 32 columns is in flight while the current ones are converted and stored
+      uint32_t va[32], vb[32];
+      tmem_ld_32x32(tacc, va);
+#pragma unroll 1
+      for (int c = 0; c < kTileN / 32; c += 2) {
+        tmem_ld_wait();
+        tmem_ld_32x32(tacc + 32 * (c + 1), vb);
+        emit(c, va);
+        tmem_ld_wait();
+        if (c + 2 < kTileN / 32) {
+          tmem_ld_32x32(tacc + 32 * (c + 2), va);
+        } else {                                         // every read of the accumulator has landed
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty);
+        }
+        emit(c + 1, vb);
       }
     }
     if (!ok && lane == 0) raise_expired(status);
