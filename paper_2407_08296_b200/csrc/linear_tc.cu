@@ -309,8 +309,10 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
 // columns are rows of X (tokens); operand A is a 128 x 64 tile of W~ that a converter thread per row writes with
 // one tcgen05.st (64 bf16 = 32 packed registers), operand B is a K-major tile of X by TMA.  Per K block the
 // shared memory then carries 80 KB (32 KB of X written and read, 8 KB of codes written and read) instead of the
-// 128 KB of the layout above.  Tensor memory: columns 0..255 the accumulator, 256..511 eight A stages of 32
-// columns, so the epilogue of a tile does not overlap the next main loop (the operand pipelines keep filling).
+// 128 KB of the layout above.  Tensor memory: columns 0..255 the accumulator, 256..383 its copy rounded to
+// bfloat16, 384..511 four A stages of 32 columns: there is no room for a second accumulator, so the epilogue first
+// parks the rounded accumulator in the copy (fast: tensor memory to registers and back), releases the accumulator
+// to the MMA, and writes the copy out beside the next tile's main loop.
 // Warp roles: 0 TMA producer (X tiles and codes), 1 MMA issuer and tensor-memory owner, 4-7 and 12-15 two
 // converter groups that take alternate K blocks (a warp reaches the lane quarter warp % 4), 8-11 epilogue.
 struct FwdSmem {
@@ -318,7 +320,10 @@ struct FwdSmem {
   static constexpr int kStages = 5;
   static constexpr int kRawBytes = kTileM * kBK;               // 8 KB of codes
   static constexpr int kRawStages = 4;
-  static constexpr int kAStages = 8, kACols = kBK / 2;         // tensor-memory stages of A, 32 columns each
+  static constexpr int kAStages = 4, kACols = kBK / 2;         // tensor-memory stages of A, 32 columns each
+  static constexpr int kCopyCol = kTileN;                      // tensor-memory columns of the accumulator's bf16 copy
+  static constexpr int kACol0 = kCopyCol + kTileN / 2;         // ... and of the first A stage
+  static_assert(kACol0 + kAStages * kACols <= 512, "tensor memory columns");
   // per epilogue warp: a 32 x 32 bf16 block on its way to being stored transposed (rows of 64 bytes)
   static constexpr int kTransRow = 64, kTransBytes = 32 * kTransRow;
   static constexpr int kTransOffset = kStages * kBBytes + kRawStages * kRawBytes;
@@ -360,7 +365,7 @@ int8_linear_forward_kernel(const __grid_constant__ LinArgs a, int32_t* __restric
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_a = tmem_base + kTileN;
+  const uint32_t tmem_a = tmem_base + S::kACol0;
 
   // here a.rows / a.mblocks count rows of W (the accumulator's rows), a.cols / a.nblocks rows of X (its columns);
   // consecutive tiles (concurrent CTAs) share the block of X
@@ -425,12 +430,41 @@ int8_linear_forward_kernel(const __grid_constant__ LinArgs a, int32_t* __restric
       const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
       if (!mbar_wait(acc_full, tcount & 1)) { ok = false; break; }
       tc_fence_after_sync();
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16);
-      auto emit = [&](int c, const uint32_t* v) {
+      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16), tcopy = tacc + S::kCopyCol;
+      // Phase 1: the accumulator is rounded to bfloat16 and parked in 128 spare columns of tensor memory, 32
+      // columns at a time with the next load in flight; then the MMA may start the next tile.
+      {
+        uint32_t va[32], vb[32];
+        auto park = [&](int c, const uint32_t* v) {
+          uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {                   // block[j][lane] = D[lane][j]
-          const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(v[j]));
-          *reinterpret_cast<uint16_t*>(trans + j * S::kTransRow + lane * 2) = *reinterpret_cast<const uint16_t*>(&h);
+          for (int i = 0; i < 16; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+            pk[i] = *reinterpret_cast<uint32_t*>(&h);
+          }
+          tmem_st_32x16(tcopy + 16 * c, pk);
+        };
+        tmem_ld_32x32(tacc, va);
+#pragma unroll 1
+        for (int c = 0; c < kTileN / 32; c += 2) {
+          tmem_ld_wait();
+          tmem_ld_32x32(tacc + 32 * (c + 1), vb);
+          park(c, va);
+          tmem_ld_wait();
+          if (c + 2 < kTileN / 32) tmem_ld_32x32(tacc + 32 * (c + 2), va);
+          park(c + 1, vb);
+        }
+        tmem_st_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty);
+      }
+      // Phase 2, beside the next tile's main loop: the copy leaves through shared memory, transposed.
+      auto emit = [&](int c, const uint32_t* pk) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {                   // block[j][lane] = D[lane][j], columns 2i and 2i + 1 in pk[i]
+          *reinterpret_cast<uint16_t*>(trans + (2 * i) * S::kTransRow + lane * 2) = (uint16_t)(pk[i] & 0xFFFFu);
+          *reinterpret_cast<uint16_t*>(trans + (2 * i + 1) * S::kTransRow + lane * 2) = (uint16_t)(pk[i] >> 16);
         }
         __syncwarp();
         const int piece = lane & 3, w0 = m0 + q * 32 + 8 * piece;   // this lane's 8 values of a row of Y start at w0
@@ -451,23 +485,16 @@ int8_linear_forward_kernel(const __grid_constant__ LinArgs a, int32_t* __restric
         }
         __syncwarp();
       };
-      // the load of the next 32 columns is in flight while the current ones are converted and stored
-      uint32_t va[32], vb[32];
-      tmem_ld_32x32(tacc, va);
+      uint32_t pa[16], pb[16];
+      tmem_ld_32x16(tcopy, pa);
 #pragma unroll 1
       for (int c = 0; c < kTileN / 32; c += 2) {
         tmem_ld_wait();
-        tmem_ld_32x32(tacc + 32 * (c + 1), vb);
-        emit(c, va);
+        tmem_ld_32x16(tcopy + 16 * (c + 1), pb);
+        emit(c, pa);
         tmem_ld_wait();
-        if (c + 2 < kTileN / 32) {
-          tmem_ld_32x32(tacc + 32 * (c + 2), va);
-        } else {                                         // every read of the accumulator has landed
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acc_empty);
-        }
-        emit(c + 1, vb);
+        if (c + 2 < kTileN / 32) tmem_ld_32x16(tcopy + 16 * (c + 2), pa);
+        emit(c + 1, pb);
       }
     }
     if (!ok && lane == 0) raise_expired(status);
