@@ -761,7 +761,8 @@ def _check_product(got: torch.Tensor, exact: np.ndarray, ref_bits: np.ndarray, a
     assert same >= 0.98, f"{name}: only {same:.4f} of the outputs round to the same bfloat16"
 
 
-@pytest.mark.parametrize("shape", [(300, 520, 1376), (1, 256, 256), (130, 300, 5461), (1000, 2048, 2048), (257, 64, 200)])
+@pytest.mark.parametrize("shape", [(300, 520, 1376), (1, 256, 256), (130, 300, 5461), (1000, 2048, 2048), (257, 64, 200),
+                                   (1, 1, 1), (7, 9, 17), (129, 127, 63)])
 def test_int8_linear_forward_and_backward(shape):
     T, m, n = shape
     W_q, X_bits, dY_bits = _linear_case(T, m, n, seed=T + 3 * m + 7 * n)
