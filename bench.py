@@ -230,49 +230,6 @@ def whole_job_throughput(ms_total, elements_per_rank, steps, world, device):
     return ms, elements_per_rank * world * steps / (ms * 1e-3)
 
 
-def build_stack(workload, device, seed=0, layers=0, moments=32):
-    """Device-resident synthetic state of the whole stack: bf16 gradients (rank-32 signal + noise),
-    INT8 weights, INT4 projections, zero moments.  Generated with torch on the device (input
-    generation, not the path); quantization goes through the library."""
-    import torch
-    from paper_2407_08296_b200 import binding as B
-    from paper_2407_08296_b200 import synth
-    specs = synth.stack_matrices(workload)
-    if layers:
-        specs = [s for s in specs if s.layer < layers]
-    gen = torch.Generator(device=device)
-    gen.manual_seed(seed)
-    items = []
-    sig = 1.0 / torch.arange(1, synth.SIGNAL_RANK + 1, device=device, dtype=torch.float32)
-    for s in specs:
-        k = min(synth.SIGNAL_RANK, s.m, s.n)
-        U = torch.linalg.qr(torch.randn(s.m, k, device=device, generator=gen))[0]
-        Vt = torch.linalg.qr(torch.randn(s.n, k, device=device, generator=gen))[0]
-        g32 = (U * sig[:k]) @ Vt.T + synth.NOISE_STD * torch.randn(s.m, s.n, device=device, generator=gen)
-        G = B.empty_matrix(s.m, s.n, torch.bfloat16, device)
-        G.copy_(g32)
-        del g32
-        w32 = B.empty_matrix(s.m, s.n, torch.float32, device)
-        w32.copy_(torch.randn(s.m, s.n, device=device, generator=gen) * synth.WEIGHT_STD)
-        W = B.quantize_int8(w32)
-        del w32
-        p32 = B.empty_matrix(s.m, s.r, torch.float32, device)
-        p32.copy_(torch.linalg.qr(torch.randn(s.m, s.r, device=device, generator=gen))[0])
-        P = B.quantize_int4(p32)
-        del p32
-        if moments == 8:        # 8-bit block-wise moments: codes and one scale per 32 columns, all zero at the start
-            M = B.zeros_matrix(s.r, s.n, torch.int8, device)
-            V = B.zeros_matrix(s.r, s.n, torch.uint8, device)
-            extra = {"M_scale": torch.zeros((s.r, (s.n + 31) // 32), dtype=torch.float32, device=device),
-                     "V_scale": torch.zeros((s.r, (s.n + 31) // 32), dtype=torch.float32, device=device)}
-        else:
-            M = B.zeros_matrix(s.r, s.n, torch.float32, device)
-            V = B.zeros_matrix(s.r, s.n, torch.float32, device)
-            extra = {}
-        items.append({"G": G, "P": P, "W": W, "M": M, "V": V, "seed": synth.matrix_seed(seed, s.index), "spec": s, **extra})
-    return specs, items
-
-
 def time_linear(items, device, tokens, peak_tflops):
     """The INT8 linear layer either side of the step (App. A), timed apart from it: forward, input gradient and
     weight gradient of one matrix of each distinct shape on `tokens` rows of synthetic activations, CUDA events
@@ -414,6 +371,7 @@ def run_ours(args):
     # every rank holds and steps its own replica of the stack: matrices are independent units, no collective
     global MOMENT_BYTES
     MOMENT_BYTES = 4.5 if args.moments == 8 else 16.0
+    from paper_2407_08296_b200.synth_device import build_stack
     specs, items = build_stack(args.workload, device, seed=rank, layers=args.layers, moments=args.moments)
     batch = B.StepPlan(items)
     elements = batch.elements

@@ -93,6 +93,7 @@ typedef struct {
   float* R;      /* r x n, pitch ldmv: projected gradient                     */
   float* N;      /* r x n, pitch ldmv: Adam direction before bfloat16 rounding */
   float* W_pre;  /* m x n, pitch W->ld: weight before requantization           */
+  uint16_t* N_b; /* r x n, pitch ldmv (elements): the bfloat16 direction as the back-projection reads it */
 } qg_debug;
 
 /* --- Sec. 3.1 / Sec. 3.3: round-to-nearest block-wise quantization ----------------------
@@ -307,18 +308,26 @@ QG_API const char* qgalore_status_string(int status);
 QG_API const char* qgalore_last_cuda_error(void);
 /* Number of kernels the library has launched from this process (for launch accounting). */
 QG_API uint64_t qgalore_launch_count(void);
-/* Test aid: 0 selects the tensor-core kernels of qgalore_project_step (the default and the
- * product path), 1 the plain CUDA-core kernels kept to cross-check them.  Not thread safe. */
+/* --- Test aids.  Declared only when QGALORE_TEST_API is defined before this header is included: they are
+ * process-global switches (not thread safe) that change what later calls do, meant for the test suite. ---- */
+#ifdef QGALORE_TEST_API
+/* 0 selects the tensor-core kernels of qgalore_project_step (the default and the product path), 1 the plain
+ * CUDA-core kernels kept to cross-check them. */
 QG_API int qgalore_debug_set_step_impl(int impl);
-
-/* Test aid: which kernels of plans created after this call run as CTA pairs (tcgen05 cta_group::2, 256 x 256
- * tiles per pair): bit 0 the back-projection, bit 1 the projection (where every rank of a chunk is a multiple of
- * 256).  0 = one CTA per 128 x 256 tile; the default is 2.  Every setting gives the same results bit for bit.
- * Not thread safe. */
+/* Which kernels of plans created after this call run as CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles per
+ * pair): bit 0 the back-projection (chunks of left-hand items only), bit 1 the projection (where every rank of a
+ * chunk is a multiple of 256).  0 = one CTA per 128 x 256 tile; the default is 2.  Every setting gives the same
+ * results bit for bit. */
 QG_API int qgalore_debug_set_pair_mode(int mask);
-/* Test aid: scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks
- * mean fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
+/* Scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks mean
+ * fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
 QG_API int qgalore_debug_set_chunk_budget(size_t bytes);
+/* Runs the bounded barrier wait every tensor-core kernel uses on a barrier that nothing ever signals, with a
+ * limit of `polls` polls (1 .. 2^20), in one small kernel that has no copy in flight and holds no tensor
+ * memory: the wait gives up, the kernel ORs QG_DEV_WAIT_EXPIRED into *status_dev and returns normally.
+ * polls_used_dev (device, optional) receives the number of polls made. */
+QG_API int qgalore_debug_expire_wait(int32_t polls, int32_t* status_dev, int32_t* polls_used_dev, void* stream);
+#endif
 
 /* Diagnostic: writes one text line per tensor-core kernel (registers per thread, thread limit, shared
  * memory) as the CUDA runtime reports them for the current device into buf (HOST, NUL-terminated). */

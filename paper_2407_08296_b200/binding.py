@@ -55,7 +55,7 @@ class _CStepItem(C.Structure):
 
 
 class _CDebug(C.Structure):
-    _fields_ = [("R", C.c_void_p), ("N", C.c_void_p), ("W_pre", C.c_void_p)]
+    _fields_ = [("R", C.c_void_p), ("N", C.c_void_p), ("W_pre", C.c_void_p), ("N_b", C.c_void_p)]
 
 
 _lib = None
@@ -108,6 +108,9 @@ def lib() -> C.CDLL:
         L.qgalore_last_cuda_error.restype = C.c_char_p
         L.qgalore_launch_count.restype = C.c_uint64
         L.qgalore_debug_set_step_impl.argtypes = [C.c_int]
+        L.qgalore_debug_set_pair_mode.argtypes = [C.c_int]
+        L.qgalore_debug_set_chunk_budget.argtypes = [sz]
+        L.qgalore_debug_expire_wait.argtypes = [i32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -302,6 +305,15 @@ def int8_linear_backward_weight(dY: torch.Tensor, X: torch.Tensor, out: torch.Te
     return out
 
 
+def _debug_struct(debug: dict) -> _CDebug:
+    """Optional taps of one step: R, N (fp32), N_b (bf16 bit patterns, same pitch as R and N), W_pre (fp32)."""
+    nb = debug.get("N_b")
+    for key in ("R", "N"):
+        if nb is not None and debug.get(key) is not None and debug[key].stride(0) != nb.stride(0):
+            raise ValueError("the N_b tap must share the row pitch of the R and N taps")
+    return _CDebug(_ptr(debug.get("R")), _ptr(debug.get("N")), _ptr(debug.get("W_pre")), _ptr(nb))
+
+
 def project_step(G: torch.Tensor, P: QTensor, W: QTensor, M: torch.Tensor, V: torch.Tensor, hyper: Hyper,
                  workspace: torch.Tensor | None = None, status: torch.Tensor | None = None,
                  debug: dict | None = None, stream=None, side: str = "left") -> None:
@@ -323,7 +335,7 @@ def project_step(G: torch.Tensor, P: QTensor, W: QTensor, M: torch.Tensor, V: to
         workspace = torch.empty(workspace_bytes(QG_OP_PROJECT_STEP, m, n, r), dtype=torch.uint8, device=G.device)
     dbg = None
     if debug:
-        dbg = _CDebug(_ptr(debug.get("R")), _ptr(debug.get("N")), _ptr(debug.get("W_pre")))
+        dbg = _debug_struct(debug)
     pc, wc, hc = P.c_struct(), W.c_struct(), hyper.c_struct()
     fn = lib().qgalore_project_step_right if right else lib().qgalore_project_step
     _check(fn(_ptr(G), _matrix_ld(G, "G"), m, n, r, C.byref(pc), C.byref(wc), _ptr(M), _ptr(V),
@@ -356,7 +368,7 @@ def project_step_item(item: dict, hyper: "Hyper", workspace: torch.Tensor | None
                                 device=item["G"].device)
     dbg = None
     if debug:
-        dbg = _CDebug(_ptr(debug.get("R")), _ptr(debug.get("N")), _ptr(debug.get("W_pre")))
+        dbg = _debug_struct(debug)
     hc = hyper.c_struct()
     _check(lib().qgalore_project_step_item(C.byref(ci), C.byref(hc), _ptr(workspace), workspace.numel(), _ptr(status),
                                            C.byref(dbg) if dbg is not None else None, _stream_ptr(stream)),
@@ -532,3 +544,13 @@ class Gate:
 
 def debug_set_step_impl(impl: int) -> None:
     _check(lib().qgalore_debug_set_step_impl(impl), "qgalore_debug_set_step_impl")
+
+
+def debug_set_pair_mode(mask: int) -> None:
+    _check(lib().qgalore_debug_set_pair_mode(mask), "qgalore_debug_set_pair_mode")
+
+
+def debug_expire_wait(polls: int, status: torch.Tensor, polls_used: torch.Tensor | None = None, stream=None) -> None:
+    """Test aid: one bounded barrier wait that nothing ever satisfies; ORs QG_DEV_WAIT_EXPIRED into ``status``."""
+    _check(lib().qgalore_debug_expire_wait(polls, _ptr(status), _ptr(polls_used), _stream_ptr(stream)),
+           "qgalore_debug_expire_wait")

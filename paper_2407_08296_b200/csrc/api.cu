@@ -41,17 +41,6 @@ int set_chunk_budget(size_t bytes);
 
 static int g_step_impl = 0;  // 0: tensor-core kernels; 1: CUDA-core kernels (validation aid)
 
-static int check_qtensor(const qg_qtensor* t, int bits) {
-  if (!t || !t->codes || !t->scales || !t->zeros) return QG_INVALID_ARGUMENT;
-  if (t->rows <= 0 || t->cols <= 0 || t->ld < t->cols) return QG_INVALID_ARGUMENT;
-  if (t->bits != bits || t->group != kGroup) return QG_INVALID_ARGUMENT;
-  if (!aligned16(t->codes) || (reinterpret_cast<uintptr_t>(t->scales) & 3u) ||
-      (reinterpret_cast<uintptr_t>(t->zeros) & 3u))
-    return QG_MISALIGNED;
-  if (t->ld % (128 / bits) != 0) return QG_MISALIGNED;      // a row of codes is a multiple of 16 bytes
-  return QG_OK;
-}
-
 }  // namespace qg
 
 using namespace qg;
@@ -388,6 +377,7 @@ static int refresh_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, in
   if (!aligned16(G) || ldg % 8 != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return QG_MISALIGNED;
   if (P_fp32 && !aligned16(P_fp32)) return QG_MISALIGNED;
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
+  if (sim_dev && !aligned4(sim_dev)) return QG_MISALIGNED;
   if (workspace_bytes < qgalore_workspace_bytes(QG_OP_REFRESH, pm, pn, b)) return QG_WORKSPACE_TOO_SMALL;
   constexpr int kJacobiSweeps = 12;
   rc = launch_refresh(G, ldg, pm, pn, r, b, iters, kJacobiSweeps, seed, P_new, P_fp32, workspace, workspace_bytes,
@@ -420,13 +410,12 @@ int qgalore_refresh_subspace_right(const uint16_t* G, int64_t ldg, int64_t m, in
 int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,
                                 void* workspace, size_t workspace_bytes, void* stream) {
   if (!sim_dev || !workspace) return QG_INVALID_ARGUMENT;
-  if (!A || !B || (A->bits != 2 && A->bits != 4 && A->bits != 8) || (B->bits != 2 && B->bits != 4 && B->bits != 8))
-    return QG_INVALID_ARGUMENT;
-  int rc = check_qtensor(A, A->bits);
+  int rc = check_projection_qtensor(A);
   if (rc != QG_OK) return rc;
-  rc = check_qtensor(B, B->bits);
+  rc = check_projection_qtensor(B);
   if (rc != QG_OK) return rc;
   if (A->rows != B->rows || A->cols != B->cols) return QG_INVALID_ARGUMENT;
+  if (!aligned4(sim_dev)) return QG_MISALIGNED;
   const int32_t c = (sim_cols <= 0 || sim_cols > A->cols) ? (int32_t)A->cols : sim_cols;
   if (A->cols > 16384) return QG_UNSUPPORTED_SHAPE;
   if (workspace_bytes < similarity_workspace_bytes(A->rows, A->cols)) return QG_WORKSPACE_TOO_SMALL;

@@ -8,6 +8,7 @@
 #include <float.h>
 #include <stdint.h>
 
+#define QGALORE_TEST_API            // the library implements the test aids the header guards
 #include "../../include/qgalore.h"
 
 namespace qg {
@@ -38,6 +39,24 @@ void count_launch(int n = 1);
   } while (0)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+// Pointer, extent and alignment rules of a quantized matrix that every entry point applies: non-null buffers,
+// positive extents, pitch >= cols, the expected code width, groups of 256; codes 16-byte aligned with rows of
+// whole 16-byte units, scales and zero points 4-byte aligned (the kernels read them as binary32 words).
+inline int check_qtensor(const qg_qtensor* t, int bits) {
+  if (!t || !t->codes || !t->scales || !t->zeros) return QG_INVALID_ARGUMENT;
+  if (t->rows <= 0 || t->cols <= 0 || t->ld < t->cols) return QG_INVALID_ARGUMENT;
+  if (t->bits != bits || t->group != 256) return QG_INVALID_ARGUMENT;
+  if (!aligned16(t->codes) || !aligned4(t->scales) || !aligned4(t->zeros)) return QG_MISALIGNED;
+  if (t->ld % (128 / bits) != 0) return QG_MISALIGNED;      // a row of codes is a multiple of 16 bytes
+  return QG_OK;
+}
+// The same for a projection matrix, whose codes may be 2, 4 or 8 bits wide (Sec. 4.4, Fig. 3).
+inline int check_projection_qtensor(const qg_qtensor* t) {
+  if (!t || (t->bits != 2 && t->bits != 4 && t->bits != 8)) return QG_INVALID_ARGUMENT;
+  return check_qtensor(t, t->bits);
+}
 #ifdef __CUDACC__
 #define QG_HD __host__ __device__
 #else

@@ -252,13 +252,14 @@ extern "C" QG_API size_t qgalore_subspace_similarity_static_max_bytes(void) { re
 extern "C" QG_API int qgalore_subspace_similarity_static(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols,
                                                          float* sim_dev, void* stream) {
   using namespace qg;
-  if (!A || !B || !sim_dev) return QG_INVALID_ARGUMENT;
-  for (const qg_qtensor* t : {A, B}) {
-    if (!t->codes || !t->scales || !t->zeros || t->rows <= 0 || t->cols <= 0 || t->ld < t->cols) return QG_INVALID_ARGUMENT;
-    if ((t->bits != 2 && t->bits != 4 && t->bits != 8) || t->group != kGroup) return QG_INVALID_ARGUMENT;
-    if (!aligned16(t->codes) || t->ld % (128 / t->bits) != 0) return QG_MISALIGNED;
-  }
+  if (!sim_dev) return QG_INVALID_ARGUMENT;
+  // exactly the rules of qgalore_subspace_similarity: what that entry point refuses, this one refuses too
+  int rc = check_projection_qtensor(A);
+  if (rc != QG_OK) return rc;
+  rc = check_projection_qtensor(B);
+  if (rc != QG_OK) return rc;
   if (A->rows != B->rows || A->cols != B->cols) return QG_INVALID_ARGUMENT;
+  if (!aligned4(sim_dev)) return QG_MISALIGNED;
   if (A->cols > 16384) return QG_UNSUPPORTED_SHAPE;
   // the shape must fit the fixed array: report it as a workspace that cannot be made larger
   if (similarity_workspace_bytes(A->rows, A->cols) > kStaticSimilarityBytes) return QG_WORKSPACE_TOO_SMALL;

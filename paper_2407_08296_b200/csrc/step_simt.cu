@@ -97,7 +97,7 @@ struct AdamEpilogue {
   StepScalars sc;
   float* M; float* V; int64_t ldmv;
   uint16_t* Nb; int64_t ldn;
-  float* dbgR; float* dbgN;
+  float* dbgR; float* dbgN; uint16_t* dbgNb;
   int64_t n;
   __device__ void operator()(int64_t i, int64_t j0, const float r8[8]) const {
     const int nvalid = (int)max((int64_t)0, min((int64_t)8, n - j0));
@@ -111,6 +111,7 @@ struct AdamEpilogue {
     }
     if (dbgR) for (int t = 0; t < nvalid; ++t) dbgR[i * ldmv + j0 + t] = r8[t];
     if (dbgN) for (int t = 0; t < nvalid; ++t) dbgN[i * ldmv + j0 + t] = n8[t];
+    if (dbgNb) for (int t = 0; t < nvalid; ++t) dbgNb[i * ldmv + j0 + t] = float_to_bf16_bits(n8[t]);
   }
 };
 
@@ -183,7 +184,7 @@ int launch_project_step_simt(const StepArgs& a, cudaStream_t st) {
     if (rc != QG_OK) return rc;
   }
   {
-    AdamEpilogue epi{a.sc, a.M, a.V, a.ldmv, Nb, ldn, a.dbg.R, a.dbg.N, a.n};
+    AdamEpilogue epi{a.sc, a.M, a.V, a.ldmv, Nb, ldn, a.dbg.R, a.dbg.N, a.dbg.N_b, a.n};
     dim3 grid((unsigned)ceil_div(a.n, kTN), (unsigned)ceil_div(a.r, kTM));
     gemm_simt_kernel<true, AdamEpilogue><<<grid, 256, 0, st>>>(Pt, a.r, a.G, a.ldg, a.r, a.n, a.m, epi);
     QG_LAUNCH_CHECK();

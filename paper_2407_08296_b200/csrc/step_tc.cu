@@ -65,6 +65,7 @@ struct alignas(64) TcProblem {
   float* dbgR;
   float* dbgN;
   float* dbgW;
+  uint16_t* dbgNb;                     // test tap: N_b with the pitch of the moments
   float* M;
   float* V;
   int8_t* w_codes;
@@ -405,7 +406,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       const int nch = min(BN / kChunk, (pn - n0 + kChunk - 1) / kChunk);
       const int cmax = pn - n0 - lcol;               // offset `off` (from n0 + lcol) is a valid column iff off < cmax
       const int64_t ldmv = p->ldmv, ldn = p->ldn;
-      float* Mr[2]; float* Vr[2]; uint16_t* Nr[2]; float* tapR[2]; float* tapN[2];
+      float* Mr[2]; float* Vr[2]; uint16_t* Nr[2]; float* tapR[2]; float* tapN[2]; uint16_t* tapNb[2];
       bool rok[2];
 #pragma unroll
       for (int a = 0; a < 2; ++a) {
@@ -416,10 +417,11 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         Nr[a] = p->nb + gr * ldn + n0 + lcol;
         tapR[a] = p->dbgR ? p->dbgR + gr * ldmv + n0 + lcol : nullptr;
         tapN[a] = p->dbgN ? p->dbgN + gr * ldmv + n0 + lcol : nullptr;
+        tapNb[a] = p->dbgNb ? p->dbgNb + gr * ldmv + n0 + lcol : nullptr;
       }
       // interior tiles (every row and column valid, no test taps) take a path without per-access predicates
       const bool s8 = S8 && p->state8 != 0;
-      const bool whole = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr;
+      const bool whole = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr && p->dbgNb == nullptr;
       const bool interior = whole && !s8;
       int8_t* M8r[2]; uint8_t* V8r[2]; float* msc[2]; float* vsc[2];
 #pragma unroll
@@ -528,10 +530,12 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
                   *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
                   if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
                   if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
+                  if (tapNb[a]) { tapNb[a][off] = __bfloat16_as_ushort(nb2.x); tapNb[a][off + 1] = __bfloat16_as_ushort(nb2.y); }
                 } else if (off < cmax) {
                   Nr[a][off] = float_to_bf16_bits(nn.x);
                   if (tapR[a]) tapR[a][off] = rr.x;
                   if (tapN[a]) tapN[a][off] = nn.x;
+                  if (tapNb[a]) tapNb[a][off] = __bfloat16_as_ushort(nb2.x);
                 }
               }
             } else if (interior) {
@@ -545,12 +549,14 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
                 *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
                 if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
                 if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
+                if (tapNb[a]) { tapNb[a][off] = __bfloat16_as_ushort(nb2.x); tapNb[a][off + 1] = __bfloat16_as_ushort(nb2.y); }
               } else if (off < cmax) {             // odd n: the last column stands alone
                 Mr[a][off] = mm.x;
                 Vr[a][off] = vv.x;
                 Nr[a][off] = float_to_bf16_bits(nn.x);
                 if (tapR[a]) tapR[a][off] = rr.x;
                 if (tapN[a]) tapN[a][off] = nn.x;
+                if (tapNb[a]) tapNb[a][off] = __bfloat16_as_ushort(nb2.x);
               }
             }
           }
@@ -1179,7 +1185,7 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   p->M = a.M; p->V = a.V; p->w_codes = reinterpret_cast<int8_t*>(a.W.codes);
   p->w_scales = a.W.scales;
   p->w_zeros = a.W.zeros;
-  p->dbgR = a.dbg.R; p->dbgN = a.dbg.N; p->dbgW = a.dbg.W_pre;
+  p->dbgR = a.dbg.R; p->dbgN = a.dbg.N; p->dbgW = a.dbg.W_pre; p->dbgNb = a.dbg.N_b;
   p->nb = w.Nb;
   p->ldmv = a.ldmv; p->ldw = a.W.ld; p->ldn = w.ldn;
   p->m = (int32_t)a.m; p->n = (int32_t)a.n; p->r = (int32_t)a.r;
@@ -1207,9 +1213,16 @@ int sm_count() {
   return n;
 }
 
+// Opts a kernel instance into its dynamic shared memory, once per device and instance (`done` is the calling
+// launcher's own flag array, one launcher per instance).
 template <class K>
-int set_smem(K kernel, int bytes) {
+int set_smem_once(K kernel, int bytes, bool* done) {
+  int dev = 0;
+  QG_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QG_UNSUPPORTED_SHAPE;
+  if (done[dev]) return QG_OK;
   QG_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  done[dev] = true;
   return QG_OK;
 }
 
@@ -1222,7 +1235,8 @@ int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedul
               int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
   using S = K1Smem<BN, CTAS>;
   auto kern = project_adam_kernel<BN, SINGLE, CTAS, S8>;
-  int rc = set_smem(kern, S::kBytes);
+  static bool smem_set[64] = {};
+  int rc = set_smem_once(kern, S::kBytes, smem_set);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
   const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
@@ -1251,7 +1265,8 @@ int launch_k2(const TcProblem* single, const TcProblem* table, const TileSchedul
               int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
   using S = typename std::conditional<CTAS == 2, K2PairSmem, K2Smem>::type;
   auto kern = backproject_sr_kernel<SINGLE, CTAS>;
-  int rc = set_smem(kern, S::kBytes);
+  static bool smem_set[64] = {};
+  int rc = set_smem_once(kern, S::kBytes, smem_set);
   if (rc != QG_OK) return rc;
   const int sms = sm_count();
   const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
@@ -1460,6 +1475,14 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     ch.k1_pairs = (g_pair_mode & 2) && ch.bn == 256;
     for (int k = i; k < j && ch.k1_pairs; ++k)
       if (items[k].r % 256 != 0) ch.k1_pairs = 0;
+    // the back-projection runs as CTA pairs when asked to, unless the chunk holds a right-hand item (the paired
+    // kernel knows the left form only); decided here, before the tile lists are made, because the lists of the
+    // two forms differ (tiles of 256 rows against tiles of 128)
+    ch.pairs = g_pair_mode & 1;
+    for (int k = i; k < j; ++k) {
+      if (items[k].right) ch.pairs = 0;
+      if (items[k].state8) ch.state8 = 1;
+    }
     size_t off = 0;
     std::vector<int2> t1, t2;
     std::vector<float> c1, c2;
@@ -1476,7 +1499,7 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       const int k1n = ch.k1_pairs ? probs[k].k1p_tiles : probs[k].k1_tiles;
       for (int t = 0; t < k1n; ++t) { t1.push_back(make_int2(k - i, t)); c1.push_back((float)ceil_div(proj_rows(a), kBK) + 6.f); }
       ch.k1p_tiles += probs[k].k1p_tiles;
-      const int k2n = (g_pair_mode & 1) ? probs[k].k2p_tiles : probs[k].k2_tiles;
+      const int k2n = ch.pairs ? probs[k].k2p_tiles : probs[k].k2_tiles;
       for (int t = 0; t < k2n; ++t) { t2.push_back(make_int2(k - i, t)); c2.push_back((float)ceil_div(a.r, kBK) + 6.f); }
       ch.k2p_tiles += probs[k].k2p_tiles;
       dq[k].P = a.P; dq[k].out = w.Pt;
@@ -1487,11 +1510,6 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     }
     if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
     else ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
-    ch.pairs = g_pair_mode & 1;
-    for (int k = i; k < j; ++k) {
-      if (items[k].right) ch.pairs = 0;              // the paired back-projection knows the left form only
-      if (items[k].state8) ch.state8 = 1;
-    }
     if (ch.pairs) ch.k2_grid = 2 * (ch.k2p_tiles < sm_count() / 2 ? ch.k2p_tiles : sm_count() / 2);   // CTA pairs
     else ch.k2_grid = ch.k2_tiles < sm_count() ? ch.k2_tiles : sm_count();
     schedule_tiles(t1, c1, ch.k1_pairs ? ch.k1_grid / 2 : ch.k1_grid, sched, &ch.k1_start_off, &ch.k1_items_off);

@@ -123,6 +123,24 @@ class GradientModel:
         return to_bf16_bits(g)
 
 
+    def sample_columns(self, step: int, a: int, b: int, width: int = 256) -> np.ndarray:
+        """Columns [a, b) of a gradient whose noise is drawn per block of ``width`` columns, each block from its
+        own stream (seed, matrix, step, block): any column range costs only its own blocks, and the full matrix
+        ``sample_columns(step, 0, n)`` is the concatenation of the ranges.  (A different gradient than
+        ``sample(step)``, with the same model; used where only a few column blocks of a large matrix are needed
+        at most steps.)  ``a`` must be a multiple of ``width``."""
+        assert a % width == 0 and 0 <= a < b <= self.n
+        sig_u = (self.U * self.sigma[None, :]).astype(np.float32)
+        out = np.empty((self.m, b - a), np.uint16)
+        for c0 in range(a, b, width):
+            cw = min(width, self.n - c0)                # the whole block is formed, then cut: the same arithmetic
+            z = _rng(self.seed, self.index, 5, step, c0 // width).standard_normal((self.m, cw), dtype=np.float32)
+            g = to_bf16_bits(sig_u @ self.V[c0:c0 + cw].T.astype(np.float32) + np.float32(NOISE_STD) * z)
+            c1 = min(c0 + cw, b)
+            out[:, c0 - a:c1 - a] = g[:, :c1 - c0]
+        return out
+
+
 def initial_weight(m: int, n: int, seed: int = 0, matrix_index: int = 0) -> np.ndarray:
     """fp32 W0 ~ N(0, 0.02^2); the caller quantizes it."""
     return (_rng(seed, matrix_index, 3).standard_normal((m, n), dtype=np.float32) * np.float32(WEIGHT_STD))

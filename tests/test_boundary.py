@@ -102,3 +102,22 @@ def test_gate_rejects_bad_arguments():
     assert L.qgalore_gate_update(0.5, 0.4, 2, None, hist, C.byref(cnt)) == B.QG_INVALID_ARGUMENT
     cnt = C.c_int32(5)
     assert L.qgalore_gate_update(0.5, 0.4, 2, C.byref(iv), hist, C.byref(cnt)) == B.QG_INVALID_ARGUMENT
+
+
+def test_both_similarity_entry_points_apply_the_same_pointer_rules():
+    # host-only: nothing is dereferenced, every call is refused before a launch
+    L = B.lib()
+    small = lambda scales=0x2000, zeros=0x3000: B._CQTensor(0x1000, scales, zeros, 64, 256, 256, 4, 256)
+    ok, bad_s, bad_z = small(), small(scales=0x2002), small(zeros=0x3001)
+    for fn, extra in ((L.qgalore_subspace_similarity_static, ()), (L.qgalore_subspace_similarity, (0x8000, 1 << 20))):
+        assert fn(C.byref(bad_s), C.byref(ok), 0, 0x4000, *extra, None) == B.QG_MISALIGNED
+        assert fn(C.byref(ok), C.byref(bad_z), 0, 0x4000, *extra, None) == B.QG_MISALIGNED
+        assert fn(C.byref(ok), C.byref(ok), 0, 0x4002, *extra, None) == B.QG_MISALIGNED
+        assert fn(C.byref(ok), C.byref(small()), 0, None, *extra, None) == B.QG_INVALID_ARGUMENT
+
+
+def test_wait_expiry_aid_validates_on_the_host():
+    L = B.lib()
+    assert L.qgalore_debug_expire_wait(0, 0x1000, None, None) == B.QG_INVALID_ARGUMENT
+    assert L.qgalore_debug_expire_wait(8, None, None, None) == B.QG_INVALID_ARGUMENT
+    assert L.qgalore_debug_expire_wait(8, 0x1002, None, None) == B.QG_MISALIGNED

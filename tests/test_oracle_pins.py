@@ -17,6 +17,38 @@ from paper_2407_08296_b200 import synth
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
 
+# ----------------------------------------------------------------------------- bfloat16 rounding
+def test_bf16_rounding_is_nearest_with_ties_to_even():
+    """The rounding point the step crosses twice (P~ and N_b).  bfloat16 keeps the top 16 bits of a binary32;
+    hand-made cases: exact values stay; 1 + 2^-8 lies midway between 0x3F80 and 0x3F81 and goes to the even
+    one, 0x3F80; 1 + 3 * 2^-8 lies midway between 0x3F81 and 0x3F82 and goes to 0x3F82 (truncation would give
+    0x3F81, round-half-up would give 0x3F81 for the first); just above and below a midpoint; negative values
+    mirror; the largest binary32 below 2 rounds up into the next binade.  Then torch's own conversion on
+    random values and on every midpoint of one binade."""
+    import torch
+    cases = [
+        (1.0, 0x3F80), (1.0 + 2.0 ** -7, 0x3F81), (-2.5, 0xC020), (0.0, 0x0000),
+        (1.0 + 2.0 ** -8, 0x3F80), (1.0 + 3 * 2.0 ** -8, 0x3F82),
+        (1.0 + 2.0 ** -8 + 2.0 ** -23, 0x3F81), (1.0 + 2.0 ** -8 - 2.0 ** -23, 0x3F80),
+        (-(1.0 + 2.0 ** -8), 0xBF80), (-(1.0 + 3 * 2.0 ** -8), 0xBF82),
+        (2.0 - 2.0 ** -23, 0x4000), (3.0e-3, 0x3B45),     # 3.0e-3 = 0x3B449BA6 in binary32: low half above 0x8000, up
+    ]
+    for value, bits in cases:
+        x = np.array([value], np.float32)
+        assert int(O.f32_to_bf16_bits(x)[0]) == bits, (value, hex(int(O.f32_to_bf16_bits(x)[0])))
+        assert int(synth.to_bf16_bits(x)[0]) == bits
+        back = O.bf16_round(x)
+        assert back.dtype == np.float32 and back.view(np.uint32)[0] == bits << 16
+        assert O.bf16_bits_to_f32(np.array([bits], np.uint16)).view(np.uint32)[0] == bits << 16
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(200000).astype(np.float32) * np.float32(s) for s in (1.0, 1e-3, 1e-20, 1e20)])
+    mids = ((np.arange(0x3F80, 0x4000, dtype=np.uint32) << np.uint32(16)) | np.uint32(0x8000)).view(np.float32)
+    x = np.concatenate([x, mids, -mids])
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(O.f32_to_bf16_bits(x), want)
+    assert np.array_equal(synth.to_bf16_bits(x), want)
+
+
 # ----------------------------------------------------------------------------- Philox
 def _kat_rows():
     rows = []

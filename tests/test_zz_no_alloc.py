@@ -50,3 +50,11 @@ def test_static_similarity_refuses_what_does_not_fit():
     q = B._CQTensor(0x1000, 0x2000, 0x3000, rows, cols, cols, 4, 256)       # never dereferenced: rejected on the host
     assert L.qgalore_subspace_similarity_static(C.byref(q), C.byref(q), 0, 0x4000, None) == B.QG_WORKSPACE_TOO_SMALL
     assert L.qgalore_subspace_similarity_static(None, C.byref(q), 0, 0x4000, None) == B.QG_INVALID_ARGUMENT
+    # the same pointer rules as the workspace-taking entry point, checked on the host: scales, zero points and the
+    # result word are read and written as 4-byte words
+    small = lambda scales=0x2000, zeros=0x3000: B._CQTensor(0x1000, scales, zeros, 64, 256, 256, 4, 256)
+    ok, bad_s, bad_z = small(), small(scales=0x2002), small(zeros=0x3001)
+    for fn, extra in ((L.qgalore_subspace_similarity_static, ()), (L.qgalore_subspace_similarity, (0x8000, 1 << 20))):
+        assert fn(C.byref(bad_s), C.byref(ok), 0, 0x4000, *extra, None) == B.QG_MISALIGNED
+        assert fn(C.byref(ok), C.byref(bad_z), 0, 0x4000, *extra, None) == B.QG_MISALIGNED
+        assert fn(C.byref(ok), C.byref(ok), 0, 0x4002, *extra, None) == B.QG_MISALIGNED
