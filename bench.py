@@ -6,6 +6,9 @@ add, stochastic-rounding requantization) over every 2-D attention/MLP matrix of 
 Prints ONE JSON line: weight elements updated per second, with the per-step roofline, the end-to-end
 figure (gradients copied from pinned host memory every step) and the CPU oracle timed beside it.
 
+With no --workload the run times BOTH stacks the target is set on: LLaMA-7B (the largest single-GPU
+configuration; the top-level keys of the line) and then LLaMA-1B (the same block under "also": {"llama1b": ...}).
+
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama1b|llama7b|...] [--impl reference]
 """
 from __future__ import annotations
@@ -83,14 +86,23 @@ def k2_alu_ops(m, n, r):
     return float(K2_ALU_OPS_PER_ELEMENT) * m * n
 
 
-# DRAM bytes per launch of the kernels from the committed ncu capture (profiles/), per weight element of
-# the captured launch, so that it scales to the launches timed here.  None = no valid capture for the
-# kernels as they stand.
-NCU_TRAFFIC_PER_ELEMENT = {
-    # profiles/project_adam_and_backproject_sr_llama1b_4layers.md: 1215.4, 526.7 and 51.3 MB over 201.3 M elements
-    "llama1b": {"project_adam": 1215.4e6 / 201.3184e6, "backproject_sr": 526.7e6 / 201.3184e6,
-                "dequant_p_grouped": 51.3e6 / 201.3184e6},
-}
+def load_ncu_traffic(kernel_revision):
+    """DRAM bytes per weight element of each kernel, per workload, from the ncu captures summarised under
+    profiles/ (read from the small table beside them).  A row counts only if it was taken on the kernels as they
+    stand: its revision tag must equal the one the library reports.  Returns {workload: {kernel: bytes/element}}."""
+    table = {}
+    path = os.path.join(ROOT, "profiles", "dram_traffic_per_element.txt")
+    if not os.path.exists(path):
+        return table
+    with open(path) as f:
+        for line in f:
+            f4 = line.split()
+            if len(f4) < 4 or line.startswith("#"):
+                continue
+            workload, kernel, per_element, revision = f4[0], f4[1], float(f4[2]), f4[3]
+            if revision == kernel_revision:
+                table.setdefault(workload, {})[kernel] = per_element
+    return table
 
 
 def stack_roofline(specs, peaks):
@@ -180,14 +192,16 @@ def oracle_sample(workload, steps, warmup):
             out = O.project_step(g, P, W, M, V, O.Hyper(step=it + 1, seed=1))
             dt = time.perf_counter() - t0
             W, M, V = out["W"], out["M"], out["V"]
-            if it >= warmup:
+            if it >= warmup or dt > 2.0:
                 best = dt if best is None else min(best, dt)
+            if dt > 2.0:                                  # a 7B-sized matrix: one step is the bounded sample
+                break
         per_step += best * count
         elements += m * n * count
         detail.append(f"{m}x{n} r{r}: {best:.3f}s x{count}")
     return (elements / per_step, per_step,
-            f"best of {steps} oracle steps (after {warmup} warm-up) on one matrix of each distinct shape, extrapolated by "
-            "shape counts (" + "; ".join(detail) + ")")
+            f"best of up to {steps} oracle steps (after {warmup} warm-up; a single step where one takes over 2 s) on one matrix "
+            "of each distinct shape, extrapolated by shape counts (" + "; ".join(detail) + ")")
 
 
 def blas_threads():
@@ -203,6 +217,7 @@ def run_reference(args):
     if rank != 0:
         return
     steps = max(1, min(args.steps, 2))
+    args.workload = args.workload or "llama7b"
     value, per_step, sample = oracle_sample(args.workload, steps, 0 if args.warmup == 0 else 1)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -348,31 +363,17 @@ def time_refresh(items, device):
     out["concurrent"] = {"streams": streams, "matrices": batch, "sequential_ms": times[0], "concurrent_ms": times[1],
                          "device_status": int(status.item())}
     out["stack_seconds_concurrent"] = total * times[1] / max(times[0], 1e-9)
+    out["stack_seconds_best"] = min(out["stack_seconds"], out["stack_seconds_concurrent"])
     return out
 
 
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
-    from paper_2407_08296_b200 import binding as B
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the Q-GaLore step has no CPU path")
-    torch.cuda.set_device(local_rank)
-    device = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=device)
-    B.lib()                                                    # fail loudly if the library is missing
-    peaks, peak_kind = load_peaks()
-
-    # every rank holds and steps its own replica of the stack: matrices are independent units, no collective
+def bench_workload(workload, args, B, torch, dist, device, world, rank, local_rank, peaks, peak_kind, extras):
+    """Times one stack and returns the keys of its result block (rank 0; None elsewhere)."""
+    from paper_2407_08296_b200.synth_device import build_stack
     global MOMENT_BYTES
     MOMENT_BYTES = 4.5 if args.moments == 8 else 16.0
-    from paper_2407_08296_b200.synth_device import build_stack
-    specs, items = build_stack(args.workload, device, seed=rank, layers=args.layers, moments=args.moments)
+    # every rank holds and steps its own replica of the stack: matrices are independent units, no collective
+    specs, items = build_stack(workload, device, seed=rank, layers=args.layers, moments=args.moments)
     batch = B.StepPlan(items)
     elements = batch.elements
     hyper = B.Hyper(rounding=B.QG_ROUND_NEAREST if args.rounding == "nearest" else B.QG_ROUND_STOCHASTIC)
@@ -458,8 +459,9 @@ def run_ours(args):
     del host_g, alt_g, plan_alt, plans, gsets
 
     # ---- per-kernel device time: a second pass of the same steps with an event pair around every launch
-    kms = [0.0, 0.0, 0.0]
-    kcount = [0, 0, 0]
+    names = list(B.STEP_KERNEL_NAMES)
+    kms = [0.0] * len(names)
+    kcount = [0] * len(names)
     for _ in range(args.steps):
         step_no += 1
         hyper.step = step_no
@@ -468,24 +470,26 @@ def run_ours(args):
         kcount = [a + b for a, b in zip(kcount, c3)]
     barrier()
 
+    block = None
     if rank == 0:
         t_roof, flops, nbytes = stack_roofline(specs, peaks)
         t_roof_nom, _, _ = stack_roofline(specs, NOMINAL)
         t_c = flops / (peaks["bf16_tflops"] * 1e12)
         t_m = nbytes / (peaks["hbm_gbs"] * 1e9)
         sec = ms_per_step * 1e-3
-        # roofline of every kernel from its live-measured duration: the bound is the slowest of the tensor
-        # pipe (sustained bf16 peak: the kernels are timed inside a long step), HBM (copy peak) and, for the
-        # requantizing epilogue, the plain ALUs (lanes x SMs x the maximum SM clock)
-        names = ["dequant_p_grouped", "project_adam", "backproject_sr"]
-        units = [dq_units, k1_units, k2_units]
-        peak_tf = peaks["bf16_tflops_sustained"]
+        # roofline of every kernel from its live-measured duration: the bound is the slowest of the tensor pipe
+        # (burst bf16 peak: the primary denominator; the sustained figure is reported beside it), HBM (copy
+        # peak) and, for the requantizing epilogue, the plain ALUs (lanes x SMs x the maximum SM clock)
+        units = {"dequant_p_grouped": dq_units, "project_adam": k1_units, "backproject_sr": k2_units}
+        peak_tf, peak_tf_sus = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
         sm_mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
         alu_peak = torch.cuda.get_device_properties(device).multi_processor_count * ALU_LANES_PER_SM_CLOCK * sm_mhz * 1e6
         per_kernel = {}
         for k, nm in enumerate(names):
-            kf = sum(units[k](sp.m, sp.n, sp.r)[0] for sp in specs) * args.steps
-            kb = sum(units[k](sp.m, sp.n, sp.r)[1] for sp in specs) * args.steps
+            if kcount[k] == 0:
+                continue
+            kf = sum(units[nm](sp.m, sp.n, sp.r)[0] for sp in specs) * args.steps
+            kb = sum(units[nm](sp.m, sp.n, sp.r)[1] for sp in specs) * args.steps
             ko = sum(k2_alu_ops(sp.m, sp.n, sp.r) for sp in specs) * args.steps if nm == "backproject_sr" else 0.0
             ksec = max(kms[k] * 1e-3, 1e-12)
             cand = {"tensor": (kf / (peak_tf * 1e12), kf / ksec / 1e12, peak_tf, "TFLOP/s"),
@@ -494,52 +498,62 @@ def run_ours(args):
             bound = max(cand, key=lambda c: cand[c][0])
             per_kernel[nm] = {"bound": bound, "achieved": cand[bound][1], "peak": cand[bound][2], "unit": cand[bound][3],
                               "frac": cand[bound][1] / cand[bound][2], "ms_per_step": kms[k] / args.steps,
+                              "launches_per_step": kcount[k] / args.steps,
                               "bound_ms_per_step": {c: cand[c][0] * 1e3 / args.steps for c in cand},
                               "flops": kf / args.steps, "bytes": kb / args.steps, "alu_ops": ko / args.steps}
-        dom = max(range(3), key=lambda k: kms[k])
-        k_flops = per_kernel[names[dom]]["flops"] * args.steps
-        k_bytes = per_kernel[names[dom]]["bytes"] * args.steps
-        roof = {key: per_kernel[names[dom]][key] for key in ("bound", "achieved", "peak", "unit")}
+            if bound == "tensor":
+                per_kernel[nm]["frac_of_sustained_peak"] = cand[bound][1] / peak_tf_sus
+        # the dominant kernel is named by what the shapes demand, not by a timing: the one whose own bound is largest
+        dom_name = max(per_kernel, key=lambda nm: max(per_kernel[nm]["bound_ms_per_step"].values()))
+        dom = names.index(dom_name)
+        k_flops = per_kernel[dom_name]["flops"] * args.steps
+        k_bytes = per_kernel[dom_name]["bytes"] * args.steps
+        roof = {key: per_kernel[dom_name][key] for key in ("bound", "achieved", "peak", "unit")}
         roof["frac"] = roof["achieved"] / roof["peak"]
-        tpe = NCU_TRAFFIC_PER_ELEMENT.get(args.workload, {}).get(names[dom]) if args.moments == 32 else None
+        if roof["bound"] == "tensor":
+            roof["frac_of_sustained_peak"] = roof["achieved"] / peak_tf_sus
+            roof["sustained_peak"] = peak_tf_sus
+        traffic = extras["traffic"].get(workload, {}) if (args.moments == 32 and not args.layers) else {}
+        tpe = traffic.get(dom_name)
         roof["traffic"] = None if tpe is None else tpe * elements * args.steps / max(kcount[dom], 1)
-        roof["kernel"] = names[dom]
+        roof["traffic_per_kernel_per_launch"] = {nm: (traffic[nm] * elements * args.steps / max(kcount[names.index(nm)], 1))
+                                                 for nm in per_kernel if nm in traffic} or None
+        roof["kernel"] = dom_name
+        roof["kernel_revision"] = extras["revision"]
         roof["launches"] = kcount[dom]
         roof["avg_launch_ms"] = kms[dom] / max(kcount[dom], 1)
         roof["algorithmic_bytes_per_launch"] = k_bytes / max(kcount[dom], 1)
         roof["algorithmic_flops_per_launch"] = k_flops / max(kcount[dom], 1)
-        roof["peak_source"] = {"tensor": peak_kind + " (sustained bf16)", "hbm": peak_kind + " (copy)",
+        roof["peak_source"] = {"tensor": peak_kind + " (burst bf16; sustained beside it)", "hbm": peak_kind + " (copy)",
                                "alu": "derived: SMs x 128 lanes x maximum SM clock"}[roof["bound"]]
         roof["per_kernel"] = per_kernel
         roof["timing"] = "separate pass of the same steps with a CUDA event pair around every launch"
-        roof["kernel_ms_per_step"] = {nm: kms[k] / args.steps for k, nm in enumerate(names)}
-        roof["kernel_share"] = {nm: kms[k] / max(sum(kms), 1e-12) for k, nm in enumerate(names)}
-        sec = ms_per_step * 1e-3
-        kernel_bound_ms = sum(max(per_kernel[nm]["bound_ms_per_step"].values()) for nm in names)
+        roof["kernel_ms_per_step"] = {nm: kms[k] / args.steps for k, nm in enumerate(names) if kcount[k]}
+        roof["kernel_share"] = {nm: kms[k] / max(sum(kms), 1e-12) for k, nm in enumerate(names) if kcount[k]}
+        kernel_bound_ms = sum(max(per_kernel[nm]["bound_ms_per_step"].values()) for nm in per_kernel)
         roof["whole_step"] = {"per_matrix_roofline_ms": t_roof * 1e3, "frac_of_per_matrix_roofline": t_roof / sec,
                               "frac_of_nominal_roofline": t_roof_nom / sec,
                               "bound": "tensor" if t_c >= t_m else "hbm",
                               "achieved_tflops": flops / sec / 1e12, "achieved_gbs": nbytes / sec / 1e9,
-                              # the three kernels run one after the other: the sum of their own bounds (each the
-                              # slowest of its tensor, HBM and ALU time) is what this design can reach at best
+                              # the kernels run one after the other: the sum of their own bounds (each the slowest
+                              # of its tensor, HBM and ALU time) is what such a design can reach at best
                               "sum_of_kernel_rooflines_ms": kernel_bound_ms,
                               "frac_of_sum_of_kernel_rooflines": kernel_bound_ms / ms_per_step}
         refresh = None if args.no_refresh else time_refresh(items, device)
         if refresh is not None:
             # the step and the refresh blended at the base interval of Sec. 4.1 (a refresh every 200 steps)
-            refresh["blended_ms_per_step_at_interval_200"] = ms_per_step + refresh["stack_seconds_concurrent"] * 1e3 / 200.0
+            refresh["blended_ms_per_step_at_interval_200"] = ms_per_step + refresh["stack_seconds_best"] * 1e3 / 200.0
         linear = time_linear(items, device, args.linear_tokens, peaks["bf16_tflops"]) if args.linear_tokens > 0 else None
         cpu = None
         if not args.no_cpu_baseline:
-            v, per_step, sample = oracle_sample(args.workload, 3, 1)
+            v, per_step, sample = oracle_sample(workload, 3, 1)
             cpu = {"value": v, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample,
                    "host_cpus": os.cpu_count()}
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": args.workload + (f"[first {args.layers} layers]" if args.layers else ""), "matrices": len(specs), "elements_per_step": elements,
-                       "rank": specs[0].r, "group": 256, "rounding": args.rounding, "moments_bits": args.moments, "l2": "inputs larger than L2 (whole stack streams each step)",
+        block = {
+            "value": value, "unit": UNIT, "ms_per_step": ms_per_step,
+            "config": {"workload": workload + (f"[first {args.layers} layers]" if args.layers else ""), "matrices": len(specs),
+                       "elements_per_step": elements, "rank": specs[0].r, "group": 256, "rounding": args.rounding,
+                       "moments_bits": args.moments, "l2": "inputs larger than L2 (whole stack streams each step)",
                        "parallelism": f"replica per GPU x{world}, no collective"},
             "roofline": roof, "cpu_baseline": cpu,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 4,
@@ -547,6 +561,45 @@ def run_ours(args):
             "gpu_launches": launches, "clocks": clocks, "device_status": status, "refresh": refresh,
             "int8_linear": linear,
         }
+    batch.close()
+    del batch, items
+    torch.cuda.empty_cache()
+    return block
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2407_08296_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the Q-GaLore step has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    B.lib()                                                    # fail loudly if the library is missing
+    peaks, peak_kind = load_peaks()
+    revision = B.kernel_revision()
+    extras = {"traffic": load_ncu_traffic(revision), "revision": revision}
+
+    # both target stacks unless one is asked for: the largest single-GPU configuration first (top level of the
+    # line), the other under "also"
+    workloads = [args.workload] if args.workload else ["llama7b", "llama1b"]
+    blocks = [bench_workload(w, args, B, torch, dist, device, world, rank, local_rank, peaks, peak_kind, extras)
+              for w in workloads]
+    if rank == 0:
+        top = blocks[0]
+        line = {"metric": METRIC, "value": top["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": top["ms_per_step"], "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic"}
+        line.update({k: v for k, v in top.items() if k not in ("value", "unit", "ms_per_step")})
+        if len(blocks) > 1:
+            line["also"] = {w: b for w, b in zip(workloads[1:], blocks[1:])}
+            line["gpu_launches"] = sum(b["gpu_launches"] for b in blocks)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -557,7 +610,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="llama1b")
+    ap.add_argument("--workload", default=None,
+                    help="llama7b | llama1b | llama350m | llama130m | llama60m_mlp; default: llama7b, then llama1b under 'also'")
     ap.add_argument("--no-refresh", action="store_true", help="skip the separate timing of the subspace refresh")
     ap.add_argument("--linear-tokens", type=int, default=8192,
                     help="rows of activations for the separate timing of the INT8 linear layer's GEMMs (0: skip)")

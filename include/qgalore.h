@@ -306,6 +306,9 @@ QG_API size_t qgalore_workspace_bytes(int op, int64_t m, int64_t n, int64_t r);
 QG_API const char* qgalore_status_string(int status);
 /* Text of the last CUDA error this thread met inside the library ("" if none). */
 QG_API const char* qgalore_last_cuda_error(void);
+/* A tag that changes whenever the kernels of the optimizer step change in a way that can move their memory traffic
+ * or timing; profiler figures taken on one revision are not quoted for another. */
+QG_API const char* qgalore_kernel_revision(void);
 /* Number of kernels the library has launched from this process (for launch accounting). */
 QG_API uint64_t qgalore_launch_count(void);
 /* --- Test aids.  Declared only when QGALORE_TEST_API is defined before this header is included: they are

@@ -107,6 +107,7 @@ def lib() -> C.CDLL:
         L.qgalore_status_string.restype = C.c_char_p
         L.qgalore_last_cuda_error.restype = C.c_char_p
         L.qgalore_launch_count.restype = C.c_uint64
+        L.qgalore_kernel_revision.restype = C.c_char_p
         L.qgalore_debug_set_step_impl.argtypes = [C.c_int]
         L.qgalore_debug_set_pair_mode.argtypes = [C.c_int]
         L.qgalore_debug_set_chunk_budget.argtypes = [sz]
@@ -213,6 +214,14 @@ class Hyper:
 
 def workspace_bytes(op: int, m: int, n: int, r: int) -> int:
     return int(lib().qgalore_workspace_bytes(op, m, n, r))
+
+
+# kernels of one plan step, in the order qgalore_plan_step_timed reports them
+STEP_KERNEL_NAMES = ("dequant_p_grouped", "project_adam", "backproject_sr")
+
+
+def kernel_revision() -> str:
+    return lib().qgalore_kernel_revision().decode()
 
 
 def launch_count() -> int:

@@ -61,6 +61,7 @@ const char* qgalore_status_string(int status) {
 }
 
 const char* qgalore_last_cuda_error(void) { return g_last_error; }
+const char* qgalore_kernel_revision(void) { return QG_STEP_KERNELS_REVISION; }
 uint64_t qgalore_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 static int quantize_common(int bits, const float* src, int64_t rows, int64_t cols, int64_t ld_src,
