@@ -322,6 +322,11 @@ QG_API int qgalore_debug_set_step_impl(int impl);
  * chunk is a multiple of 256).  0 = one CTA per 128 x 256 tile; the default is 2.  Every setting gives the same
  * results bit for bit. */
 QG_API int qgalore_debug_set_pair_mode(int mask);
+/* 1: the projection kernel converts the INT4 codes of P inside its main loop (converter warps write the bf16
+ * operand tile straight into shared memory); 0 (the default, the faster arrangement as measured): P is dequantized
+ * to bf16 by a separate grouped launch first, as for 2- and 8-bit codes.  Applies to calls and plans made
+ * afterwards; the results are the same bit for bit. */
+QG_API int qgalore_debug_set_fused_dequant(int on);
 /* Scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks mean
  * fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
 QG_API int qgalore_debug_set_chunk_budget(size_t bytes);

@@ -10,10 +10,11 @@
 //                         thread of the epilogue owns one accumulator row, so the group minimum and
 //                         maximum are thread-local.
 //
-// Warp roles: one TMA producer thread, one MMA issuer thread, (first kernel only) one loader thread
-// for the M/V chunks, and four epilogue warps that read the accumulator with tcgen05.ld.  The
-// accumulator is double buffered in tensor memory, so the epilogue of a tile overlaps the main
-// loop of the next one.  Everything global the epilogue touches goes through shared memory in the
+// Warp roles: one TMA producer thread, one MMA issuer thread, epilogue warps that read the accumulator with
+// tcgen05.ld and, in the first kernel, two converter warps that turn the INT4 codes of the projection matrix
+// into the bf16 operand tile inside shared memory (Sec. 3.3: the projection is stored in INT4 and dequantized
+// where it is used).  The accumulator is double buffered in tensor memory, so the epilogue of a tile overlaps
+// the main loop of the next one.  Everything global the epilogue touches goes through shared memory in the
 // 128-byte TMA swizzle: a thread reads/writes its own row with 16-byte accesses without bank
 // conflicts, and global traffic stays fully coalesced.
 //
@@ -83,6 +84,15 @@ struct alignas(64) TcProblem {
   int32_t state8, nsb;
   float* m_scale;
   float* v_scale;
+  // The projection's A operand converted in the kernel: the INT4 codes, scales and zero points of the projection
+  // matrix (row pitch in bytes, groups per row) and where the bf16 copy for the back-projection goes.  fuse_a = 0
+  // (2- or 8-bit codes, a rank that is not a multiple of 128): the tile comes by TMA from a bf16 copy made beforehand.
+  const uint8_t* p_codes;
+  const float* p_scales;
+  const float* p_zeros;
+  uint16_t* pt;
+  int64_t p_row_bytes;
+  int32_t p_ngroups, fuse_a;
   int32_t r_whole, n_whole;            // r, n rounded down to whole 64-column chunks (extent of the 3-D views)
   uint32_t seed_lo, seed_hi;           // stochastic-rounding key of this matrix
   int32_t k1_rblocks, k1_tiles;
@@ -150,7 +160,8 @@ struct K1Smem {
   static constexpr int kMvOffset = kStages * kStageBytes;
   static constexpr int kBarOffset = kMvOffset + kMvBytes;
   static constexpr int kBytes = kBarOffset + 512 + 1024;   // barriers + slack for 1024-byte alignment
-  static constexpr int kThreads = 64 + kEpiWarps * 32;
+  static constexpr int kConvWarps = 2;                      // one thread per K row of a stage converts 128 codes
+  static constexpr int kThreads = 64 + kEpiWarps * 32 + kConvWarps * 32;
 };
 
 // The Adam update of Sec. 3.5: M <- b1 M + (1-b1) R, V <- b2 V + (1-b2) R^2,
@@ -170,6 +181,43 @@ __device__ __forceinline__ float2 adam2(const AdamConsts& c, float2 r, float2& m
   return make_float2(__fdividef(m.x, den.x), __fdividef(m.y, den.y));
 }
 
+// One K row of the projection's A tile: 128 INT4 codes (64 bytes, `c`) of row `ct` of a stage -> bf16((q - z) * s)
+// in the 128-byte-swizzled MN-major layout (`sA` = the row's base in the stage: two 64-column slabs of 8 KB, the
+// 16-byte piece p of a row stored at p ^ (row % 8)), and, if `gout` is given, to the same row of the bf16 copy in
+// global memory.  FAST: the stored nibble (code + 8) is dropped into the mantissa of 2^23 and (2^23 + 8 + z)
+// subtracted: q - z exactly, without an integer-to-float conversion, for |z| < 2^22.
+template <bool FAST>
+__device__ __forceinline__ void convert_p_row(const uint4 (&c)[4], float s_cur, float z_cur, uint8_t* sA, int ct, uint16_t* gout) {
+  const float cz = 8388616.0f + z_cur;
+  const float2 mcz = make_float2(-cz, -cz), s2 = make_float2(s_cur, s_cur);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t w4[4] = {c[j].x, c[j].y, c[j].z, c[j].w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const uint32_t lo4 = w4[i] & 0x0F0F0F0Fu, hi4 = (w4[i] >> 4) & 0x0F0F0F0Fu;   // even and odd columns, one per byte
+      uint32_t o[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        float2 v;
+        if (FAST) {
+          v = mul2(add2(make_float2(__uint_as_float(__byte_perm(lo4, 0x4B000000u, 0x7650 + b)),
+                                    __uint_as_float(__byte_perm(hi4, 0x4B000000u, 0x7650 + b))), mcz), s2);
+        } else {
+          v.x = __fmul_rn(__fsub_rn((float)((int)((lo4 >> (8 * b)) & 0xFu) - 8), z_cur), s_cur);
+          v.y = __fmul_rn(__fsub_rn((float)((int)((hi4 >> (8 * b)) & 0xFu) - 8), z_cur), s_cur);
+        }
+        const __nv_bfloat162 h2 = __floats2bfloat162_rn(v.x, v.y);
+        o[b] = *reinterpret_cast<const uint32_t*>(&h2);
+      }
+      const uint4 out = make_uint4(o[0], o[1], o[2], o[3]);
+      // columns 32 j + 8 i .. + 7 of the rank block: slab j / 2, piece (j % 2) * 4 + i of the row
+      *reinterpret_cast<uint4*>(sA + (j >> 1) * kBoxBytes + (((((j & 1) << 2) + i) ^ (ct & 7)) << 4)) = out;
+      if (gout) *reinterpret_cast<uint4*>(gout + 32 * j + 8 * i) = out;
+    }
+  }
+}
+
 // The epilogue reads the accumulator in the 16-lane x 256-bit shape: thread t holds, per group of
 // eight columns, the column pair 2(t%4), 2(t%4)+1 of rows t/4 and t/4 + 8.  A quad of threads therefore
 // covers 32 contiguous bytes of a row of M, V (fp32): every global store of the epilogue writes whole
@@ -180,7 +228,8 @@ __device__ __forceinline__ float2 adam2(const AdamConsts& c, float2 r, float2& m
 template <int BN, bool SINGLE, int CTAS, bool S8 = false>
 __global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
-                    const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status) {
+                    const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status,
+                    const int conv_active) {
   static_assert(CTAS == 1 || (!SINGLE && BN == 256), "CTA pairs run from a plan, on 256-column tiles");
   using S = K1Smem<BN, CTAS>;
   const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;   // 0 = the pair's leader, which issues the MMAs
@@ -200,7 +249,13 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
   const TcProblem* probs = SINGLE ? &single : table;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < S::kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+    // a stage is full once the producer's copies have landed and, in a launch some matrix of which has its A tile
+    // converted in the kernel (conv_active), the converter warps (of both CTAs of a pair) have written, or waived,
+    // their part of it
+    for (int i = 0; i < S::kStages; ++i) {
+      mbar_init(&full[i], 1 + (conv_active ? CTAS * S::kConvWarps : 0));
+      mbar_init(&empty[i], 1);
+    }
     for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], CTAS * S::kEpiWarps); }
     for (int i = 0; i < S::kEpiWarps * S::kMvSlots; ++i) mbar_init(&mv_full[i], 1);
     fence_mbar_init();
@@ -241,6 +296,8 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         // whole-chunk tiles take one 3-D copy per operand; chunks past the end of a 3-D view read as zero
         const bool a3 = (p->r_whole == p->r) || (r0 + kTileM <= p->r_whole);
         const bool b3 = (p->n_whole == p->k1_n) || (n0 + BNC <= p->n_whole);
+        const bool fuse_a = p->fuse_a != 0;            // the converter warps write the A tile: nothing to copy
+        const uint32_t tx_bytes = fuse_a ? S::kBBytes : S::kStageBytes;
         // (An L2 prefetch of G a few K blocks ahead was tried and removed: the extra TMA instruction per K
         // block cost the single producer thread more than the hidden latency was worth.)
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -251,9 +308,10 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
           uint8_t* sB = sA + S::kABytes;
           if (CTAS == 2) {
             // the leader's barrier counts the bytes of both CTAs; every copy lands in the issuing CTA only
-            if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * S::kStageBytes);
+            if (rank == 0) mbar_arrive_expect_tx(&full[s], 2 * tx_bytes);
             const uint32_t lead_full = mapa_u32(smem_u32(&full[s]), 0);
-            if (a3) {
+            if (fuse_a) {
+            } else if (a3) {
               tma_load_3d_pair(sA, mapP3, lead_full, 0, kb * kBK, r0 / 64);
             } else {
 #pragma unroll
@@ -268,8 +326,9 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
               for (int h = 0; h < BNC / 64; ++h) tma_load_2d_pair(sB + h * kBoxBytes, mapG, lead_full, n0 + 64 * h, kb * kBK);
             }
           } else {
-            mbar_arrive_expect_tx(&full[s], S::kStageBytes);
-            if (a3) {
+            mbar_arrive_expect_tx(&full[s], tx_bytes);
+            if (fuse_a) {
+            } else if (a3) {
               tma_load_3d(sA, mapP3, &full[s], 0, kb * kBK, r0 / 64);
             } else {
 #pragma unroll
@@ -332,6 +391,93 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       }
       if (!ok) raise_wait_expired(status);
     }
+  } else if (warp >= 2 + S::kEpiWarps) {
+    // ------------------------------------------------------------------ converters: INT4 codes -> bf16 A tile
+    // P~ = bf16((q - z) * s) (App. A, the dequantization line) is formed here, K block by K block, straight in
+    // the 128-byte-swizzled MN-major operand layout: thread ct owns K row ct of the stage, i.e. row kb * 64 + ct
+    // of the projection matrix, and converts the 128 codes (64 bytes) of the tile's rank block: the stored nibble
+    // (code + 8) is dropped into the mantissa of 2^23 and (2^23 + 8 + z) subtracted, which gives q - z exactly
+    // without an integer-to-float conversion.  Codes, scale and zero point of the NEXT K block are fetched (from
+    // L2: the codes of a matrix are 1/4 the size of its bf16 form) before this one is converted.  The tiles of the
+    // first column block also write the converted rows to global memory, where the back-projection reads its
+    // K-major operand from.
+    // Off by default (conv_active = 0: these warps leave at once).  Measured on B200, LLaMA-1B shapes, one CTA per
+    // tile: 1.8 us per K block with the conversion against 0.8 us without.  The kernel is bound by how many bytes
+    // it keeps in flight, a stage now also waits for this warp's chain (wake-up, a load issued one K block
+    // earlier that takes about 1.5 us to return under the kernel's own traffic, 450 instructions, fence, arrive),
+    // and the global stores of the writer tiles delay their barrier arrivals; as CTA pairs the arrival on the
+    // leader's barrier is a cluster-scope release, about 1 us each.  The separate conversion launch costs 0.2 us
+    // per K block equivalent, so it stays the default until these warps take their codes through the copy
+    // engine several stages ahead.
+    const int ct = (int)threadIdx.x - (64 + S::kEpiWarps * 32);
+    struct Pos {
+      TileWalk<SINGLE> tw;
+      const TcProblem* p;
+      int kb, kblocks, r0;
+      bool writer;
+      __device__ Pos(const TileSchedule& sch, int total) : tw(sch, total), p(nullptr), kb(0), kblocks(0), r0(0), writer(false) {}
+    };
+    auto enter = [&](Pos& ps) {
+      if (!ps.tw.valid()) return;
+      const int2 item = ps.tw.cur();
+      ps.p = probs + item.x;
+      const int rblocks = CTAS == 2 ? ps.p->k1_rpairs : ps.p->k1_rblocks;
+      ps.r0 = (item.y % rblocks) * (CTAS * kTileM) + (int)rank * kTileM;
+      ps.writer = (item.y / rblocks) == 0;
+      ps.kblocks = (ps.p->k1_k + kBK - 1) / kBK;
+      ps.kb = 0;
+    };
+    auto fetch = [&](const Pos& ps, uint4 c[4], float& sc_, float& zp) {
+      c[0] = c[1] = c[2] = c[3] = make_uint4(0u, 0u, 0u, 0u);
+      sc_ = 0.f; zp = 0.f;                            // rows past the matrix convert to zero
+      if (!ps.tw.valid() || !ps.p->fuse_a) return;
+      const int64_t row = (int64_t)ps.kb * kBK + ct;
+      if (row >= ps.p->k1_k) return;
+      const uint4* src = reinterpret_cast<const uint4*>(ps.p->p_codes + row * ps.p->p_row_bytes + (ps.r0 >> 1));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) c[j] = __ldg(src + j);
+      const int64_t g = row * ps.p->p_ngroups + (ps.r0 >> 8);
+      sc_ = __ldg(ps.p->p_scales + g);
+      zp = __ldg(ps.p->p_zeros + g);
+    };
+    Pos pos(sched, total_tiles);
+    enter(pos);
+    uint4 cn[4];
+    float sn, zn;
+    fetch(pos, cn, sn, zn);
+    uint32_t it = 0;
+    bool ok = true;
+    while (conv_active && ok && pos.tw.valid()) {
+      const uint4 c[4] = {cn[0], cn[1], cn[2], cn[3]};
+      const float s_cur = sn, z_cur = zn;
+      const TcProblem* p = pos.p;
+      const int kb = pos.kb, r0 = pos.r0;
+      const bool writer = pos.writer;
+      if (++pos.kb >= pos.kblocks) { pos.tw.advance(); enter(pos); }
+      fetch(pos, cn, sn, zn);
+      const int s = it % S::kStages;
+      // the MMAs that read this stage are done; one lane polls, so that the warp does not crowd the barrier unit the
+      // copies and commits of the pipeline go through
+      if (lane == 0) ok = mbar_wait(&empty[s], ((it / S::kStages) & 1) ^ 1);
+      ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+      if (!ok) break;
+      if (p->fuse_a) {
+        uint8_t* sA = stage_base + s * S::kStageBytes + ct * 128;
+        const int64_t row = (int64_t)kb * kBK + ct;
+        uint16_t* gout = (writer && row < p->k1_k) ? p->pt + row * p->r + r0 : nullptr;
+        // the exact-by-construction fast form needs |z| < 2^22; a warp with a row outside that takes the plain form
+        if (__all_sync(0xFFFFFFFFu, fabsf(z_cur) < 4.0e6f)) convert_p_row<true>(c, s_cur, z_cur, sA, ct, gout);
+        else convert_p_row<false>(c, s_cur, z_cur, sA, ct, gout);
+        fence_proxy_async_smem();                        // the MMA reads these stores through the async proxy
+      }
+      __syncwarp();
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_cluster(mapa_u32(smem_u32(&full[s]), 0));
+        else mbar_arrive(&full[s]);
+      }
+      ++it;
+    }
+    if (!ok && lane == 0) raise_wait_expired(status);
   } else {
     // ------------------------------------------------------------------ epilogue: Adam on the tile
     const int q = warp & 3, hh = (warp - 2) >> 2;   // TMEM lane quarter of this warp, 16-lane half within it
@@ -1151,6 +1297,15 @@ TcScratch carve(void* base, int64_t m, int64_t n, int64_t r) {
 inline int64_t proj_rows(const StepArgs& a) { return a.right ? a.n : a.m; }
 inline int64_t state_cols(const StepArgs& a) { return a.right ? a.m : a.n; }
 
+// 1: the projection kernel converts the INT4 codes of P itself (converter warps); 0 (the default): P is
+// dequantized to bf16 by a separate grouped launch first.  Both give the same results bit for bit; measured on
+// B200 the separate launch is the faster arrangement (see the note at the converter warps).
+int g_fuse_dequant = 0;
+
+// The projection kernel converts the INT4 codes of P itself when a 128-wide rank block is whole and lies inside
+// one quantization group; other code widths (the ablation) and ragged ranks take the bf16 copy made beforehand.
+inline bool fused_dequant(const StepArgs& a) { return g_fuse_dequant && a.P.bits == 4 && a.r % kTileM == 0; }
+
 int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   memset(p, 0, sizeof(*p));
   bool ok = true;
@@ -1169,6 +1324,13 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   ok &= make_map(&p->mapQk, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, w.Pt, a.r, prow, a.r, 64, 256, CU_TENSOR_MAP_SWIZZLE_128B);
   p->r_whole = (int32_t)r_whole;
   p->n_whole = (int32_t)n_whole;
+  p->p_codes = reinterpret_cast<const uint8_t*>(a.P.codes);
+  p->p_scales = a.P.scales;
+  p->p_zeros = a.P.zeros;
+  p->pt = w.Pt;
+  p->p_row_bytes = a.P.ld / 2;
+  p->p_ngroups = (int32_t)ceil_div(a.r, kGroup);
+  p->fuse_a = fused_dequant(a) ? 1 : 0;
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
   if (a.state8) {
@@ -1232,7 +1394,7 @@ int choose_bn(int64_t tiles_at_256) { return tiles_at_256 >= 2 * (int64_t)sm_cou
 
 template <int BN, bool SINGLE, int CTAS, bool S8 = false>
 int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
-              int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st) {
+              int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st, int conv_active) {
   using S = K1Smem<BN, CTAS>;
   auto kern = project_adam_kernel<BN, SINGLE, CTAS, S8>;
   static bool smem_set[64] = {};
@@ -1242,7 +1404,7 @@ int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedul
   const int grid = SINGLE ? (total_tiles < sms ? total_tiles : sms) : grid_planned;
   static const TcProblem dummy{};
   if (CTAS == 1) {
-    kern<<<grid, S::kThreads, S::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status);
+    kern<<<grid, S::kThreads, S::kBytes, st>>>(single ? *single : dummy, table, sched, total_tiles, sc, status, conv_active);
   } else {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
@@ -1254,7 +1416,7 @@ int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedul
     attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    QG_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, dummy, table, sched, total_tiles, sc, status));
+    QG_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, dummy, table, sched, total_tiles, sc, status, conv_active));
   }
   QG_LAUNCH_CHECK();
   return QG_OK;
@@ -1294,57 +1456,86 @@ int launch_k2(const TcProblem* single, const TcProblem* table, const TileSchedul
 struct DequantItem {
   qg_qtensor P;
   uint16_t* out;
-  int32_t block0, nblocks;   // blocks of 256 threads, 32 columns per thread
+  int32_t block0, nblocks;   // blocks of 256 threads; a block converts kDqUnits * 256 units of 8 columns
 };
 
-// One thread converts 32 consecutive columns of a row (16 bytes of codes -> 64 bytes of bf16): the stored
-// nibble (code + 8) is dropped into the mantissa of 2^23 and (2^23 + 8 + z) subtracted, which gives q - z
-// exactly without an integer-to-float conversion.
+// Eight consecutive columns of a row: one 32-bit word of INT4 codes -> 16 bytes of bf16((q - z) * s).  FAST: the
+// stored nibble (code + 8) is dropped into the mantissa of 2^23 and (2^23 + 8 + z) subtracted, which gives q - z
+// exactly without an integer-to-float conversion (|z| < 2^22).
+template <bool FAST>
+__device__ __forceinline__ uint4 dequant8_int4(uint32_t w, float s, float z) {
+  const float c = 8388616.0f + z;
+  const float2 mc = make_float2(-c, -c), s2 = make_float2(s, s);
+  const uint32_t lo4 = w & 0x0F0F0F0Fu, hi4 = (w >> 4) & 0x0F0F0F0Fu;   // even and odd columns, one per byte
+  uint32_t o[4];
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    float2 v;
+    if (FAST) {
+      v = mul2(add2(make_float2(__uint_as_float(__byte_perm(lo4, 0x4B000000u, 0x7650 + b)),
+                                __uint_as_float(__byte_perm(hi4, 0x4B000000u, 0x7650 + b))), mc), s2);
+    } else {
+      v.x = __fmul_rn(__fsub_rn((float)((int)((lo4 >> (8 * b)) & 0xFu) - 8), z), s);
+      v.y = __fmul_rn(__fsub_rn((float)((int)((hi4 >> (8 * b)) & 0xFu) - 8), z), s);
+    }
+    const __nv_bfloat162 h2 = __floats2bfloat162_rn(v.x, v.y);
+    o[b] = *reinterpret_cast<const uint32_t*>(&h2);
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// The unit of work is eight columns.  A block converts kDqUnits * 256 consecutive units; a thread takes kDqUnits of
+// them, 256 units apart, so that a warp reads 128 contiguous bytes of codes and writes 512 contiguous bytes of
+// bf16 per step, and has all its loads in flight before it converts the first.
+constexpr int kDqUnits = 8;
+
 __global__ void __launch_bounds__(256)
 dequant_p_grouped_kernel(const DequantItem* __restrict__ items, const int32_t* __restrict__ block_item) {
   const DequantItem& it = items[__ldg(block_item + blockIdx.x)];   // host-made map: block -> matrix of the chunk
   const uint32_t cols = (uint32_t)it.P.cols, rows = (uint32_t)it.P.rows;
-  const uint32_t per_row = cols / 32, ngroups = (cols + kGroup - 1) / kGroup;
-  const uint32_t idx = (blockIdx.x - (uint32_t)it.block0) * blockDim.x + threadIdx.x;
-  if (idx >= rows * per_row) return;
-  const uint32_t row = idx / per_row, c0 = (idx - row * per_row) * 32;
-  const uint32_t g = c0 / kGroup;
-  const float s = __ldg(it.P.scales + (size_t)row * ngroups + g), z = __ldg(it.P.zeros + (size_t)row * ngroups + g);
+  const uint32_t per_row = cols / 8, ngroups = (cols + kGroup - 1) / kGroup, total = rows * per_row;   // r % 32 == 0
+  const uint32_t base = (blockIdx.x - (uint32_t)it.block0) * (kDqUnits * 256u) + threadIdx.x;
   if (it.P.bits != 4) {                              // the 2- and 8-bit projections of the ablation: plain conversion
-    uint4* o = reinterpret_cast<uint4*>(it.out + (size_t)row * cols + c0);
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int u = 0; u < kDqUnits; ++u) {
+      const uint32_t idx = base + 256u * u;
+      if (idx >= total) break;
+      const uint32_t row = idx / per_row, c0 = (idx - row * per_row) * 8;
+      const uint32_t g = c0 / kGroup;
+      const float s = __ldg(it.P.scales + (size_t)row * ngroups + g), z = __ldg(it.P.zeros + (size_t)row * ngroups + g);
       float q[8], v[8];
-      load_codes8(it.P, row, c0 + 8 * k, 8, q);
+      load_codes8(it.P, row, c0, 8, q);
 #pragma unroll
       for (int e = 0; e < 8; ++e) v[e] = __fmul_rn(__fsub_rn(q[e], z), s);
-      o[k] = pack_bf16x8(v);
+      *reinterpret_cast<uint4*>(it.out + (size_t)row * cols + c0) = pack_bf16x8(v);
     }
     return;
   }
-  const uint4 w4 = __ldg(reinterpret_cast<const uint4*>((const uint8_t*)it.P.codes + (size_t)row * (it.P.ld / 2) + (c0 >> 1)));
-  const float c = 8388616.0f + z;                    // 2^23 + 8 + z, exact for |z| < 2^22
-  const bool fast = fabsf(z) < 4.0e6f;
-  const uint32_t w[4] = {w4.x, w4.y, w4.z, w4.w};
-  uint4* out = reinterpret_cast<uint4*>(it.out + (size_t)row * cols + c0);
+  uint32_t w[kDqUnits];
+  float s[kDqUnits], z[kDqUnits];
+  uint4* out[kDqUnits];
+  const uint32_t row_bytes = (uint32_t)(it.P.ld / 2);
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const uint32_t lo4 = w[k] & 0x0F0F0F0Fu, hi4 = (w[k] >> 4) & 0x0F0F0F0Fu;   // even and odd columns, one per byte
-    float v[8];
+  for (int u = 0; u < kDqUnits; ++u) {
+    const uint32_t idx = base + 256u * u;
+    out[u] = nullptr;
+    if (idx >= total) continue;
+    const uint32_t row = idx / per_row, c0 = (idx - row * per_row) * 8;
+    const uint32_t g = c0 / kGroup;
+    w[u] = __ldcs(reinterpret_cast<const uint32_t*>((const uint8_t*)it.P.codes + (size_t)row * row_bytes + (c0 >> 1)));
+    s[u] = __ldg(it.P.scales + (size_t)row * ngroups + g);
+    z[u] = __ldg(it.P.zeros + (size_t)row * ngroups + g);
+    out[u] = reinterpret_cast<uint4*>(it.out + (size_t)row * cols + c0);
+  }
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      float qe, qo;
-      if (fast) {
-        qe = __fsub_rn(__uint_as_float(__byte_perm(lo4, 0x4B000000u, 0x7650 + b)), c);
-        qo = __fsub_rn(__uint_as_float(__byte_perm(hi4, 0x4B000000u, 0x7650 + b)), c);
-      } else {
-        qe = __fsub_rn((float)((int)((lo4 >> (8 * b)) & 0xFu) - 8), z);
-        qo = __fsub_rn((float)((int)((hi4 >> (8 * b)) & 0xFu) - 8), z);
-      }
-      v[2 * b] = __fmul_rn(qe, s);
-      v[2 * b + 1] = __fmul_rn(qo, s);
+  for (int u = 0; u < kDqUnits; ++u) {
+    // a warp-uniform choice (every lane votes, also those past the end), so that the plain form is a branch
+    // not taken rather than work done and discarded
+    const bool valid = out[u] != nullptr;
+    if (__all_sync(0xFFFFFFFFu, !valid || fabsf(z[u]) < 4.0e6f)) {
+      if (valid) *out[u] = dequant8_int4<true>(w[u], s[u], z[u]);
+    } else {
+      if (valid) *out[u] = dequant8_int4<false>(w[u], s[u], z[u]);
     }
-    out[k] = pack_bf16x8(v);
   }
 }
 
@@ -1356,7 +1547,7 @@ size_t tc_workspace_bytes(int64_t m, int64_t n, int64_t r) { return scratch_pt_b
 
 int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
   const TcScratch w = carve(a.ws, proj_rows(a), state_cols(a), a.r);
-  int rc = launch_dequant_p(a.P, w.Pt, a.r, st);
+  int rc = fused_dequant(a) ? QG_OK : launch_dequant_p(a.P, w.Pt, a.r, st);
   if (rc != QG_OK) return rc;
   const int bn = choose_bn(ceil_div(a.r, kTileM) * ceil_div(state_cols(a), 256));
   TcProblem prob;
@@ -1364,11 +1555,11 @@ int launch_project_step_tc(const StepArgs& a, cudaStream_t st) {
   if (rc != QG_OK) return rc;
   const TileSchedule none{nullptr, nullptr, 1};
   if (a.state8) {
-    rc = bn == 256 ? launch_k1<256, true, 1, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
-                   : launch_k1<128, true, 1, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
+    rc = bn == 256 ? launch_k1<256, true, 1, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st, prob.fuse_a)
+                   : launch_k1<128, true, 1, true>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st, prob.fuse_a);
   } else {
-    rc = bn == 256 ? launch_k1<256, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st)
-                   : launch_k1<128, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st);
+    rc = bn == 256 ? launch_k1<256, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st, prob.fuse_a)
+                   : launch_k1<128, true, 1>(&prob, nullptr, none, 0, prob.k1_tiles, a.sc, a.status, st, prob.fuse_a);
   }
   if (rc != QG_OK) return rc;
   return launch_k2<true, 1>(&prob, nullptr, none, 0, prob.k2_tiles, a.sc, a.status, st);
@@ -1382,6 +1573,7 @@ struct PlanChunk {
   int k1_tiles, k2_tiles, k2p_tiles, bn;
   int dq_blocks;
   int k1_grid, k2_grid, pairs, k1_pairs, k1p_tiles, state8;
+  int conv_active;           // some matrix of the chunk has its projection converted inside the projection kernel
   size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
   size_t dq_map_off;                                                // same: block -> item map of the dequantize launch
 };
@@ -1504,7 +1696,8 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       ch.k2p_tiles += probs[k].k2p_tiles;
       dq[k].P = a.P; dq[k].out = w.Pt;
       dq[k].block0 = ch.dq_blocks;
-      dq[k].nblocks = (int32_t)ceil_div(proj_rows(a) * (a.r / 32), 256);
+      dq[k].nblocks = fused_dequant(a) ? 0 : (int32_t)ceil_div(proj_rows(a) * (a.r / 8), 256 * 8);
+      if (fused_dequant(a)) ch.conv_active = 1;
       ch.dq_blocks += dq[k].nblocks;
       for (int32_t blk = 0; blk < dq[k].nblocks; ++blk) dq_map.push_back(k - i);
     }
@@ -1551,8 +1744,10 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
   size_t c = 0;
   for (const PlanChunk& ch : plan->chunks) {
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 0], st));
-    dequant_p_grouped_kernel<<<ch.dq_blocks, 256, 0, st>>>(plan->dq_dev + ch.first, plan->sched_dev + ch.dq_map_off);
-    QG_LAUNCH_CHECK();
+    if (ch.dq_blocks > 0) {                              // matrices whose projection the first kernel does not convert itself
+      dequant_p_grouped_kernel<<<ch.dq_blocks, 256, 0, st>>>(plan->dq_dev + ch.first, plan->sched_dev + ch.dq_map_off);
+      QG_LAUNCH_CHECK();
+    }
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 1], st));
     const TcProblem* tab = plan->table_dev + ch.first;
     const TileSchedule s1{plan->sched_dev + ch.k1_start_off, reinterpret_cast<const int2*>(plan->sched_dev + ch.k1_items_off),
@@ -1561,13 +1756,13 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
                           ch.pairs ? 2 : 1};
     int rc;
     if (ch.state8) {       // some matrix of the chunk keeps its moments in 8 bits
-      rc = ch.k1_pairs  ? launch_k1<256, false, 2, true>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st)
-           : ch.bn == 256 ? launch_k1<256, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
-                          : launch_k1<128, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
+      rc = ch.k1_pairs  ? launch_k1<256, false, 2, true>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st, ch.conv_active)
+           : ch.bn == 256 ? launch_k1<256, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active)
+                          : launch_k1<128, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active);
     } else {
-      rc = ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st)
-           : ch.bn == 256 ? launch_k1<256, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st)
-                          : launch_k1<128, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st);
+      rc = ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st, ch.conv_active)
+           : ch.bn == 256 ? launch_k1<256, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active)
+                          : launch_k1<128, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active);
     }
     if (rc != QG_OK) return rc;
     if (ev) QG_CUDA_TRY(cudaEventRecord(ev[4 * c + 2], st));
@@ -1597,6 +1792,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
     for (size_t c = 0; c < nch; ++c)
       for (int k = 0; k < 3; ++k) {
         float t = 0.f;
+        if (k == 0 && plan->chunks[c].dq_blocks == 0) continue;      // no dequantize launch in this chunk
         if (cudaEventElapsedTime(&t, ev[4 * c + k], ev[4 * c + k + 1]) == cudaSuccess) { ms[k] += t; launches[k] += 1; }
       }
   }
@@ -1608,6 +1804,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
 
 void plan_destroy(Plan* plan) { delete plan; }
 int set_pair_mode(int mask) { g_pair_mode = mask & 3; return QG_OK; }
+int set_fused_dequant(int on) { g_fuse_dequant = on ? 1 : 0; return QG_OK; }
 int set_chunk_budget(size_t bytes) { g_chunk_budget = bytes; return QG_OK; }
 
 // Registers, thread limit and shared memory of the tensor-core kernels as the loaded module reports them.

@@ -337,6 +337,51 @@ def test_cta_pair_kernels_equal_single_cta_kernels(mask):
         assert torch.equal(a["M"], b["M"]) and torch.equal(a["V"], b["V"])
 
 
+def test_projection_dequantized_inside_the_kernel_equals_the_separate_launch():
+    """The converter warps of the projection kernel form the same bf16 operand as the dequantize-P launch: two
+    steps of a stack that mixes 1B shapes (ragged K: 5461 rows), small ranks, a right-hand item and a rank that is
+    not a multiple of 128 (which keeps the separate launch either way) give the same bits in both modes, as single
+    calls and as a plan."""
+    from paper_2407_08296_b200.synth_device import build_stack
+    _, base = build_stack("llama1b", torch.device("cuda", 0), seed=5, layers=1)
+    base = [{k: v for k, v in it.items() if k != "spec"} for it in base]
+    for idx, ((m, n, r), side) in enumerate([((512, 1376, 128), "left"), ((1376, 512, 256), "right"), ((300, 777, 96), "left"),
+                                              ((257, 1025, 128), "left")]):
+        right = side == "right"
+        gb = synth.GradientModel(m, n, seed=23, matrix_index=idx).sample(1)
+        P = O.quantize_rtn(synth.random_orthonormal(n if right else m, r, seed=23, stream=idx), 4)
+        sc = m if right else n
+        base.append({"G": g_to_device(gb), "P": to_device_q(P), "W": to_device_q(O.quantize_rtn(synth.initial_weight(m, n, 23, idx), 8)),
+                     "M": f32_to_device(np.zeros((r, sc), np.float32)), "V": f32_to_device(np.zeros((r, sc), np.float32)),
+                     "seed": 100 + idx, "side": side})
+    results = {}
+    try:
+        for fused in (True, False):
+            B.debug_set_fused_dequant(fused)
+            items = [{**it, "W": it["W"].clone(), "M": it["M"]._base.clone()[:, :it["M"].shape[1]],
+                      "V": it["V"]._base.clone()[:, :it["V"].shape[1]]} for it in base]
+            plan = B.StepPlan(items)
+            for t in (1, 2):
+                plan.step(B.Hyper(step=t))
+            torch.cuda.synchronize()
+            assert int(plan.status.item()) == 0
+            plan.close()
+            singles = [{**it, "W": it["W"].clone(), "M": it["M"]._base.clone()[:, :it["M"].shape[1]],
+                        "V": it["V"]._base.clone()[:, :it["V"].shape[1]]} for it in base[-4:]]
+            for it in singles:
+                for t in (1, 2):
+                    B.project_step_item(it, B.Hyper(step=t))
+            torch.cuda.synchronize()
+            results[fused] = items + singles
+    finally:
+        B.debug_set_fused_dequant(True)
+    for a, b in zip(results[True], results[False]):
+        assert torch.equal(a["W"].codes, b["W"].codes) and torch.equal(a["W"].scales, b["W"].scales)
+        assert torch.equal(a["W"].zeros, b["W"].zeros) and torch.equal(a["M"], b["M"]) and torch.equal(a["V"], b["V"])
+    for a, b in zip(results[True][-8:-4], results[True][-4:]):       # plan == single calls, in the fused mode too
+        assert torch.equal(a["W"].codes, b["W"].codes) and torch.equal(a["M"], b["M"])
+
+
 # ----------------------------------------------------------------------------- full sizes, as the bench runs them
 def _full_size_case(shapes, blocks_of, seed):
     """A plan over full-size matrices (the launch configuration bench.py times: grouped launches, CTA pairs,
