@@ -290,81 +290,51 @@ def time_linear(items, device, tokens, peak_tflops):
 
 
 def time_refresh(items, device):
-    """The occasional subspace refresh (Sec. 3.5), timed apart from the step: one matrix of each distinct
-    shape (12 subspace iterations on a block of 2r columns, Rayleigh-Ritz, INT4), CUDA events around the second
-    of two calls, extrapolated to the stack by the shape counts.  Also the similarity to the random projection
-    the stack was built with, as the gate would see it."""
+    """The occasional subspace refresh (Sec. 3.5), timed apart from the step (12 subspace iterations on a block of
+    2r columns, Rayleigh-Ritz, INT4): per distinct shape, one matrix alone (the latency of a refresh) and a batch of
+    up to eight matrices of that shape in one qgalore_refresh_subspace_batched call (how a stack is refreshed),
+    CUDA events around the second of two calls each; extrapolated to the stack by the shape counts.  Also the
+    similarity to the random projection the stack was built with, as the gate would see it."""
     import torch
     from paper_2407_08296_b200 import binding as B
-    first, counts = {}, {}
+    groups = {}
     for it in items:
         sp = it["spec"]
-        key = (sp.m, sp.n, sp.r)
-        counts[key] = counts.get(key, 0) + 1
-        first.setdefault(key, it)
-    per_shape, total = [], 0.0
-    for (m, n, r), it in first.items():
+        groups.setdefault((sp.m, sp.n, sp.r), []).append(it)
+    per_shape, total_single, total_batched = [], 0.0, 0.0
+    stream = torch.cuda.current_stream()
+    for (m, n, r), group in groups.items():
         block = min((2 * r + 63) // 64 * 64, min(m, n) // 64 * 64)
-        ws = torch.empty(B.workspace_bytes(B.QG_OP_REFRESH, m, n, block), dtype=torch.uint8, device=device)
+        nb = min(8, len(group))
+        per = B.workspace_bytes(B.QG_OP_REFRESH, m, n, block)
+        ws = torch.empty(per * nb, dtype=torch.uint8, device=device)
         sim = torch.zeros(1, dtype=torch.float32, device=device)
         status = torch.zeros(1, dtype=torch.int32, device=device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        stream = torch.cuda.current_stream()
         for rep in range(2):
             e0.record(stream)
-            B.refresh_subspace(it["G"], r, iters=12, seed=1, P_prev=it["P"], sim=sim, workspace=ws, status=status)
+            B.refresh_subspace(group[0]["G"], r, iters=12, seed=1, P_prev=group[0]["P"], sim=sim, workspace=ws, status=status)
             e1.record(stream)
             torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        per_shape.append({"shape": f"{m}x{n} r{r}", "count": counts[(m, n, r)], "ms": ms, "block": block,
+        ms_single = e0.elapsed_time(e1)
+        batch = [{"G": it["G"], "seed": 1 + k, "P_new": B.dense_projection(m, r, 4, device)} for k, it in enumerate(group[:nb])]
+        for rep in range(2):
+            e0.record(stream)
+            B.refresh_subspace_batched(batch, r, iters=12, workspace=ws, status=status)
+            e1.record(stream)
+            torch.cuda.synchronize()
+        ms_batch = e0.elapsed_time(e1)
+        count = len(group)
+        per_shape.append({"shape": f"{m}x{n} r{r}", "count": count, "ms": ms_single, "block": block, "batch": nb,
+                          "batch_ms": ms_batch, "ms_per_matrix_batched": ms_batch / nb,
                           "similarity_to_previous": float(sim.item()), "device_status": int(status.item())})
-        total += ms * counts[(m, n, r)] * 1e-3
-        del ws
-    out = {"iters": 12, "per_shape": per_shape, "stack_seconds": total,
-           "note": "not part of the timed step; one matrix per distinct shape, extrapolated by shape counts"}
-    # several matrices at once on several streams (each with its own scratch): the refresh is a long chain of
-    # small kernels, so independent matrices fill each other's gaps.  The first `batch` matrices of the stack,
-    # timed once one after the other and once round-robin over `streams` streams; the ratio scales the figure above.
-    streams, batch = 4, min(8, len(items))
-    some = items[:batch]
-    side = [torch.cuda.Stream(device=device) for _ in range(streams)]
-    wss, outs = [], []
-    for k in range(streams):
-        need = max(B.workspace_bytes(B.QG_OP_REFRESH, it["spec"].m, it["spec"].n,
-                                     min((2 * it["spec"].r + 63) // 64 * 64, min(it["spec"].m, it["spec"].n) // 64 * 64))
-                   for it in some)
-        wss.append(torch.empty(need, dtype=torch.uint8, device=device))
-    for it in some:
-        sp = it["spec"]
-        ng = (sp.r + 255) // 256
-        outs.append(B.QTensor(torch.full((sp.m, sp.r // 2), 0x88, dtype=torch.uint8, device=device),
-                              torch.zeros((sp.m, ng), dtype=torch.float32, device=device),
-                              torch.zeros((sp.m, ng), dtype=torch.float32, device=device), sp.m, sp.r, sp.r, 4))
-    status = torch.zeros(1, dtype=torch.int32, device=device)
-    main = torch.cuda.current_stream()
-    times = []
-    for concurrent in (False, True):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record(main)
-        for k, (it, pq) in enumerate(zip(some, outs)):
-            s = side[k % streams] if concurrent else main
-            if concurrent:
-                s.wait_stream(main)
-            with torch.cuda.stream(s):
-                B.refresh_subspace(it["G"], it["spec"].r, iters=12, seed=1, P_new=pq, workspace=wss[k % streams], status=status,
-                                   stream=s)
-        if concurrent:
-            for s in side:
-                main.wait_stream(s)
-        e1.record(main)
-        torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1))
-    out["concurrent"] = {"streams": streams, "matrices": batch, "sequential_ms": times[0], "concurrent_ms": times[1],
-                         "device_status": int(status.item())}
-    out["stack_seconds_concurrent"] = total * times[1] / max(times[0], 1e-9)
-    out["stack_seconds_best"] = min(out["stack_seconds"], out["stack_seconds_concurrent"])
-    return out
+        total_single += ms_single * count * 1e-3
+        total_batched += ms_batch / nb * count * 1e-3
+        del ws, batch
+        torch.cuda.empty_cache()
+    return {"iters": 12, "per_shape": per_shape, "stack_seconds": total_single, "stack_seconds_batched": total_batched,
+            "stack_seconds_best": min(total_single, total_batched),
+            "note": "not part of the timed step; per distinct shape one matrix alone and a batch of up to 8, extrapolated by shape counts"}
 
 
 def bench_workload(workload, args, B, torch, dist, device, world, rank, local_rank, peaks, peak_kind, extras):

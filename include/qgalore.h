@@ -239,6 +239,31 @@ QG_API int qgalore_refresh_subspace_right(const uint16_t* G, int64_t ldg, int64_
                                    void* workspace, size_t workspace_bytes,
                                    int32_t* status_dev, void* stream);
 
+/* --- Sec. 3.5, the refresh of several matrices of ONE shape in one call (with a fixed interval every matrix of a
+ * stack is due in the same step; under the adaptive schedule of Sec. 3.2, those whose interval has run out).
+ * The matrices are refreshed in batches: every kernel launch, and every grid barrier of the eigen-iteration,
+ * serves all matrices of a batch, so that a stack costs far less than its matrices one after the other.
+ *   items      HOST; per matrix: the gradient and its pitch, the seed of its start block, where the new
+ *              projection goes (P_new, ld == r) and optionally the fp32 vectors (P_fp32), the previous projection
+ *              (P_prev, may be NULL) and the device word that receives the similarity to it (sim_dev, may be NULL)
+ *   m, n, r    the shape and rank all items share; ldg must be the same for all items as well
+ *   side       QG_SIDE_LEFT: top-r left singular vectors (P_new is m x r); QG_SIDE_RIGHT: right ones (n x r)
+ *   workspace  at least qgalore_workspace_bytes(QG_OP_REFRESH, ...) bytes (the extents as for the single-matrix
+ *              call); a batch holds as many matrices as fit (up to 8), so count times that amount is the useful
+ *              maximum.  256-byte aligned.
+ * Results are those of the single-matrix call on each item (same seed, same arithmetic, bit for bit). */
+typedef struct {
+  const uint16_t* G; int64_t ldg;
+  uint64_t seed;
+  qg_qtensor P_new;
+  float* P_fp32;
+  const qg_qtensor* P_prev;
+  float* sim_dev;
+} qg_refresh_item;
+QG_API int qgalore_refresh_subspace_batched(const qg_refresh_item* items, int32_t count, int64_t m, int64_t n, int64_t r,
+                                     int32_t iters, int32_t oversample_cols, int32_t side, int32_t sim_cols,
+                                     void* workspace, size_t workspace_bytes, int32_t* status_dev, void* stream);
+
 /* --- Sec. 3.2: cosine similarity between adjacent projection matrices -------------------
  * *sim_dev = sum_{j < c} |<a_j, b_j>| / (||A[:, :c]||_F ||B[:, :c]||_F), c = sim_cols
  * (<= 0 means all columns), on the dequantized INT4 matrices A and B (same shape).

@@ -54,6 +54,11 @@ class _CStepItem(C.Structure):
                 ("M_scale", C.c_void_p), ("V_scale", C.c_void_p)]
 
 
+class _CRefreshItem(C.Structure):
+    _fields_ = [("G", C.c_void_p), ("ldg", C.c_int64), ("seed", C.c_uint64), ("P_new", _CQTensor), ("P_fp32", C.c_void_p),
+                ("P_prev", C.POINTER(_CQTensor)), ("sim_dev", C.c_void_p)]
+
+
 class _CDebug(C.Structure):
     _fields_ = [("R", C.c_void_p), ("N", C.c_void_p), ("W_pre", C.c_void_p), ("N_b", C.c_void_p)]
 
@@ -96,6 +101,8 @@ def lib() -> C.CDLL:
         L.qgalore_refresh_subspace.argtypes = [vp, i64, i64, i64, i64, i32, i32, C.c_uint64, qp, vp, qp, i32, vp,
                                                vp, sz, vp, vp]
         L.qgalore_refresh_subspace_right.argtypes = L.qgalore_refresh_subspace.argtypes
+        L.qgalore_refresh_subspace_batched.argtypes = [C.POINTER(_CRefreshItem), i32, i64, i64, i64, i32, i32, i32, i32, vp, sz,
+                                                       vp, vp]
         L.qgalore_subspace_similarity.argtypes = [qp, qp, i32, vp, vp, sz, vp]
         L.qgalore_subspace_similarity_static.argtypes = [qp, qp, i32, vp, vp]
         L.qgalore_subspace_similarity_static_max_bytes.restype = sz
@@ -503,6 +510,51 @@ def refresh_subspace(G: torch.Tensor, r: int, iters: int = 12, oversample_cols: 
               workspace.numel() * workspace.element_size(), _ptr(status),
               _stream_ptr(stream)), "qgalore_refresh_subspace_right" if right else "qgalore_refresh_subspace")
     return P_new
+
+
+def dense_projection(rows: int, r: int, bits: int = 4, device="cuda") -> QTensor:
+    """An empty quantized rows x r projection with ld == r, the layout the refresh writes."""
+    ng = (r + GROUP - 1) // GROUP
+    per_byte = {8: 1, 4: 2, 2: 4}[bits]
+    fill = {8: 0, 4: 0x88, 2: 0xAA}[bits]
+    codes = torch.full((rows, r // per_byte), fill, dtype=torch.int8 if bits == 8 else torch.uint8, device=device)
+    return QTensor(codes, torch.zeros((rows, ng), dtype=torch.float32, device=device),
+                   torch.zeros((rows, ng), dtype=torch.float32, device=device), rows, r, r, bits)
+
+
+def refresh_subspace_batched(items: list[dict], r: int, iters: int = 12, oversample_cols: int | None = None, sim_cols: int = 0,
+                             workspace: torch.Tensor | None = None, max_batch: int = 8, status: torch.Tensor | None = None,
+                             stream=None, side: str = "left") -> list[QTensor]:
+    """The refresh of several matrices of one shape in one call (Sec. 3.5).  items: dicts with G and seed, and
+    optionally P_new, P_fp32, P_prev and sim (a 1-element device tensor).  Returns the new projections."""
+    m, n = items[0]["G"].shape
+    right = side == "right"
+    pm, pn_ = (n, m) if right else (m, n)
+    if oversample_cols is None:
+        block = min((2 * r + 63) // 64 * 64, min(m, n) // 64 * 64)
+        oversample_cols = max(block - r, 0)
+    dev = items[0]["G"].device
+    table = (_CRefreshItem * len(items))()
+    keep, out = [], []
+    for k, it in enumerate(items):
+        G = it["G"]
+        if tuple(G.shape) != (m, n):
+            raise ValueError("a batch holds matrices of one shape")
+        P_new = it.get("P_new") or dense_projection(pm, r, 4, dev)
+        out.append(P_new)
+        prev = it.get("P_prev")
+        prev_c = prev.c_struct() if prev is not None else None
+        keep.append(prev_c)
+        table[k] = _CRefreshItem(_ptr(G), _matrix_ld(G, "G"), int(it.get("seed", 0)), P_new.c_struct(), _ptr(it.get("P_fp32")),
+                                 C.pointer(prev_c) if prev_c is not None else None, _ptr(it.get("sim")))
+    if workspace is None:
+        per = workspace_bytes(QG_OP_REFRESH, pm, pn_, r + oversample_cols)
+        workspace = torch.empty(per * max(1, min(max_batch, len(items))), dtype=torch.uint8, device=dev)
+    _check(lib().qgalore_refresh_subspace_batched(table, len(items), m, n, r, iters, oversample_cols,
+                                                  QG_SIDE_RIGHT if right else QG_SIDE_LEFT, sim_cols, _ptr(workspace),
+                                                  workspace.numel(), _ptr(status), _stream_ptr(stream)),
+           "qgalore_refresh_subspace_batched")
+    return out
 
 
 def subspace_similarity(A: QTensor, B: QTensor, sim_cols: int = 0, out: torch.Tensor | None = None,

@@ -27,6 +27,8 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
                    uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
                    cudaStream_t st, bool transposed);
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b);
+int launch_refresh_batched(const RefreshJob* jobs, int count, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
+                           void* ws, size_t ws_bytes, int32_t* status, cudaStream_t st, bool transposed);
 struct Plan;
 size_t plan_table_bytes(const StepArgs* items, int32_t count);
 int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t table_bytes, void* workspace,
@@ -354,59 +356,85 @@ void qgalore_plan_destroy(qg_plan* plan) {
   delete plan;
 }
 
-static int refresh_impl(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
-                        int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
-                        const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
-                        size_t workspace_bytes, int32_t* status_dev, void* stream, bool right) {
-  if (!G || !workspace || m <= 0 || n <= 0 || r <= 0 || ldg < n || iters < 0 || oversample_cols < 0)
+// Argument rules of a refresh, for one matrix or a batch of one shape; on success enqueues everything.
+static int refresh_impl(const qg_refresh_item* items, int32_t count, int64_t m, int64_t n, int64_t r, int32_t iters,
+                        int32_t oversample_cols, int32_t sim_cols, void* workspace, size_t workspace_bytes,
+                        int32_t* status_dev, void* stream, bool right) {
+  if (!items || count <= 0 || !workspace || m <= 0 || n <= 0 || r <= 0 || iters < 0 || oversample_cols < 0)
     return QG_INVALID_ARGUMENT;
   // the matrix whose LEFT singular vectors are wanted: G, or G^T for the right-hand projection
   const int64_t pm = right ? n : m, pn = right ? m : n;
-  if (!P_new || (P_new->bits != 2 && P_new->bits != 4 && P_new->bits != 8)) return QG_INVALID_ARGUMENT;
-  int rc = check_qtensor(P_new, P_new->bits);
-  if (rc != QG_OK) return rc;
-  if (P_new->rows != pm || P_new->cols != r || P_new->ld != r) return QG_INVALID_ARGUMENT;
-  if (P_prev) {
-    if (P_prev->bits != 2 && P_prev->bits != 4 && P_prev->bits != 8) return QG_INVALID_ARGUMENT;
-    rc = check_qtensor(P_prev, P_prev->bits);
-    if (rc != QG_OK) return rc;
-    if (P_prev->rows != pm || P_prev->cols != r) return QG_INVALID_ARGUMENT;
-  }
   const int64_t b = r + oversample_cols;
   // the block is handled in panels of 64 columns and cannot be wider than the matrix is tall or wide
   if (r % 32 != 0 || b % 64 != 0 || b > m || b > n || b > 4096 || m > (1ll << 31) - 1 || n > (1ll << 31) - 1)
     return QG_UNSUPPORTED_SHAPE;
-  if (!aligned16(G) || ldg % 8 != 0 || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return QG_MISALIGNED;
-  if (P_fp32 && !aligned16(P_fp32)) return QG_MISALIGNED;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return QG_MISALIGNED;
   if (status_dev && (reinterpret_cast<uintptr_t>(status_dev) & 3u)) return QG_MISALIGNED;
-  if (sim_dev && !aligned4(sim_dev)) return QG_MISALIGNED;
+  std::vector<RefreshJob> jobs((size_t)count);
+  for (int32_t i = 0; i < count; ++i) {
+    const qg_refresh_item& it = items[i];
+    if (!it.G || it.ldg < n || it.ldg != items[0].ldg) return QG_INVALID_ARGUMENT;
+    int rc = check_projection_qtensor(&it.P_new);
+    if (rc != QG_OK) return rc;
+    if (it.P_new.rows != pm || it.P_new.cols != r || it.P_new.ld != r) return QG_INVALID_ARGUMENT;
+    if (it.P_prev) {
+      rc = check_projection_qtensor(it.P_prev);
+      if (rc != QG_OK) return rc;
+      if (it.P_prev->rows != pm || it.P_prev->cols != r) return QG_INVALID_ARGUMENT;
+    }
+    if (!aligned16(it.G) || it.ldg % 8 != 0) return QG_MISALIGNED;
+    if (it.P_fp32 && !aligned16(it.P_fp32)) return QG_MISALIGNED;
+    if (it.sim_dev && !aligned4(it.sim_dev)) return QG_MISALIGNED;
+    jobs[(size_t)i] = RefreshJob{it.G, it.ldg, it.seed, &it.P_new, it.P_fp32};
+  }
   if (workspace_bytes < qgalore_workspace_bytes(QG_OP_REFRESH, pm, pn, b)) return QG_WORKSPACE_TOO_SMALL;
   constexpr int kJacobiSweeps = 12;
-  rc = launch_refresh(G, ldg, pm, pn, r, b, iters, kJacobiSweeps, seed, P_new, P_fp32, workspace, workspace_bytes,
-                      status_dev, (cudaStream_t)stream, right);
+  int rc = launch_refresh_batched(jobs.data(), count, pm, pn, r, b, iters, kJacobiSweeps, workspace, workspace_bytes, status_dev,
+                                  (cudaStream_t)stream, right);
   if (rc != QG_OK) return rc;
-  if (P_prev && sim_dev) {
-    const int32_t c = (sim_cols <= 0 || sim_cols > r) ? (int32_t)r : sim_cols;
-    // the refresh has finished with its scratch by the time this runs on the same stream
-    return launch_similarity(P_prev, P_new, c, sim_dev, workspace, (cudaStream_t)stream);
+  for (int32_t i = 0; i < count; ++i) {
+    const qg_refresh_item& it = items[i];
+    if (it.P_prev && it.sim_dev) {
+      const int32_t c = (sim_cols <= 0 || sim_cols > r) ? (int32_t)r : sim_cols;
+      // the refresh has finished with its scratch by the time this runs on the same stream
+      rc = launch_similarity(it.P_prev, &it.P_new, c, it.sim_dev, workspace, (cudaStream_t)stream);
+      if (rc != QG_OK) return rc;
+    }
   }
   return QG_OK;
+}
+
+static int refresh_single(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
+                          int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
+                          const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
+                          size_t workspace_bytes, int32_t* status_dev, void* stream, bool right) {
+  if (!P_new) return QG_INVALID_ARGUMENT;
+  const qg_refresh_item item{G, ldg, seed, *P_new, P_fp32, P_prev, sim_dev};
+  return refresh_impl(&item, 1, m, n, r, iters, oversample_cols, sim_cols, workspace, workspace_bytes, status_dev, stream, right);
+}
+
+int qgalore_refresh_subspace_batched(const qg_refresh_item* items, int32_t count, int64_t m, int64_t n, int64_t r,
+                                     int32_t iters, int32_t oversample_cols, int32_t side, int32_t sim_cols, void* workspace,
+                                     size_t workspace_bytes, int32_t* status_dev, void* stream) {
+  if (side != QG_SIDE_LEFT && side != QG_SIDE_RIGHT) return QG_INVALID_ARGUMENT;
+  return refresh_impl(items, count, m, n, r, iters, oversample_cols, sim_cols, workspace, workspace_bytes, status_dev, stream,
+                      side == QG_SIDE_RIGHT);
 }
 
 int qgalore_refresh_subspace(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
                              int32_t oversample_cols, uint64_t seed, const qg_qtensor* P_new, float* P_fp32,
                              const qg_qtensor* P_prev, int32_t sim_cols, float* sim_dev, void* workspace,
                              size_t workspace_bytes, int32_t* status_dev, void* stream) {
-  return refresh_impl(G, ldg, m, n, r, iters, oversample_cols, seed, P_new, P_fp32, P_prev, sim_cols, sim_dev, workspace,
-                      workspace_bytes, status_dev, stream, false);
+  return refresh_single(G, ldg, m, n, r, iters, oversample_cols, seed, P_new, P_fp32, P_prev, sim_cols, sim_dev, workspace,
+                        workspace_bytes, status_dev, stream, false);
 }
 
 int qgalore_refresh_subspace_right(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int32_t iters,
                                    int32_t oversample_cols, uint64_t seed, const qg_qtensor* Q_new, float* Q_fp32,
                                    const qg_qtensor* Q_prev, int32_t sim_cols, float* sim_dev, void* workspace,
                                    size_t workspace_bytes, int32_t* status_dev, void* stream) {
-  return refresh_impl(G, ldg, m, n, r, iters, oversample_cols, seed, Q_new, Q_fp32, Q_prev, sim_cols, sim_dev, workspace,
-                      workspace_bytes, status_dev, stream, true);
+  return refresh_single(G, ldg, m, n, r, iters, oversample_cols, seed, Q_new, Q_fp32, Q_prev, sim_cols, sim_dev, workspace,
+                        workspace_bytes, status_dev, stream, true);
 }
 
 int qgalore_subspace_similarity(const qg_qtensor* A, const qg_qtensor* B, int32_t sim_cols, float* sim_dev,

@@ -251,6 +251,14 @@ struct StepArgs {
 int launch_dequant_p(const qg_qtensor& P, uint16_t* out, int64_t ld_out, cudaStream_t st);
 
 
+// refresh.cu: one matrix of a batched subspace refresh
+struct RefreshJob {
+  const uint16_t* G; int64_t ldg;
+  uint64_t seed;
+  const qg_qtensor* P_new;
+  float* P_fp32;           // optional
+};
+
 // linear_tc.cu: the INT8 linear layer of App. A.  mode 0: D (T x m) = act (X, T x n) W~^T; mode 1: D (T x n) =
 // act (dY, T x m) W~; mode 2: D (m x n) = act^T (dY, T x m) act2 (X, T x n), W unused.  All bf16, row-major.
 int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint16_t* act2, int64_t ld_act2,

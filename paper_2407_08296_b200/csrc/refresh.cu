@@ -14,6 +14,11 @@
 // round-robin pair ordering: all sweeps in one cooperative launch, a grid barrier between rounds of b/2 disjoint pairs.  Each column of P is then
 // given the sign that makes its largest entry positive, and P is quantized to INT4 (Quant_4).
 //
+// Several matrices of one shape are refreshed together (a "batch", up to kMaxBatch): every launch carries a matrix
+// index beside its tile index and reads its operands from small pointer tables passed by value, so the few
+// thousand small launches and the ~9000 grid barriers of the eigen-iteration are paid once per batch instead of
+// once per matrix.
+//
 // The arithmetic is plain fp32/fp64 on the CUDA cores: the singular values next to the r-th one sit in the
 // noise bulk of the gradient with relative gaps of 1e-4..1e-3, and resolving that subspace to 1e-2 rad
 // needs fp32-faithful products (bf16 tensor-core products do not get there).
@@ -35,18 +40,38 @@ constexpr int kMaxSweeps = 32;
 constexpr int kGT = 64;       // GEMM tile (square), 16 x 16 threads, 4 x 4 outputs each
 constexpr int kGK = 16;
 
+constexpr int kMaxBatch = 8;  // matrices refreshed together
+// One pointer per matrix of a batch, passed to the kernels by value.
+template <class T>
+struct Ptrs {
+  T* p[kMaxBatch];
+};
+template <class T, class U>
+Ptrs<T> offset_ptrs(const Ptrs<U>& src, int nb, int64_t off) {
+  Ptrs<T> out{};
+  for (int i = 0; i < nb; ++i) out.p[i] = src.p[i] + off;
+  return out;
+}
+
 __device__ __forceinline__ float ld_as_float(const uint16_t* p, int64_t i) { return bf16_bits_to_float(p[i]); }
 __device__ __forceinline__ float ld_as_float(const float* p, int64_t i) { return p[i]; }
 
 // C[M x N] = alpha * A * B + beta * C.  A(i, k) = A[i * sa_m + k * sa_k], B(k, j) = B[k * sb_k + j * sb_n],
 // C(i, j) = C[i * ldc + j].  TA is uint16_t (bfloat16 bits) or float; ACC/TC float or double.
-// With k_slice < K the grid's z index selects a slice of K, and slice z writes its bare partial sums to
-// part + z * M * N (row-major M x N) instead of C: products with a small result and a long K (the Gram
-// matrices and projection coefficients of the orthonormalisation) would otherwise keep a handful of SMs busy.
+// The grid's z index is (matrix of the batch) * slices + (slice of K).  With more than one slice, slice z writes
+// its bare partial sums to part + z * M * N (row-major M x N) instead of C: products with a small result and a
+// long K (the Gram matrices and projection coefficients of the orthonormalisation) would otherwise keep a
+// handful of SMs busy.
 template <class TA, class ACC, class TC>
 __global__ void __launch_bounds__(256)
-gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* __restrict__ B, int64_t sb_k, int64_t sb_n,
-            TC* __restrict__ C, int64_t ldc, int M, int N, int K, ACC alpha, ACC beta, int k_slice, ACC* __restrict__ part) {
+gemm_kernel(const Ptrs<const TA> Ab, int64_t sa_m, int64_t sa_k, const Ptrs<const float> Bb, int64_t sb_k, int64_t sb_n,
+            const Ptrs<TC> Cb, int64_t ldc, int M, int N, int K, ACC alpha, ACC beta, int k_slice, int slices,
+            const Ptrs<ACC> partb) {
+  const int mat = (int)blockIdx.z / slices, slice = (int)blockIdx.z % slices;
+  const TA* __restrict__ A = Ab.p[mat];
+  const float* __restrict__ B = Bb.p[mat];
+  TC* __restrict__ C = Cb.p[mat];
+  ACC* __restrict__ part = slices > 1 ? partb.p[mat] : nullptr;
   __shared__ __align__(16) float As[kGK][kGT + 4];
   __shared__ __align__(16) float Bs[kGK][kGT + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -57,8 +82,8 @@ gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* _
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = (ACC)0;
   const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
-  const int k_begin = (int)blockIdx.z * k_slice;
-  if (k_slice < K) K = min(K, k_begin + k_slice);
+  const int k_begin = slice * k_slice;
+  if (slices > 1) K = min(K, k_begin + k_slice);
   for (int k0 = k_begin; k0 < K; k0 += kGK) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
@@ -93,7 +118,7 @@ gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* _
       const int64_t gn = n0 + tx * 4 + j;
       if (gn >= N) continue;
       if (part != nullptr) {
-        part[((int64_t)blockIdx.z * M + gm) * N + gn] = acc[i][j];
+        part[((int64_t)slice * M + gm) * N + gn] = acc[i][j];
         continue;
       }
       TC* c = C + gm * ldc + gn;
@@ -106,7 +131,9 @@ gemm_kernel(const TA* __restrict__ A, int64_t sa_m, int64_t sa_k, const float* _
 // C = alpha * (sum of the slices' partial sums, in slice order) + beta * C
 template <class ACC, class TC>
 __global__ void __launch_bounds__(256)
-gemm_reduce_kernel(const ACC* __restrict__ part, int slices, TC* __restrict__ C, int64_t ldc, int M, int N, ACC alpha, ACC beta) {
+gemm_reduce_kernel(const Ptrs<ACC> partb, int slices, const Ptrs<TC> Cb, int64_t ldc, int M, int N, ACC alpha, ACC beta) {
+  const ACC* __restrict__ part = partb.p[blockIdx.y];
+  TC* __restrict__ C = Cb.p[blockIdx.y];
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)M * N) return;
   ACC s = (ACC)0;
@@ -129,13 +156,15 @@ constexpr int kSplitTiles = 160;         // products with fewer output tiles tha
 constexpr int kSplitMinK = 128;          // ... into slices no shorter than this
 constexpr int64_t kSplitScratch = 32 << 20;  // bytes of partial sums a product may use
 
-// `part` (kSplitScratch bytes, or null) lets a product with few output tiles and a long K run as slices.
+// One product per matrix of the batch.  `part` (kSplitScratch bytes per matrix, or null tables) lets a product
+// with few output tiles and a long K run as slices.
 template <class TA, class ACC, class TC>
-int gemm(const TA* A, int64_t sa_m, int64_t sa_k, const float* B, int64_t sb_k, int64_t sb_n, TC* C, int64_t ldc, int64_t M,
-         int64_t N, int64_t K, ACC alpha, ACC beta, cudaStream_t st, void* part = nullptr) {
+int gemm(int nb, const Ptrs<const TA>& A, int64_t sa_m, int64_t sa_k, const Ptrs<const float>& B, int64_t sb_k, int64_t sb_n,
+         const Ptrs<TC>& C, int64_t ldc, int64_t M, int64_t N, int64_t K, ACC alpha, ACC beta, cudaStream_t st,
+         const Ptrs<void>* part = nullptr) {
   if (M <= 0 || N <= 0) return QG_OK;
   dim3 grid((unsigned)ceil_div(N, kGT), (unsigned)ceil_div(M, kGT));
-  const int64_t tiles = (int64_t)grid.x * grid.y;
+  const int64_t tiles = (int64_t)grid.x * grid.y * nb;
   int64_t slices = 1;
   if (part != nullptr && tiles < kSplitTiles && K >= 2 * kSplitMinK) {
     slices = ceil_div(2 * (int64_t)refresh_sm_count(), tiles);
@@ -143,26 +172,34 @@ int gemm(const TA* A, int64_t sa_m, int64_t sa_k, const float* B, int64_t sb_k, 
     const int64_t fit = kSplitScratch / (M * N * (int64_t)sizeof(ACC));
     if (slices > fit) slices = fit;
   }
+  Ptrs<ACC> pt{};
   if (slices <= 1) {
+    grid.z = (unsigned)nb;
     gemm_kernel<TA, ACC, TC><<<grid, 256, 0, st>>>(A, sa_m, sa_k, B, sb_k, sb_n, C, ldc, (int)M, (int)N, (int)K, alpha, beta,
-                                                   (int)K, nullptr);
+                                                   (int)K, 1, pt);
     QG_LAUNCH_CHECK();
     return QG_OK;
   }
+  for (int i = 0; i < nb; ++i) pt.p[i] = reinterpret_cast<ACC*>(part->p[i]);
   const int64_t k_slice = round_up(ceil_div(K, slices), kGK);
-  grid.z = (unsigned)ceil_div(K, k_slice);
+  const int nslices = (int)ceil_div(K, k_slice);
+  grid.z = (unsigned)(nslices * nb);
   gemm_kernel<TA, ACC, TC><<<grid, 256, 0, st>>>(A, sa_m, sa_k, B, sb_k, sb_n, C, ldc, (int)M, (int)N, (int)K, alpha, beta,
-                                                 (int)k_slice, reinterpret_cast<ACC*>(part));
+                                                 (int)k_slice, nslices, pt);
   QG_LAUNCH_CHECK();
-  gemm_reduce_kernel<ACC, TC><<<(unsigned)ceil_div(M * N, 256), 256, 0, st>>>(reinterpret_cast<const ACC*>(part), (int)grid.z, C,
-                                                                              ldc, (int)M, (int)N, alpha, beta);
+  gemm_reduce_kernel<ACC, TC><<<dim3((unsigned)ceil_div(M * N, 256), (unsigned)nb), 256, 0, st>>>(pt, nslices, C, ldc, (int)M, (int)N,
+                                                                                                  alpha, beta);
   QG_LAUNCH_CHECK();
   return QG_OK;
 }
 
 // ---- Gaussian start block: Q[i][j] ~ N(0, 1) from Philox4x32-10 (counter (j / 4, i, 0, 0x51)) and Box-Muller
 __global__ void __launch_bounds__(256)
-gaussian_kernel(float* __restrict__ Q, int64_t ld, int64_t rows, int64_t cols, uint32_t seed_lo, uint32_t seed_hi) {
+gaussian_kernel(const Ptrs<float> Qb, int64_t ld, int64_t rows, int64_t cols, const Ptrs<const void> seeds) {
+  float* __restrict__ Q = Qb.p[blockIdx.y];
+  // the seed of matrix y travels in the pointer table's slot (a 64-bit value, not an address)
+  const uint64_t seed = (uint64_t)reinterpret_cast<uintptr_t>(seeds.p[blockIdx.y]);
+  const uint32_t seed_lo = (uint32_t)seed, seed_hi = (uint32_t)(seed >> 32);
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int64_t quads = cols / 4;
   if (idx >= rows * quads) return;
@@ -183,7 +220,9 @@ gaussian_kernel(float* __restrict__ Q, int64_t ld, int64_t rows, int64_t cols, u
 // One shared array holds both triangles: L below and on the diagonal, the transpose of L^-1 above it
 // (A[j][i] = (L^-1)[i][j] for i > j); the diagonal of L^-1 is kept apart.
 __global__ void __launch_bounds__(256)
-chol64_inverse_kernel(const float* __restrict__ S, float* __restrict__ Linv, int32_t* __restrict__ status) {
+chol64_inverse_kernel(const Ptrs<const float> Sb, const Ptrs<float> Linvb, int32_t* __restrict__ status) {
+  const float* __restrict__ S = Sb.p[blockIdx.x];
+  float* __restrict__ Linv = Linvb.p[blockIdx.x];
   __shared__ double A[kPanel][kPanel + 1];
   __shared__ double xd[kPanel];
   const int t = threadIdx.x;
@@ -267,32 +306,36 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* count, unsigned int* 
   return __syncthreads_and(ok) != 0;
 }
 
-// All sweeps in one cooperative launch.  A team of 128 threads takes a pair of rows, NE elements of each row
-// per thread, kept in registers between the three inner products and the rotation; four teams per CTA move
-// in step.  A grid barrier follows every round (the next round pairs the rows differently).  Rows move
-// between SMs from round to round, so they are read and written through L2 (.cg).  The sweep's largest
-// normalised inner product is collected in off[sweep]; the iteration stops after the first sweep whose value
-// is <= tol and flags QG_DEV_NOT_CONVERGED if none is.
+// All sweeps of all matrices of a batch in one cooperative launch.  A team of 128 threads takes a pair of rows of
+// one matrix, NE elements of each row per thread, kept in registers between the three inner products and the
+// rotation; four teams per CTA move in step.  A grid barrier follows every round (the next round pairs the rows
+// differently); a round covers that round's pairs of every matrix, so the barriers are shared by the batch.
+// Rows move between SMs from round to round, so they are read and written through L2 (.cg).  The sweep's
+// largest normalised inner product of matrix i is collected in off[i][sweep]; a matrix stops rotating after its
+// first sweep whose value is <= tol, the launch ends when all have, and QG_DEV_NOT_CONVERGED is flagged if one
+// never does.
 constexpr int kTeam = 128, kTeamsPerCta = 4;
 template <int NE>
-__global__ void __launch_bounds__(kTeam * kTeamsPerCta, 1)
-jacobi_sweeps_kernel(double* __restrict__ T, int b, int sweeps, double tol, unsigned long long* __restrict__ off,
+__global__ void __launch_bounds__(kTeam * kTeamsPerCta, NE <= 8 ? 2 : 1)   // two CTAs per SM while the rows fit 64 registers
+jacobi_sweeps_kernel(const Ptrs<double> Tb, int nb, int b, int sweeps, double tol, const Ptrs<unsigned long long> offb,
                      unsigned int* __restrict__ sync_words, int32_t* __restrict__ status) {
   __shared__ double red[kTeamsPerCta][3][kTeam / 32];
+  __shared__ double s_worst[kTeamsPerCta][kMaxBatch];
   const int team = threadIdx.x / kTeam, tt = threadIdx.x % kTeam, tw = tt >> 5, lane = threadIdx.x & 31;
-  const int pairs = b / 2, batch = (int)gridDim.x * kTeamsPerCta;
+  const int pairs = b / 2, jobs = pairs * nb, batch = (int)gridDim.x * kTeamsPerCta;
   unsigned int gen = 0;
-  bool converged = false;
-  for (int sw = 0; sw < sweeps && !converged; ++sw) {
-    double worst = 0.0;
+  uint32_t active = (1u << nb) - 1u;                // matrices still rotating
+  for (int sw = 0; sw < sweeps && active != 0u; ++sw) {
+    if (tt < kMaxBatch) s_worst[team][tt] = 0.0;
     for (int rnd = 0; rnd < b - 1; ++rnd) {
-      for (int k0 = 0; k0 < pairs; k0 += batch) {
+      for (int k0 = 0; k0 < jobs; k0 += batch) {
         const int k = k0 + (int)blockIdx.x * kTeamsPerCta + team;
-        const bool live = k < pairs;
+        const int mat = k < jobs ? k / pairs : 0;
+        const bool live = k < jobs && ((active >> mat) & 1u);
         int p = 0, q = 0;
-        if (live) tournament_pair(b, rnd, k, p, q);
-        double* tp = T + (int64_t)p * b;
-        double* tq = T + (int64_t)q * b;
+        if (live) tournament_pair(b, rnd, k - mat * pairs, p, q);
+        double* tp = Tb.p[mat] + (int64_t)p * b;
+        double* tq = Tb.p[mat] + (int64_t)q * b;
         double x[NE], y[NE];
         double a = 0.0, c = 0.0, d = 0.0;
 #pragma unroll
@@ -310,7 +353,7 @@ jacobi_sweeps_kernel(double* __restrict__ T, int b, int sweeps, double tol, unsi
           d += __shfl_xor_sync(0xFFFFFFFFu, d, o);
           c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
         }
-        __syncthreads();                               // the previous batch has read `red`
+        __syncthreads();                               // the previous job has read `red`
         if (lane == 0) { red[team][0][tw] = a; red[team][1][tw] = d; red[team][2][tw] = c; }
         __syncthreads();
         a = red[team][0][0] + red[team][0][1] + red[team][0][2] + red[team][0][3];
@@ -318,7 +361,7 @@ jacobi_sweeps_kernel(double* __restrict__ T, int b, int sweeps, double tol, unsi
         c = red[team][2][0] + red[team][2][1] + red[team][2][2] + red[team][2][3];
         const double denom = sqrt(a * d);
         const double rel = denom > 0.0 ? fabs(c) / denom : 0.0;
-        worst = fmax(worst, rel);
+        if (live && tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], rel);
         if (live && rel >= 1e-15) {
           const double zeta = (d - a) / (2.0 * c);
           const double tn = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
@@ -333,32 +376,38 @@ jacobi_sweeps_kernel(double* __restrict__ T, int b, int sweeps, double tol, unsi
           }
         }
       }
-      if (rnd == b - 2 && tt == 0 && worst > 0.0) {
+      if (rnd == b - 2) {
+        __syncthreads();
         // only ever compared, so the monotone integer view of a non-negative double serves atomicMax
-        atomicMax(off + sw, (unsigned long long)__double_as_longlong(worst));
+        if (tt < nb && s_worst[team][tt] > 0.0)
+          atomicMax(offb.p[tt] + sw, (unsigned long long)__double_as_longlong(s_worst[team][tt]));
       }
       if (!grid_barrier(sync_words, sync_words + 1, gen)) {
         if (threadIdx.x == 0 && status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
         return;
       }
     }
-    converged = __longlong_as_double((long long)__ldcg(off + sw)) <= tol;
+    for (int i = 0; i < nb; ++i)
+      if (((active >> i) & 1u) && __longlong_as_double((long long)__ldcg(offb.p[i] + sw)) <= tol) active &= ~(1u << i);
+    __syncthreads();                                 // s_worst is cleared at the top of the next sweep
   }
-  if (!converged && blockIdx.x == 0 && threadIdx.x == 0 && status) atomicOr(status, QG_DEV_NOT_CONVERGED);
+  if (active != 0u && blockIdx.x == 0 && threadIdx.x == 0 && status) atomicOr(status, QG_DEV_NOT_CONVERGED);
 }
 
 template <int NE>
-int launch_jacobi(double* T, int64_t b, int sweeps, double tol, unsigned long long* off, unsigned int* sync_words,
-                  int32_t* status, cudaStream_t st) {
+int launch_jacobi(const Ptrs<double>& T, int nb, int64_t b, int sweeps, double tol, const Ptrs<unsigned long long>& off,
+                  unsigned int* sync_words, int32_t* status, cudaStream_t st) {
   // one cooperative launch, never more CTAs than are resident at once
   int per_sm = 0;
   QG_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_sweeps_kernel<NE>, kTeam * kTeamsPerCta, 0));
   const int64_t resident = (int64_t)per_sm * refresh_sm_count();
   if (resident < 1) { note_cuda_error(cudaErrorCooperativeLaunchTooLarge, "jacobi_sweeps_kernel occupancy"); return QG_CUDA_ERROR; }
-  int64_t grid = ceil_div(b / 2, kTeamsPerCta);
+  int64_t grid = ceil_div(b / 2 * nb, kTeamsPerCta);
   if (grid > resident) grid = resident;
   int bi = (int)b;
-  void* args[] = {&T, &bi, &sweeps, &tol, &off, &sync_words, &status};
+  Ptrs<double> Tc = T;
+  Ptrs<unsigned long long> offc = off;
+  void* args[] = {&Tc, &nb, &bi, &sweeps, &tol, &offc, &sync_words, &status};
   QG_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)jacobi_sweeps_kernel<NE>, dim3((unsigned)grid), dim3(kTeam * kTeamsPerCta),
                                           args, 0, st));
   count_launch();
@@ -367,8 +416,9 @@ int launch_jacobi(double* T, int64_t b, int sweeps, double tol, unsigned long lo
 
 // lambda_j = norm of row j of the rotated T (= |eigenvalue j|); rank_j = its position in descending order
 __global__ void __launch_bounds__(128)
-row_norm_kernel(const double* __restrict__ T, int b, double* __restrict__ lam) {
-  const double* row = T + (int64_t)blockIdx.x * b;
+row_norm_kernel(const Ptrs<const double> Tb, int b, const Ptrs<double> lamb) {
+  const double* row = Tb.p[blockIdx.y] + (int64_t)blockIdx.x * b;
+  double* __restrict__ lam = lamb.p[blockIdx.y];
   double s = 0.0;
   for (int i = threadIdx.x; i < b; i += blockDim.x) s += row[i] * row[i];
   __shared__ double red[4];
@@ -381,7 +431,10 @@ row_norm_kernel(const double* __restrict__ T, int b, double* __restrict__ lam) {
 
 // Xsel[i][rank_j] = X[i][j] = T[j][i] / lambda_j for the r largest lambda_j
 __global__ void __launch_bounds__(256)
-select_top_kernel(const double* __restrict__ T, const double* __restrict__ lam, int b, int r, float* __restrict__ Xsel) {
+select_top_kernel(const Ptrs<const double> Tb, const Ptrs<const double> lamb, int b, int r, const Ptrs<float> Xselb) {
+  const double* __restrict__ T = Tb.p[blockIdx.y];
+  const double* __restrict__ lam = lamb.p[blockIdx.y];
+  float* __restrict__ Xsel = Xselb.p[blockIdx.y];
   const int j = blockIdx.x;
   const double lj = lam[j];
   __shared__ int s_rank;
@@ -402,7 +455,9 @@ select_top_kernel(const double* __restrict__ T, const double* __restrict__ lam, 
 
 // Each column of P gets the sign that makes its largest-magnitude entry positive; optional copy to P_out.
 __global__ void __launch_bounds__(256)
-sign_fix_kernel(float* __restrict__ P, int64_t m, int r, float* __restrict__ P_out) {
+sign_fix_kernel(const Ptrs<float> Pb, int64_t m, int r, const Ptrs<float> P_outb) {
+  float* __restrict__ P = Pb.p[blockIdx.y];
+  float* __restrict__ P_out = P_outb.p[blockIdx.y];
   const int j = blockIdx.x;
   float best = 0.f, bestv = 0.f;
   for (int64_t i = threadIdx.x; i < m; i += blockDim.x) {
@@ -453,31 +508,53 @@ size_t carve_refresh(void* base, int64_t m, int64_t n, int64_t b, int64_t r, Ref
   return off;
 }
 
-// Q <- orthonormal basis of the columns of Y (m x b, both pitch b), panel by panel.
-int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cudaStream_t st) {
+// The workspaces of the matrices of one batch, and pointer tables into them.
+struct Batch {
+  int nb;
+  RefreshWs w[kMaxBatch];
+  template <class T, class F>
+  Ptrs<T> tab(F field, int64_t off = 0) const {
+    Ptrs<T> t{};
+    for (int i = 0; i < nb; ++i) t.p[i] = field(w[i]) + off;
+    return t;
+  }
+};
+#define QG_TAB(T, member) bt.tab<T>([](const RefreshWs& x) { return x.member; })
+#define QG_TAB_OFF(T, member, off) bt.tab<T>([](const RefreshWs& x) { return x.member; }, (off))
+
+// Q <- orthonormal basis of the columns of Y (m x b, both pitch b), panel by panel, for every matrix of the batch.
+int orthonormalize(const Batch& bt, int64_t m, int64_t b, int32_t* status, cudaStream_t st) {
+  const int nb = bt.nb;
+  Ptrs<void> part{};
+  for (int i = 0; i < nb; ++i) part.p[i] = bt.w[i].part;
+  const Ptrs<const float> Q = QG_TAB(const float, Q);
+  const Ptrs<float> Cb = QG_TAB(float, Cb), S = QG_TAB(float, S), Linv = QG_TAB(float, Linv), Wp = QG_TAB(float, Wp);
+  const Ptrs<const float> Cbc = QG_TAB(const float, Cb), Sc = QG_TAB(const float, S), Linvc = QG_TAB(const float, Linv),
+                          Wpc = QG_TAB(const float, Wp);
   for (int64_t j0 = 0; j0 < b; j0 += kPanel) {
-    float* Yj = w.Y + j0;
-    float* Qj = w.Q + j0;
+    const Ptrs<float> Yj = QG_TAB_OFF(float, Y, j0), Qj = QG_TAB_OFF(float, Q, j0);
+    const Ptrs<const float> Yjc = QG_TAB_OFF(const float, Y, j0);
     int rc;
     for (int pass = 0; pass < 2 && j0 > 0; ++pass) {
       // C = Q[:, :j0]^T Yj   (j0 x 64);   Yj -= Q[:, :j0] C
-      rc = gemm<float, float, float>(w.Q, 1, b, Yj, b, 1, w.Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st, w.part);
+      rc = gemm<float, float, float>(nb, Q, 1, b, Yjc, b, 1, Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st, &part);
       if (rc != QG_OK) return rc;
-      rc = gemm<float, float, float>(w.Q, b, 1, w.Cb, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st, w.part);
+      rc = gemm<float, float, float>(nb, Q, b, 1, Cbc, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st, &part);
       if (rc != QG_OK) return rc;
     }
     // two rounds of Cholesky QR on the panel: Yj -> Wp -> Qj
-    const float* src = Yj; int64_t lds = b;
-    float* dst = w.Wp; int64_t ldd = kPanel;
     for (int pass = 0; pass < 2; ++pass) {
-      rc = gemm<float, float, float>(src, 1, lds, src, lds, 1, w.S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st, w.part);
+      const Ptrs<const float>& src = pass == 0 ? Yjc : Wpc;
+      const int64_t lds = pass == 0 ? b : kPanel;
+      const Ptrs<float>& dst = pass == 0 ? Wp : Qj;
+      const int64_t ldd = pass == 0 ? kPanel : b;
+      rc = gemm<float, float, float>(nb, src, 1, lds, src, lds, 1, S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st, &part);
       if (rc != QG_OK) return rc;
-      chol64_inverse_kernel<<<1, 256, 0, st>>>(w.S, w.Linv, status);
+      chol64_inverse_kernel<<<nb, 256, 0, st>>>(Sc, Linv, status);
       QG_LAUNCH_CHECK();
       // dst = src * Linv^T:  B(k, j) = Linv[j][k]
-      rc = gemm<float, float, float>(src, lds, 1, w.Linv, 1, kPanel, dst, ldd, m, kPanel, kPanel, 1.f, 0.f, st);
+      rc = gemm<float, float, float>(nb, src, lds, 1, Linvc, 1, kPanel, dst, ldd, m, kPanel, kPanel, 1.f, 0.f, st);
       if (rc != QG_OK) return rc;
-      src = w.Wp; lds = kPanel; dst = Qj; ldd = b;
     }
   }
   return QG_OK;
@@ -487,48 +564,64 @@ int orthonormalize(const RefreshWs& w, int64_t m, int64_t b, int32_t* status, cu
 
 size_t refresh_workspace_bytes(int64_t m, int64_t n, int64_t b) { return carve_refresh(nullptr, m, n, b, b, nullptr); }
 
-// `transposed`: the singular vectors wanted are the RIGHT ones of G, i.e. the left ones of G^T; G is then read
-// with its two strides swapped and (m, n) below are the extents of G^T.
-int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
-                   uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
-                   cudaStream_t st, bool transposed) {
+// One batch (at most kMaxBatch matrices of one shape).  `transposed`: the singular vectors wanted are the RIGHT ones
+// of G, i.e. the left ones of G^T; G is then read with its two strides swapped and (m, n) are the extents of G^T.
+static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
+                         char* ws, size_t ws_stride, int32_t* status, cudaStream_t st, bool transposed) {
+  Batch bt{};
+  bt.nb = nb;
+  Ptrs<const uint16_t> G{};
+  Ptrs<const void> seeds{};
+  Ptrs<float> P_out{};
+  int64_t ldg = jobs[0].ldg;
+  for (int i = 0; i < nb; ++i) {
+    carve_refresh(ws + (size_t)i * ws_stride, m, n, b, r, &bt.w[i]);
+    G.p[i] = jobs[i].G;
+    seeds.p[i] = reinterpret_cast<const void*>((uintptr_t)jobs[i].seed);
+    P_out.p[i] = jobs[i].P_fp32;
+    if (jobs[i].ldg != ldg) return QG_INVALID_ARGUMENT;          // one pitch per batch (the caller groups by it)
+  }
   const int64_t rs = transposed ? 1 : ldg, cs = transposed ? ldg : 1;   // strides between rows / columns of the matrix
-  RefreshWs w;
-  if (carve_refresh(ws, m, n, b, r, &w) > ws_bytes) return QG_WORKSPACE_TOO_SMALL;
+  const Ptrs<const float> Q = QG_TAB(const float, Q), Z = QG_TAB(const float, Z), Xsel = QG_TAB(const float, Xsel);
+  const Ptrs<float> Y = QG_TAB(float, Y), Zw = QG_TAB(float, Z), P32 = QG_TAB(float, P32);
   int rc;
   // start block
   {
     const int64_t threads = m * (b / 4);
-    gaussian_kernel<<<(unsigned)ceil_div(threads, 256), 256, 0, st>>>(w.Y, b, m, b, (uint32_t)seed, (uint32_t)(seed >> 32));
+    gaussian_kernel<<<dim3((unsigned)ceil_div(threads, 256), (unsigned)nb), 256, 0, st>>>(Y, b, m, b, seeds);
     QG_LAUNCH_CHECK();
-    rc = orthonormalize(w, m, b, status, st);
+    rc = orthonormalize(bt, m, b, status, st);
     if (rc != QG_OK) return rc;
   }
   for (int it = 0; it <= iters; ++it) {
     // Z = G^T Q
-    rc = gemm<uint16_t, float, float>(G, cs, rs, w.Q, b, 1, w.Z, b, n, b, m, 1.f, 0.f, st);
+    rc = gemm<uint16_t, float, float>(nb, G, cs, rs, Q, b, 1, Zw, b, n, b, m, 1.f, 0.f, st);
     if (rc != QG_OK) return rc;
     if (it == iters) break;
     // Y = G Z
-    rc = gemm<uint16_t, float, float>(G, rs, cs, w.Z, b, 1, w.Y, b, m, b, n, 1.f, 0.f, st);
+    rc = gemm<uint16_t, float, float>(nb, G, rs, cs, Z, b, 1, Y, b, m, b, n, 1.f, 0.f, st);
     if (rc != QG_OK) return rc;
-    rc = orthonormalize(w, m, b, status, st);
+    rc = orthonormalize(bt, m, b, status, st);
     if (rc != QG_OK) return rc;
   }
   // Rayleigh-Ritz: T = Z^T Z in fp64, eigenvectors by one-sided Jacobi
-  rc = gemm<float, double, double>(w.Z, 1, b, w.Z, b, 1, w.T, b, b, b, n, 1.0, 0.0, st);
+  const Ptrs<double> T = QG_TAB(double, T), lam = QG_TAB(double, lam);
+  rc = gemm<float, double, double>(nb, Z, 1, b, Z, b, 1, T, b, b, b, n, 1.0, 0.0, st);
   if (rc != QG_OK) return rc;
   if (sweeps > kMaxSweeps) sweeps = kMaxSweeps;
-  QG_CUDA_TRY(cudaMemsetAsync(w.off, 0, kMaxSweeps * 8, st));
-  QG_CUDA_TRY(cudaMemsetAsync(w.done, 0, 8, st));
+  Ptrs<unsigned long long> off{};
+  for (int i = 0; i < nb; ++i) {
+    QG_CUDA_TRY(cudaMemsetAsync(bt.w[i].off, 0, kMaxSweeps * 8, st));
+    off.p[i] = reinterpret_cast<unsigned long long*>(bt.w[i].off);
+  }
+  QG_CUDA_TRY(cudaMemsetAsync(bt.w[0].done, 0, 8, st));
   {
-    unsigned long long* off = reinterpret_cast<unsigned long long*>(w.off);
-    unsigned int* sync_words = reinterpret_cast<unsigned int*>(w.done);
+    unsigned int* sync_words = reinterpret_cast<unsigned int*>(bt.w[0].done);
     // the iteration converges quadratically at the end: a sweep that met nothing above 1e-5 leaves ~1e-10
     constexpr double kTol = 1e-5;
-    // Refreshes of several matrices may run on several streams at once (their many small kernels overlap
-    // well), but two grids whose CTAs wait for one another must never be half resident together: each
-    // cooperative launch waits for the previous one of this process on the device, whatever its stream.
+    // Refreshes may run on several streams at once (their many small kernels overlap well), but two grids whose
+    // CTAs wait for one another must never be half resident together: each cooperative launch waits for the
+    // previous one of this process on the device, whatever its stream.
     std::lock_guard<std::mutex> lock(g_coop_mutex);
     int dev = 0;
     QG_CUDA_TRY(cudaGetDevice(&dev));
@@ -539,22 +632,50 @@ int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t
       if (!g_coop_done[dev]) QG_CUDA_TRY(cudaEventCreateWithFlags(&g_coop_done[dev], cudaEventDisableTiming));
       else QG_CUDA_TRY(cudaStreamWaitEvent(st, g_coop_done[dev], 0));
     }
-    if (b <= 8 * kTeam) rc = launch_jacobi<8>(w.T, b, sweeps, kTol, off, sync_words, status, st);
-    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(w.T, b, sweeps, kTol, off, sync_words, status, st);
-    else rc = launch_jacobi<32>(w.T, b, sweeps, kTol, off, sync_words, status, st);
+    if (b <= 8 * kTeam) rc = launch_jacobi<8>(T, nb, b, sweeps, kTol, off, sync_words, status, st);
+    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(T, nb, b, sweeps, kTol, off, sync_words, status, st);
+    else rc = launch_jacobi<32>(T, nb, b, sweeps, kTol, off, sync_words, status, st);
     if (rc != QG_OK) return rc;
     if (chain) QG_CUDA_TRY(cudaEventRecord(g_coop_done[dev], st));
   }
-  row_norm_kernel<<<(unsigned)b, 128, 0, st>>>(w.T, (int)b, w.lam);
+  const Ptrs<const double> Tc = QG_TAB(const double, T), lamc = QG_TAB(const double, lam);
+  row_norm_kernel<<<dim3((unsigned)b, (unsigned)nb), 128, 0, st>>>(Tc, (int)b, lam);
   QG_LAUNCH_CHECK();
-  select_top_kernel<<<(unsigned)b, 256, 0, st>>>(w.T, w.lam, (int)b, (int)r, w.Xsel);
+  select_top_kernel<<<dim3((unsigned)b, (unsigned)nb), 256, 0, st>>>(Tc, lamc, (int)b, (int)r, QG_TAB(float, Xsel));
   QG_LAUNCH_CHECK();
   // P = Q Xsel
-  rc = gemm<float, float, float>(w.Q, b, 1, w.Xsel, r, 1, w.P32, r, m, r, b, 1.f, 0.f, st);
+  rc = gemm<float, float, float>(nb, Q, b, 1, Xsel, r, 1, P32, r, m, r, b, 1.f, 0.f, st);
   if (rc != QG_OK) return rc;
-  sign_fix_kernel<<<(unsigned)r, 256, 0, st>>>(w.P32, m, (int)r, P_fp32);
+  sign_fix_kernel<<<dim3((unsigned)r, (unsigned)nb), 256, 0, st>>>(P32, m, (int)r, P_out);
   QG_LAUNCH_CHECK();
-  return launch_quantize_rtn(P_new->bits, w.P32, m, r, r, P_new, st);
+  for (int i = 0; i < nb; ++i) {
+    rc = launch_quantize_rtn(jobs[i].P_new->bits, bt.w[i].P32, m, r, r, jobs[i].P_new, st);
+    if (rc != QG_OK) return rc;
+  }
+  return QG_OK;
+}
+
+// `count` matrices of one shape, in batches of as many as the workspace holds (at most kMaxBatch).
+int launch_refresh_batched(const RefreshJob* jobs, int count, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
+                           void* ws, size_t ws_bytes, int32_t* status, cudaStream_t st, bool transposed) {
+  const size_t stride = refresh_workspace_bytes(m, n, b);
+  int64_t fit = (int64_t)(ws_bytes / stride);
+  if (fit < 1) return QG_WORKSPACE_TOO_SMALL;
+  if (fit > kMaxBatch) fit = kMaxBatch;
+  for (int first = 0; first < count; first += (int)fit) {
+    const int nb = count - first < (int)fit ? count - first : (int)fit;
+    const int rc = refresh_batch(jobs + first, nb, m, n, r, b, iters, sweeps, reinterpret_cast<char*>(ws), stride, status, st,
+                                 transposed);
+    if (rc != QG_OK) return rc;
+  }
+  return QG_OK;
+}
+
+int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
+                   uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
+                   cudaStream_t st, bool transposed) {
+  const RefreshJob job{G, ldg, seed, P_new, P_fp32};
+  return launch_refresh_batched(&job, 1, m, n, r, b, iters, sweeps, ws, ws_bytes, status, st, transposed);
 }
 
 }  // namespace qg

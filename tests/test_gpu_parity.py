@@ -156,6 +156,34 @@ def test_refresh_replayed_from_a_cuda_graph_gives_the_same_codes():
     assert torch.equal(P_new.codes, want.codes) and torch.equal(P_new.zeros, want.zeros)
 
 
+@pytest.mark.parametrize("side,m,n,r,max_batch", [("left", 512, 768, 128, 8), ("left", 320, 256, 64, 2), ("right", 768, 320, 64, 3)])
+def test_batched_refresh_equals_single_calls(side, m, n, r, max_batch):
+    """Five matrices of one shape refreshed in one call (in batches of max_batch: 5, 2 + 2 + 1, 3 + 2) give, matrix by
+    matrix, the codes, the vectors and the similarity of five single calls."""
+    right = side == "right"
+    pm = n if right else m
+    gms = [synth.GradientModel(m, n, seed=40, matrix_index=i) for i in range(5)]
+    Gs = [g_to_device(gm.sample(1)) for gm in gms]
+    prev = [B.refresh_subspace(g_to_device(gm.sample(2)), r, seed=9, side=side) for gm in gms]
+    single, items = [], []
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for i, G in enumerate(Gs):
+        P32 = torch.zeros((pm, r), dtype=torch.float32, device="cuda")
+        sim = torch.zeros(1, dtype=torch.float32, device="cuda")
+        Pn = B.refresh_subspace(G, r, seed=100 + i, P_fp32=P32, P_prev=prev[i], sim_cols=8, sim=sim, status=status, side=side)
+        single.append((Pn, P32, sim))
+        items.append({"G": G, "seed": 100 + i, "P_fp32": torch.zeros((pm, r), dtype=torch.float32, device="cuda"), "P_prev": prev[i],
+                      "sim": torch.zeros(1, dtype=torch.float32, device="cuda")})
+    got = B.refresh_subspace_batched(items, r, sim_cols=8, max_batch=max_batch, status=status, side=side)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for (Pn, P32, sim), it, Pb in zip(single, items, got):
+        assert torch.equal(Pn.codes, Pb.codes) and torch.equal(Pn.scales, Pb.scales) and torch.equal(Pn.zeros, Pb.zeros)
+        assert torch.equal(P32, it["P_fp32"]) and torch.equal(sim, it["sim"])
+    with pytest.raises((B.QgError, ValueError)):      # one shape per call
+        B.refresh_subspace_batched([items[0], {"G": g_to_device(synth.GradientModel(m, n + 64, seed=1).sample(1)), "seed": 1}], r)
+
+
 def test_refresh_rejects_bad_block_widths():
     dG = torch.zeros((128, 256), dtype=torch.int16, device="cuda")
     with pytest.raises(B.QgError) as e:
