@@ -87,11 +87,13 @@ def k2_alu_ops(m, n, r):
 
 
 def load_ncu_traffic(kernel_revision):
-    """DRAM bytes per weight element of each kernel, per workload, from the ncu captures summarised under
-    profiles/ (read from the small table beside them).  A row counts only if it was taken on the kernels as they
-    stand: its revision tag must equal the one the library reports.  Returns {workload: {kernel: bytes/element}}."""
+    """Measured DRAM bytes over algorithmic bytes of each kernel, per workload, from the ncu captures summarised
+    under profiles/ (read from the small table beside them).  A row counts only if it was taken on the kernels as
+    they stand: its revision tag must equal the one the library reports.  The captures are of small cases (a few
+    layers); every kernel streams each byte once, so its traffic grows in proportion to its algorithmic bytes and
+    the ratio carries over to a full launch.  Returns {workload: {kernel: ratio}}."""
     table = {}
-    path = os.path.join(ROOT, "profiles", "dram_traffic_per_element.txt")
+    path = os.path.join(ROOT, "profiles", "dram_traffic_ratio.txt")
     if not os.path.exists(path):
         return table
     with open(path) as f:
@@ -99,9 +101,9 @@ def load_ncu_traffic(kernel_revision):
             f4 = line.split()
             if len(f4) < 4 or line.startswith("#"):
                 continue
-            workload, kernel, per_element, revision = f4[0], f4[1], float(f4[2]), f4[3]
+            workload, kernel, ratio, revision = f4[0], f4[1], float(f4[2]), f4[3]
             if revision == kernel_revision:
-                table.setdefault(workload, {})[kernel] = per_element
+                table.setdefault(workload, {})[kernel] = ratio
     return table
 
 
@@ -483,10 +485,12 @@ def bench_workload(workload, args, B, torch, dist, device, world, rank, local_ra
         if roof["bound"] == "tensor":
             roof["frac_of_sustained_peak"] = roof["achieved"] / peak_tf_sus
             roof["sustained_peak"] = peak_tf_sus
-        traffic = extras["traffic"].get(workload, {}) if (args.moments == 32 and not args.layers) else {}
+        # measured DRAM traffic per launch = (ratio from the committed ncu capture) x (algorithmic bytes per launch)
+        traffic = extras["traffic"].get(workload, {}) if args.moments == 32 else {}
         tpe = traffic.get(dom_name)
-        roof["traffic"] = None if tpe is None else tpe * elements * args.steps / max(kcount[dom], 1)
-        roof["traffic_per_kernel_per_launch"] = {nm: (traffic[nm] * elements * args.steps / max(kcount[names.index(nm)], 1))
+        roof["traffic"] = None if tpe is None else tpe * k_bytes / max(kcount[dom], 1)
+        roof["traffic_over_algorithmic"] = tpe
+        roof["traffic_per_kernel_per_launch"] = {nm: traffic[nm] * per_kernel[nm]["bytes"] * args.steps / max(kcount[names.index(nm)], 1)
                                                  for nm in per_kernel if nm in traffic} or None
         roof["kernel"] = dom_name
         roof["kernel_revision"] = extras["revision"]
