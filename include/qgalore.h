@@ -352,6 +352,9 @@ QG_API int qgalore_debug_set_pair_mode(int mask);
  * to bf16 by a separate grouped launch first, as for 2- and 8-bit codes.  Applies to calls and plans made
  * afterwards; the results are the same bit for bit. */
 QG_API int qgalore_debug_set_fused_dequant(int on);
+/* 1 (the default): the early iterations of a refresh take their two products with the gradient on the tensor cores
+ * (the iterate split into three bfloat16 planes); 0: every product on the CUDA cores. */
+QG_API int qgalore_debug_set_refresh_tensor_cores(int on);
 /* Scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks mean
  * fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
 QG_API int qgalore_debug_set_chunk_budget(size_t bytes);

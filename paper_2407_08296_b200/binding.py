@@ -118,6 +118,7 @@ def lib() -> C.CDLL:
         L.qgalore_debug_set_step_impl.argtypes = [C.c_int]
         L.qgalore_debug_set_pair_mode.argtypes = [C.c_int]
         L.qgalore_debug_set_fused_dequant.argtypes = [C.c_int]
+        L.qgalore_debug_set_refresh_tensor_cores.argtypes = [C.c_int]
         L.qgalore_debug_set_chunk_budget.argtypes = [sz]
         L.qgalore_debug_expire_wait.argtypes = [i32, vp, vp, vp]
         _lib = L
@@ -614,6 +615,10 @@ def debug_set_pair_mode(mask: int) -> None:
 
 def debug_set_fused_dequant(on: bool) -> None:
     _check(lib().qgalore_debug_set_fused_dequant(1 if on else 0), "qgalore_debug_set_fused_dequant")
+
+
+def debug_set_refresh_tensor_cores(on: bool) -> None:
+    _check(lib().qgalore_debug_set_refresh_tensor_cores(1 if on else 0), "qgalore_debug_set_refresh_tensor_cores")
 
 
 def debug_expire_wait(polls: int, status: torch.Tensor, polls_used: torch.Tensor | None = None, stream=None) -> None:

@@ -29,11 +29,20 @@
 
 namespace qg {
 
+// refresh_tc.cu: the tensor-core route of the two products with the gradient
+size_t split_planes_bytes(int64_t K, int64_t N);
+bool split_gemm_supported(const uint16_t* A, int64_t sa_m, int64_t sa_k, int64_t M, int64_t N, int64_t K);
+int launch_split_gemm(const uint16_t* A, int64_t sa_m, int64_t sa_k, const float* B, int64_t ldb, float* D, int64_t ldd,
+                      int64_t M, int64_t N, int64_t K, uint16_t* planes, int32_t* status, cudaStream_t st);
+
 namespace {
 
 constexpr int kCoopDevices = 64;
 std::mutex g_coop_mutex;
 cudaEvent_t g_coop_done[kCoopDevices] = {};   // completion of the last cooperative launch, per device ordinal
+
+// Test aid: 0 keeps every product of the refresh on the CUDA cores.
+int g_refresh_tc = 1;
 
 constexpr int kPanel = 64;    // columns orthonormalised together
 constexpr int kMaxSweeps = 32;
@@ -482,6 +491,7 @@ sign_fix_kernel(const Ptrs<float> Pb, int64_t m, int r, const Ptrs<float> P_outb
 struct RefreshWs {
   float *Q, *Y, *Z, *Wp, *Cb, *S, *Linv, *Xsel, *P32;
   void* part;      // partial sums of sliced products
+  uint16_t* planes;  // the three bfloat16 planes of an iterate, for the tensor-core products
   double *T, *lam, *off;
   int32_t* done;
 };
@@ -504,6 +514,7 @@ size_t carve_refresh(void* base, int64_t m, int64_t n, int64_t b, int64_t r, Ref
   t.Xsel = (float*)take((size_t)b * r * 4);
   t.P32 = (float*)take((size_t)m * r * 4);
   t.part = take((size_t)kSplitScratch);
+  t.planes = (uint16_t*)take(split_planes_bytes(m > n ? m : n, b));
   if (w) *w = t;
   return off;
 }
@@ -593,14 +604,36 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
     rc = orthonormalize(bt, m, b, status, st);
     if (rc != QG_OK) return rc;
   }
+  // The two products with the gradient go to the tensor cores (bfloat16 gradient times an iterate split into three
+  // bfloat16 planes, fp32 accumulation: refresh_tc.cu), one launch per matrix, where shape and strides allow it.
+  // Their rounding differs from the CUDA-core kernel's only in the order of an fp32 accumulation; errors made in
+  // an early iteration are damped by the later ones, and the last full iteration and the product that feeds the
+  // Rayleigh-Ritz step keep the CUDA-core kernel, whose accumulation is not biased toward zero.
+  const bool tc_z = g_refresh_tc && split_gemm_supported(G.p[0], cs, rs, n, b, m);   // Z = X^T Q: A(i, k) = X[k][i]
+  const bool tc_y = g_refresh_tc && split_gemm_supported(G.p[0], rs, cs, m, b, n);   // Y = X Z:   A(i, k) = X[i][k]
   for (int it = 0; it <= iters; ++it) {
+    const bool early = it + 1 < iters;
     // Z = G^T Q
-    rc = gemm<uint16_t, float, float>(nb, G, cs, rs, Q, b, 1, Zw, b, n, b, m, 1.f, 0.f, st);
-    if (rc != QG_OK) return rc;
+    if (tc_z && early) {
+      for (int i = 0; i < nb; ++i) {
+        rc = launch_split_gemm(G.p[i], cs, rs, bt.w[i].Q, b, bt.w[i].Z, b, n, b, m, bt.w[i].planes, status, st);
+        if (rc != QG_OK) return rc;
+      }
+    } else {
+      rc = gemm<uint16_t, float, float>(nb, G, cs, rs, Q, b, 1, Zw, b, n, b, m, 1.f, 0.f, st);
+      if (rc != QG_OK) return rc;
+    }
     if (it == iters) break;
     // Y = G Z
-    rc = gemm<uint16_t, float, float>(nb, G, rs, cs, Z, b, 1, Y, b, m, b, n, 1.f, 0.f, st);
-    if (rc != QG_OK) return rc;
+    if (tc_y && early) {
+      for (int i = 0; i < nb; ++i) {
+        rc = launch_split_gemm(G.p[i], rs, cs, bt.w[i].Z, b, bt.w[i].Y, b, m, b, n, bt.w[i].planes, status, st);
+        if (rc != QG_OK) return rc;
+      }
+    } else {
+      rc = gemm<uint16_t, float, float>(nb, G, rs, cs, Z, b, 1, Y, b, m, b, n, 1.f, 0.f, st);
+      if (rc != QG_OK) return rc;
+    }
     rc = orthonormalize(bt, m, b, status, st);
     if (rc != QG_OK) return rc;
   }
@@ -670,6 +703,8 @@ int launch_refresh_batched(const RefreshJob* jobs, int count, int64_t m, int64_t
   }
   return QG_OK;
 }
+
+int set_refresh_tc(int on) { g_refresh_tc = on ? 1 : 0; return QG_OK; }
 
 int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
                    uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,
