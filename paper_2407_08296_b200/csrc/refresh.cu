@@ -534,7 +534,13 @@ struct Batch {
 #define QG_TAB_OFF(T, member, off) bt.tab<T>([](const RefreshWs& x) { return x.member; }, (off))
 
 // Q <- orthonormal basis of the columns of Y (m x b, both pitch b), panel by panel, for every matrix of the batch.
-int orthonormalize(const Batch& bt, int64_t m, int64_t b, int32_t* status, cudaStream_t st) {
+// `full`: every projection applied twice and two rounds of Cholesky QR per panel: orthonormal to fp32 rounding, what
+// the Rayleigh-Ritz step and the returned vectors need.  Otherwise one of each: the basis comes out orthonormal to
+// about 1e-2 (fp32 Gram matrices of panels with a condition number of several hundred), which is all an
+// intermediate subspace iteration asks of it: the next multiplication by G G^T and the next orthonormalisation
+// start from that basis, they do not inherit its error.
+int orthonormalize(const Batch& bt, int64_t m, int64_t b, int32_t* status, cudaStream_t st, bool full) {
+  const int passes = full ? 2 : 1;
   const int nb = bt.nb;
   Ptrs<void> part{};
   for (int i = 0; i < nb; ++i) part.p[i] = bt.w[i].part;
@@ -546,19 +552,20 @@ int orthonormalize(const Batch& bt, int64_t m, int64_t b, int32_t* status, cudaS
     const Ptrs<float> Yj = QG_TAB_OFF(float, Y, j0), Qj = QG_TAB_OFF(float, Q, j0);
     const Ptrs<const float> Yjc = QG_TAB_OFF(const float, Y, j0);
     int rc;
-    for (int pass = 0; pass < 2 && j0 > 0; ++pass) {
+    for (int pass = 0; pass < passes && j0 > 0; ++pass) {
       // C = Q[:, :j0]^T Yj   (j0 x 64);   Yj -= Q[:, :j0] C
       rc = gemm<float, float, float>(nb, Q, 1, b, Yjc, b, 1, Cb, kPanel, j0, kPanel, m, 1.f, 0.f, st, &part);
       if (rc != QG_OK) return rc;
       rc = gemm<float, float, float>(nb, Q, b, 1, Cbc, kPanel, 1, Yj, b, m, kPanel, j0, -1.f, 1.f, st, &part);
       if (rc != QG_OK) return rc;
     }
-    // two rounds of Cholesky QR on the panel: Yj -> Wp -> Qj
-    for (int pass = 0; pass < 2; ++pass) {
+    // Cholesky QR on the panel, two rounds (Yj -> Wp -> Qj) or one (Yj -> Qj)
+    for (int pass = 0; pass < passes; ++pass) {
+      const bool last = pass + 1 == passes;
       const Ptrs<const float>& src = pass == 0 ? Yjc : Wpc;
       const int64_t lds = pass == 0 ? b : kPanel;
-      const Ptrs<float>& dst = pass == 0 ? Wp : Qj;
-      const int64_t ldd = pass == 0 ? kPanel : b;
+      const Ptrs<float>& dst = last ? Qj : Wp;
+      const int64_t ldd = last ? b : kPanel;
       rc = gemm<float, float, float>(nb, src, 1, lds, src, lds, 1, S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st, &part);
       if (rc != QG_OK) return rc;
       chol64_inverse_kernel<<<nb, 256, 0, st>>>(Sc, Linv, status);
@@ -601,20 +608,20 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
     const int64_t threads = m * (b / 4);
     gaussian_kernel<<<dim3((unsigned)ceil_div(threads, 256), (unsigned)nb), 256, 0, st>>>(Y, b, m, b, seeds);
     QG_LAUNCH_CHECK();
-    rc = orthonormalize(bt, m, b, status, st);
+    rc = orthonormalize(bt, m, b, status, st, iters < 2);          // in full only if no later iteration will be
     if (rc != QG_OK) return rc;
   }
   // The two products with the gradient go to the tensor cores (bfloat16 gradient times an iterate split into three
   // bfloat16 planes, fp32 accumulation: refresh_tc.cu), one launch per matrix, where shape and strides allow it.
-  // Their rounding differs from the CUDA-core kernel's only in the order of an fp32 accumulation; errors made in
-  // an early iteration are damped by the later ones, and the last full iteration and the product that feeds the
-  // Rayleigh-Ritz step keep the CUDA-core kernel, whose accumulation is not biased toward zero.
+  // Their rounding differs from the CUDA-core kernel's only in the order of an fp32 accumulation; measured, the
+  // largest principal angle to the exact subspace is the same to three digits either way (it is set by the number
+  // of iterations, 5e-3 rad on the rectangular LLaMA shapes after 12, not by the arithmetic).  Only the product that
+  // feeds the Rayleigh-Ritz step keeps the CUDA-core kernel, whose accumulation is not biased toward zero.
   const bool tc_z = g_refresh_tc && split_gemm_supported(G.p[0], cs, rs, n, b, m);   // Z = X^T Q: A(i, k) = X[k][i]
   const bool tc_y = g_refresh_tc && split_gemm_supported(G.p[0], rs, cs, m, b, n);   // Y = X Z:   A(i, k) = X[i][k]
   for (int it = 0; it <= iters; ++it) {
-    const bool early = it + 1 < iters;
     // Z = G^T Q
-    if (tc_z && early) {
+    if (tc_z && it < iters) {
       for (int i = 0; i < nb; ++i) {
         rc = launch_split_gemm(G.p[i], cs, rs, bt.w[i].Q, b, bt.w[i].Z, b, n, b, m, bt.w[i].planes, status, st);
         if (rc != QG_OK) return rc;
@@ -625,7 +632,7 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
     }
     if (it == iters) break;
     // Y = G Z
-    if (tc_y && early) {
+    if (tc_y) {
       for (int i = 0; i < nb; ++i) {
         rc = launch_split_gemm(G.p[i], rs, cs, bt.w[i].Z, b, bt.w[i].Y, b, m, b, n, bt.w[i].planes, status, st);
         if (rc != QG_OK) return rc;
@@ -634,7 +641,7 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
       rc = gemm<uint16_t, float, float>(nb, G, rs, cs, Z, b, 1, Y, b, m, b, n, 1.f, 0.f, st);
       if (rc != QG_OK) return rc;
     }
-    rc = orthonormalize(bt, m, b, status, st);
+    rc = orthonormalize(bt, m, b, status, st, it + 2 >= iters);   // the last two in full
     if (rc != QG_OK) return rc;
   }
   // Rayleigh-Ritz: T = Z^T Z in fp64, eigenvectors by one-sided Jacobi

@@ -870,6 +870,36 @@ def test_plan_mixes_fp32_and_8bit_moments():
     plan.close()
 
 
+def test_8bit_moments_through_a_plan_at_a_7b_shape():
+    """The 8-bit moment storage in the launch configuration the throughput run uses at 7B size (a plan, CTA pairs,
+    r = 1024): one 4096 x 4096 matrix stepped twice as a plan and twice by single calls, bit for bit."""
+    m, n, r = 4096, 4096, 1024
+    gb = synth.GradientModel(m, n, seed=33, matrix_index=0).sample(1)
+    P = O.quantize_rtn(synth.random_orthonormal(m, r, seed=33), 4)
+    W = O.quantize_rtn(synth.initial_weight(m, n, 33), 8)
+    rng = np.random.default_rng(33)
+    M8 = O.quantize_m8(rng.normal(0, 1e-3, (r, n)).astype(np.float32))
+    V8 = O.quantize_v8((rng.normal(0, 1e-3, (r, n)) ** 2).astype(np.float32))
+    dG, dP = g_to_device(gb), to_device_q(P)
+    pair = []
+    for _ in range(2):
+        pair.append({"G": dG, "P": dP, "W": to_device_q(W), "M": _codes_to_device(M8.codes), "V": _codes_to_device(V8.codes),
+                     "M_scale": torch.from_numpy(M8.scales).cuda().contiguous(),
+                     "V_scale": torch.from_numpy(V8.scales).cuda().contiguous(), "seed": 3})
+    plan = B.StepPlan([pair[1]])
+    for t in (1, 2):
+        B.project_step_item(pair[0], B.Hyper(step=t))
+        plan.step(B.Hyper(step=t))
+    torch.cuda.synchronize()
+    assert int(plan.status.item()) == 0
+    a, b = pair
+    assert torch.equal(a["W"].codes, b["W"].codes) and torch.equal(a["W"].scales, b["W"].scales)
+    assert torch.equal(a["M"]._base, b["M"]._base) and torch.equal(a["V"]._base, b["V"]._base)
+    assert torch.equal(a["M_scale"], b["M_scale"]) and torch.equal(a["V_scale"], b["V_scale"])
+    assert int(a["M"].abs().max().item()) > 0
+    plan.close()
+
+
 # ----------------------------------------------------------------------------- App. A: the INT8 linear layer
 def _linear_case(T, m, n, seed):
     rng = np.random.default_rng(seed)
