@@ -144,7 +144,10 @@ __device__ __forceinline__ float sqrt_approx(float x) {
 // ============================================================================================
 // Kernel 1: projection + Adam
 // ============================================================================================
-template <int BN, int CTAS = 1>
+// MVS: slots of the M/V rings (0: three while a stage is at most 32 KB, else two).  Fewer slots leave room for one
+// more operand stage, which pays when the main loop is long (LLaMA-7B: K = 4096 .. 11008) and costs a little when it
+// is short.
+template <int BN, int CTAS = 1, int MVS = 0>
 struct K1Smem {
   static constexpr int kABytes = 2 * kBoxBytes;            // 128 (r) x 64 (m) bf16
   static constexpr int kBBytes = (BN / 64 / CTAS) * kBoxBytes;   // this CTA's share of BN (n) x 64 (m) bf16
@@ -152,7 +155,7 @@ struct K1Smem {
   static constexpr int kEpiWarps = 8;                      // 4 lane quarters x 2 halves of 16 lanes
   // every epilogue warp stages its own 16 rows x 32 columns of M and of V per accumulator chunk, kMvSlots
   // chunks deep, through TMA
-  static constexpr int kMvSlots = kStageBytes > 32 * 1024 ? 2 : 3;
+  static constexpr int kMvSlots = MVS > 0 ? MVS : (kStageBytes > 32 * 1024 ? 2 : 3);
   static constexpr int kMvArrayBytes = 16 * kChunk * 4;    // 2 KB: one array's piece of a chunk
   static constexpr int kMvSlotBytes = 2 * kMvArrayBytes;   // M then V
   static constexpr int kMvBytes = kEpiWarps * kMvSlots * kMvSlotBytes;
@@ -225,13 +228,13 @@ __device__ __forceinline__ void convert_p_row(const uint4 (&c)[4], float s_cur, 
 // TMA, several chunks ahead (see the epilogue).
 // S8: the instance that also knows the 8-bit storage of the moments (it costs registers, so launches whose
 // matrices all keep fp32 moments take the instance without it).
-template <int BN, bool SINGLE, int CTAS, bool S8 = false>
+template <int BN, bool SINGLE, int CTAS, bool S8 = false, int MVS = 0>
 __global__ void __launch_bounds__(K1Smem<BN>::kThreads, 1)
 project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* __restrict__ table,
                     const TileSchedule sched, int total_tiles, const StepScalars sc, int32_t* __restrict__ status,
                     const int conv_active) {
   static_assert(CTAS == 1 || (!SINGLE && BN == 256), "CTA pairs run from a plan, on 256-column tiles");
-  using S = K1Smem<BN, CTAS>;
+  using S = K1Smem<BN, CTAS, MVS>;
   const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;   // 0 = the pair's leader, which issues the MMAs
   constexpr int BNC = BN / CTAS;                 // columns of the B tile this CTA stages
   extern __shared__ uint8_t smem_raw[];
@@ -1392,11 +1395,11 @@ int set_smem_once(K kernel, int bytes, bool* done) {
 // but only pays once there are enough tiles to occupy every SM.
 int choose_bn(int64_t tiles_at_256) { return tiles_at_256 >= 2 * (int64_t)sm_count() ? 256 : 128; }
 
-template <int BN, bool SINGLE, int CTAS, bool S8 = false>
+template <int BN, bool SINGLE, int CTAS, bool S8 = false, int MVS = 0>
 int launch_k1(const TcProblem* single, const TcProblem* table, const TileSchedule& sched, int grid_planned,
               int total_tiles, const StepScalars& sc, int32_t* status, cudaStream_t st, int conv_active) {
-  using S = K1Smem<BN, CTAS>;
-  auto kern = project_adam_kernel<BN, SINGLE, CTAS, S8>;
+  using S = K1Smem<BN, CTAS, MVS>;
+  auto kern = project_adam_kernel<BN, SINGLE, CTAS, S8, MVS>;
   static bool smem_set[64] = {};
   int rc = set_smem_once(kern, S::kBytes, smem_set);
   if (rc != QG_OK) return rc;
@@ -1574,6 +1577,7 @@ struct PlanChunk {
   int dq_blocks;
   int k1_grid, k2_grid, pairs, k1_pairs, k1p_tiles, state8;
   int conv_active;           // some matrix of the chunk has its projection converted inside the projection kernel
+  int k1_deep;               // long main loops (on average 48 K blocks or more per tile): five operand stages, two M/V slots
   size_t k1_start_off, k1_items_off, k2_start_off, k2_items_off;   // int32 offsets into the schedule buffer
   size_t dq_map_off;                                                // same: block -> item map of the dequantize launch
 };
@@ -1701,6 +1705,11 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
       ch.dq_blocks += dq[k].nblocks;
       for (int32_t blk = 0; blk < dq[k].nblocks; ++blk) dq_map.push_back(k - i);
     }
+    {
+      double kb_sum = 0.0;
+      for (float c : c1) kb_sum += (double)c - 6.0;
+      ch.k1_deep = !c1.empty() && kb_sum / (double)c1.size() >= 48.0;
+    }
     if (ch.k1_pairs) ch.k1_grid = 2 * (ch.k1p_tiles < sm_count() / 2 ? ch.k1p_tiles : sm_count() / 2);
     else ch.k1_grid = ch.k1_tiles < sm_count() ? ch.k1_tiles : sm_count();
     if (ch.pairs) ch.k2_grid = 2 * (ch.k2p_tiles < sm_count() / 2 ? ch.k2p_tiles : sm_count() / 2);   // CTA pairs
@@ -1760,7 +1769,8 @@ int plan_step(const Plan* plan, const StepScalars& sc, int32_t* status, cudaStre
            : ch.bn == 256 ? launch_k1<256, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active)
                           : launch_k1<128, false, 1, true>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active);
     } else {
-      rc = ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st, ch.conv_active)
+      rc = (ch.k1_pairs && ch.k1_deep) ? launch_k1<256, false, 2, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st, ch.conv_active)
+           : ch.k1_pairs  ? launch_k1<256, false, 2>(nullptr, tab, s1, ch.k1_grid, ch.k1p_tiles, sc, status, st, ch.conv_active)
            : ch.bn == 256 ? launch_k1<256, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active)
                           : launch_k1<128, false, 1>(nullptr, tab, s1, ch.k1_grid, ch.k1_tiles, sc, status, st, ch.conv_active);
     }
