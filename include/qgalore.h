@@ -344,8 +344,8 @@ QG_API uint64_t qgalore_launch_count(void);
 QG_API int qgalore_debug_set_step_impl(int impl);
 /* Which kernels of plans created after this call run as CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles per
  * pair): bit 0 the back-projection (chunks of left-hand items only), bit 1 the projection (where every rank of a
- * chunk is a multiple of 256).  0 = one CTA per 128 x 256 tile; the default is 2.  Every setting gives the same
- * results bit for bit. */
+ * chunk is a multiple of 256), bit 2 the back-projection in chunks whose ranks average 1024 or more.  0 = one CTA
+ * per 128 x 256 tile; the default is 6.  Every setting gives the same results bit for bit. */
 QG_API int qgalore_debug_set_pair_mode(int mask);
 /* 1: the projection kernel converts the INT4 codes of P inside its main loop (converter warps write the bf16
  * operand tile straight into shared memory); 0 (the default, the faster arrangement as measured): P is dequantized

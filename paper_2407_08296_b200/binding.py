@@ -609,6 +609,9 @@ def debug_set_step_impl(impl: int) -> None:
     _check(lib().qgalore_debug_set_step_impl(impl), "qgalore_debug_set_step_impl")
 
 
+DEFAULT_PAIR_MODE = 6
+
+
 def debug_set_pair_mode(mask: int) -> None:
     _check(lib().qgalore_debug_set_pair_mode(mask), "qgalore_debug_set_pair_mode")
 

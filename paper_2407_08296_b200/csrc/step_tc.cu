@@ -1618,9 +1618,11 @@ void schedule_tiles(const std::vector<int2>& tiles, const std::vector<float>& co
     for (int t : per_cta[(size_t)c]) { buf.push_back(tiles[t].x); buf.push_back(tiles[t].y); }
 }
 
-// bit 0: the back-projection of a plan runs as CTA pairs (cta_group::2); bit 1: the projection does.  Read when a
-// plan is created.
-int g_pair_mode = 2;
+// bit 0: the back-projection of a plan runs as CTA pairs (cta_group::2); bit 1: the projection does; bit 2: the
+// back-projection does where it pays, i.e. in chunks whose ranks average 1024 or more (measured on LLaMA-7B under
+// the power cap: 13.9-14.2 ms against 15.1 unpaired, the halved operand traffic buys clock; on LLaMA-1B, r = 512,
+// pairs are 3 % slower).  Read when a plan is created.
+int g_pair_mode = 6;
 
 // Scratch is shared by the matrices of a chunk; a chunk is a run of consecutive items whose P~ and N_b fit
 // both the caller's workspace and this budget.  Few, long launches win: with two or three tiles per CTA the
@@ -1675,6 +1677,11 @@ int plan_create(const StepArgs* items, int32_t count, void* table_dev, size_t ta
     // kernel knows the left form only); decided here, before the tile lists are made, because the lists of the
     // two forms differ (tiles of 256 rows against tiles of 128)
     ch.pairs = g_pair_mode & 1;
+    if (g_pair_mode & 4) {
+      int64_t rsum = 0;
+      for (int k = i; k < j; ++k) rsum += items[k].r;
+      if (rsum >= (int64_t)1024 * (j - i)) ch.pairs = 1;
+    }
     for (int k = i; k < j; ++k) {
       if (items[k].right) ch.pairs = 0;
       if (items[k].state8) ch.state8 = 1;
@@ -1813,7 +1820,7 @@ int plan_step_timed(const Plan* plan, const StepScalars& sc, int32_t* status, cu
 }
 
 void plan_destroy(Plan* plan) { delete plan; }
-int set_pair_mode(int mask) { g_pair_mode = mask & 3; return QG_OK; }
+int set_pair_mode(int mask) { g_pair_mode = mask & 7; return QG_OK; }
 int set_fused_dequant(int on) { g_fuse_dequant = on ? 1 : 0; return QG_OK; }
 int set_chunk_budget(size_t bytes) { g_chunk_budget = bytes; return QG_OK; }
 

@@ -358,7 +358,7 @@ def test_cta_pair_kernels_equal_single_cta_kernels(mask):
             plan.close()
             results.append(items)
     finally:
-        set_mode(2)                                        # the library's default
+        set_mode(B.DEFAULT_PAIR_MODE)
     for a, b in zip(*results):
         assert torch.equal(a["W"].codes, b["W"].codes)
         assert torch.equal(a["W"].scales, b["W"].scales) and torch.equal(a["W"].zeros, b["W"].zeros)
@@ -678,7 +678,7 @@ def test_plan_mixes_projection_sides():
         single.append((dW1, dM1, dV1))
         items.append({"G": dG, "P": dP, "W": to_device_q(W), "M": f32_to_device(M), "V": f32_to_device(V), "seed": idx,
                       "side": side})
-    for pair_mode in (2, 0, 1, 3):      # 1 and 3 ask for the paired back-projection, which a chunk with a right-hand item declines
+    for pair_mode in (2, 0, 1, 3, 6):   # 1 and 3 ask for the paired back-projection, which a chunk with a right-hand item declines
         B.debug_set_pair_mode(pair_mode)
         try:
             fresh = [{**it, "W": it["W"].clone(), "M": it["M"]._base.clone()[:, :it["M"].shape[1]],
@@ -692,7 +692,7 @@ def test_plan_mixes_projection_sides():
                 assert torch.equal(dM1._base, it["M"]._base) and torch.equal(dV1._base, it["V"]._base)
             plan.close()
         finally:
-            B.debug_set_pair_mode(2)
+            B.debug_set_pair_mode(B.DEFAULT_PAIR_MODE)
 
 
 @pytest.mark.parametrize("m,n,r", [(320, 256, 64), (1376, 512, 128), (5461, 2048, 512)])
