@@ -135,6 +135,17 @@ __device__ __forceinline__ void raise_wait_expired(int32_t* status) {
 
 constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it leaves an integer in the low mantissa bits
 
+__device__ __forceinline__ float min3(float a, float b, float c) {
+  float d;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 __device__ __forceinline__ float sqrt_approx(float x) {
   float y;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -508,24 +519,32 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     const uint32_t swz = (uint32_t)(lane >> 2), half8 = (uint32_t)(lane & 1) * 8u, unit0 = (uint32_t)((lane >> 1) & 1);
     const uint32_t row_off = (uint32_t)(lane >> 2) * 128u;
 
+    // With 8-bit moments a warp takes all 32 rows of its lane quarter and every second chunk (a thread then holds
+    // one whole 32-element block of a row); with fp32 moments 16 rows and every chunk.
     struct Cursor {                                  // a (tile, chunk) position in this CTA's work list
       TileWalk<SINGLE> tw;
       const TcProblem* p;
-      int c, nch, x0, y0;
-      __device__ Cursor(const TileSchedule& sch, int total) : tw(sch, total), p(nullptr), c(0), nch(0), x0(0), y0(0) {}
+      int c, cstep, nch, x0, y0;
+      __device__ Cursor(const TileSchedule& sch, int total) : tw(sch, total), p(nullptr), c(0), cstep(1), nch(0), x0(0), y0(0) {}
     };
     auto enter_tile = [&](Cursor& cu) {
-      if (!cu.tw.valid()) return;
-      const int2 item = cu.tw.cur();
-      cu.p = probs + item.x;
-      const int rblocks = CTAS == 2 ? cu.p->k1_rpairs : cu.p->k1_rblocks;
-      cu.y0 = (item.y % rblocks) * (CTAS * kTileM) + (int)rank * kTileM + wrow;
-      cu.x0 = (item.y / rblocks) * BN;
-      cu.nch = min(BN / kChunk, (cu.p->k1_n - cu.x0 + kChunk - 1) / kChunk);
-      cu.c = 0;
+      while (cu.tw.valid()) {
+        const int2 item = cu.tw.cur();
+        cu.p = probs + item.x;
+        const bool t8 = S8 && cu.p->state8 != 0;
+        const int rblocks = CTAS == 2 ? cu.p->k1_rpairs : cu.p->k1_rblocks;
+        cu.y0 = (item.y % rblocks) * (CTAS * kTileM) + (int)rank * kTileM + (t8 ? q * 32 : wrow);
+        cu.x0 = (item.y / rblocks) * BN;
+        cu.nch = min(BN / kChunk, (cu.p->k1_n - cu.x0 + kChunk - 1) / kChunk);
+        cu.c = t8 ? hh : 0;
+        cu.cstep = t8 ? 2 : 1;
+        if (cu.c < cu.nch) return;
+        cu.tw.advance();                             // a one-chunk tile has nothing for the warp of the odd chunks
+      }
     };
     auto next_chunk = [&](Cursor& cu) {
-      if (++cu.c >= cu.nch) { cu.tw.advance(); enter_tile(cu); }
+      cu.c += cu.cstep;
+      if (cu.c >= cu.nch) { cu.tw.advance(); enter_tile(cu); }
     };
     Cursor ld(sched, total_tiles);                   // the next chunk to request
     enter_tile(ld);
@@ -533,7 +552,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
     auto request = [&]() {                           // one lane: the two copies of chunk `ld` into slot ld_slot
       if (lane == 0) {
         uint8_t* dst = mv_base + ld_slot * S::kMvSlotBytes;
-        mbar_arrive_expect_tx(&my_full[ld_slot], (S8 && ld.p->state8) ? 2 * 16 * kChunk : S::kMvSlotBytes);
+        mbar_arrive_expect_tx(&my_full[ld_slot], (S8 && ld.p->state8) ? 2 * 32 * kChunk : S::kMvSlotBytes);
         tma_load_2d(dst, &ld.p->mapM, &my_full[ld_slot], ld.x0 + kChunk * ld.c, ld.y0);
         tma_load_2d(dst + S::kMvArrayBytes, &ld.p->mapV, &my_full[ld_slot], ld.x0 + kChunk * ld.c, ld.y0);
       }
@@ -571,30 +590,155 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
       // interior tiles (every row and column valid, no test taps) take a path without per-access predicates
       const bool s8 = S8 && p->state8 != 0;
       const bool whole = (r0 + kTileM <= p->r) && (n0 + BN <= pn) && p->dbgR == nullptr && p->dbgN == nullptr && p->dbgNb == nullptr;
-      const bool interior = whole && !s8;
-      int8_t* M8r[2]; uint8_t* V8r[2]; float* msc[2]; float* vsc[2];
+      const bool interior = whole;
+      const uint32_t ab = tcount & 1;
+      if (s8) {
+        // ---- 8-bit moments: thread = one row of the lane quarter, chunk = one 32-element block of that row
+        const int64_t gr = r0 + q * 32 + lane;
+        const bool rok8 = gr < p->r;
+        int8_t* M8 = reinterpret_cast<int8_t*>(p->M) + gr * ldmv + n0;
+        uint8_t* V8 = reinterpret_cast<uint8_t*>(p->V) + gr * ldmv + n0;
+        float* msc = p->m_scale + gr * p->nsb;
+        float* vsc = p->v_scale + gr * p->nsb;
+        uint16_t* Nrow = p->nb + gr * ldn + n0;
+        float* tR = p->dbgR ? p->dbgR + gr * ldmv + n0 : nullptr;
+        float* tN = p->dbgN ? p->dbgN + gr * ldmv + n0 : nullptr;
+        uint16_t* tNb = p->dbgNb ? p->dbgNb + gr * ldmv + n0 : nullptr;
+        const int cvalid = pn - n0;                  // columns of the tile inside the matrix
+        float ms_next = 0.f, vs_next = 0.f;          // the block scales, fetched one chunk ahead
+        auto fetch_scales = [&](int c) {
+          const int blk = (n0 + kChunk * c) >> 5;
+          ms_next = rok8 ? __ldg(msc + blk) : 0.f;
+          vs_next = rok8 ? __ldg(vsc + blk) : 0.f;
+        };
+        if (hh < nch) fetch_scales(hh);
+        ok = __all_sync(0xFFFFFFFFu, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
+        if (!ok) break;
+        tc_fence_after_sync();
+        auto release_acc = [&]() {                   // every read of this accumulator buffer has landed
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            if (CTAS == 2) mbar_arrive_cluster(mapa_u32(smem_u32(&acc_empty[ab]), 0));
+            else mbar_arrive(&acc_empty[ab]);
+          }
+        };
+        if (hh >= nch) release_acc();
+#pragma unroll 1
+        for (int c = hh; c < nch; c += 2) {
+          ok = __all_sync(0xFFFFFFFFu, mbar_wait(&my_full[slot], slot_phase));
+          if (!ok) break;
+          --in_flight;
+          // the 32 + 32 codes of the thread's block (rows of 32 bytes, no swizzle)
+          const uint4* src8 = reinterpret_cast<const uint4*>(mv_base + slot * S::kMvSlotBytes + lane * kChunk);
+          const uint4 mc4[2] = {src8[0], src8[1]};
+          const uint4 vc4[2] = {src8[S::kMvArrayBytes / 16], src8[S::kMvArrayBytes / 16 + 1]};
+          const float ms = ms_next, vs = vs_next;
+          if (c + 2 < nch) fetch_scales(c + 2);
+          if (++slot == (uint32_t)S::kMvSlots) { slot = 0; slot_phase ^= 1u; }
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (ld.tw.valid()) request();
+
+          uint32_t acc[32];
+          tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + ab * BN + c * kChunk, acc);
+          tmem_ld_wait();
+          if (c + 2 >= nch) release_acc();
+
+          const uint32_t mw[8] = {mc4[0].x, mc4[0].y, mc4[0].z, mc4[0].w, mc4[1].x, mc4[1].y, mc4[1].z, mc4[1].w};
+          const uint32_t vw[8] = {vc4[0].x, vc4[0].y, vc4[0].z, vc4[0].w, vc4[1].x, vc4[1].y, vc4[1].z, vc4[1].w};
+          const float stepm = __fmul_rn(ms, 1.0f / 127.0f);
+          const float2 stepm2 = make_float2(stepm, stepm), vs2 = make_float2(vs, vs);
+          const float2 c255 = make_float2(1.0f / 255.0f, 1.0f / 255.0f);
+          const float2 bias_m = make_float2(-8388736.0f, -8388736.0f), bias_v = make_float2(-8388608.0f, -8388608.0f);
+          const bool chunk_whole = rok8 && kChunk * c + kChunk <= cvalid;
+          const bool taps = tR != nullptr || tN != nullptr || tNb != nullptr;
+          float2 mm[16], vv[16];
+          float mxm = 0.f, mxv = 0.f;
+          uint32_t nbq[4];                            // the bf16 direction of eight columns, stored 16 bytes at a time
 #pragma unroll
-      for (int a = 0; a < 2; ++a) {
-        const int64_t gr = r0 + lrow + 8 * a;
-        M8r[a] = reinterpret_cast<int8_t*>(p->M) + gr * ldmv + n0 + lcol;
-        V8r[a] = reinterpret_cast<uint8_t*>(p->V) + gr * ldmv + n0 + lcol;
-        msc[a] = p->m_scale + gr * p->nsb;
-        vsc[a] = p->v_scale + gr * p->nsb;
+          for (int k = 0; k < 8; ++k) {               // word k: columns 4k .. 4k+3 of the block
+            const uint32_t mcw = mw[k] ^ 0x80808080u;
+            uint32_t* nbw = nbq + 2 * (k & 1);
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+              const int j = 2 * k + b;                // column pair 2j, 2j+1
+              // a byte dropped into the mantissa of 2^23 is the float 2^23 + byte: no integer-to-float conversion
+              const float2 mq = make_float2(__uint_as_float(__byte_perm(mcw, 0x4B000000u, 0x7650 + 2 * b)),
+                                            __uint_as_float(__byte_perm(mcw, 0x4B000000u, 0x7651 + 2 * b)));
+              mm[j] = mul2(add2(mq, bias_m), stepm2);                                   // code = byte - 128
+              const float2 vq = make_float2(__uint_as_float(__byte_perm(vw[k], 0x4B000000u, 0x7650 + 2 * b)),
+                                            __uint_as_float(__byte_perm(vw[k], 0x4B000000u, 0x7651 + 2 * b)));
+              const float2 w = mul2(add2(vq, bias_v), c255);
+              vv[j] = mul2(mul2(w, w), vs2);
+              const float2 rr = make_float2(__uint_as_float(acc[2 * j]), __uint_as_float(acc[2 * j + 1]));
+              const float2 nn = adam2(ac, rr, mm[j], vv[j]);
+              const __nv_bfloat162 nb2 = __floats2bfloat162_rn(nn.x, nn.y);
+              nbw[b] = *reinterpret_cast<const uint32_t*>(&nb2);
+              mxm = max3(mxm, fabsf(mm[j].x), fabsf(mm[j].y));
+              mxv = max3(mxv, vv[j].x, vv[j].y);
+              if (taps && rok8) {
+                const int off = kChunk * c + 2 * j;
+#pragma unroll
+                for (int e = 0; e < 2; ++e)
+                  if (off + e < cvalid) {
+                    if (tR) tR[off + e] = e ? rr.y : rr.x;
+                    if (tN) tN[off + e] = e ? nn.y : nn.x;
+                    if (tNb) tNb[off + e] = (uint16_t)(nbw[b] >> (16 * e));
+                  }
+              }
+            }
+            if (chunk_whole) {
+              if (k & 1) *reinterpret_cast<uint4*>(Nrow + kChunk * c + 4 * (k - 1)) = make_uint4(nbq[0], nbq[1], nbq[2], nbq[3]);
+            } else if (rok8) {
+#pragma unroll
+              for (int e = 0; e < 4; ++e)
+                if (kChunk * c + 4 * k + e < cvalid) Nrow[kChunk * c + 4 * k + e] = (uint16_t)(nbw[e >> 1] >> (16 * (e & 1)));
+            }
+          }
+          // 8-bit storage of the new moments: scale = the block's largest |M'| resp. V'; M' linear in [-127, 127],
+          // V' by the square-root law in [0, 255]; every operation a single binary32 one, as on the reference side.
+          // Reciprocals and roots by the approximate units (a few ulp): a code can differ from the correctly
+          // rounded one only when the scaled value sits within ~1e-5 of a rounding boundary.
+          const float invm = mxm > 0.f ? __fdividef(127.0f, mxm) : 0.f;
+          const float invv = mxv > 0.f ? __fdividef(1.0f, mxv) : 0.f;
+          if (!rok8) continue;
+          const int blk = (n0 + kChunk * c) >> 5;
+          if (kChunk * c < cvalid) { msc[blk] = mxm; vsc[blk] = mxv; }
+          uint32_t mo[8], vo[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            // rint(t) sits in the low mantissa bits of t + 1.5 * 2^23; |t| <= 127 (+ a few ulp) resp. 0 <= t <= 255
+            // by construction of the scales, so the low byte is the code
+            uint32_t mq4[4], vq4[4];
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+              const float2 m2 = mm[2 * k + b], v2 = vv[2 * k + b];
+              mq4[2 * b] = __float_as_uint(__fadd_rn(__fmul_rn(m2.x, invm), kMagic));
+              mq4[2 * b + 1] = __float_as_uint(__fadd_rn(__fmul_rn(m2.y, invm), kMagic));
+              vq4[2 * b] = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(v2.x, invv)), 255.0f), kMagic));
+              vq4[2 * b + 1] = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(v2.y, invv)), 255.0f), kMagic));
+            }
+            mo[k] = __byte_perm(__byte_perm(mq4[0], mq4[1], 0x0040), __byte_perm(mq4[2], mq4[3], 0x0040), 0x5410);
+            vo[k] = __byte_perm(__byte_perm(vq4[0], vq4[1], 0x0040), __byte_perm(vq4[2], vq4[3], 0x0040), 0x5410);
+          }
+          if (chunk_whole) {
+            uint4* md = reinterpret_cast<uint4*>(M8 + kChunk * c);
+            uint4* vd = reinterpret_cast<uint4*>(V8 + kChunk * c);
+            md[0] = make_uint4(mo[0], mo[1], mo[2], mo[3]); md[1] = make_uint4(mo[4], mo[5], mo[6], mo[7]);
+            vd[0] = make_uint4(vo[0], vo[1], vo[2], vo[3]); vd[1] = make_uint4(vo[4], vo[5], vo[6], vo[7]);
+          } else {
+#pragma unroll
+            for (int e = 0; e < kChunk; ++e)
+              if (kChunk * c + e < cvalid) {
+                M8[kChunk * c + e] = (int8_t)((mo[e >> 2] >> (8 * (e & 3))) & 0xFFu);
+                V8[kChunk * c + e] = (uint8_t)((vo[e >> 2] >> (8 * (e & 3))) & 0xFFu);
+              }
+          }
+        }
+        continue;
       }
 
-      // 8-bit moments: the block scales of the thread's two rows, fetched one chunk ahead
-      float ms_next[2] = {0.f, 0.f}, vs_next[2] = {0.f, 0.f};
-      auto fetch_scales = [&](int c) {
-        const int blk = (n0 + kChunk * c) >> 5;
-#pragma unroll
-        for (int a = 0; a < 2; ++a) {
-          ms_next[a] = rok[a] ? __ldg(msc[a] + blk) : 0.f;
-          vs_next[a] = rok[a] ? __ldg(vsc[a] + blk) : 0.f;
-        }
-      };
-      if (s8) fetch_scales(0);
-
-      const uint32_t ab = tcount & 1;
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(&acc_full[ab], (tcount >> 1) & 1));
       if (!ok) break;
       tc_fence_after_sync();
@@ -606,33 +750,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
         if (!ok) break;
         --in_flight;
         float2 sm[8], sv[8];
-        if (s8) {
-          // codes of the thread's column pairs (rows of 32 bytes, no swizzle) and the block scales of its two rows
-          const uint8_t* src8 = mv_base + slot * S::kMvSlotBytes + (lane >> 2) * kChunk + 2 * (lane & 3);
-          const float ms_cur[2] = {ms_next[0], ms_next[1]}, vs_cur[2] = {vs_next[0], vs_next[1]};
-          if (c + 1 < nch) fetch_scales(c + 1);
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            const float ms = ms_cur[a], vs = vs_cur[a];
-            const float stepm = __fmul_rn(ms, 1.0f / 127.0f);
-            const float2 stepm2 = make_float2(stepm, stepm), vs2 = make_float2(vs, vs);
-            const float2 c255 = make_float2(1.0f / 255.0f, 1.0f / 255.0f);
-            const float2 bias_m = make_float2(-8388736.0f, -8388736.0f), bias_v = make_float2(-8388608.0f, -8388608.0f);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              // a byte dropped into the mantissa of 2^23 is the float 2^23 + byte: no integer-to-float conversion
-              const uint32_t mc = (uint32_t)*reinterpret_cast<const uint16_t*>(src8 + a * 8 * kChunk + 8 * k) ^ 0x8080u;
-              const uint32_t vc = *reinterpret_cast<const uint16_t*>(src8 + S::kMvArrayBytes + a * 8 * kChunk + 8 * k);
-              const float2 mq = make_float2(__uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7650)),
-                                            __uint_as_float(__byte_perm(mc, 0x4B000000u, 0x7651)));
-              sm[2 * k + a] = mul2(add2(mq, bias_m), stepm2);                         // code = byte - 128
-              const float2 vq = make_float2(__uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7650)),
-                                            __uint_as_float(__byte_perm(vc, 0x4B000000u, 0x7651)));
-              const float2 w = mul2(add2(vq, bias_v), c255);
-              sv[2 * k + a] = mul2(mul2(w, w), vs2);
-            }
-          }
-        } else {
+        {
           const uint8_t* src = mv_base + slot * S::kMvSlotBytes + row_off + half8;
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
@@ -669,25 +787,7 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
             const float2 rr = make_float2(__uint_as_float(acc[4 * k + 2 * a]), __uint_as_float(acc[4 * k + 2 * a + 1]));
             const float2 nn = adam2(ac, rr, mm, vv);
             const __nv_bfloat162 nb2 = __floats2bfloat162_rn(nn.x, nn.y);
-            if (s8) {                                 // the new moments wait for their block's scale
-              sm[2 * k + a] = mm;
-              sv[2 * k + a] = vv;
-              if (whole) {
-                *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
-              } else if (rok[a]) {
-                if (off + 1 < cmax) {
-                  *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
-                  if (tapR[a]) { tapR[a][off] = rr.x; tapR[a][off + 1] = rr.y; }
-                  if (tapN[a]) { tapN[a][off] = nn.x; tapN[a][off + 1] = nn.y; }
-                  if (tapNb[a]) { tapNb[a][off] = __bfloat16_as_ushort(nb2.x); tapNb[a][off + 1] = __bfloat16_as_ushort(nb2.y); }
-                } else if (off < cmax) {
-                  Nr[a][off] = float_to_bf16_bits(nn.x);
-                  if (tapR[a]) tapR[a][off] = rr.x;
-                  if (tapN[a]) tapN[a][off] = nn.x;
-                  if (tapNb[a]) tapNb[a][off] = __bfloat16_as_ushort(nb2.x);
-                }
-              }
-            } else if (interior) {
+            if (interior) {
               __stcs(reinterpret_cast<float2*>(Mr[a] + off), mm);
               __stcs(reinterpret_cast<float2*>(Vr[a] + off), vv);
               *reinterpret_cast<__nv_bfloat162*>(Nr[a] + off) = nb2;
@@ -709,49 +809,6 @@ project_adam_kernel(const __grid_constant__ TcProblem single, const TcProblem* _
               }
             }
           }
-        if (s8) {
-          // 8-bit storage of the new moments: the chunk's 32 columns of a row are one block, held by the four
-          // threads of a quad.  Scale = the block's largest |M'| resp. V'; M' linear in [-127, 127], V' by the
-          // square-root law in [0, 255]; every operation a single binary32 one, as on the reference side.
-          const int blk = (n0 + kChunk * c) >> 5;
-#pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            float mxm = 0.f, mxv = 0.f;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              mxm = fmaxf(mxm, fmaxf(fabsf(sm[2 * k + a].x), fabsf(sm[2 * k + a].y)));
-              mxv = fmaxf(mxv, fmaxf(sv[2 * k + a].x, sv[2 * k + a].y));
-            }
-            mxm = fmaxf(mxm, __shfl_xor_sync(0xFFFFFFFFu, mxm, 1));
-            mxv = fmaxf(mxv, __shfl_xor_sync(0xFFFFFFFFu, mxv, 1));
-            mxm = fmaxf(mxm, __shfl_xor_sync(0xFFFFFFFFu, mxm, 2));
-            mxv = fmaxf(mxv, __shfl_xor_sync(0xFFFFFFFFu, mxv, 2));
-            // reciprocals and roots by the approximate units (a few ulp): a code can differ from the correctly
-            // rounded one only when the scaled value sits within ~1e-5 of a rounding boundary
-            const float invm = mxm > 0.f ? __fdividef(127.0f, mxm) : 0.f;
-            const float invv = mxv > 0.f ? __fdividef(1.0f, mxv) : 0.f;
-            if (!rok[a]) continue;
-            if ((lane & 3) == 0 && kChunk * c < pn - n0) { msc[a][blk] = mxm; vsc[a][blk] = mxv; }
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const int off = kChunk * c + 8 * k;
-              const float2 mm = sm[2 * k + a], vv = sv[2 * k + a];
-              // rint(t) sits in the low mantissa bits of t + 1.5 * 2^23; |t| <= 127 (+ a few ulp) resp. 0 <= t <= 255
-              // by construction of the scales, so the low byte is the code
-              const uint32_t m0q = __float_as_uint(__fadd_rn(__fmul_rn(mm.x, invm), kMagic));
-              const uint32_t m1q = __float_as_uint(__fadd_rn(__fmul_rn(mm.y, invm), kMagic));
-              const uint32_t v0q = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(vv.x, invv)), 255.0f), kMagic));
-              const uint32_t v1q = __float_as_uint(__fadd_rn(__fmul_rn(sqrt_approx(__fmul_rn(vv.y, invv)), 255.0f), kMagic));
-              if (whole || off + 1 < cmax) {
-                *reinterpret_cast<uint16_t*>(M8r[a] + off) = (uint16_t)__byte_perm(m0q, m1q, 0x0040);
-                *reinterpret_cast<uint16_t*>(V8r[a] + off) = (uint16_t)__byte_perm(v0q, v1q, 0x0040);
-              } else if (off < cmax) {
-                M8r[a][off] = (int8_t)(m0q & 0xFFu);
-                V8r[a][off] = (uint8_t)(v0q & 0xFFu);
-              }
-            }
-          }
-        }
       }
     }
     if (!ok) {
@@ -859,17 +916,6 @@ __device__ __forceinline__ uint32_t pack_sat_s8x4(int c0, int c1, int c2, int c3
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(c3), "r"(c2), "r"(0));
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(c1), "r"(c0), "r"(hi));
   return out;
-}
-
-__device__ __forceinline__ float min3(float a, float b, float c) {
-  float d;
-  asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
 }
 
 // Philox4x32-10 with the ten round keys given (key schedule hoisted out of the per-block calls) and
@@ -1337,8 +1383,8 @@ int fill_problem(const StepArgs& a, const TcScratch& w, TcProblem* p, int bn) {
   ok &= make_map(&p->mapW, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.W.codes, a.n, a.m, a.W.ld, 128, kTileM,
                  CU_TENSOR_MAP_SWIZZLE_128B);
   if (a.state8) {
-    ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.M, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
-    ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.V, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
+    ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.M, scol, a.r, a.ldmv, kChunk, 32, CU_TENSOR_MAP_SWIZZLE_NONE);
+    ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a.V, scol, a.r, a.ldmv, kChunk, 32, CU_TENSOR_MAP_SWIZZLE_NONE);
   } else {
     ok &= make_map(&p->mapM, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.M, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
     ok &= make_map(&p->mapV, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.V, scol, a.r, a.ldmv, kChunk, 16, CU_TENSOR_MAP_SWIZZLE_128B);
