@@ -6,11 +6,12 @@
 //
 //   Q <- orth(Gaussian m x b)
 //   repeat iters times:   Z = G^T Q  (n x b);   Y = G Z  (m x b);   Q <- orth(Y)
-//   Z = G^T Q;   T = Z^T Z  (b x b, fp64);   T = X diag(lambda) X^T;   P = Q X[:, top r]
+//   Z = G^T Q;   T = Z^T Z  (b x b, summed in fp64);   T = X diag(lambda) X^T;   P = Q X[:, top r]
 //
 // Everything heavy is a GEMM (one generic fp32 kernel, fp64 accumulation for T).  orth() is block
 // Gram-Schmidt over panels of 64 columns, each projection done twice, the panel itself by two rounds of
-// Cholesky QR.  The eigenvectors of T come from a one-sided (Hestenes) Jacobi iteration in fp64 with a
+// Cholesky QR.  The eigenvectors of T come from a one-sided (Hestenes) Jacobi iteration (rows kept in fp32, every
+// sum and rotation angle in fp64: the result is INT4 in the end, and a round is bound by the bytes it moves) with a
 // round-robin pair ordering: all sweeps in one cooperative launch, a grid barrier between rounds of b/2 disjoint pairs.  Each column of P is then
 // given the sign that makes its largest entry positive, and P is quantized to INT4 (Quant_4).
 //
@@ -46,6 +47,7 @@ int g_refresh_tc = 1;
 
 constexpr int kPanel = 64;    // columns orthonormalised together
 constexpr int kMaxSweeps = 32;
+constexpr int64_t kJacobiBytes = 64ll << 20;   // Rayleigh-Ritz matrices rotated by one launch: half of L2
 constexpr int kGT = 64;       // GEMM tile (square), 16 x 16 threads, 4 x 4 outputs each
 constexpr int kGK = 16;
 
@@ -280,7 +282,7 @@ chol64_inverse_kernel(const Ptrs<const float> Sb, const Ptrs<float> Linvb, int32
   }
 }
 
-// ---- one-sided (Hestenes) Jacobi on the rows of the symmetric b x b fp64 matrix T: rows are rotated in
+// ---- one-sided (Hestenes) Jacobi on the rows of the symmetric b x b matrix T (binary32): rows are rotated in
 // pairs until they are mutually orthogonal.  Then row j is lambda_j x_j^T (from T X = X Lambda), so the
 // eigenvectors are the normalised rows and no second matrix has to follow the rotations.  Round `rnd` of a
 // sweep pairs the b indices by the round-robin tournament schedule.
@@ -291,26 +293,26 @@ __device__ __forceinline__ void tournament_pair(int nitems, int rnd, int k, int&
   if (p > q) { const int t = p; p = q; q = t; }
 }
 
-// Barrier across the CTAs of a cooperative launch (all resident at once): a counter that only grows and a
-// generation word.  The wait is bounded; when it runs out the caller flags the status word and every CTA
-// leaves.  `gen` counts the barriers this CTA has passed.
+// Barrier across the CTAs of a cooperative launch (all resident at once): one counter that only grows.  A CTA
+// arrives with a release-add that returns nothing and then polls the counter itself with acquire loads until all
+// gridDim.x arrivals of this generation are in: one trip to L2 to arrive and one to see the last arrival, no
+// hand-over through a second word.  The wait is bounded; when it runs out the caller flags the status word and
+// every CTA leaves.  `gen` counts the barriers this CTA has passed.
 constexpr uint32_t kGridWaitPolls = 1u << 24;
-__device__ __forceinline__ bool grid_barrier(unsigned int* count, unsigned int* generation, unsigned int& gen) {
+__device__ __forceinline__ bool grid_barrier(unsigned int* count, unsigned int& gen) {
   __syncthreads();
   int ok = 1;
   ++gen;
   if (threadIdx.x == 0) {
-    __threadfence();
-    if (atomicAdd(count, 1u) + 1u == gen * gridDim.x) {
-      __threadfence();
-      atomicExch(generation, gen);
-    } else {
-      uint32_t polls = 0;
-      while (*reinterpret_cast<volatile unsigned int*>(generation) < gen) {
-        if (++polls >= kGridWaitPolls) { ok = 0; break; }
-      }
+    const unsigned int target = gen * gridDim.x;
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(count), "r"(1u) : "memory");
+    uint32_t polls = 0;
+    unsigned int seen;
+    for (;;) {
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(count) : "memory");
+      if (seen >= target) break;
+      if (++polls >= kGridWaitPolls) { ok = 0; break; }
     }
-    __threadfence();
   }
   return __syncthreads_and(ok) != 0;
 }
@@ -325,8 +327,8 @@ __device__ __forceinline__ bool grid_barrier(unsigned int* count, unsigned int* 
 // never does.
 constexpr int kTeam = 128, kTeamsPerCta = 4;
 template <int NE>
-__global__ void __launch_bounds__(kTeam * kTeamsPerCta, NE <= 8 ? 2 : 1)   // two CTAs per SM while the rows fit 64 registers
-jacobi_sweeps_kernel(const Ptrs<double> Tb, int nb, int b, int sweeps, double tol, const Ptrs<unsigned long long> offb,
+__global__ void __launch_bounds__(kTeam * kTeamsPerCta, NE <= 16 ? 2 : 1)   // two CTAs per SM while the rows fit 64 registers
+jacobi_sweeps_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol, const Ptrs<unsigned long long> offb,
                      unsigned int* __restrict__ sync_words, int32_t* __restrict__ status) {
   __shared__ double red[kTeamsPerCta][3][kTeam / 32];
   __shared__ double s_worst[kTeamsPerCta][kMaxBatch];
@@ -343,19 +345,22 @@ jacobi_sweeps_kernel(const Ptrs<double> Tb, int nb, int b, int sweeps, double to
         const bool live = k < jobs && ((active >> mat) & 1u);
         int p = 0, q = 0;
         if (live) tournament_pair(b, rnd, k - mat * pairs, p, q);
-        double* tp = Tb.p[mat] + (int64_t)p * b;
-        double* tq = Tb.p[mat] + (int64_t)q * b;
-        double x[NE], y[NE];
-        double a = 0.0, c = 0.0, d = 0.0;
+        float* tp = Tb.p[mat] + (int64_t)p * b;
+        float* tq = Tb.p[mat] + (int64_t)q * b;
+        float x[NE], y[NE];
 #pragma unroll
         for (int e = 0; e < NE; ++e) {
           const int i = tt + kTeam * e;
           const bool in = live && i < b;
-          x[e] = in ? __ldcg(tp + i) : 0.0;
-          y[e] = in ? __ldcg(tq + i) : 0.0;
+          x[e] = in ? __ldcg(tp + i) : 0.f;
+          y[e] = in ? __ldcg(tq + i) : 0.f;
         }
+        // the thread's few products in binary32 (each exact to 2^-24 of itself), everything summed across
+        // threads in binary64
+        float af = 0.f, cf = 0.f, df = 0.f;
 #pragma unroll
-        for (int e = 0; e < NE; ++e) { a += x[e] * x[e]; d += y[e] * y[e]; c += x[e] * y[e]; }
+        for (int e = 0; e < NE; ++e) { af = fmaf(x[e], x[e], af); df = fmaf(y[e], y[e], df); cf = fmaf(x[e], y[e], cf); }
+        double a = (double)af, c = (double)cf, d = (double)df;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
@@ -371,16 +376,17 @@ jacobi_sweeps_kernel(const Ptrs<double> Tb, int nb, int b, int sweeps, double to
         const double denom = sqrt(a * d);
         const double rel = denom > 0.0 ? fabs(c) / denom : 0.0;
         if (live && tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], rel);
-        if (live && rel >= 1e-15) {
+        if (live && rel >= 1e-9) {
           const double zeta = (d - a) / (2.0 * c);
           const double tn = (zeta >= 0.0 ? 1.0 : -1.0) / (fabs(zeta) + sqrt(1.0 + zeta * zeta));
-          const double cs = 1.0 / sqrt(1.0 + tn * tn), sn = cs * tn;
+          const double csd = 1.0 / sqrt(1.0 + tn * tn);
+          const float cs = (float)csd, sn = (float)(csd * tn);
 #pragma unroll
           for (int e = 0; e < NE; ++e) {
             const int i = tt + kTeam * e;
             if (i < b) {
-              __stcg(tp + i, cs * x[e] - sn * y[e]);
-              __stcg(tq + i, sn * x[e] + cs * y[e]);
+              __stcg(tp + i, fmaf(cs, x[e], -sn * y[e]));
+              __stcg(tq + i, fmaf(sn, x[e], cs * y[e]));
             }
           }
         }
@@ -391,7 +397,7 @@ jacobi_sweeps_kernel(const Ptrs<double> Tb, int nb, int b, int sweeps, double to
         if (tt < nb && s_worst[team][tt] > 0.0)
           atomicMax(offb.p[tt] + sw, (unsigned long long)__double_as_longlong(s_worst[team][tt]));
       }
-      if (!grid_barrier(sync_words, sync_words + 1, gen)) {
+      if (!grid_barrier(sync_words, gen)) {
         if (threadIdx.x == 0 && status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
         return;
       }
@@ -404,7 +410,7 @@ jacobi_sweeps_kernel(const Ptrs<double> Tb, int nb, int b, int sweeps, double to
 }
 
 template <int NE>
-int launch_jacobi(const Ptrs<double>& T, int nb, int64_t b, int sweeps, double tol, const Ptrs<unsigned long long>& off,
+int launch_jacobi(const Ptrs<float>& T, int nb, int64_t b, int sweeps, double tol, const Ptrs<unsigned long long>& off,
                   unsigned int* sync_words, int32_t* status, cudaStream_t st) {
   // one cooperative launch, never more CTAs than are resident at once
   int per_sm = 0;
@@ -414,7 +420,7 @@ int launch_jacobi(const Ptrs<double>& T, int nb, int64_t b, int sweeps, double t
   int64_t grid = ceil_div(b / 2 * nb, kTeamsPerCta);
   if (grid > resident) grid = resident;
   int bi = (int)b;
-  Ptrs<double> Tc = T;
+  Ptrs<float> Tc = T;
   Ptrs<unsigned long long> offc = off;
   void* args[] = {&Tc, &nb, &bi, &sweeps, &tol, &offc, &sync_words, &status};
   QG_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)jacobi_sweeps_kernel<NE>, dim3((unsigned)grid), dim3(kTeam * kTeamsPerCta),
@@ -425,11 +431,11 @@ int launch_jacobi(const Ptrs<double>& T, int nb, int64_t b, int sweeps, double t
 
 // lambda_j = norm of row j of the rotated T (= |eigenvalue j|); rank_j = its position in descending order
 __global__ void __launch_bounds__(128)
-row_norm_kernel(const Ptrs<const double> Tb, int b, const Ptrs<double> lamb) {
-  const double* row = Tb.p[blockIdx.y] + (int64_t)blockIdx.x * b;
+row_norm_kernel(const Ptrs<const float> Tb, int b, const Ptrs<double> lamb) {
+  const float* row = Tb.p[blockIdx.y] + (int64_t)blockIdx.x * b;
   double* __restrict__ lam = lamb.p[blockIdx.y];
   double s = 0.0;
-  for (int i = threadIdx.x; i < b; i += blockDim.x) s += row[i] * row[i];
+  for (int i = threadIdx.x; i < b; i += blockDim.x) s += (double)row[i] * (double)row[i];
   __shared__ double red[4];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
@@ -440,8 +446,8 @@ row_norm_kernel(const Ptrs<const double> Tb, int b, const Ptrs<double> lamb) {
 
 // Xsel[i][rank_j] = X[i][j] = T[j][i] / lambda_j for the r largest lambda_j
 __global__ void __launch_bounds__(256)
-select_top_kernel(const Ptrs<const double> Tb, const Ptrs<const double> lamb, int b, int r, const Ptrs<float> Xselb) {
-  const double* __restrict__ T = Tb.p[blockIdx.y];
+select_top_kernel(const Ptrs<const float> Tb, const Ptrs<const double> lamb, int b, int r, const Ptrs<float> Xselb) {
+  const float* __restrict__ T = Tb.p[blockIdx.y];
   const double* __restrict__ lam = lamb.p[blockIdx.y];
   float* __restrict__ Xsel = Xselb.p[blockIdx.y];
   const int j = blockIdx.x;
@@ -459,7 +465,7 @@ select_top_kernel(const Ptrs<const double> Tb, const Ptrs<const double> lamb, in
   const int rank = s_rank;
   if (rank >= r) return;
   const double inv = lj > 0.0 ? 1.0 / lj : 0.0;
-  for (int i = threadIdx.x; i < b; i += blockDim.x) Xsel[(int64_t)i * r + rank] = (float)(T[(int64_t)j * b + i] * inv);
+  for (int i = threadIdx.x; i < b; i += blockDim.x) Xsel[(int64_t)i * r + rank] = (float)((double)T[(int64_t)j * b + i] * inv);
 }
 
 // Each column of P gets the sign that makes its largest-magnitude entry positive; optional copy to P_out.
@@ -492,7 +498,8 @@ struct RefreshWs {
   float *Q, *Y, *Z, *Wp, *Cb, *S, *Linv, *Xsel, *P32;
   void* part;      // partial sums of sliced products
   uint16_t* planes;  // the three bfloat16 planes of an iterate, for the tensor-core products
-  double *T, *lam, *off;
+  float* T;        // the Rayleigh-Ritz matrix, then its rotated rows
+  double *lam, *off;
   int32_t* done;
 };
 
@@ -500,7 +507,7 @@ size_t carve_refresh(void* base, int64_t m, int64_t n, int64_t b, int64_t r, Ref
   size_t off = 0;
   auto take = [&](size_t bytes) { void* p = base ? (char*)base + off : nullptr; off += (size_t)round_up((int64_t)bytes, 256); return p; };
   RefreshWs t{};
-  t.T = (double*)take((size_t)b * b * 8);
+  t.T = (float*)take((size_t)b * b * 4);
   t.lam = (double*)take((size_t)b * 8);
   t.off = (double*)take(kMaxSweeps * 8);     // largest normalised inner product of each sweep
   t.done = (int32_t*)take(8);               // the two words of the grid barrier
@@ -644,18 +651,25 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
     rc = orthonormalize(bt, m, b, status, st, it + 2 >= iters);   // the last two in full
     if (rc != QG_OK) return rc;
   }
-  // Rayleigh-Ritz: T = Z^T Z in fp64, eigenvectors by one-sided Jacobi
-  const Ptrs<double> T = QG_TAB(double, T), lam = QG_TAB(double, lam);
-  rc = gemm<float, double, double>(nb, Z, 1, b, Z, b, 1, T, b, b, b, n, 1.0, 0.0, st);
+  // Rayleigh-Ritz: T = Z^T Z (accumulated in binary64, kept in binary32), eigenvectors by one-sided Jacobi
+  const Ptrs<float> T = QG_TAB(float, T);
+  const Ptrs<double> lam = QG_TAB(double, lam);
+  rc = gemm<float, double, float>(nb, Z, 1, b, Z, b, 1, T, b, b, b, n, 1.0, 0.0, st);
   if (rc != QG_OK) return rc;
   if (sweeps > kMaxSweeps) sweeps = kMaxSweeps;
-  Ptrs<unsigned long long> off{};
-  for (int i = 0; i < nb; ++i) {
-    QG_CUDA_TRY(cudaMemsetAsync(bt.w[i].off, 0, kMaxSweeps * 8, st));
-    off.p[i] = reinterpret_cast<unsigned long long*>(bt.w[i].off);
-  }
-  QG_CUDA_TRY(cudaMemsetAsync(bt.w[0].done, 0, 8, st));
-  {
+  for (int i = 0; i < nb; ++i) QG_CUDA_TRY(cudaMemsetAsync(bt.w[i].off, 0, kMaxSweeps * 8, st));
+  // A round reads and writes every row once, so the matrices rotated together should stay in L2 together: at most
+  // kJacobiBytes of them per cooperative launch.
+  const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(nb, kJacobiBytes / (b * b * 4)));
+  for (int first = 0; first < nb; first += per_launch) {
+    const int cnt = std::min(per_launch, nb - first);
+    Ptrs<float> Tsub{};
+    Ptrs<unsigned long long> off{};
+    for (int i = 0; i < cnt; ++i) {
+      Tsub.p[i] = bt.w[first + i].T;
+      off.p[i] = reinterpret_cast<unsigned long long*>(bt.w[first + i].off);
+    }
+    QG_CUDA_TRY(cudaMemsetAsync(bt.w[0].done, 0, 8, st));
     unsigned int* sync_words = reinterpret_cast<unsigned int*>(bt.w[0].done);
     // the iteration converges quadratically at the end: a sweep that met nothing above 1e-5 leaves ~1e-10
     constexpr double kTol = 1e-5;
@@ -672,13 +686,14 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
       if (!g_coop_done[dev]) QG_CUDA_TRY(cudaEventCreateWithFlags(&g_coop_done[dev], cudaEventDisableTiming));
       else QG_CUDA_TRY(cudaStreamWaitEvent(st, g_coop_done[dev], 0));
     }
-    if (b <= 8 * kTeam) rc = launch_jacobi<8>(T, nb, b, sweeps, kTol, off, sync_words, status, st);
-    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(T, nb, b, sweeps, kTol, off, sync_words, status, st);
-    else rc = launch_jacobi<32>(T, nb, b, sweeps, kTol, off, sync_words, status, st);
+    if (b <= 8 * kTeam) rc = launch_jacobi<8>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    else if (b <= 16 * kTeam) rc = launch_jacobi<16>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    else rc = launch_jacobi<32>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     if (rc != QG_OK) return rc;
     if (chain) QG_CUDA_TRY(cudaEventRecord(g_coop_done[dev], st));
   }
-  const Ptrs<const double> Tc = QG_TAB(const double, T), lamc = QG_TAB(const double, lam);
+  const Ptrs<const float> Tc = QG_TAB(const float, T);
+  const Ptrs<const double> lamc = QG_TAB(const double, lam);
   row_norm_kernel<<<dim3((unsigned)b, (unsigned)nb), 128, 0, st>>>(Tc, (int)b, lam);
   QG_LAUNCH_CHECK();
   select_top_kernel<<<dim3((unsigned)b, (unsigned)nb), 256, 0, st>>>(Tc, lamc, (int)b, (int)r, QG_TAB(float, Xsel));
