@@ -44,6 +44,8 @@ cudaEvent_t g_coop_done[kCoopDevices] = {};   // completion of the last cooperat
 
 // Test aid: 0 keeps every product of the refresh on the CUDA cores.
 int g_refresh_tc = 1;
+// Test aid: 0 rotates the rows of the Rayleigh-Ritz matrix pair by pair through L2 for every shape.
+int g_jacobi_blocks = 1;
 
 constexpr int kPanel = 64;    // columns orthonormalised together
 constexpr int kMaxSweeps = 32;
@@ -83,8 +85,9 @@ gemm_kernel(const Ptrs<const TA> Ab, int64_t sa_m, int64_t sa_k, const Ptrs<cons
   const float* __restrict__ B = Bb.p[mat];
   TC* __restrict__ C = Cb.p[mat];
   ACC* __restrict__ part = slices > 1 ? partb.p[mat] : nullptr;
-  __shared__ __align__(16) float As[kGK][kGT + 4];
-  __shared__ __align__(16) float Bs[kGK][kGT + 4];
+  // two buffers per operand: the loads of the next K step are in flight (in registers) while this one is multiplied
+  __shared__ __align__(16) float As[2][kGK][kGT + 4];
+  __shared__ __align__(16) float Bs[2][kGK][kGT + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const int64_t m0 = (int64_t)blockIdx.y * kGT, n0 = (int64_t)blockIdx.x * kGT;
   ACC acc[4][4];
@@ -95,29 +98,48 @@ gemm_kernel(const Ptrs<const TA> Ab, int64_t sa_m, int64_t sa_k, const Ptrs<cons
   const bool a_m_fast = (sa_m == 1), b_n_fast = (sb_n == 1);
   const int k_begin = slice * k_slice;
   if (slices > 1) K = min(K, k_begin + k_slice);
-  for (int k0 = k_begin; k0 < K; k0 += kGK) {
+  float ra[4], rb[4];
+  auto fetch = [&](int k0) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       int mm, kk;
       if (a_m_fast) { mm = tid & 63; kk = (tid >> 6) + 4 * e; } else { kk = tid & 15; mm = (tid >> 4) + 16 * e; }
       const int64_t gm = m0 + mm, gk = k0 + kk;
-      As[kk][mm] = (gm < M && gk < K) ? ld_as_float(A, gm * sa_m + gk * sa_k) : 0.f;
+      ra[e] = (gm < M && gk < K) ? ld_as_float(A, gm * sa_m + gk * sa_k) : 0.f;
       int nn, kb;
       if (b_n_fast) { nn = tid & 63; kb = (tid >> 6) + 4 * e; } else { kb = tid & 15; nn = (tid >> 4) + 16 * e; }
       const int64_t gn = n0 + nn, gkb = k0 + kb;
-      Bs[kb][nn] = (gn < N && gkb < K) ? B[gkb * sb_k + gn * sb_n] : 0.f;
+      rb[e] = (gn < N && gkb < K) ? B[gkb * sb_k + gn * sb_n] : 0.f;
     }
-    __syncthreads();
+  };
+  auto stash = [&](int buf) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      int mm, kk;
+      if (a_m_fast) { mm = tid & 63; kk = (tid >> 6) + 4 * e; } else { kk = tid & 15; mm = (tid >> 4) + 16 * e; }
+      As[buf][kk][mm] = ra[e];
+      int nn, kb;
+      if (b_n_fast) { nn = tid & 63; kb = (tid >> 6) + 4 * e; } else { kb = tid & 15; nn = (tid >> 4) + 16 * e; }
+      Bs[buf][kb][nn] = rb[e];
+    }
+  };
+  if (k_begin < K) { fetch(k_begin); stash(0); }
+  __syncthreads();
+  int buf = 0;
+  for (int k0 = k_begin; k0 < K; k0 += kGK, buf ^= 1) {
+    const bool more = k0 + kGK < K;
+    if (more) fetch(k0 + kGK);
 #pragma unroll
     for (int kk = 0; kk < kGK; ++kk) {
-      const float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float4 a4 = *reinterpret_cast<const float4*>(&As[buf][kk][ty * 4]);
+      const float4 b4 = *reinterpret_cast<const float4*>(&Bs[buf][kk][tx * 4]);
       const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] += (ACC)a[i] * (ACC)b[j];
     }
+    if (more) stash(buf ^ 1);      // nobody reads that buffer before the barrier below
     __syncthreads();
   }
 #pragma unroll
@@ -225,60 +247,80 @@ gaussian_kernel(const Ptrs<float> Qb, int64_t ld, int64_t rows, int64_t cols, co
   *reinterpret_cast<float4*>(Q + i * ld + 4 * jq) = make_float4(r0 * c0, r0 * s0, r1 * c1, r1 * s1);
 }
 
-// ---- Cholesky factor of a 64 x 64 Gram matrix and the inverse of the factor, one CTA of 256 threads, fp64.
-// S (row-major fp32) = L L^T;  Linv = L^-1 (lower triangular, row-major fp32).  A non-positive pivot raises
+// ---- Cholesky factor of a 64 x 64 Gram matrix and the inverse of the factor, ONE WARP per matrix, binary32.
+// S (row-major) = L L^T;  Linv = L^-1 (lower triangular, row-major).  A non-positive pivot raises
 // QG_DEV_BAD_FACTOR and is replaced by a tiny positive number so that the run continues with finite values.
-// One shared array holds both triangles: L below and on the diagonal, the transpose of L^-1 above it
-// (A[j][i] = (L^-1)[i][j] for i > j); the diagonal of L^-1 is kept apart.
-__global__ void __launch_bounds__(256)
+// The factorisation is a chain of 64 dependent steps whatever runs it, so it is laid out for the shortest step:
+// lane r keeps rows r and r + 32 in registers, the pivot and the column under it travel by shuffles, every loop is
+// unrolled (all register indices are constants), and nothing touches memory until L is complete.  The inverse is
+// then taken column-wise (lane c owns columns c and c + 32) by forward substitution with L broadcast from shared
+// memory.  Binary32 is enough here: S itself comes from a binary32 product, and where the basis has to be
+// orthonormal to rounding the panel goes through this twice.
+__global__ void __launch_bounds__(32)
 chol64_inverse_kernel(const Ptrs<const float> Sb, const Ptrs<float> Linvb, int32_t* __restrict__ status) {
+  static_assert(kPanel == 64, "two rows and two columns per lane");
   const float* __restrict__ S = Sb.p[blockIdx.x];
   float* __restrict__ Linv = Linvb.p[blockIdx.x];
-  __shared__ double A[kPanel][kPanel + 1];
-  __shared__ double xd[kPanel];
-  const int t = threadIdx.x;
-  for (int e = t; e < kPanel * kPanel; e += 256) A[e / kPanel][e % kPanel] = (double)S[e];
-  __syncthreads();
-  // right-looking factorisation: thread (i, g) owns the entries L[i][j] with j = k + 1 + g, k + 5 + g, ...
-  {
-    const int i = t & 63, g = t >> 6;
-    for (int k = 0; k < kPanel; ++k) {
-      double d = A[k][k];
-      if (!(d > 0.0)) { if (t == 0 && status) atomicOr(status, QG_DEV_BAD_FACTOR); d = 1e-30; }
-      const double dk = sqrt(d);
-      __syncthreads();                                 // everyone has read the pivot
-      if (g == 0) {
-        if (i == k) A[k][k] = dk;
-        else if (i > k) A[i][k] /= dk;
-      }
-      __syncthreads();
-      if (i > k) {
-        const double lik = A[i][k];
-        for (int j = k + 1 + g; j <= i; j += 4) A[i][j] -= lik * A[j][k];
-      }
-      __syncthreads();
+  __shared__ float Ls[kPanel][kPanel + 1];
+  __shared__ float rds[kPanel];                  // 1 / L[i][i]
+  const int lane = threadIdx.x;
+  float a0[32], a1[64];                          // row `lane` (its lower triangle ends at column 31) and row `lane + 32`
+#pragma unroll
+  for (int j = 0; j < 32; j += 4) {
+    const float4 v = *reinterpret_cast<const float4*>(S + lane * kPanel + j);
+    a0[j] = v.x; a0[j + 1] = v.y; a0[j + 2] = v.z; a0[j + 3] = v.w;
+  }
+#pragma unroll
+  for (int j = 0; j < 64; j += 4) {
+    const float4 v = *reinterpret_cast<const float4*>(S + (lane + 32) * kPanel + j);
+    a1[j] = v.x; a1[j + 1] = v.y; a1[j + 2] = v.z; a1[j + 3] = v.w;
+  }
+  bool bad = false;
+  // right-looking factorisation; entries right of a row's diagonal hold values that are never read
+#pragma unroll
+  for (int k = 0; k < kPanel; ++k) {
+    float piv = __shfl_sync(0xFFFFFFFFu, k < 32 ? a0[k & 31] : a1[k], k & 31);
+    if (!(piv > 0.f)) { bad = true; piv = 1e-30f; }
+    float inv = rsqrtf(piv);
+    inv = inv * fmaf(-0.5f * piv * inv, inv, 1.5f);        // one Newton step: the reciprocal root to rounding
+    if (lane == (k & 31)) rds[k] = inv;
+    float l0 = 0.f;
+    if (k < 32) { l0 = (lane == k) ? piv * inv : a0[k & 31] * inv; a0[k & 31] = l0; }
+    const float l1 = (k >= 32 && lane + 32 == k) ? piv * inv : a1[k] * inv;
+    a1[k] = l1;
+#pragma unroll
+    for (int j = k + 1; j < kPanel; ++j) {
+      const float ljk = __shfl_sync(0xFFFFFFFFu, j < 32 ? l0 : l1, j & 31);
+      if (j < 32) a0[j & 31] = fmaf(-l0, ljk, a0[j & 31]);
+      a1[j] = fmaf(-l1, ljk, a1[j]);
     }
   }
-  // forward substitution, row by row: X[i][j] = -(sum_{k=j}^{i-1} L[i][k] X[k][j]) / L[i][i] for j < i.
-  // Four neighbouring lanes share a column j and split the sum.
-  {
-    const int j = t >> 2, part = t & 3;
-    if (t < kPanel) xd[t] = 1.0 / A[t][t];
-    __syncthreads();
-    for (int i = 1; i < kPanel; ++i) {
-      double sum = 0.0;
-      if (j < i) {
-        for (int k = j + part; k < i; k += 4) sum += A[i][k] * (k == j ? xd[j] : A[j][k]);
-      }
-      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-      sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);
-      if (j < i && part == 0) A[j][i] = -sum * xd[i];   // column i of the upper triangle: read by later rows only
-      __syncthreads();
+  if (bad && lane == 0 && status) atomicOr(status, QG_DEV_BAD_FACTOR);
+#pragma unroll
+  for (int j = 0; j < 32; ++j) Ls[lane][j] = a0[j];
+#pragma unroll
+  for (int j = 0; j < 64; ++j) Ls[lane + 32][j] = a1[j];
+  __syncwarp();
+  // X = L^-1, column c (rows c..63) in x0, column c + 32 (rows c + 32..63) in x1:
+  // X[i][c] = ([i == c] - sum_{k < i} L[i][k] X[k][c]) / L[i][i], with X[k][c] = 0 above the diagonal
+  float x0[64], x1[32];
+#pragma unroll
+  for (int i = 0; i < kPanel; ++i) {
+    float s0 = (i == lane) ? 1.f : 0.f, s0b = 0.f, s1 = (i == lane + 32) ? 1.f : 0.f, s1b = 0.f;
+#pragma unroll
+    for (int k = 0; k < i; ++k) {
+      const float lik = Ls[i][k];
+      if (k & 1) s0b = fmaf(-lik, x0[k], s0b); else s0 = fmaf(-lik, x0[k], s0);
+      if (k >= 32) { if (k & 1) s1b = fmaf(-lik, x1[k - 32], s1b); else s1 = fmaf(-lik, x1[k - 32], s1); }
     }
+    const float rd = rds[i];
+    x0[i] = (i >= lane) ? (s0 + s0b) * rd : 0.f;
+    if (i >= 32) x1[i - 32] = (i >= lane + 32) ? (s1 + s1b) * rd : 0.f;
   }
-  for (int e = t; e < kPanel * kPanel; e += 256) {
-    const int i = e / kPanel, j = e % kPanel;
-    Linv[e] = (float)(i == j ? xd[i] : (i > j ? A[j][i] : 0.0));
+#pragma unroll
+  for (int i = 0; i < kPanel; ++i) {
+    Linv[i * kPanel + lane] = x0[i];
+    Linv[i * kPanel + lane + 32] = i >= 32 ? x1[i - 32] : 0.f;
   }
 }
 
@@ -429,6 +471,209 @@ int launch_jacobi(const Ptrs<float>& T, int nb, int64_t b, int sweeps, double to
   return QG_OK;
 }
 
+// ---- the same iteration with the rows in blocks of eight.  A sweep first rotates the pairs INSIDE every block
+// (seven short rounds through L2, as above), then runs a round-robin tournament over the blocks: a CTA takes a pair
+// of blocks (I, J), every team of 64 threads keeps one row of I in registers, the rows of J sit in shared memory,
+// and eight inner rounds rotate every row of I against every row of J.  A row pair thus moves through L2 once per
+// eight rotations and a grid barrier separates b/8 - 1 rounds instead of b - 1: rounds of the plain form move every
+// matrix of the batch through L2 once per rotation and are bound by exactly that.
+constexpr int kBlkRows = 8, kBlkTeam = 64, kBlkThreads = kBlkRows * kBlkTeam;
+
+// One rotation of the rows x, y (NE elements each per thread) held by a team; all teams of the CTA call it together.
+// Returns the normalised inner product the pair had; `rotated` tells whether x and y changed.
+template <int NE>
+__device__ __forceinline__ double team_rotate(float (&x)[NE], float (&y)[NE], bool live, double (*red)[2], int tw, int lane,
+                                              bool& rotated) {
+  // the thread's few products in binary32 (each exact to 2^-24 of itself), everything summed across threads in
+  // binary64
+  float af = 0.f, cf = 0.f, df = 0.f;
+#pragma unroll
+  for (int e = 0; e < NE; ++e) { af = fmaf(x[e], x[e], af); df = fmaf(y[e], y[e], df); cf = fmaf(x[e], y[e], cf); }
+  double a = (double)af, c = (double)cf, d = (double)df;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+    d += __shfl_xor_sync(0xFFFFFFFFu, d, o);
+    c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+  }
+  if (lane == 0) { red[0][tw] = a; red[1][tw] = d; red[2][tw] = c; }
+  __syncthreads();
+  a = red[0][0] + red[0][1];
+  d = red[1][0] + red[1][1];
+  c = red[2][0] + red[2][1];
+  // The sums are binary64; the angle is formed from them in binary32 (the difference d - a first, in binary64):
+  // the rows it turns are binary32, and the six dependent divisions and roots of the binary64 form were a third
+  // of a rotation's time.
+  const double ad = a * d;
+  const float rel_f = ad > 0.0 ? fabsf((float)c) * rsqrtf((float)a) * rsqrtf((float)d) : 0.f;
+  const double rel = (double)rel_f;
+  rotated = live && rel_f >= 1e-9f;
+  if (rotated) {
+    const float zeta = __fdividef((float)(d - a), 2.0f * (float)c);
+    const float az = fabsf(zeta);
+    // tan = sign(zeta) / (|zeta| + sqrt(1 + zeta^2)); for |zeta| beyond 2^60 the square overflows and tan = 1 / (2 zeta)
+    const float tn = az < 1.0e18f ? copysignf(__fdividef(1.0f, az + sqrtf(fmaf(zeta, zeta, 1.0f))), zeta) : __fdividef(0.5f, zeta);
+    const float cs = rsqrtf(fmaf(tn, tn, 1.0f)), sn = cs * tn;
+#pragma unroll
+    for (int e = 0; e < NE; ++e) {
+      const float xn = fmaf(cs, x[e], -sn * y[e]);
+      y[e] = fmaf(sn, x[e], cs * y[e]);
+      x[e] = xn;
+    }
+  }
+  return live ? rel : 0.0;
+}
+
+template <int NE>
+__global__ void __launch_bounds__(kBlkThreads, NE <= 16 ? 2 : 1)
+jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol, const Ptrs<unsigned long long> offb,
+                    unsigned int* __restrict__ sync_words, int32_t* __restrict__ status) {
+  extern __shared__ float rows_j[];                  // the eight rows of block J, b floats each
+  __shared__ double red[kBlkRows][3][2];
+  __shared__ double s_worst[kBlkRows][kMaxBatch];
+  const int team = threadIdx.x / kBlkTeam, tt = threadIdx.x % kBlkTeam, tw = tt >> 5, lane = threadIdx.x & 31;
+  const int nblk = b / kBlkRows, half = nblk / 2;
+  const int cta_jobs = nb * half;                    // block pairs per outer round; also eight within-block pairs each
+  unsigned int gen = 0;
+  uint32_t active = (1u << nb) - 1u;                 // matrices still rotating
+  for (int sw = 0; sw < sweeps && active != 0u; ++sw) {
+    if (tt < kMaxBatch) s_worst[team][tt] = 0.0;
+    __syncthreads();
+    // ---- the pairs inside every block: round `rnd` of the tournament of its eight rows, four pairs per block
+    for (int rnd = 0; rnd < kBlkRows - 1; ++rnd) {
+      for (int j0 = 0; j0 < cta_jobs; j0 += (int)gridDim.x) {
+        const int k = (j0 + (int)blockIdx.x) * kBlkRows + team;     // pair index: (matrix, block, pair of the round)
+        const int per_mat = nblk * (kBlkRows / 2);
+        const bool in_range = j0 + (int)blockIdx.x < cta_jobs;
+        const int mat = in_range ? k / per_mat : 0;
+        const bool live = in_range && ((active >> mat) & 1u);
+        int p = 0, q = 0;
+        if (live) {
+          const int rem = k - mat * per_mat;
+          tournament_pair(kBlkRows, rnd, rem % (kBlkRows / 2), p, q);
+          p += (rem / (kBlkRows / 2)) * kBlkRows;
+          q += (rem / (kBlkRows / 2)) * kBlkRows;
+        }
+        float* tp = Tb.p[mat] + (int64_t)p * b;
+        float* tq = Tb.p[mat] + (int64_t)q * b;
+        float x[NE], y[NE];
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+          const int i = tt + kBlkTeam * e;
+          const bool in = live && i < b;
+          x[e] = in ? __ldcg(tp + i) : 0.f;
+          y[e] = in ? __ldcg(tq + i) : 0.f;
+        }
+        bool rotated;
+        const double rel = team_rotate<NE>(x, y, live, red[team], tw, lane, rotated);
+        if (live && tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], rel);
+        if (rotated) {
+#pragma unroll
+          for (int e = 0; e < NE; ++e) {
+            const int i = tt + kBlkTeam * e;
+            if (i < b) { __stcg(tp + i, x[e]); __stcg(tq + i, y[e]); }
+          }
+        }
+        __syncthreads();                               // `red` is free again
+      }
+      if (!grid_barrier(sync_words, gen)) {
+        if (threadIdx.x == 0 && status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
+        return;
+      }
+    }
+    // ---- the pairs between blocks: round `orr` of the tournament of the blocks
+    for (int orr = 0; orr < nblk - 1; ++orr) {
+      for (int job = (int)blockIdx.x; job < cta_jobs; job += (int)gridDim.x) {
+        const int mat = job / half;
+        if (!((active >> mat) & 1u)) continue;         // the same for every thread of the CTA
+        int bi = 0, bj = 0;
+        tournament_pair(nblk, orr, job - mat * half, bi, bj);
+        float* ti = Tb.p[mat] + ((int64_t)bi * kBlkRows + team) * b;   // this team's row of block I
+        float* tj = Tb.p[mat] + ((int64_t)bj * kBlkRows + team) * b;   // the row of block J it brings in and takes out
+        float x[NE], y[NE];
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+          const int i = tt + kBlkTeam * e;
+          x[e] = i < b ? __ldcg(ti + i) : 0.f;
+          if (i < b) rows_j[team * b + i] = __ldcg(tj + i);
+        }
+        __syncthreads();
+        double worst = 0.0;
+#pragma unroll 1
+        for (int sft = 0; sft < kBlkRows; ++sft) {
+          float* yr = rows_j + ((team + sft) & (kBlkRows - 1)) * b;
+#pragma unroll
+          for (int e = 0; e < NE; ++e) {
+            const int i = tt + kBlkTeam * e;
+            y[e] = i < b ? yr[i] : 0.f;
+          }
+          bool rotated;
+          worst = fmax(worst, team_rotate<NE>(x, y, true, red[team], tw, lane, rotated));
+          if (rotated) {
+#pragma unroll
+            for (int e = 0; e < NE; ++e) {
+              const int i = tt + kBlkTeam * e;
+              if (i < b) yr[i] = y[e];
+            }
+          }
+          __syncthreads();                             // the next round reads another team's row; `red` is free
+        }
+        if (tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], worst);
+#pragma unroll
+        for (int e = 0; e < NE; ++e) {
+          const int i = tt + kBlkTeam * e;
+          if (i < b) { __stcg(ti + i, x[e]); __stcg(tj + i, rows_j[team * b + i]); }
+        }
+        __syncthreads();                               // rows_j may be refilled
+      }
+      if (orr == nblk - 2) {
+        __syncthreads();
+        // only ever compared, so the monotone integer view of a non-negative double serves atomicMax
+        if (tt < nb && s_worst[team][tt] > 0.0)
+          atomicMax(offb.p[tt] + sw, (unsigned long long)__double_as_longlong(s_worst[team][tt]));
+      }
+      if (!grid_barrier(sync_words, gen)) {
+        if (threadIdx.x == 0 && status) atomicOr(status, QG_DEV_WAIT_EXPIRED);
+        return;
+      }
+    }
+    for (int i = 0; i < nb; ++i)
+      if (((active >> i) & 1u) && __longlong_as_double((long long)__ldcg(offb.p[i] + sw)) <= tol) active &= ~(1u << i);
+    __syncthreads();                                 // s_worst is cleared at the top of the next sweep
+  }
+  if (active != 0u && blockIdx.x == 0 && threadIdx.x == 0 && status) atomicOr(status, QG_DEV_NOT_CONVERGED);
+}
+
+// Opts the instance into its dynamic shared memory once per device.
+template <int NE>
+int launch_jacobi_block(const Ptrs<float>& T, int nb, int64_t b, int sweeps, double tol, const Ptrs<unsigned long long>& off,
+                        unsigned int* sync_words, int32_t* status, cudaStream_t st) {
+  const int smem = (int)(kBlkRows * b * sizeof(float));
+  static bool smem_set[kCoopDevices] = {};
+  int dev = 0;
+  QG_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kCoopDevices) return QG_UNSUPPORTED_SHAPE;
+  if (!smem_set[dev]) {
+    QG_CUDA_TRY(cudaFuncSetAttribute(jacobi_block_kernel<NE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBlkRows * NE * kBlkTeam * 4));
+    smem_set[dev] = true;
+  }
+  // one cooperative launch, never more CTAs than are resident at once
+  int per_sm = 0;
+  QG_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, jacobi_block_kernel<NE>, kBlkThreads, smem));
+  const int64_t resident = (int64_t)per_sm * refresh_sm_count();
+  if (resident < 1) { note_cuda_error(cudaErrorCooperativeLaunchTooLarge, "jacobi_block_kernel occupancy"); return QG_CUDA_ERROR; }
+  int64_t grid = (b / kBlkRows / 2) * nb;
+  if (grid > resident) grid = resident;
+  int bi = (int)b;
+  Ptrs<float> Tc = T;
+  Ptrs<unsigned long long> offc = off;
+  void* args[] = {&Tc, &nb, &bi, &sweeps, &tol, &offc, &sync_words, &status};
+  QG_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)jacobi_block_kernel<NE>, dim3((unsigned)grid), dim3(kBlkThreads), args,
+                                          (size_t)smem, st));
+  count_launch();
+  return QG_OK;
+}
+
 // lambda_j = norm of row j of the rotated T (= |eigenvalue j|); rank_j = its position in descending order
 __global__ void __launch_bounds__(128)
 row_norm_kernel(const Ptrs<const float> Tb, int b, const Ptrs<double> lamb) {
@@ -575,7 +820,7 @@ int orthonormalize(const Batch& bt, int64_t m, int64_t b, int32_t* status, cudaS
       const int64_t ldd = last ? b : kPanel;
       rc = gemm<float, float, float>(nb, src, 1, lds, src, lds, 1, S, kPanel, kPanel, kPanel, m, 1.f, 0.f, st, &part);
       if (rc != QG_OK) return rc;
-      chol64_inverse_kernel<<<nb, 256, 0, st>>>(Sc, Linv, status);
+      chol64_inverse_kernel<<<nb, 32, 0, st>>>(Sc, Linv, status);
       QG_LAUNCH_CHECK();
       // dst = src * Linv^T:  B(k, j) = Linv[j][k]
       rc = gemm<float, float, float>(nb, src, lds, 1, Linvc, 1, kPanel, dst, ldd, m, kPanel, kPanel, 1.f, 0.f, st);
@@ -686,7 +931,10 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
       if (!g_coop_done[dev]) QG_CUDA_TRY(cudaEventCreateWithFlags(&g_coop_done[dev], cudaEventDisableTiming));
       else QG_CUDA_TRY(cudaStreamWaitEvent(st, g_coop_done[dev], 0));
     }
-    if (b <= 8 * kTeam) rc = launch_jacobi<8>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    // rows in blocks of eight where the block count is even and a block fits shared memory; else row by row
+    if (g_jacobi_blocks && b % (2 * kBlkRows) == 0 && b <= 16 * kBlkTeam) rc = launch_jacobi_block<16>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    else if (g_jacobi_blocks && b % (2 * kBlkRows) == 0 && b <= 32 * kBlkTeam) rc = launch_jacobi_block<32>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    else if (b <= 8 * kTeam) rc = launch_jacobi<8>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     else if (b <= 16 * kTeam) rc = launch_jacobi<16>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     else rc = launch_jacobi<32>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     if (rc != QG_OK) return rc;
