@@ -16,7 +16,7 @@ namespace qg {
 constexpr int kGroup = 256;  // Sec. 3.1: block size 256
 
 // Bumped whenever a change to the step's kernels can move their DRAM traffic or timing (see qgalore_kernel_revision).
-#define QG_STEP_KERNELS_REVISION "step-2026-11-28c"
+#define QG_STEP_KERNELS_REVISION "step-2026-11-30a"
 
 // ----------------------------------------------------------------------------- host plumbing
 void note_cuda_error(cudaError_t e, const char* where);
