@@ -212,7 +212,7 @@ QG_API int qgalore_plan_step_timed(const qg_plan* plan, const qg_hyper* h, int32
  * Top-r left singular vectors of G (bf16, m x n, pitch ldg) by block subspace iteration on G G^T with a
  * block of b = r + oversample_cols columns (`iters` multiplications by G G^T, each followed by a block
  * Gram-Schmidt orthonormalisation) and a Rayleigh-Ritz step (eigenvectors of the projected b x b matrix by
- * a Jacobi iteration in fp64), then Quant_4 into P_new.  Each column carries the sign that makes its
+ * a Jacobi iteration on binary32 rows with binary64 sums), then Quant_4 into P_new.  Each column carries the sign that makes its
  * largest-magnitude entry positive.
  *   P_new      INT4, m x r, ld == r; written
  *   P_fp32     optional (may be NULL): m x r fp32, pitch r, receives the vectors before quantization
