@@ -149,8 +149,10 @@ QG_API int qgalore_project_step_right(const uint16_t* G, int64_t ldg, int64_t m,
  * Every item is one independent matrix with its own buffers and its own stochastic-rounding
  * seed; lr, alpha, the Adam constants and the step index come from h (h->seed is ignored).
  * items is HOST memory.  The workspace (qgalore_workspace_bytes_batched) is shared by the
- * items, which are processed in order on `stream`.  Validation covers every item before
- * anything is enqueued. */
+ * items, which are processed in order on `stream`, three launches per matrix.  Validation covers
+ * every item before anything is enqueued.  This call is for lists that change from call to call;
+ * a list that is stepped repeatedly belongs in a plan (below), which prepares the descriptors once
+ * and runs a whole chunk of matrices per launch (LLaMA-1B stack: 3.2 ms per step as a plan). */
 typedef struct {
   const uint16_t* G; int64_t ldg, m, n, r;
   qg_qtensor P, W;
