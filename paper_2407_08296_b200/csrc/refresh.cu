@@ -479,6 +479,16 @@ int launch_jacobi(const Ptrs<float>& T, int nb, int64_t b, int sweeps, double to
 // matrix of the batch through L2 once per rotation and are bound by exactly that.
 constexpr int kBlkRows = 8, kBlkTeam = 64, kBlkThreads = kBlkRows * kBlkTeam;
 
+// A thread of a team holds NE elements of a row in groups of four consecutive ones: group g covers elements
+// 256 g + 4 tt .. + 3 (tt = its index in the team of 64), so rows move as 16-byte pieces everywhere.
+__device__ __forceinline__ int blk_elem(int g, int tt) { return 256 * g + 4 * tt; }
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 // One rotation of the rows x, y (NE elements each per thread) held by a team; all teams of the CTA call it together.
 // Returns the normalised inner product the pair had; `rotated` tells whether x and y changed.
 template <int NE>
@@ -528,12 +538,16 @@ template <int NE>
 __global__ void __launch_bounds__(kBlkThreads, NE <= 16 ? 2 : 1)
 jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol, const Ptrs<unsigned long long> offb,
                     unsigned int* __restrict__ sync_words, int32_t* __restrict__ status) {
-  extern __shared__ float rows_j[];                  // the eight rows of block J, b floats each
+  // three sets of eight rows of b floats: the rows of block J of this job and of the next one (the copy engine brings
+  // the next job's rows in while this one rotates), and the rows of block I of the next job
+  extern __shared__ __align__(16) float blk_smem[];
   __shared__ double red[kBlkRows][3][2];
   __shared__ double s_worst[kBlkRows][kMaxBatch];
   const int team = threadIdx.x / kBlkTeam, tt = threadIdx.x % kBlkTeam, tw = tt >> 5, lane = threadIdx.x & 31;
   const int nblk = b / kBlkRows, half = nblk / 2;
   const int cta_jobs = nb * half;                    // block pairs per outer round; also eight within-block pairs each
+  const int set = kBlkRows * b;
+  float* const rows_i_next = blk_smem + 2 * set;
   unsigned int gen = 0;
   uint32_t active = (1u << nb) - 1u;                 // matrices still rotating
   for (int sw = 0; sw < sweeps && active != 0u; ++sw) {
@@ -558,20 +572,25 @@ jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol,
         float* tq = Tb.p[mat] + (int64_t)q * b;
         float x[NE], y[NE];
 #pragma unroll
-        for (int e = 0; e < NE; ++e) {
-          const int i = tt + kBlkTeam * e;
+        for (int g = 0; g < NE / 4; ++g) {
+          const int i = blk_elem(g, tt);
           const bool in = live && i < b;
-          x[e] = in ? __ldcg(tp + i) : 0.f;
-          y[e] = in ? __ldcg(tq + i) : 0.f;
+          const float4 vx = in ? __ldcg(reinterpret_cast<const float4*>(tp + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 vy = in ? __ldcg(reinterpret_cast<const float4*>(tq + i)) : make_float4(0.f, 0.f, 0.f, 0.f);
+          x[4 * g] = vx.x; x[4 * g + 1] = vx.y; x[4 * g + 2] = vx.z; x[4 * g + 3] = vx.w;
+          y[4 * g] = vy.x; y[4 * g + 1] = vy.y; y[4 * g + 2] = vy.z; y[4 * g + 3] = vy.w;
         }
         bool rotated;
         const double rel = team_rotate<NE>(x, y, live, red[team], tw, lane, rotated);
         if (live && tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], rel);
         if (rotated) {
 #pragma unroll
-          for (int e = 0; e < NE; ++e) {
-            const int i = tt + kBlkTeam * e;
-            if (i < b) { __stcg(tp + i, x[e]); __stcg(tq + i, y[e]); }
+          for (int g = 0; g < NE / 4; ++g) {
+            const int i = blk_elem(g, tt);
+            if (i < b) {
+              __stcg(reinterpret_cast<float4*>(tp + i), make_float4(x[4 * g], x[4 * g + 1], x[4 * g + 2], x[4 * g + 3]));
+              __stcg(reinterpret_cast<float4*>(tq + i), make_float4(y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]));
+            }
           }
         }
         __syncthreads();                               // `red` is free again
@@ -583,48 +602,84 @@ jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol,
     }
     // ---- the pairs between blocks: round `orr` of the tournament of the blocks
     for (int orr = 0; orr < nblk - 1; ++orr) {
-      for (int job = (int)blockIdx.x; job < cta_jobs; job += (int)gridDim.x) {
+      // the jobs of this CTA in this round whose matrix still rotates, in order; `fetch` starts the copies of a job's
+      // sixteen rows (the team's row of block I into rows_i_next, its row of block J into set `buf`)
+      auto next_job = [&](int job) {
+        while (job < cta_jobs && !((active >> (job / half)) & 1u)) job += (int)gridDim.x;
+        return job;
+      };
+      auto rows_of = [&](int job, float*& ti, float*& tj) {
         const int mat = job / half;
-        if (!((active >> mat) & 1u)) continue;         // the same for every thread of the CTA
         int bi = 0, bj = 0;
         tournament_pair(nblk, orr, job - mat * half, bi, bj);
-        float* ti = Tb.p[mat] + ((int64_t)bi * kBlkRows + team) * b;   // this team's row of block I
-        float* tj = Tb.p[mat] + ((int64_t)bj * kBlkRows + team) * b;   // the row of block J it brings in and takes out
-        float x[NE], y[NE];
+        ti = Tb.p[mat] + ((int64_t)bi * kBlkRows + team) * b;   // this team's row of block I
+        tj = Tb.p[mat] + ((int64_t)bj * kBlkRows + team) * b;   // the row of block J it brings in and takes out
+      };
+      auto fetch = [&](int job, int buf) {
+        float *ti, *tj;
+        rows_of(job, ti, tj);
 #pragma unroll
-        for (int e = 0; e < NE; ++e) {
-          const int i = tt + kBlkTeam * e;
-          x[e] = i < b ? __ldcg(ti + i) : 0.f;
-          if (i < b) rows_j[team * b + i] = __ldcg(tj + i);
+        for (int g = 0; g < NE / 4; ++g) {
+          const int i = blk_elem(g, tt);
+          if (i < b) {
+            cp_async_16(rows_i_next + team * b + i, ti + i);
+            cp_async_16(blk_smem + buf * set + team * b + i, tj + i);
+          }
         }
-        __syncthreads();
+        cp_async_commit();
+      };
+      int job = next_job((int)blockIdx.x), buf = 0;
+      if (job < cta_jobs) fetch(job, 0);
+      while (job < cta_jobs) {
+        const int mat = job / half;
+        const int nxt = next_job(job + (int)gridDim.x);
+        float *ti, *tj;
+        rows_of(job, ti, tj);
+        float* const rows_j = blk_smem + buf * set;
+        cp_async_wait_all();
+        float x[NE], y[NE];
+        // the thread's own pieces of its row of block I: the very bytes its own copies wrote
+#pragma unroll
+        for (int g = 0; g < NE / 4; ++g) {
+          const int i = blk_elem(g, tt);
+          const float4 v = i < b ? *reinterpret_cast<const float4*>(rows_i_next + team * b + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+          x[4 * g] = v.x; x[4 * g + 1] = v.y; x[4 * g + 2] = v.z; x[4 * g + 3] = v.w;
+        }
+        __syncthreads();                               // every team's row of block J has landed
+        if (nxt < cta_jobs) fetch(nxt, buf ^ 1);       // rows of the same round: nobody writes them before their job
         double worst = 0.0;
 #pragma unroll 1
         for (int sft = 0; sft < kBlkRows; ++sft) {
           float* yr = rows_j + ((team + sft) & (kBlkRows - 1)) * b;
 #pragma unroll
-          for (int e = 0; e < NE; ++e) {
-            const int i = tt + kBlkTeam * e;
-            y[e] = i < b ? yr[i] : 0.f;
+          for (int g = 0; g < NE / 4; ++g) {
+            const int i = blk_elem(g, tt);
+            const float4 v = i < b ? *reinterpret_cast<const float4*>(yr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            y[4 * g] = v.x; y[4 * g + 1] = v.y; y[4 * g + 2] = v.z; y[4 * g + 3] = v.w;
           }
           bool rotated;
           worst = fmax(worst, team_rotate<NE>(x, y, true, red[team], tw, lane, rotated));
           if (rotated) {
 #pragma unroll
-            for (int e = 0; e < NE; ++e) {
-              const int i = tt + kBlkTeam * e;
-              if (i < b) yr[i] = y[e];
+            for (int g = 0; g < NE / 4; ++g) {
+              const int i = blk_elem(g, tt);
+              if (i < b) *reinterpret_cast<float4*>(yr + i) = make_float4(y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]);
             }
           }
           __syncthreads();                             // the next round reads another team's row; `red` is free
         }
         if (tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], worst);
 #pragma unroll
-        for (int e = 0; e < NE; ++e) {
-          const int i = tt + kBlkTeam * e;
-          if (i < b) { __stcg(ti + i, x[e]); __stcg(tj + i, rows_j[team * b + i]); }
+        for (int g = 0; g < NE / 4; ++g) {
+          const int i = blk_elem(g, tt);
+          if (i < b) {
+            __stcg(reinterpret_cast<float4*>(ti + i), make_float4(x[4 * g], x[4 * g + 1], x[4 * g + 2], x[4 * g + 3]));
+            __stcg(reinterpret_cast<float4*>(tj + i), *reinterpret_cast<const float4*>(rows_j + team * b + i));
+          }
         }
-        __syncthreads();                               // rows_j may be refilled
+        __syncthreads();                               // set `buf` may be refilled by the job after next
+        job = nxt;
+        buf ^= 1;
       }
       if (orr == nblk - 2) {
         __syncthreads();
@@ -648,13 +703,13 @@ jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol,
 template <int NE>
 int launch_jacobi_block(const Ptrs<float>& T, int nb, int64_t b, int sweeps, double tol, const Ptrs<unsigned long long>& off,
                         unsigned int* sync_words, int32_t* status, cudaStream_t st) {
-  const int smem = (int)(kBlkRows * b * sizeof(float));
+  const int smem = (int)(3 * kBlkRows * b * sizeof(float));
   static bool smem_set[kCoopDevices] = {};
   int dev = 0;
   QG_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= kCoopDevices) return QG_UNSUPPORTED_SHAPE;
   if (!smem_set[dev]) {
-    QG_CUDA_TRY(cudaFuncSetAttribute(jacobi_block_kernel<NE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBlkRows * NE * kBlkTeam * 4));
+    QG_CUDA_TRY(cudaFuncSetAttribute(jacobi_block_kernel<NE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 3 * kBlkRows * NE * kBlkTeam * 4));
     smem_set[dev] = true;
   }
   // one cooperative launch, never more CTAs than are resident at once
@@ -903,9 +958,12 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
   if (rc != QG_OK) return rc;
   if (sweeps > kMaxSweeps) sweeps = kMaxSweeps;
   for (int i = 0; i < nb; ++i) QG_CUDA_TRY(cudaMemsetAsync(bt.w[i].off, 0, kMaxSweeps * 8, st));
-  // A round reads and writes every row once, so the matrices rotated together should stay in L2 together: at most
-  // kJacobiBytes of them per cooperative launch.
-  const int per_launch = (int)std::max<int64_t>(1, std::min<int64_t>(nb, kJacobiBytes / (b * b * 4)));
+  // A round of the row-by-row form reads and writes every row once, so the matrices rotated together should stay in
+  // L2 together: at most kJacobiBytes of them per cooperative launch.
+  const bool blocks = g_jacobi_blocks && b % (2 * kBlkRows) == 0 && b <= 32 * kBlkTeam;
+  // (the block form moves a row through L2 once per eight rotations and takes the whole batch in one launch: more
+  // jobs per round leave fewer CTAs idle at its end)
+  const int per_launch = blocks ? nb : (int)std::max<int64_t>(1, std::min<int64_t>(nb, kJacobiBytes / (b * b * 4)));
   for (int first = 0; first < nb; first += per_launch) {
     const int cnt = std::min(per_launch, nb - first);
     Ptrs<float> Tsub{};
@@ -932,8 +990,8 @@ static int refresh_batch(const RefreshJob* jobs, int nb, int64_t m, int64_t n, i
       else QG_CUDA_TRY(cudaStreamWaitEvent(st, g_coop_done[dev], 0));
     }
     // rows in blocks of eight where the block count is even and a block fits shared memory; else row by row
-    if (g_jacobi_blocks && b % (2 * kBlkRows) == 0 && b <= 16 * kBlkTeam) rc = launch_jacobi_block<16>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
-    else if (g_jacobi_blocks && b % (2 * kBlkRows) == 0 && b <= 32 * kBlkTeam) rc = launch_jacobi_block<32>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    if (blocks && b <= 16 * kBlkTeam) rc = launch_jacobi_block<16>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
+    else if (blocks) rc = launch_jacobi_block<32>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     else if (b <= 8 * kTeam) rc = launch_jacobi<8>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     else if (b <= 16 * kTeam) rc = launch_jacobi<16>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
     else rc = launch_jacobi<32>(Tsub, cnt, b, sweeps, kTol, off, sync_words, status, st);
