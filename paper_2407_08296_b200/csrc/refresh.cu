@@ -492,8 +492,8 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 // One rotation of the rows x, y (NE elements each per thread) held by a team; all teams of the CTA call it together.
 // Returns the normalised inner product the pair had; `rotated` tells whether x and y changed.
 template <int NE>
-__device__ __forceinline__ double team_rotate(float (&x)[NE], float (&y)[NE], bool live, double (*red)[2], int tw, int lane,
-                                              bool& rotated) {
+__device__ __forceinline__ double team_rotate(float (&x)[NE], float (&y)[NE], bool live, double (*red)[2], int team, int tw,
+                                              int lane, bool& rotated) {
   // the thread's few products in binary32 (each exact to 2^-24 of itself), everything summed across threads in
   // binary64
   float af = 0.f, cf = 0.f, df = 0.f;
@@ -507,7 +507,9 @@ __device__ __forceinline__ double team_rotate(float (&x)[NE], float (&y)[NE], bo
     c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
   }
   if (lane == 0) { red[0][tw] = a; red[1][tw] = d; red[2][tw] = c; }
-  __syncthreads();
+  // only the two warps of the team meet here (named barrier 1 + team): the teams of a CTA drift apart within a
+  // round, so that one team's loads and multiplications overlap another's reductions
+  asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(kBlkTeam) : "memory");
   a = red[0][0] + red[0][1];
   d = red[1][0] + red[1][1];
   c = red[2][0] + red[2][1];
@@ -581,7 +583,7 @@ jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol,
           y[4 * g] = vy.x; y[4 * g + 1] = vy.y; y[4 * g + 2] = vy.z; y[4 * g + 3] = vy.w;
         }
         bool rotated;
-        const double rel = team_rotate<NE>(x, y, live, red[team], tw, lane, rotated);
+        const double rel = team_rotate<NE>(x, y, live, red[team], team, tw, lane, rotated);
         if (live && tt == 0) s_worst[team][mat] = fmax(s_worst[team][mat], rel);
         if (rotated) {
 #pragma unroll
@@ -658,7 +660,7 @@ jacobi_block_kernel(const Ptrs<float> Tb, int nb, int b, int sweeps, double tol,
             y[4 * g] = v.x; y[4 * g + 1] = v.y; y[4 * g + 2] = v.z; y[4 * g + 3] = v.w;
           }
           bool rotated;
-          worst = fmax(worst, team_rotate<NE>(x, y, true, red[team], tw, lane, rotated));
+          worst = fmax(worst, team_rotate<NE>(x, y, true, red[team], team, tw, lane, rotated));
           if (rotated) {
 #pragma unroll
             for (int g = 0; g < NE / 4; ++g) {
