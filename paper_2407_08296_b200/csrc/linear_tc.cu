@@ -51,10 +51,14 @@ struct LinArgs {
 template <int MODE>
 struct LinSmem {
   static constexpr bool kConvert = MODE != kWeightGrad;
-  static constexpr int kABytes = kTileM * kBK * 2;             // 16 KB
+  // The input gradient takes TWO row blocks of dY per tile of W: a converted B tile then serves two MMAs, which
+  // halves, per flop, the shared-memory traffic of the conversion (codes in, codes read, bf16 written) that bounds
+  // this product.  Both accumulators together fill tensor memory, so its epilogue does not overlap the next main loop.
+  static constexpr int kMT = MODE == kInputGrad ? 2 : 1;
+  static constexpr int kABytes = kMT * kTileM * kBK * 2;       // 16 KB per row block
   static constexpr int kBBytes = kTileN * kBK * 2;             // 32 KB
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kStages = kConvert ? 3 : 4;
+  static constexpr int kStages = kConvert ? 2 : 4;
   static constexpr int kRawBytes = kTileN * kBK;               // one INT8 tile: 16 KB
   static constexpr int kRawStages = kConvert ? 3 : 0;
   static constexpr int kBarOffset = kStages * kStageBytes + kRawStages * kRawBytes;
@@ -136,7 +140,7 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; ok && t < total; t += gridDim.x) {
-        const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
+        const int m0 = (t % a.mblocks) * (S::kMT * kTileM), n0 = (t / a.mblocks) * kTileN;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
           const int s = it % S::kStages;
           if (!mbar_wait(&empty[s], ((it / S::kStages) & 1) ^ 1)) { ok = false; break; }
@@ -147,7 +151,9 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
             tma_load_3d(sA + S::kABytes, &a.mapB, &full[s], 0, kb * kBK, n0 / 64);
           } else {
             mbar_arrive_expect_tx(&full[s], S::kABytes);
-            tma_load_2d(sA, &a.mapA, &full[s], kb * kBK, m0);
+#pragma unroll
+            for (int h = 0; h < S::kMT; ++h)       // rows past the matrix read as zero
+              tma_load_2d(sA + h * (S::kABytes / S::kMT), &a.mapA, &full[s], kb * kBK, m0 + h * kTileM);
           }
         }
       }
@@ -167,8 +173,11 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
-        const uint32_t ab = tcount & 1;
-        if (!mbar_wait(&acc_empty[ab], ((tcount >> 1) & 1) ^ 1)) { ok = false; break; }
+        // one row block per tile: two accumulators of 256 columns take alternate tiles; two row blocks per tile: the
+        // tile's two accumulators are the whole of tensor memory and barrier 0 alone paces the tiles
+        const uint32_t ab = S::kMT == 1 ? (tcount & 1) : 0u;
+        const uint32_t use = S::kMT == 1 ? (tcount >> 1) : tcount;
+        if (!mbar_wait(&acc_empty[ab], (use & 1) ^ 1)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + ab * kTileN;
         for (int kb = 0; kb < kblocks; ++kb, ++it) {
@@ -178,7 +187,11 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
           const uint64_t da = desc_a0 + (uint64_t)((s * S::kStageBytes) >> 4);
           const uint64_t db = desc_b0 + (uint64_t)((s * S::kStageBytes) >> 4);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) umma_bf16(d_tmem, da + k * astep, db + k * bstep, idesc, (kb | k) != 0);
+          for (int h = 0; h < S::kMT; ++h)
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k)
+              umma_bf16(d_tmem + h * kTileN, da + (uint64_t)((h * (S::kABytes / S::kMT)) >> 4) + k * astep, db + k * bstep, idesc,
+                        (kb | k) != 0);
           umma_commit(&empty[s]);
         }
         if (ok) umma_commit(&acc_full[ab]);
@@ -208,19 +221,21 @@ int8_linear_kernel(const __grid_constant__ LinArgs a, int32_t* __restrict__ stat
     uint32_t tcount = 0;
     bool ok = true;
     for (int t = blockIdx.x; ok && t < total; t += gridDim.x, ++tcount) {
-      const int m0 = (t % a.mblocks) * kTileM, n0 = (t / a.mblocks) * kTileN;
-      const uint32_t ab = tcount & 1;
-      if (!mbar_wait(&acc_full[ab], (tcount >> 1) & 1)) { ok = false; break; }
+      const int m0 = (t % a.mblocks) * (S::kMT * kTileM), n0 = (t / a.mblocks) * kTileN;
+      const uint32_t ab = S::kMT == 1 ? (tcount & 1) : 0u;
+      const uint32_t use = S::kMT == 1 ? (tcount >> 1) : tcount;
+      if (!mbar_wait(&acc_full[ab], use & 1)) { ok = false; break; }
       tc_fence_after_sync();
-      const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + ab * kTileN;
-      const int row = m0 + q * 32 + lane;
-      uint16_t* drow = a.D + (int64_t)row * a.ldd;
 #pragma unroll 1
-      for (int c = 0; c < kTileN / 32; ++c) {
+      for (int cc = 0; cc < S::kMT * (kTileN / 32); ++cc) {
+        const int h = cc / (kTileN / 32), c = cc % (kTileN / 32);      // row block of the tile, 32-column piece
+        const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (ab + h) * kTileN;
+        const int row = m0 + h * kTileM + q * 32 + lane;
+        uint16_t* drow = a.D + (int64_t)row * a.ldd;
         uint32_t v[32];
         tmem_ld_32x32(tacc + 32 * c, v);
         tmem_ld_wait();
-        if (c == kTileN / 32 - 1) {                    // every read of this accumulator has landed
+        if (cc == S::kMT * (kTileN / 32) - 1) {        // every read of this tile's accumulators has landed
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(&acc_empty[ab]);
@@ -558,7 +573,14 @@ template <int MODE>
 int launch_mode(const LinArgs& args, int32_t* status, cudaStream_t st) {
   using S = LinSmem<MODE>;
   auto kern = int8_linear_kernel<MODE>;
-  QG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
+  static bool smem_set[64] = {};                     // opted into its shared memory, per device
+  int dev = 0;
+  QG_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QG_UNSUPPORTED_SHAPE;
+  if (!smem_set[dev]) {
+    QG_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kBytes));
+    smem_set[dev] = true;
+  }
   const int total = args.mblocks * args.nblocks;
   const int sms = device_sms();
   kern<<<total < sms ? total : sms, S::kThreads, S::kBytes, st>>>(args, status);
@@ -599,7 +621,9 @@ int launch_int8_linear(int mode, const uint16_t* act, int64_t ld_act, const uint
     }
   }
   if (!ok) return QG_CUDA_ERROR;
-  a.mblocks = (a.rows + kTileM - 1) / kTileM;
+  // tiles per column of tiles: the input gradient's tiles are two row blocks high
+  const int tile_rows = mode == kInputGrad ? LinSmem<kInputGrad>::kMT * kTileM : kTileM;
+  a.mblocks = (a.rows + tile_rows - 1) / tile_rows;
   a.nblocks = (a.cols + kTileN - 1) / kTileN;
   if ((int64_t)a.mblocks * a.nblocks > (int64_t)1 << 30) return QG_UNSUPPORTED_SHAPE;   // the tile index is an int
   if (mode == kForward) {
