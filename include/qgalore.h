@@ -357,6 +357,10 @@ QG_API int qgalore_debug_set_fused_dequant(int on);
 /* 1 (the default): the early iterations of a refresh take their two products with the gradient on the tensor cores
  * (the iterate split into three bfloat16 planes); 0: every product on the CUDA cores. */
 QG_API int qgalore_debug_set_refresh_tensor_cores(int on);
+/* 1 (the default): the eigen-iteration of a refresh handles the rows of the projected matrix in blocks of eight
+ * kept in shared memory and registers (block widths up to 2048); 0: row by row through L2, the form wider blocks
+ * take.  Applies to calls made afterwards; both meet the same accuracy bound, their results differ in the last bits. */
+QG_API int qgalore_debug_set_jacobi_blocks(int on);
 /* Scratch bytes a chunk of a plan may use (plans created afterwards; at least 1 MiB).  Larger chunks mean
  * fewer, longer launches; smaller ones keep the bf16 direction between the two kernels inside L2. */
 QG_API int qgalore_debug_set_chunk_budget(size_t bytes);

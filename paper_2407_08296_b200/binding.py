@@ -117,6 +117,7 @@ def lib() -> C.CDLL:
         L.qgalore_kernel_revision.restype = C.c_char_p
         L.qgalore_debug_set_step_impl.argtypes = [C.c_int]
         L.qgalore_debug_set_pair_mode.argtypes = [C.c_int]
+        L.qgalore_debug_set_jacobi_blocks.argtypes = [C.c_int]
         L.qgalore_debug_set_fused_dequant.argtypes = [C.c_int]
         L.qgalore_debug_set_refresh_tensor_cores.argtypes = [C.c_int]
         L.qgalore_debug_set_chunk_budget.argtypes = [sz]
@@ -610,6 +611,10 @@ def debug_set_step_impl(impl: int) -> None:
 
 
 DEFAULT_PAIR_MODE = 6
+
+
+def debug_set_jacobi_blocks(on: bool) -> None:
+    _check(lib().qgalore_debug_set_jacobi_blocks(1 if on else 0), "qgalore_debug_set_jacobi_blocks")
 
 
 def debug_set_pair_mode(mask: int) -> None:

@@ -41,6 +41,7 @@ int tc_kernel_info(char* buf, size_t cap);
 int set_pair_mode(int mask);
 int set_fused_dequant(int on);
 int set_refresh_tc(int on);
+int set_jacobi_blocks(int on);
 int set_chunk_budget(size_t bytes);
 
 static int g_step_impl = 0;  // 0: tensor-core kernels; 1: CUDA-core kernels (validation aid)
@@ -479,6 +480,7 @@ int qgalore_debug_kernel_info(char* buf, size_t capacity) {
 int qgalore_debug_set_pair_mode(int mask) { return set_pair_mode(mask); }
 int qgalore_debug_set_fused_dequant(int on) { return set_fused_dequant(on); }
 int qgalore_debug_set_refresh_tensor_cores(int on) { return set_refresh_tc(on); }
+int qgalore_debug_set_jacobi_blocks(int on) { return set_jacobi_blocks(on); }
 int qgalore_debug_set_chunk_budget(size_t bytes) { return bytes >= (1u << 20) ? set_chunk_budget(bytes) : QG_INVALID_ARGUMENT; }
 
 /* Test aid: selects the CUDA-core (1) or the tensor-core (0) kernels of qgalore_project_step. */

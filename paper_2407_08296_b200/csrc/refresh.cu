@@ -1035,6 +1035,7 @@ int launch_refresh_batched(const RefreshJob* jobs, int count, int64_t m, int64_t
 }
 
 int set_refresh_tc(int on) { g_refresh_tc = on ? 1 : 0; return QG_OK; }
+int set_jacobi_blocks(int on) { g_jacobi_blocks = on ? 1 : 0; return QG_OK; }
 
 int launch_refresh(const uint16_t* G, int64_t ldg, int64_t m, int64_t n, int64_t r, int64_t b, int iters, int sweeps,
                    uint64_t seed, const qg_qtensor* P_new, float* P_fp32, void* ws, size_t ws_bytes, int32_t* status,

@@ -114,6 +114,17 @@ def test_refresh_subspace_matches_exact_svd(m, n, r):
     run_refresh_case(m, n, r, seed=m + r)
 
 
+def test_refresh_with_the_row_by_row_eigen_iteration():
+    # blocks wider than 2048 columns do not fit the block form of the Jacobi iteration and take the row-by-row form;
+    # here the same form is selected on a small shape
+    B.debug_set_jacobi_blocks(False)
+    try:
+        run_refresh_case(768, 768, 256, seed=1024)
+        run_refresh_case(512, 1376, 128, seed=640)
+    finally:
+        B.debug_set_jacobi_blocks(True)
+
+
 def test_refresh_reports_similarity_with_previous_projection():
     m, n, r = 256, 512, 64
     gm = synth.GradientModel(m, n, seed=9, matrix_index=0)
