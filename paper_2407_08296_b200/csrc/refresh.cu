@@ -8,21 +8,23 @@
 //   repeat iters times:   Z = G^T Q  (n x b);   Y = G Z  (m x b);   Q <- orth(Y)
 //   Z = G^T Q;   T = Z^T Z  (b x b, summed in fp64);   T = X diag(lambda) X^T;   P = Q X[:, top r]
 //
-// Everything heavy is a GEMM (one generic fp32 kernel, fp64 accumulation for T).  orth() is block
-// Gram-Schmidt over panels of 64 columns, each projection done twice, the panel itself by two rounds of
-// Cholesky QR.  The eigenvectors of T come from a one-sided (Hestenes) Jacobi iteration (rows kept in fp32, every
-// sum and rotation angle in fp64: the result is INT4 in the end, and a round is bound by the bytes it moves) with a
-// round-robin pair ordering: all sweeps in one cooperative launch, a grid barrier between rounds of b/2 disjoint pairs.  Each column of P is then
-// given the sign that makes its largest entry positive, and P is quantized to INT4 (Quant_4).
+// The products with G run on the tensor cores (refresh_tc.cu: the fp32 iterate split into three bfloat16 planes,
+// every product exact, fp32 accumulation); everything else is a generic fp32 GEMM kernel on the CUDA cores (fp64
+// accumulation for T).  orth() is block Gram-Schmidt over panels of 64 columns with Cholesky QR of the panel: every
+// projection twice and two rounds of Cholesky QR in the last iterations, one of each before.  The eigenvectors of T
+// come from a one-sided (Hestenes) Jacobi iteration (rows kept in fp32, every sum in fp64: the result is INT4 in the
+// end) over blocks of eight rows held on the SM, all sweeps in one cooperative launch with a grid barrier between the
+// rounds of the tournament of blocks.  Each column of P is then given the sign that makes its largest entry positive,
+// and P is quantized to INT4 (Quant_4).
 //
 // Several matrices of one shape are refreshed together (a "batch", up to kMaxBatch): every launch carries a matrix
 // index beside its tile index and reads its operands from small pointer tables passed by value, so the few
-// thousand small launches and the ~9000 grid barriers of the eigen-iteration are paid once per batch instead of
+// thousand small launches and the grid barriers of the eigen-iteration (about 1200) are paid once per batch instead of
 // once per matrix.
 //
-// The arithmetic is plain fp32/fp64 on the CUDA cores: the singular values next to the r-th one sit in the
-// noise bulk of the gradient with relative gaps of 1e-4..1e-3, and resolving that subspace to 1e-2 rad
-// needs fp32-faithful products (bf16 tensor-core products do not get there).
+// The singular values next to the r-th one sit in the noise bulk of the gradient with relative gaps of 1e-4..1e-3,
+// and resolving that subspace to 1e-2 rad needs fp32-faithful products: plain bf16 tensor-core products of the
+// iterate do not get there, the three-plane split does.
 #include <cmath>
 #include <mutex>
 
